@@ -1,0 +1,390 @@
+/*
+ * nm_oracle.c -- TEST INFRASTRUCTURE, NOT PRODUCT CODE.
+ *
+ * A plain, slow, scalar CPU statement of what the N:M low-bit path computes,
+ * written from the paper (arxiv 2206.15014) so that the CUDA library can be
+ * checked against it.  It shares no code, header, table or helper with the
+ * CUDA path and is only ever called from tests, from the smoke check and from
+ * the benchmark's CPU-baseline leg.
+ *
+ * Conventions (kept:group, i.e. "2:4" keeps n=2 of every m=4):
+ *   W, U        fp32 [out, in] row-major (nn.Linear layout); groups of m run
+ *               along `in`, the reduction dimension.
+ *   values      kept integer codes, ascending position inside each group,
+ *               row-major [out, in*n/m]; 8-bit: one byte each; 4-bit: two's
+ *               complement nibbles, even element in bits 3:0, odd in bits 7:4.
+ *   meta        position-in-group of each kept element; 2-bit fields for m=4,
+ *               4-bit fields for m=8, LSB first in element order, packed into
+ *               little-endian u32 words, each row padded to whole words.
+ *               n == m has no metadata.
+ *   scales      fp32 [out], one per output channel.
+ *
+ * Parity status of the pieces:
+ *   projection (Eq. 3, Sec. 3.2), ADMM-Max scale (Sec. 3.3.1), quantiser
+ *   (Eq. 5), dequantisation (Eq. 4), integer linear layer (Sec. 5.3): pinned by
+ *   the CPU tests (brute-force Euclidean projection, idempotence, scale
+ *   invariance under pruning, textbook absmax quantisation, int64 numpy matmul,
+ *   double-precision epilogue, the paper's Table 1 / Table 4 size accounting).
+ *   The byte-level packing of values and metadata is this library's own
+ *   convention (the paper specifies none): parity unpinned beyond the
+ *   pack -> unpack round trip and the 2-index-bits-per-kept-value accounting.
+ */
+#include <math.h>
+#include <stddef.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+#ifdef _OPENMP
+#include <omp.h>
+#endif
+
+#define ORACLE_OK 0
+#define ORACLE_ERR_SHAPE -1
+#define ORACLE_ERR_NONFINITE -2
+#define ORACLE_ERR_OVERFLOW -3
+
+static int g_threads = 1;
+
+/* Number of OpenMP threads used by the row loops (1 = serial). */
+void oracle_set_threads(int t) { g_threads = t < 1 ? 1 : t; }
+int oracle_get_threads(void) { return g_threads; }
+int oracle_max_threads(void)
+{
+#ifdef _OPENMP
+    return omp_get_num_procs();
+#else
+    return 1;
+#endif
+}
+
+static int field_bits(int m) { return m == 4 ? 2 : 4; }
+
+static int shape_ok(int out, int in, int n, int m, int bits)
+{
+    if (out < 0 || in < 0 || n < 1 || m < 1 || n > m) return 0;
+    if (bits != 4 && bits != 8) return 0;
+    if (n != m && m != 4 && m != 8) return 0;
+    if (in % m) return 0;
+    if (((long long)(in / m) * n * bits) % 8) return 0;
+    return 1;
+}
+
+/* Bytes of one packed row of values / words of one row of metadata. */
+static size_t values_row_bytes(int in, int n, int m, int bits)
+{
+    return (size_t)(in / m) * n * bits / 8;
+}
+static size_t meta_row_words(int in, int n, int m)
+{
+    if (n == m) return 0;
+    size_t row_bits = (size_t)(in / m) * n * field_bits(m);
+    return (row_bits + 31) / 32;
+}
+
+int oracle_packed_sizes(int out, int in, int n, int m, int bits, size_t *values_bytes,
+                        size_t *meta_bytes)
+{
+    if (!shape_ok(out, in, n, m, bits)) return ORACLE_ERR_SHAPE;
+    *values_bytes = (size_t)out * values_row_bytes(in, n, m, bits);
+    *meta_bytes = (size_t)out * meta_row_words(in, n, m) * 4;
+    return ORACLE_OK;
+}
+
+/*
+ * Support of the Euclidean projection of one group onto "at most n non-zeros
+ * out of m" (Eq. 2-3; Sec. 3.2: keep the largest entries of each contiguous
+ * group).  The largest are the largest in magnitude -- that is what minimises
+ * the Frobenius distance.  Equal magnitudes: the lower index is kept.  A stable
+ * insertion sort by descending |v| gives exactly that order.  keep[] receives
+ * the n chosen positions in ascending order.
+ */
+static void group_support(const float *v, int n, int m, int *keep)
+{
+    int idx[64];
+    for (int i = 0; i < m; ++i) idx[i] = i;
+    for (int i = 1; i < m; ++i) {
+        int cur = idx[i];
+        float a = fabsf(v[cur]);
+        int j = i - 1;
+        while (j >= 0 && fabsf(v[idx[j]]) < a) { /* strict: equal keys keep their order */
+            idx[j + 1] = idx[j];
+            --j;
+        }
+        idx[j + 1] = cur;
+    }
+    /* first n of the sorted order, then ascending by position */
+    for (int i = 0; i < n; ++i) keep[i] = idx[i];
+    for (int i = 1; i < n; ++i) {
+        int cur = keep[i], j = i - 1;
+        while (j >= 0 && keep[j] > cur) {
+            keep[j + 1] = keep[j];
+            --j;
+        }
+        keep[j + 1] = cur;
+    }
+}
+
+/*
+ * ADMM-Max scale of one output channel (Sec. 3.3.1, "Minimize Error on the
+ * Largest Parameter"): the largest magnitude of W+U divided by the largest
+ * integer code 2^(b-1)-1.  An all-zero channel gets scale 1.
+ */
+static float row_scale(const float *v, int in, int bits)
+{
+    float a = 0.0f;
+    for (int k = 0; k < in; ++k) {
+        float t = fabsf(v[k]);
+        if (t > a) a = t;
+    }
+    float qmax = (float)((1 << (bits - 1)) - 1);
+    return a == 0.0f ? 1.0f : a / qmax;
+}
+
+/* Eq. 5 with offset 0: clamp(round(x / s), -2^(b-1), 2^(b-1)-1), round = half to even. */
+static int quantise(float x, float s, int bits)
+{
+    int hi = (1 << (bits - 1)) - 1, lo = -(1 << (bits - 1));
+    float r = nearbyintf(x / s); /* default rounding mode: to nearest, ties to even */
+    if (r > (float)hi) return hi;
+    if (r < (float)lo) return lo;
+    return (int)r;
+}
+
+static int row_finite(const float *v, int in)
+{
+    for (int k = 0; k < in; ++k)
+        if (!isfinite(v[k])) return 0;
+    return 1;
+}
+
+/*
+ * Joint projection of Sec. 3.3.1 (last paragraph): sparsity constraint, then
+ * quantisation constraint, scale from ADMM-Max.  V = W + U is the Z-update's
+ * argument (Eq. 3); U may be NULL.
+ */
+int oracle_project_pack(const float *W, const float *U, int out, int in, int n, int m, int bits,
+                        uint8_t *values, uint32_t *meta, float *scales)
+{
+    if (!shape_ok(out, in, n, m, bits)) return ORACLE_ERR_SHAPE;
+    const size_t vrb = values_row_bytes(in, n, m, bits);
+    const size_t mrw = meta_row_words(in, n, m);
+    const int fb = field_bits(m);
+    int status = ORACLE_OK;
+#pragma omp parallel for schedule(static) num_threads(g_threads)
+    for (int r = 0; r < out; ++r) {
+        float *v = (float *)malloc(sizeof(float) * (size_t)(in > 0 ? in : 1));
+        for (int k = 0; k < in; ++k) {
+            float w = W[(size_t)r * in + k];
+            v[k] = U ? w + U[(size_t)r * in + k] : w;
+        }
+        if (!row_finite(v, in)) {
+#pragma omp atomic write
+            status = ORACLE_ERR_NONFINITE;
+        }
+        float s = row_scale(v, in, bits);
+        scales[r] = s;
+        uint8_t *vrow = values + (size_t)r * vrb;
+        uint32_t *mrow = meta ? meta + (size_t)r * mrw : NULL;
+        memset(vrow, 0, vrb);
+        if (mrow) memset(mrow, 0, mrw * 4);
+        size_t e = 0; /* index of the kept element inside the row */
+        for (int g = 0; g < in / m; ++g) {
+            int keep[64];
+            group_support(v + (size_t)g * m, n, m, keep);
+            for (int i = 0; i < n; ++i, ++e) {
+                int q = quantise(v[(size_t)g * m + keep[i]], s, bits);
+                if (bits == 8) {
+                    vrow[e] = (uint8_t)(int8_t)q;
+                } else {
+                    uint8_t nib = (uint8_t)(q & 0xF);
+                    vrow[e / 2] |= (e & 1) ? (uint8_t)(nib << 4) : nib;
+                }
+                if (mrow) {
+                    size_t bit = e * (size_t)fb;
+                    mrow[bit / 32] |= (uint32_t)keep[i] << (bit % 32);
+                }
+            }
+        }
+        free(v);
+    }
+    return status;
+}
+
+/* Inverse of the packing: dense integer codes [out, in], zero where pruned. */
+int oracle_unpack(const uint8_t *values, const uint32_t *meta, int out, int in, int n, int m,
+                  int bits, int8_t *Wq)
+{
+    if (!shape_ok(out, in, n, m, bits)) return ORACLE_ERR_SHAPE;
+    const size_t vrb = values_row_bytes(in, n, m, bits);
+    const size_t mrw = meta_row_words(in, n, m);
+    const int fb = field_bits(m);
+    for (int r = 0; r < out; ++r) {
+        const uint8_t *vrow = values + (size_t)r * vrb;
+        const uint32_t *mrow = meta ? meta + (size_t)r * mrw : NULL;
+        int8_t *drow = Wq + (size_t)r * in;
+        memset(drow, 0, (size_t)in);
+        size_t e = 0;
+        for (int g = 0; g < in / m; ++g) {
+            for (int i = 0; i < n; ++i, ++e) {
+                int q;
+                if (bits == 8) {
+                    q = (int8_t)vrow[e];
+                } else {
+                    int nib = (vrow[e / 2] >> ((e & 1) ? 4 : 0)) & 0xF;
+                    q = nib >= 8 ? nib - 16 : nib;
+                }
+                int pos = i;
+                if (n != m) {
+                    size_t bit = e * (size_t)fb;
+                    pos = (int)((mrow[bit / 32] >> (bit % 32)) & ((1u << fb) - 1u));
+                }
+                drow[(size_t)g * m + pos] = (int8_t)q;
+            }
+        }
+    }
+    return ORACLE_OK;
+}
+
+/* Sparsity projection alone (Eq. 3): Z = Pi_S(W + U) as dense fp32. */
+int oracle_project_dense(const float *W, const float *U, int out, int in, int n, int m, float *Z)
+{
+    if (n < 1 || n > m || m > 64 || in % m) return ORACLE_ERR_SHAPE;
+    for (int r = 0; r < out; ++r)
+        for (int g = 0; g < in / m; ++g) {
+            float v[64];
+            int keep[64];
+            size_t base = (size_t)r * in + (size_t)g * m;
+            for (int i = 0; i < m; ++i) {
+                v[i] = U ? W[base + i] + U[base + i] : W[base + i];
+                Z[base + i] = 0.0f;
+            }
+            group_support(v, n, m, keep);
+            for (int i = 0; i < n; ++i) Z[base + keep[i]] = v[keep[i]];
+        }
+    return ORACLE_OK;
+}
+
+/* Per-channel ADMM-Max scales of an fp32 matrix (Sec. 3.3.1). */
+int oracle_row_scales(const float *V, int out, int in, int bits, float *scales)
+{
+    for (int r = 0; r < out; ++r) scales[r] = row_scale(V + (size_t)r * in, in, bits);
+    return ORACLE_OK;
+}
+
+/*
+ * STE forward pass (Sec. 3.3.2): the weight the forward pass sees is the
+ * dequantised quantised one, x_d = s * x_q (Eq. 4 with o = 0), here applied to
+ * an fp32 matrix Z elementwise with the given per-row scales.
+ */
+int oracle_fake_quant(const float *Z, int out, int in, int bits, const float *scales, float *Zq)
+{
+    for (int r = 0; r < out; ++r)
+        for (int k = 0; k < in; ++k) {
+            size_t i = (size_t)r * in + k;
+            Zq[i] = scales[r] * (float)quantise(Z[i], scales[r], bits);
+        }
+    return ORACLE_OK;
+}
+
+/*
+ * Integer linear layer (Sec. 5.3): 8-bit activations times weights widened to
+ * 8 bits, exact integer accumulation, then dequantisation (Eq. 4):
+ *   acc[t,o] = sum_k X[t,k] * Wq[o,k]          (int64, every k, zeros included)
+ *   y[t,o]   = fma((float)acc, sx * sw[o], bias[o])
+ * ACC (nullable) receives the accumulators as int32.
+ */
+int oracle_int_linear(const int8_t *X, int tokens, const int8_t *Wq, int out, int in, float sx,
+                      const float *sw, const float *bias, int32_t *ACC, float *Y)
+{
+    int status = ORACLE_OK;
+#pragma omp parallel for schedule(static) num_threads(g_threads)
+    for (int t = 0; t < tokens; ++t) {
+        const int8_t *x = X + (size_t)t * in;
+        for (int o = 0; o < out; ++o) {
+            const int8_t *w = Wq + (size_t)o * in;
+            int64_t acc = 0;
+            for (int k = 0; k < in; ++k) acc += (int64_t)x[k] * (int64_t)w[k];
+            if (acc > INT32_MAX || acc < INT32_MIN) {
+#pragma omp atomic write
+                status = ORACLE_ERR_OVERFLOW;
+            }
+            if (ACC) ACC[(size_t)t * out + o] = (int32_t)acc;
+            if (Y) {
+                float c = sx * sw[o];
+                float b = bias ? bias[o] : 0.0f;
+                Y[(size_t)t * out + o] = fmaf((float)(int32_t)acc, c, b);
+            }
+        }
+    }
+    return status;
+}
+
+/*
+ * The same accumulators, summed over the kept positions only, walking the
+ * packed form: "only computing half the operations" (Sec. 5.3) must not change
+ * the result.
+ */
+int oracle_int_linear_kept(const int8_t *X, int tokens, const uint8_t *values, const uint32_t *meta,
+                           int out, int in, int n, int m, int bits, int32_t *ACC)
+{
+    if (!shape_ok(out, in, n, m, bits)) return ORACLE_ERR_SHAPE;
+    const size_t vrb = values_row_bytes(in, n, m, bits);
+    const size_t mrw = meta_row_words(in, n, m);
+    const int fb = field_bits(m);
+    for (int t = 0; t < tokens; ++t)
+        for (int o = 0; o < out; ++o) {
+            const uint8_t *vrow = values + (size_t)o * vrb;
+            const uint32_t *mrow = meta ? meta + (size_t)o * mrw : NULL;
+            int64_t acc = 0;
+            size_t e = 0;
+            for (int g = 0; g < in / m; ++g)
+                for (int i = 0; i < n; ++i, ++e) {
+                    int q;
+                    if (bits == 8) {
+                        q = (int8_t)vrow[e];
+                    } else {
+                        int nib = (vrow[e / 2] >> ((e & 1) ? 4 : 0)) & 0xF;
+                        q = nib >= 8 ? nib - 16 : nib;
+                    }
+                    int pos = i;
+                    if (n != m) {
+                        size_t bit = e * (size_t)fb;
+                        pos = (int)((mrow[bit / 32] >> (bit % 32)) & ((1u << fb) - 1u));
+                    }
+                    acc += (int64_t)X[(size_t)t * in + (size_t)g * m + pos] * q;
+                }
+            ACC[(size_t)t * out + o] = (int32_t)acc;
+        }
+    return ORACLE_OK;
+}
+
+/*
+ * Dynamic per-tensor symmetric 8-bit activation quantiser: Eq. 5 with b = 8 and
+ * the scale chosen as for ADMM-Max over the whole tensor (max|y| / 127).
+ */
+int oracle_quantize_act(const float *Y, size_t count, int8_t *Xq, float *sx)
+{
+    float a = 0.0f;
+    for (size_t i = 0; i < count; ++i) {
+        float t = fabsf(Y[i]);
+        if (t > a) a = t;
+    }
+    float s = a == 0.0f ? 1.0f : a / 127.0f;
+    *sx = s;
+    for (size_t i = 0; i < count; ++i) Xq[i] = (int8_t)quantise(Y[i], s, 8);
+    return ORACLE_OK;
+}
+
+/*
+ * Storage accounting behind the paper's size columns (Table 1, Table 4): bits
+ * per dense parameter of an n:m sparse b-bit matrix = value bits of the kept
+ * entries plus index bits per kept entry.  index_bits < 0 selects this
+ * library's field width (2 for m=4, 4 for m=8); the paper's tables correspond
+ * to index_bits = 2 at m = 4.
+ */
+double oracle_bits_per_param(int n, int m, int bits, int index_bits)
+{
+    if (n == m) return (double)bits;
+    int ib = index_bits < 0 ? field_bits(m) : index_bits;
+    return ((double)n / (double)m) * (double)(bits + ib);
+}
