@@ -1,0 +1,172 @@
+/*
+ * nmsparse.h -- C ABI of the B200 (sm_100a) N:M-sparse low-bit integer linear layer and of the
+ * projection / quantise / pack step that produces its weights.
+ *
+ * The operations are those of "Compressing Pre-trained Transformers via Low-Bit NxM Sparsity"
+ * (arxiv 2206.15014).  Patterns are written kept:group -- "2:4" keeps n = 2 of every m = 4
+ * consecutive weights (the paper writes the same pattern "4:2").
+ *
+ * General rules for every entry point
+ *   - Pointers are DEVICE pointers unless the comment says "host".  The caller owns every buffer;
+ *     the library allocates nothing and keeps no pointer after a call returns.
+ *   - Calls enqueue work on `stream` (a cudaStream_t passed as void*, NULL = default stream) and
+ *     return without synchronising, unless stated.
+ *   - Return value: NM_OK or a negative NM_ERR_* code detected on the host; nothing is enqueued
+ *     when an error is returned.  Conditions only the device can see (non-finite weights, a bounded
+ *     wait that expired) are OR-ed as NM_STATUS_* bits into the optional `status` device word,
+ *     which the caller zeroes beforehand and reads with nm_poll_status().
+ *   - No exceptions, no exit(), no output to stdout/stderr.
+ *
+ * Layouts
+ *   W, U     fp32 [out, in] row-major (nn.Linear layout).  Groups of m run along `in`, the reduction
+ *            dimension.  `in` must be a multiple of m and of 4; rows must start 16-byte aligned.
+ *   values   kept integer codes in ascending position inside each group, row-major
+ *            [out, in*n/m].  bits = 8: one int8 per code.  bits = 4: two's-complement nibbles, even
+ *            element in bits 3:0 and odd element in bits 7:4 of a byte.
+ *   meta     position-in-group of each kept code: 2-bit fields for m = 4, 4-bit fields for m = 8,
+ *            least-significant field first in element order, in little-endian u32 words; every row
+ *            is padded with zero bits to a whole number of words.  n == m (dense) has no metadata.
+ *   scales   fp32 [out], one symmetric scale per output channel.
+ *   X        int8 [tokens, in] row-major;  Y fp32 [tokens, out] row-major.
+ */
+#ifndef NMSPARSE_H_
+#define NMSPARSE_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define NM_OK 0
+#define NM_ERR_NULL (-1)        /* a required pointer is NULL */
+#define NM_ERR_SHAPE (-2)       /* n < 1, n > m, in % m != 0, negative size, row not a whole number of bytes */
+#define NM_ERR_UNSUPPORTED (-3) /* m not in {4, 8} (unless n == m), bits not in {4, 8}, size beyond a stated limit */
+#define NM_ERR_ALIGN (-4)       /* pointer or row pitch not aligned as the call requires */
+#define NM_ERR_WORKSPACE (-5)   /* workspace missing or smaller than nm_*_workspace_bytes() */
+#define NM_ERR_CUDA (-6)        /* a CUDA runtime / driver call failed (see nm_last_cuda_error) */
+#define NM_ERR_NONFINITE (-7)   /* reported by nm_poll_status: NaN or Inf met in W + U */
+#define NM_ERR_TIMEOUT (-8)     /* reported by nm_poll_status: a bounded device-side wait expired */
+
+#define NM_STATUS_NONFINITE 1u /* bit in the device status word */
+#define NM_STATUS_TIMEOUT 2u   /* bit in the device status word */
+
+/* A packed weight matrix: host struct holding device pointers (see "Layouts"). */
+typedef struct nm_packed_t {
+    int32_t out, in; /* output channels, input features (reduction length) */
+    int32_t n, m;    /* kept : group; n == m means dense */
+    int32_t bits;    /* 8 or 4 */
+    const void *values;
+    const void *meta; /* NULL iff n == m */
+} nm_packed_t;
+
+/* One matrix of a batched projection (host struct, device pointers). */
+typedef struct nm_pack_job_t {
+    const float *W;
+    const float *U; /* NULL: project W alone */
+    int32_t out, in, n, m, bits;
+    void *values;
+    void *meta; /* NULL iff n == m */
+    float *scales;
+} nm_pack_job_t;
+
+/*
+ * Sizes in bytes of `values` and `meta` for an [out, in] matrix (host only, touches no device).
+ * Storage accounting of Table 1 / Table 4: value bits plus index bits per kept weight.
+ */
+int nm_packed_sizes(int out, int in, int n, int m, int bits, size_t *values_bytes,
+                    size_t *meta_bytes);
+
+/*
+ * N:M magnitude projection + per-output-channel symmetric quantisation + packing of one matrix.
+ *   V = W + U                          argument of the ADMM Z-update, Eq. 3 (U may be NULL)
+ *   support = the n largest |v| of every group of m, equal magnitudes -> lower index kept
+ *                                      (Euclidean projection onto the N:M constraint, Sec. 3.2)
+ *   s[r] = max_k |V[r,k]| / (2^(bits-1) - 1),  s[r] = 1 for an all-zero row
+ *                                      (ADMM-Max scale, Sec. 3.3.1)
+ *   q = clamp(rne(v / s[r]), -2^(bits-1), 2^(bits-1) - 1)      (Eq. 5, offset 0)
+ * The same arithmetic is the forward fake-quantisation of STE-QAT (Sec. 3.3.2): s * q.
+ * Accepted: (n, m) in {1:4, 2:4, 1:8, 2:8, 4:8} or n == m; bits in {4, 8}; in <= 32768.
+ * W, U, values 16-byte aligned, meta and scales 4-byte aligned.
+ * Sets NM_STATUS_NONFINITE in *status (nullable) when W + U holds NaN/Inf; outputs of such rows are
+ * unspecified.  One pass over W and U; outputs are written once.
+ */
+int nm_project_pack(const float *W, const float *U, int out, int in, int n, int m, int bits,
+                    void *values, void *meta, float *scales, uint32_t *status, void *stream);
+
+/*
+ * The same for a list of matrices with as few launches as their (n, m, bits) allow (one when all
+ * jobs share them).  `jobs` is a host array; `ws` is device scratch of at least
+ * nm_pack_workspace_bytes(njobs) bytes, 16-byte aligned, which must stay untouched until the
+ * enqueued work has finished.  The host array may be reused as soon as the call returns.
+ */
+int nm_project_pack_batched(const nm_pack_job_t *jobs, int njobs, void *ws, size_t ws_bytes,
+                            uint32_t *status, void *stream);
+size_t nm_pack_workspace_bytes(int njobs);
+
+/*
+ * Integer N:M linear layer (Sec. 5.3: 8-bit activations, weights of <= 8 bits widened to 8 bits for
+ * the multipliers, N:M skipping the pruned half of the products) with the dequantisation of Eq. 4
+ * fused in:
+ *   acc[t,o] = sum_k X[t,k] * Wq[o,k]              exact, int32
+ *   Y[t,o]   = fma((float)acc[t,o], sx * sw[o], bias[o])      fp32; bias NULL = 0
+ * W is a host struct; sw = per-channel scales from nm_project_pack; sx = activation scale.
+ * 2:4, 1:4, 2:8 and 1:8 weights run on the sparse tensor-core path, 4:8 and dense weights on the
+ * dense path after decompression in shared memory.  Shape and alignment requirements are those
+ * nm_int_linear_check() tests; X and values 16-byte aligned; Y, sw, bias 4-byte aligned.
+ * `ws`/`ws_bytes`: device scratch of nm_int_linear_workspace_bytes() (may be 0 -> ws may be NULL).
+ */
+int nm_int_linear(const int8_t *X, int tokens, const nm_packed_t *W, float sx, const float *sw,
+                  const float *bias, float *Y, void *ws, size_t ws_bytes, uint32_t *status,
+                  void *stream);
+
+/*
+ * The same with the activation scale read from device memory (*sx_dev), so that a chain of layers
+ * needs no host round trip, and with an optional running maximum: when absmax_out is not NULL the
+ * kernel folds max|Y| into *absmax_out (a float the caller zeroes first; updated atomically).
+ */
+int nm_int_linear_dsx(const int8_t *X, int tokens, const nm_packed_t *W, const float *sx_dev,
+                      const float *sw, const float *bias, float *Y, float *absmax_out, void *ws,
+                      size_t ws_bytes, uint32_t *status, void *stream);
+
+/* The raw int32 accumulators acc[t,o] (row-major [tokens, out]) of the same product, no epilogue. */
+int nm_int_linear_acc(const int8_t *X, int tokens, const nm_packed_t *W, int32_t *ACC, void *ws,
+                      size_t ws_bytes, uint32_t *status, void *stream);
+
+size_t nm_int_linear_workspace_bytes(int tokens, int out, int in, int n, int m, int bits);
+
+/* Host-only validation of a linear-layer problem: NM_OK or the error nm_int_linear would return. */
+int nm_int_linear_check(int tokens, int out, int in, int n, int m, int bits);
+
+/*
+ * Dynamic per-tensor symmetric 8-bit activation quantiser (Eq. 5 with bits = 8; the activations
+ * of the integer layers are 8 bit, Sec. 5.3):
+ *   nm_absmax:        *absmax = max(*absmax, max_i |Y[i]|)   (caller zeroes *absmax first)
+ *   nm_quantize_act:  sx = *absmax / 127 (1 if *absmax == 0);  Xq[i] = clamp(rne(Y[i] / sx), -128, 127)
+ *                     *sx_out (nullable) receives sx.
+ * Y and Xq must be 16-byte aligned.
+ */
+int nm_absmax(const float *Y, size_t count, float *absmax, void *stream);
+int nm_quantize_act(const float *Y, size_t count, const float *absmax, int8_t *Xq, float *sx_out,
+                    void *stream);
+
+/*
+ * Synchronises `stream`, reads the device status word and returns NM_OK, NM_ERR_NONFINITE,
+ * NM_ERR_TIMEOUT or NM_ERR_CUDA.  `status` may be NULL (then only the stream is checked).
+ */
+int nm_poll_status(const uint32_t *status, void *stream);
+
+/* Text for an NM_* code (static storage). */
+const char *nm_strerror(int code);
+
+/* Text of the last CUDA error this thread met inside the library (static storage, "" if none). */
+const char *nm_last_cuda_error(void);
+
+/* Library version, major * 100 + minor. */
+int nm_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* NMSPARSE_H_ */

@@ -1,0 +1,80 @@
+// Host-only entry points of the nmsparse C ABI: sizes, validation, status polling, error text.
+#include "common.cuh"
+#include <stdio.h>
+#include <string.h>
+
+namespace nm {
+
+static thread_local char g_last_error[256] = "";
+
+int record_cuda_error(cudaError_t e, const char* where) {
+    snprintf(g_last_error, sizeof(g_last_error), "%s: %s", where, cudaGetErrorString(e));
+    (void)cudaGetLastError();  // reset the last-error slot so later calls start clean
+    return NM_ERR_CUDA;
+}
+
+int record_text_error(const char* text) {
+    snprintf(g_last_error, sizeof(g_last_error), "%s", text);
+    return NM_ERR_CUDA;
+}
+
+int check_pattern(int out, int in, int n, int m, int bits) {
+    if (out < 0 || in < 0 || n < 1 || m < 1 || n > m) return NM_ERR_SHAPE;
+    if (bits != 4 && bits != 8) return NM_ERR_UNSUPPORTED;
+    if (n != m) {
+        if (m != 4 && m != 8) return NM_ERR_UNSUPPORTED;
+        if (!((m == 4 && (n == 1 || n == 2)) || (m == 8 && (n == 1 || n == 2 || n == 4))))
+            return NM_ERR_UNSUPPORTED;
+    }
+    if (in % m) return NM_ERR_SHAPE;
+    if (((long long)(in / m) * n * bits) % 8) return NM_ERR_SHAPE;
+    return NM_OK;
+}
+
+}  // namespace nm
+
+extern "C" {
+
+int nm_packed_sizes(int out, int in, int n, int m, int bits, size_t* values_bytes,
+                    size_t* meta_bytes) {
+    if (!values_bytes || !meta_bytes) return NM_ERR_NULL;
+    int rc = nm::check_pattern(out, in, n, m, bits);
+    if (rc != NM_OK) return rc;
+    *values_bytes = (size_t)out * nm::values_row_bytes(in, n, m, bits);
+    *meta_bytes = (size_t)out * nm::meta_row_words(in, n, m) * 4;
+    return NM_OK;
+}
+
+int nm_poll_status(const uint32_t* status, void* stream) {
+    cudaStream_t s = (cudaStream_t)stream;
+    cudaError_t e = cudaStreamSynchronize(s);
+    if (e != cudaSuccess) return nm::record_cuda_error(e, "cudaStreamSynchronize");
+    if (!status) return NM_OK;
+    uint32_t h = 0;
+    e = cudaMemcpy(&h, status, sizeof(h), cudaMemcpyDeviceToHost);
+    if (e != cudaSuccess) return nm::record_cuda_error(e, "cudaMemcpy(status)");
+    if (h & NM_STATUS_TIMEOUT) return NM_ERR_TIMEOUT;
+    if (h & NM_STATUS_NONFINITE) return NM_ERR_NONFINITE;
+    return NM_OK;
+}
+
+const char* nm_strerror(int code) {
+    switch (code) {
+        case NM_OK: return "ok";
+        case NM_ERR_NULL: return "a required pointer is NULL";
+        case NM_ERR_SHAPE: return "invalid shape or N:M pattern";
+        case NM_ERR_UNSUPPORTED: return "pattern, bit width or size not supported";
+        case NM_ERR_ALIGN: return "pointer or row pitch not aligned as required";
+        case NM_ERR_WORKSPACE: return "workspace missing or too small";
+        case NM_ERR_CUDA: return "a CUDA call failed (see nm_last_cuda_error)";
+        case NM_ERR_NONFINITE: return "NaN or Inf met in W + U";
+        case NM_ERR_TIMEOUT: return "a bounded device-side wait expired";
+        default: return "unknown nmsparse code";
+    }
+}
+
+const char* nm_last_cuda_error(void) { return nm::g_last_error; }
+
+int nm_version(void) { return 100; }
+
+}  // extern "C"

@@ -1,0 +1,390 @@
+// N:M magnitude projection + per-channel symmetric quantisation + packing (one HBM pass).
+//
+// Work decomposition: a warp owns a chunk of 1024 consecutive weights of one row; a row is
+// covered by 1, 2, 4 ... 32 warps of the same block.  Loads are coalesced 16-byte accesses
+// (lane l, step j -> float4 number j*32+l of the chunk); the sum V = W + U goes through a
+// swizzled shared-memory tile so that afterwards every lane holds 32 CONSECUTIVE values (8 groups
+// of 4 or 4 groups of 8).  From there everything is lane-local: the lane's share of the packed
+// values and of the metadata is a whole number of bytes, written with one vector store each.
+#include "common.cuh"
+#include <cuda_runtime.h>
+#include <vector>
+#include <algorithm>
+
+namespace nm {
+
+struct PackJobDev {
+    const float* W;
+    const float* U;
+    uint8_t* values;
+    uint32_t* meta;
+    float* scales;
+    int out, in;
+    int wpr_log2;         // log2(warps per row)
+    unsigned unit_begin;  // first block of this job inside the launch
+    unsigned vrow_bytes;  // bytes of one row of values
+    unsigned mrow_words;  // words of one row of metadata
+};
+
+static constexpr int kPackMinWarps = 4;
+
+__device__ __forceinline__ float4 ld_stream(const float4* p) { return __ldcs(p); }
+
+// Bit mask of the positions kept in one group: position i is kept iff fewer than N others beat it,
+// where j beats i when |v_j| > |v_i|, or |v_j| == |v_i| and j < i.
+template <int N, int M>
+__device__ __forceinline__ unsigned keep_mask(const float* a) {
+    int rank[M];
+#pragma unroll
+    for (int i = 0; i < M; ++i) rank[i] = 0;
+#pragma unroll
+    for (int i = 0; i < M; ++i)
+#pragma unroll
+        for (int j = i + 1; j < M; ++j) {
+            bool ge = a[i] >= a[j];  // i (the lower index) beats j on >=, j beats i otherwise
+            rank[j] += ge ? 1 : 0;
+            rank[i] += ge ? 0 : 1;
+        }
+    unsigned mask = 0;
+#pragma unroll
+    for (int i = 0; i < M; ++i) mask |= (rank[i] < N ? 1u : 0u) << i;
+    return mask;
+}
+
+template <int BITS>
+__device__ __forceinline__ unsigned quantise_code(float v, float s) {
+    constexpr int hi = (1 << (BITS - 1)) - 1, lo = -(1 << (BITS - 1));
+    int q = __float2int_rn(__fdiv_rn(v, s));  // IEEE division, round half to even
+    q = max(lo, min(hi, q));
+    return (unsigned)q & ((1u << BITS) - 1u);
+}
+
+template <int NBYTES>
+__device__ __forceinline__ void store_bytes_vec(uint8_t* dst, const unsigned* w) {
+    if constexpr (NBYTES == 2) *reinterpret_cast<uint16_t*>(dst) = (uint16_t)w[0];
+    else if constexpr (NBYTES == 4) *reinterpret_cast<uint32_t*>(dst) = w[0];
+    else if constexpr (NBYTES == 8) *reinterpret_cast<uint2*>(dst) = make_uint2(w[0], w[1]);
+    else if constexpr (NBYTES == 16) *reinterpret_cast<uint4*>(dst) = make_uint4(w[0], w[1], w[2], w[3]);
+    else {
+        static_assert(NBYTES == 32, "unexpected lane share");
+        reinterpret_cast<uint4*>(dst)[0] = make_uint4(w[0], w[1], w[2], w[3]);
+        reinterpret_cast<uint4*>(dst)[1] = make_uint4(w[4], w[5], w[6], w[7]);
+    }
+}
+
+template <int MAXBYTES>
+__device__ __forceinline__ void store_bytes_slow(uint8_t* dst, const unsigned* w, int nbytes) {
+#pragma unroll
+    for (int i = 0; i < MAXBYTES; ++i)
+        if (i < nbytes) dst[i] = (uint8_t)(w[i >> 2] >> ((i & 3) * 8));
+}
+
+// N == M: dense (quantise only, no metadata), processed in groups of 4.
+template <int N, int M, int BITS, int MAXT>
+__global__ void __launch_bounds__(MAXT) pack_kernel(const PackJobDev* __restrict__ jobs, int njobs,
+                                                    PackJobDev single, uint32_t* status) {
+    constexpr bool kDense = (N == M);
+    constexpr int G = 32 / M;                          // groups per lane
+    constexpr int F = (M == 4) ? 2 : 4;                // metadata field width
+    constexpr int VBITS = G * N * BITS;                // value bits per lane (16 .. 256)
+    constexpr int VWORDS = (VBITS + 31) / 32;
+    constexpr int MBITS = kDense ? 0 : G * N * F;      // metadata bits per lane (0, 16, 32, 64)
+    constexpr int MWORDS = kDense ? 1 : (MBITS + 31) / 32;
+
+    extern __shared__ float4 tile[];  // [warps][256] float4, then [warps] floats for the row maximum
+    const int warps = blockDim.x >> 5;
+    float* red = reinterpret_cast<float*>(tile + warps * 256);
+
+    PackJobDev job;
+    if (jobs) {
+        int lo = 0, hi = njobs - 1;  // last job whose unit_begin <= blockIdx.x
+        while (lo < hi) {
+            int mid = (lo + hi + 1) >> 1;
+            if (jobs[mid].unit_begin <= blockIdx.x) lo = mid; else hi = mid - 1;
+        }
+        job = jobs[lo];
+    } else {
+        job = single;
+    }
+
+    const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+    const int wpr = 1 << job.wpr_log2;
+    const int row_in_block = w >> job.wpr_log2, chunk = w & (wpr - 1);
+    const int rows_per_block = warps >> job.wpr_log2;
+    const long long row = (long long)(blockIdx.x - job.unit_begin) * rows_per_block + row_in_block;
+    const bool row_ok = row < job.out;
+    const int in4 = job.in >> 2;
+
+    // ---- load V = W + U (coalesced), running |max| and non-finite detector -------------------
+    float4* mytile = tile + w * 256;
+    float amax = 0.0f, poison = 0.0f;
+    {
+        const float4* W4 = reinterpret_cast<const float4*>(job.W) + (row_ok ? row * in4 : 0);
+        const float4* U4 = job.U ? reinterpret_cast<const float4*>(job.U) + (row_ok ? row * in4 : 0) : nullptr;
+        float4 v[8];
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            int f = chunk * 256 + j * 32 + lane;
+            v[j] = (row_ok && f < in4) ? ld_stream(W4 + f) : make_float4(0.f, 0.f, 0.f, 0.f);
+        }
+        if (U4) {
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+                int f = chunk * 256 + j * 32 + lane;
+                if (row_ok && f < in4) {
+                    float4 u = ld_stream(U4 + f);
+                    v[j].x = __fadd_rn(v[j].x, u.x); v[j].y = __fadd_rn(v[j].y, u.y);
+                    v[j].z = __fadd_rn(v[j].z, u.z); v[j].w = __fadd_rn(v[j].w, u.w);
+                }
+            }
+        }
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            amax = fmaxf(amax, fmaxf(fmaxf(fabsf(v[j].x), fabsf(v[j].y)), fmaxf(fabsf(v[j].z), fabsf(v[j].w))));
+            poison = __fmaf_rn(v[j].x, 0.0f, poison); poison = __fmaf_rn(v[j].y, 0.0f, poison);
+            poison = __fmaf_rn(v[j].z, 0.0f, poison); poison = __fmaf_rn(v[j].w, 0.0f, poison);
+            int fl = j * 32 + lane, owner = fl >> 3, jj = fl & 7;
+            mytile[owner * 8 + (jj ^ (owner & 7))] = v[j];
+        }
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, o));
+    const bool bad = __any_sync(0xffffffffu, poison != poison) || !(amax <= 3.402823466e+38f);
+    if (bad && lane == 0 && status) atomicOr(status, NM_STATUS_NONFINITE);
+    if (wpr > 1) {
+        if (lane == 0) red[w] = amax;
+        __syncthreads();
+        for (int c = 0; c < wpr; ++c) amax = fmaxf(amax, red[row_in_block * wpr + c]);
+    } else {
+        __syncwarp();
+    }
+
+    // ---- ADMM-Max scale ---------------------------------------------------------------------
+    constexpr float qmax = (float)((1 << (BITS - 1)) - 1);
+    const float s = (amax == 0.0f) ? 1.0f : __fdiv_rn(amax, qmax);
+    if (row_ok && chunk == 0 && lane == 0) job.scales[row] = s;
+
+    // ---- this lane's 32 consecutive values ----------------------------------------------------
+    float v[32];
+#pragma unroll
+    for (int jj = 0; jj < 8; ++jj) {
+        float4 t = mytile[lane * 8 + (jj ^ (lane & 7))];
+        v[jj * 4 + 0] = t.x; v[jj * 4 + 1] = t.y; v[jj * 4 + 2] = t.z; v[jj * 4 + 3] = t.w;
+    }
+    const int lane_first = chunk * 1024 + lane * 32;             // first column of this lane
+    const int nvals = max(0, min(32, job.in - lane_first));      // columns inside the row
+    if (!row_ok || nvals == 0) return;
+
+    unsigned vw[VWORDS], mw[MWORDS];
+#pragma unroll
+    for (int i = 0; i < VWORDS; ++i) vw[i] = 0;
+#pragma unroll
+    for (int i = 0; i < MWORDS; ++i) mw[i] = 0;
+
+#pragma unroll
+    for (int g = 0; g < G; ++g) {
+        if (g * M < nvals) {
+            if constexpr (kDense) {
+#pragma unroll
+                for (int p = 0; p < M; ++p) {
+                    const int pos = (g * M + p) * BITS;
+                    vw[pos >> 5] |= quantise_code<BITS>(v[g * M + p], s) << (pos & 31);
+                }
+            } else {
+                float a[M];
+#pragma unroll
+                for (int p = 0; p < M; ++p) a[p] = fabsf(v[g * M + p]);
+                const unsigned mask = keep_mask<N, M>(a);
+                // compaction: slot c receives the c-th kept position (ascending)
+                float sel[N];
+                unsigned selp[N];
+#pragma unroll
+                for (int c = 0; c < N; ++c) { sel[c] = 0.0f; selp[c] = 0; }
+#pragma unroll
+                for (int p = 0; p < M; ++p) {
+                    const bool kept = (mask >> p) & 1u;
+                    const int before = __popc(mask & ((1u << p) - 1u));
+#pragma unroll
+                    for (int c = 0; c < N; ++c) {
+                        // position p can only land in slot c if c <= p and enough positions remain
+                        if (c <= p && (M - p) >= (N - c)) {
+                            const bool hit = kept && before == c;
+                            sel[c] = hit ? v[g * M + p] : sel[c];
+                            selp[c] = hit ? (unsigned)p : selp[c];
+                        }
+                    }
+                }
+#pragma unroll
+                for (int c = 0; c < N; ++c) {
+                    const int vpos = (g * N + c) * BITS, mpos = (g * N + c) * F;
+                    vw[vpos >> 5] |= quantise_code<BITS>(sel[c], s) << (vpos & 31);
+                    mw[mpos >> 5] |= selp[c] << (mpos & 31);
+                }
+            }
+        }
+    }
+
+    // ---- stores -----------------------------------------------------------------------------
+    const int lane_global = chunk * 32 + lane;
+    const bool full = (nvals == 32);
+    {
+        constexpr int LB = VBITS / 8;
+        uint8_t* dst = job.values + (size_t)row * job.vrow_bytes + (size_t)lane_global * LB;
+        if (full && (job.vrow_bytes % LB) == 0) store_bytes_vec<LB>(dst, vw);
+        else store_bytes_slow<LB>(dst, vw, nvals / M * N * BITS / 8);
+    }
+    if constexpr (!kDense) {
+        constexpr int MB = MBITS / 8;
+        const unsigned lane_off = (unsigned)lane_global * MB;
+        const unsigned row_bytes = job.mrow_words * 4u;
+        uint8_t* dst = reinterpret_cast<uint8_t*>(job.meta + (size_t)row * job.mrow_words) + lane_off;
+        const bool last = (lane_first + 32 >= job.in);  // lane holding the end of the row
+        if (full && !last) {
+            store_bytes_vec<MB>(dst, mw);
+        } else {
+            // the last lane also writes the zero padding up to the row's word boundary
+            const unsigned wpad[3] = {mw[0], MWORDS > 1 ? mw[MWORDS - 1] : 0u, 0u};
+            store_bytes_slow<MB + 4>(dst, wpad, (int)min(row_bytes - lane_off, (unsigned)(MB + 4)));
+        }
+    }
+}
+
+// ---------------------------------------------------------------------------------------------
+// host side
+// ---------------------------------------------------------------------------------------------
+using PackFn = void (*)(const PackJobDev*, int, PackJobDev, uint32_t*);
+
+template <int N, int M>
+static PackFn pick_bits(int bits, int warps) {
+    if (warps <= kPackMinWarps)
+        return bits == 8 ? (PackFn)pack_kernel<N, M, 8, 128> : (PackFn)pack_kernel<N, M, 4, 128>;
+    return bits == 8 ? (PackFn)pack_kernel<N, M, 8, 1024> : (PackFn)pack_kernel<N, M, 4, 1024>;
+}
+
+static PackFn pick_kernel(int n, int m, int bits, int warps) {
+    if (n == m) return pick_bits<4, 4>(bits, warps);
+    if (m == 4) return n == 1 ? pick_bits<1, 4>(bits, warps) : pick_bits<2, 4>(bits, warps);
+    if (n == 1) return pick_bits<1, 8>(bits, warps);
+    if (n == 2) return pick_bits<2, 8>(bits, warps);
+    return pick_bits<4, 8>(bits, warps);
+}
+
+static int validate_job(const nm_pack_job_t& j) {
+    int rc = check_pattern(j.out, j.in, j.n, j.m, j.bits);
+    if (rc != NM_OK) return rc;
+    if (!j.W || !j.values || !j.scales) return NM_ERR_NULL;
+    if (j.n != j.m && !j.meta) return NM_ERR_NULL;
+    if (j.in % 4) return NM_ERR_SHAPE;
+    if (j.n == j.m && j.in % 4) return NM_ERR_SHAPE;
+    if (j.in > 32768) return NM_ERR_UNSUPPORTED;
+    if (!aligned(j.W, 16) || (j.U && !aligned(j.U, 16)) || !aligned(j.values, 16) ||
+        (j.meta && !aligned(j.meta, 4)) || !aligned(j.scales, 4))
+        return NM_ERR_ALIGN;
+    return NM_OK;
+}
+
+static int wpr_log2_of(int in) {
+    int chunks = (in + 1023) / 1024, l = 0;
+    while ((1 << l) < chunks) ++l;
+    return l;
+}
+
+static PackJobDev to_dev(const nm_pack_job_t& j) {
+    PackJobDev d;
+    d.W = j.W; d.U = j.U; d.values = (uint8_t*)j.values; d.meta = (uint32_t*)j.meta; d.scales = j.scales;
+    d.out = j.out; d.in = j.in; d.wpr_log2 = wpr_log2_of(j.in); d.unit_begin = 0;
+    d.vrow_bytes = (unsigned)values_row_bytes(j.in, j.n, j.m, j.bits);
+    d.mrow_words = (unsigned)meta_row_words(j.in, j.n, j.m);
+    return d;
+}
+
+static int launch(PackFn fn, const PackJobDev* jobs_dev, int njobs, const PackJobDev& single,
+                  unsigned blocks, int warps, uint32_t* status, cudaStream_t stream) {
+    size_t smem = (size_t)warps * (256 * sizeof(float4) + sizeof(float));
+    if (smem > 48 * 1024)
+        NM_CUDA_TRY(cudaFuncSetAttribute((const void*)fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    fn<<<blocks, warps * 32, smem, stream>>>(jobs_dev, njobs, single, status);
+    NM_CUDA_TRY(cudaGetLastError());
+    return NM_OK;
+}
+
+}  // namespace nm
+
+extern "C" {
+
+int nm_project_pack(const float* W, const float* U, int out, int in, int n, int m, int bits,
+                    void* values, void* meta, float* scales, uint32_t* status, void* stream) {
+    nm_pack_job_t j{W, U, out, in, n, m, bits, values, meta, scales};
+    int rc = nm::validate_job(j);
+    if (rc != NM_OK) return rc;
+    if (out == 0 || in == 0) return NM_OK;
+    nm::PackJobDev d = nm::to_dev(j);
+    int warps = std::max(nm::kPackMinWarps, 1 << d.wpr_log2);
+    int rows_per_block = warps >> d.wpr_log2;
+    unsigned blocks = (unsigned)((out + rows_per_block - 1) / rows_per_block);
+    return nm::launch(nm::pick_kernel(n, m, bits, warps), nullptr, 0, d, blocks, warps, status, (cudaStream_t)stream);
+}
+
+size_t nm_pack_workspace_bytes(int njobs) {
+    return njobs <= 0 ? 0 : (size_t)njobs * sizeof(nm::PackJobDev);
+}
+
+int nm_project_pack_batched(const nm_pack_job_t* jobs, int njobs, void* ws, size_t ws_bytes,
+                            uint32_t* status, void* stream) {
+    if (njobs < 0) return NM_ERR_SHAPE;
+    if (njobs == 0) return NM_OK;
+    if (!jobs) return NM_ERR_NULL;
+    if (!ws || ws_bytes < nm_pack_workspace_bytes(njobs)) return NM_ERR_WORKSPACE;
+    if (!nm::aligned(ws, 16)) return NM_ERR_ALIGN;
+    for (int i = 0; i < njobs; ++i) {
+        int rc = nm::validate_job(jobs[i]);
+        if (rc != NM_OK) return rc;
+    }
+    // Group jobs that can share one launch: same (n == m ? dense : n, m), bits and block size.
+    struct Key { int n, m, bits, warps; };
+    std::vector<Key> keys;
+    std::vector<std::vector<int>> groups;
+    for (int i = 0; i < njobs; ++i) {
+        const nm_pack_job_t& j = jobs[i];
+        if (j.out == 0 || j.in == 0) continue;
+        Key k{j.n == j.m ? 4 : j.n, j.n == j.m ? 4 : j.m, j.bits,
+              std::max(nm::kPackMinWarps, 1 << nm::wpr_log2_of(j.in))};
+        size_t g = 0;
+        for (; g < keys.size(); ++g)
+            if (keys[g].n == k.n && keys[g].m == k.m && keys[g].bits == k.bits && keys[g].warps == k.warps) break;
+        if (g == keys.size()) { keys.push_back(k); groups.emplace_back(); }
+        groups[g].push_back(i);
+    }
+    std::vector<nm::PackJobDev> table;
+    table.reserve(njobs);
+    std::vector<unsigned> group_blocks(keys.size());
+    std::vector<size_t> group_first(keys.size());
+    for (size_t g = 0; g < keys.size(); ++g) {
+        unsigned blocks = 0;
+        group_first[g] = table.size();
+        for (int i : groups[g]) {
+            nm::PackJobDev d = nm::to_dev(jobs[i]);
+            int rows_per_block = keys[g].warps >> d.wpr_log2;
+            d.unit_begin = blocks;
+            unsigned long long nb = ((unsigned long long)d.out + rows_per_block - 1) / rows_per_block;
+            if (blocks + nb > 0x7fffffffull) return NM_ERR_UNSUPPORTED;
+            blocks += (unsigned)nb;
+            table.push_back(d);
+        }
+        group_blocks[g] = blocks;
+    }
+    cudaStream_t s = (cudaStream_t)stream;
+    // Pageable-source async copies are staged before the call returns, so `table` may go away.
+    NM_CUDA_TRY(cudaMemcpyAsync(ws, table.data(), table.size() * sizeof(nm::PackJobDev),
+                                cudaMemcpyHostToDevice, s));
+    for (size_t g = 0; g < keys.size(); ++g) {
+        const nm::PackJobDev* dev = reinterpret_cast<const nm::PackJobDev*>(ws) + group_first[g];
+        int rc = nm::launch(nm::pick_kernel(keys[g].n, keys[g].m, keys[g].bits, keys[g].warps), dev,
+                            (int)groups[g].size(), nm::PackJobDev{}, group_blocks[g], keys[g].warps,
+                            status, s);
+        if (rc != NM_OK) return rc;
+    }
+    return NM_OK;
+}
+
+}  // extern "C"
