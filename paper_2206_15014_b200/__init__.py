@@ -1,0 +1,174 @@
+"""Python binding of libnmsparse.so: argument marshalling only.
+
+Every function has the name and the argument order of its C entry point (include/nmsparse.h) and
+takes torch CUDA tensors (used purely as device buffers) or plain integers.  All arithmetic runs in
+the library's CUDA kernels.  There is no CPU fallback: importing this package fails when the
+library has not been built (run ``python -m paper_2206_15014_b200.build``).
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libnmsparse.so")
+
+if not os.path.exists(LIB_PATH):
+    raise ImportError(
+        f"{LIB_PATH} is missing: build it with `python -m paper_2206_15014_b200.build` "
+        "(there is no fallback path)")
+
+_lib = ctypes.CDLL(LIB_PATH)
+
+NM_OK = 0
+NM_ERR_NULL, NM_ERR_SHAPE, NM_ERR_UNSUPPORTED, NM_ERR_ALIGN = -1, -2, -3, -4
+NM_ERR_WORKSPACE, NM_ERR_CUDA, NM_ERR_NONFINITE, NM_ERR_TIMEOUT = -5, -6, -7, -8
+
+EXPORTS = (
+    "nm_packed_sizes", "nm_project_pack", "nm_project_pack_batched", "nm_pack_workspace_bytes",
+    "nm_int_linear", "nm_int_linear_dsx", "nm_int_linear_acc", "nm_int_linear_workspace_bytes",
+    "nm_int_linear_check", "nm_absmax", "nm_quantize_act", "nm_poll_status", "nm_strerror",
+    "nm_last_cuda_error", "nm_version",
+)
+
+
+class nm_packed_t(ctypes.Structure):
+    _fields_ = [("out", ctypes.c_int32), ("in_", ctypes.c_int32), ("n", ctypes.c_int32),
+                ("m", ctypes.c_int32), ("bits", ctypes.c_int32), ("values", ctypes.c_void_p),
+                ("meta", ctypes.c_void_p)]
+
+
+class nm_pack_job_t(ctypes.Structure):
+    _fields_ = [("W", ctypes.c_void_p), ("U", ctypes.c_void_p), ("out", ctypes.c_int32),
+                ("in_", ctypes.c_int32), ("n", ctypes.c_int32), ("m", ctypes.c_int32),
+                ("bits", ctypes.c_int32), ("values", ctypes.c_void_p), ("meta", ctypes.c_void_p),
+                ("scales", ctypes.c_void_p)]
+
+
+_vp, _i, _sz, _f = ctypes.c_void_p, ctypes.c_int, ctypes.c_size_t, ctypes.c_float
+_lib.nm_packed_sizes.argtypes = [_i] * 5 + [ctypes.POINTER(_sz), ctypes.POINTER(_sz)]
+_lib.nm_project_pack.argtypes = [_vp, _vp, _i, _i, _i, _i, _i, _vp, _vp, _vp, _vp, _vp]
+_lib.nm_project_pack_batched.argtypes = [ctypes.POINTER(nm_pack_job_t), _i, _vp, _sz, _vp, _vp]
+_lib.nm_pack_workspace_bytes.argtypes = [_i]
+_lib.nm_pack_workspace_bytes.restype = _sz
+_lib.nm_int_linear.argtypes = [_vp, _i, ctypes.POINTER(nm_packed_t), _f, _vp, _vp, _vp, _vp, _sz, _vp, _vp]
+_lib.nm_int_linear_dsx.argtypes = [_vp, _i, ctypes.POINTER(nm_packed_t), _vp, _vp, _vp, _vp, _vp, _vp, _sz, _vp, _vp]
+_lib.nm_int_linear_acc.argtypes = [_vp, _i, ctypes.POINTER(nm_packed_t), _vp, _vp, _sz, _vp, _vp]
+_lib.nm_int_linear_workspace_bytes.argtypes = [_i] * 6
+_lib.nm_int_linear_workspace_bytes.restype = _sz
+_lib.nm_int_linear_check.argtypes = [_i] * 6
+_lib.nm_absmax.argtypes = [_vp, _sz, _vp, _vp]
+_lib.nm_quantize_act.argtypes = [_vp, _sz, _vp, _vp, _vp, _vp]
+_lib.nm_poll_status.argtypes = [_vp, _vp]
+_lib.nm_strerror.argtypes = [_i]
+_lib.nm_strerror.restype = ctypes.c_char_p
+_lib.nm_last_cuda_error.restype = ctypes.c_char_p
+
+
+class NmError(RuntimeError):
+    def __init__(self, code, where):
+        self.code = code
+        extra = nm_last_cuda_error() if code == NM_ERR_CUDA else ""
+        super().__init__(f"{where}: {nm_strerror(code)} ({code}) {extra}".strip())
+
+
+def _chk(code, where):
+    if code != NM_OK:
+        raise NmError(code, where)
+
+
+def _ptr(t):
+    return None if t is None else ctypes.c_void_p(t.data_ptr())
+
+
+def _stream(stream=None):
+    if stream is None:
+        import torch
+        return ctypes.c_void_p(torch.cuda.current_stream().cuda_stream)
+    return ctypes.c_void_p(int(stream))
+
+
+def nm_strerror(code):
+    return _lib.nm_strerror(int(code)).decode()
+
+
+def nm_last_cuda_error():
+    return _lib.nm_last_cuda_error().decode()
+
+
+def nm_version():
+    return int(_lib.nm_version())
+
+
+def nm_packed_sizes(out, in_, n, m, bits):
+    vb, mb = _sz(), _sz()
+    _chk(_lib.nm_packed_sizes(out, in_, n, m, bits, ctypes.byref(vb), ctypes.byref(mb)), "nm_packed_sizes")
+    return vb.value, mb.value
+
+
+def nm_project_pack(W, U, out, in_, n, m, bits, values, meta, scales, status=None, stream=None):
+    _chk(_lib.nm_project_pack(_ptr(W), _ptr(U), out, in_, n, m, bits, _ptr(values), _ptr(meta),
+                              _ptr(scales), _ptr(status), _stream(stream)), "nm_project_pack")
+
+
+def nm_pack_workspace_bytes(njobs):
+    return int(_lib.nm_pack_workspace_bytes(njobs))
+
+
+def make_pack_jobs(jobs):
+    """jobs: iterable of (W, U|None, n, m, bits, values, meta|None, scales) -> ctypes job array."""
+    jobs = list(jobs)
+    arr = (nm_pack_job_t * len(jobs))()
+    for a, (W, U, n, m, bits, values, meta, scales) in zip(arr, jobs):
+        a.W, a.U = W.data_ptr(), (U.data_ptr() if U is not None else None)
+        a.out, a.in_, a.n, a.m, a.bits = W.shape[0], W.shape[1], n, m, bits
+        a.values, a.meta, a.scales = values.data_ptr(), (meta.data_ptr() if meta is not None else None), scales.data_ptr()
+    return arr
+
+
+def nm_project_pack_batched(job_array, njobs, ws, ws_bytes, status=None, stream=None):
+    _chk(_lib.nm_project_pack_batched(job_array, njobs, _ptr(ws), ws_bytes, _ptr(status), _stream(stream)),
+         "nm_project_pack_batched")
+
+
+def make_packed(out, in_, n, m, bits, values, meta):
+    return nm_packed_t(out, in_, n, m, bits, values.data_ptr(), meta.data_ptr() if meta is not None else None)
+
+
+def nm_int_linear_workspace_bytes(tokens, out, in_, n, m, bits):
+    return int(_lib.nm_int_linear_workspace_bytes(tokens, out, in_, n, m, bits))
+
+
+def nm_int_linear_check(tokens, out, in_, n, m, bits):
+    return int(_lib.nm_int_linear_check(tokens, out, in_, n, m, bits))
+
+
+def nm_int_linear(X, tokens, W, sx, sw, bias, Y, ws=None, ws_bytes=0, status=None, stream=None):
+    _chk(_lib.nm_int_linear(_ptr(X), tokens, ctypes.byref(W), float(sx), _ptr(sw), _ptr(bias), _ptr(Y),
+                            _ptr(ws), ws_bytes, _ptr(status), _stream(stream)), "nm_int_linear")
+
+
+def nm_int_linear_dsx(X, tokens, W, sx_dev, sw, bias, Y, absmax_out=None, ws=None, ws_bytes=0,
+                      status=None, stream=None):
+    _chk(_lib.nm_int_linear_dsx(_ptr(X), tokens, ctypes.byref(W), _ptr(sx_dev), _ptr(sw), _ptr(bias),
+                                _ptr(Y), _ptr(absmax_out), _ptr(ws), ws_bytes, _ptr(status),
+                                _stream(stream)), "nm_int_linear_dsx")
+
+
+def nm_int_linear_acc(X, tokens, W, ACC, ws=None, ws_bytes=0, status=None, stream=None):
+    _chk(_lib.nm_int_linear_acc(_ptr(X), tokens, ctypes.byref(W), _ptr(ACC), _ptr(ws), ws_bytes,
+                                _ptr(status), _stream(stream)), "nm_int_linear_acc")
+
+
+def nm_absmax(Y, count, absmax, stream=None):
+    _chk(_lib.nm_absmax(_ptr(Y), count, _ptr(absmax), _stream(stream)), "nm_absmax")
+
+
+def nm_quantize_act(Y, count, absmax, Xq, sx_out=None, stream=None):
+    _chk(_lib.nm_quantize_act(_ptr(Y), count, _ptr(absmax), _ptr(Xq), _ptr(sx_out), _stream(stream)),
+         "nm_quantize_act")
+
+
+def nm_poll_status(status=None, stream=None):
+    """Synchronises the stream and returns the NM_* code held in the device status word."""
+    return int(_lib.nm_poll_status(_ptr(status), _stream(stream)))

@@ -1,0 +1,414 @@
+// Integer N:M linear layer on tcgen05 tensor cores with the dequantisation epilogue fused in.
+//
+// The sparse operand of tcgen05.mma.sp is A, so the kernel computes D = Wq * X^T: a tile is
+// 128 output channels (TMEM lanes) x BN tokens (TMEM columns).  In TMEM one lane therefore holds
+// one output channel, whose scale and bias are per-thread constants in the epilogue, and for a
+// fixed token the 32 lanes of a warp hold 32 consecutive channels = one coalesced 128-byte store
+// into the row-major Y[tokens, out].
+//
+// One persistent CTA per SM walks a contiguous range of tiles ordered output-tile-major, so the
+// weight tile (and its metadata) changes at most a few times per CTA.
+//   warp 0      TMA producer: X tile and W tile of every 128-wide k-block into a ring of stages
+//   warp 1      allocates TMEM, issues tcgen05.mma[.sp] (one elected lane), commits to mbarriers
+//   warps 2-5   copy the index metadata of the current 128 output channels into TMEM
+//               (tcgen05.st, once per output tile, whole K), then run the epilogue of tile i
+//               (tcgen05.ld -> fma -> global) while the MMAs of tile i+1 fill the other accumulator
+// Every mbarrier wait is bounded; on expiry the CTA raises NM_STATUS_TIMEOUT, drains and exits.
+#include "common.cuh"
+#include "sm100_ptx.cuh"
+#include <cuda.h>
+#include <cuda_runtime.h>
+#include <mutex>
+
+namespace nm {
+
+constexpr int kBM = 128;            // output channels per tile (MMA M)
+constexpr int kKB = 128;            // reduction elements per pipeline stage
+constexpr int kGemmThreads = 192;   // 6 warps
+constexpr int kTmemCols = 512;
+constexpr int kSmemLimit = 232448;  // 227 KB of dynamic shared memory per CTA
+constexpr int kSmemTail = 1024;     // barriers, TMEM slot, abort flag
+constexpr long long kWaitLimit = 1ll << 31;  // SM clocks (about a second)
+
+enum { EPI_F32 = 0, EPI_ACC = 1 };
+
+struct GemmParams {
+    int tokens, out, in;
+    int n_tok_tiles, n_tiles, kblocks;
+    const uint32_t* meta;  // canonical metadata [out, mrow_words] (sparse modes)
+    int mrow_words;
+    const float* sw;
+    const float* bias;
+    const float* sx_dev;
+    float sx_host;
+    float* Y;
+    int32_t* ACC;
+    float* absmax;
+    uint32_t* status;
+};
+
+template <bool SPARSE, int BN>
+struct GemmCfg {
+    static constexpr int A_ROW = SPARSE ? 64 : 128;   // bytes of one weight row per stage
+    static constexpr int A_BYTES = kBM * A_ROW;
+    static constexpr int B_BYTES = BN * 128;
+    static constexpr int STAGE = A_BYTES + B_BYTES;
+    static constexpr int STAGES = (kSmemLimit - kSmemTail - 1024) / STAGE;
+    static constexpr int SMEM = STAGES * STAGE + kSmemTail + 1024;
+    static constexpr int META_COL = 2 * BN;           // first TMEM column of the metadata
+    static constexpr int META_COLS = kTmemCols - 2 * BN;
+    static_assert(STAGES >= 3, "pipeline too shallow");
+    static_assert(BN % 32 == 0 && BN >= 32 && BN <= 256, "token tile");
+};
+
+template <bool SPARSE, int BN, int EPI>
+__global__ void __launch_bounds__(kGemmThreads, 1)
+nm_gemm_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant__ CUtensorMap tmap_x,
+               const GemmParams p) {
+    using Cfg = GemmCfg<SPARSE, BN>;
+    constexpr int S = Cfg::STAGES;
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = reinterpret_cast<uint8_t*>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+    uint64_t* bars = reinterpret_cast<uint64_t*>(smem + S * Cfg::STAGE);
+    // bars[0..S) full, [S..2S) empty, then acc_full[2], acc_empty[2], meta_ready, drained
+    const uint32_t bar0 = ptx::smem_u32(bars);
+    auto full_bar = [&](int s) { return bar0 + 8u * s; };
+    auto empty_bar = [&](int s) { return bar0 + 8u * (S + s); };
+    auto acc_full_bar = [&](int b) { return bar0 + 8u * (2 * S + b); };
+    auto acc_empty_bar = [&](int b) { return bar0 + 8u * (2 * S + 2 + b); };
+    const uint32_t meta_bar = bar0 + 8u * (2 * S + 4);
+    const uint32_t drained_bar = bar0 + 8u * (2 * S + 5);
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * S + 6);
+    volatile uint32_t* abort_flag = tmem_slot + 1;
+    volatile uint32_t* never_flag = tmem_slot + 2;  // stays 0: for the drain waits after an abort
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int per = p.n_tiles / gridDim.x, rem = p.n_tiles % gridDim.x;
+    const int tile_begin = blockIdx.x * per + min((int)blockIdx.x, rem);
+    const int tile_count = per + ((int)blockIdx.x < rem ? 1 : 0);
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < S; ++s) { ptx::mbar_init(full_bar(s), 1); ptx::mbar_init(empty_bar(s), 1); }
+        for (int b = 0; b < 2; ++b) { ptx::mbar_init(acc_full_bar(b), 1); ptx::mbar_init(acc_empty_bar(b), 4); }
+        ptx::mbar_init(meta_bar, 4);
+        ptx::mbar_init(drained_bar, 1);
+        *abort_flag = 0;
+        *never_flag = 0;
+        ptx::fence_mbar_init();
+        ptx::prefetch_tensormap(&tmap_w);
+        ptx::prefetch_tensormap(&tmap_x);
+    }
+    if (warp == 1) {
+        ptx::tmem_alloc(ptx::smem_u32(tmem_slot), kTmemCols);
+        ptx::tmem_relinquish();
+    }
+    ptx::tc_fence_before();
+    __syncthreads();
+    ptx::tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+
+    auto raise_timeout = [&]() {
+        *abort_flag = 1;
+        if (p.status) atomicOr(p.status, NM_STATUS_TIMEOUT);
+    };
+
+    if (warp == 0) {
+        // ------------------------------ TMA producer ------------------------------------------
+        if (lane == 0) {
+            uint32_t it = 0;
+            bool ok = true;
+            for (int i = 0; i < tile_count && ok; ++i) {
+                const int tile = tile_begin + i;
+                const int n0 = (tile / p.n_tok_tiles) * kBM, t0 = (tile % p.n_tok_tiles) * BN;
+                for (int kb = 0; kb < p.kblocks; ++kb, ++it) {
+                    const int s = it % S;
+                    if (!ptx::mbar_wait_bounded(empty_bar(s), ((it / S) & 1u) ^ 1u, abort_flag, kWaitLimit)) {
+                        raise_timeout(); ok = false; break;
+                    }
+                    const uint32_t a_dst = ptx::smem_u32(smem + s * Cfg::STAGE);
+                    ptx::mbar_expect_tx(full_bar(s), Cfg::STAGE);
+                    ptx::tma_load_2d(a_dst, &tmap_w, kb * Cfg::A_ROW, n0, full_bar(s));
+                    ptx::tma_load_2d(a_dst + Cfg::A_BYTES, &tmap_x, kb * 128, t0, full_bar(s));
+                }
+            }
+            if (!ok) {
+                // let copies already in flight land before the CTA goes away
+                const uint32_t first = it > (uint32_t)S ? it - S : 0;
+                for (uint32_t j = first; j < it; ++j)
+                    ptx::mbar_wait_bounded(full_bar(j % S), (j / S) & 1u, never_flag, kWaitLimit >> 4);
+            }
+        }
+    } else if (warp == 1) {
+        // ------------------------------ MMA issuer ---------------------------------------------
+        if (lane == 0) {
+            constexpr uint32_t idesc = ptx::idesc_i8(kBM, BN, SPARSE);
+            uint32_t it = 0, meta_phase = 0;
+            int prev_out_tile = -1;
+            bool ok = true;
+            for (int i = 0; i < tile_count && ok; ++i) {
+                const int tile = tile_begin + i, out_tile = tile / p.n_tok_tiles, buf = i & 1;
+                if (SPARSE && out_tile != prev_out_tile) {
+                    if (!ptx::mbar_wait_bounded(meta_bar, meta_phase, abort_flag, kWaitLimit)) { raise_timeout(); ok = false; break; }
+                    meta_phase ^= 1u;
+                    prev_out_tile = out_tile;
+                }
+                if (!ptx::mbar_wait_bounded(acc_empty_bar(buf), ((i >> 1) & 1u) ^ 1u, abort_flag, kWaitLimit)) { raise_timeout(); ok = false; break; }
+                ptx::tc_fence_after();
+                const uint32_t d_tmem = tmem_base + buf * BN;
+                for (int kb = 0; kb < p.kblocks; ++kb, ++it) {
+                    const int s = it % S;
+                    if (!ptx::mbar_wait_bounded(full_bar(s), (it / S) & 1u, abort_flag, kWaitLimit)) { raise_timeout(); ok = false; break; }
+                    ptx::tc_fence_after();
+                    const uint32_t a_addr = ptx::smem_u32(smem + s * Cfg::STAGE), b_addr = a_addr + Cfg::A_BYTES;
+                    if constexpr (SPARSE) {
+#pragma unroll
+                        for (int j = 0; j < 2; ++j)  // 64 logical k each: 32 stored bytes of A, 64 of B
+                            ptx::mma_sp_i8(d_tmem, ptx::smem_desc_kmajor(a_addr + 32 * j, 64, ptx::kSwizzle64),
+                                           ptx::smem_desc_kmajor(b_addr + 64 * j, 128, ptx::kSwizzle128),
+                                           tmem_base + Cfg::META_COL + kb * 4 + 2 * j, idesc, (kb | j) != 0);
+                    } else {
+#pragma unroll
+                        for (int j = 0; j < 4; ++j)  // 32 k each
+                            ptx::mma_i8(d_tmem, ptx::smem_desc_kmajor(a_addr + 32 * j, 128, ptx::kSwizzle128),
+                                        ptx::smem_desc_kmajor(b_addr + 32 * j, 128, ptx::kSwizzle128), idesc, (kb | j) != 0);
+                    }
+                    ptx::tc_commit(empty_bar(s));  // stage reusable once these MMAs have read it
+                }
+                if (ok) ptx::tc_commit(acc_full_bar(buf));
+            }
+            // everything issued has retired before TMEM is released
+            ptx::tc_commit(drained_bar);
+            ptx::mbar_wait_bounded(drained_bar, 0, never_flag, kWaitLimit);
+        }
+    } else {
+        // ------------------------------ metadata + epilogue warps ------------------------------
+        const int q = warp & 3, row = q * 32 + lane;
+        const uint32_t lane_taddr = tmem_base + ((uint32_t)(q * 32) << 16);
+        const float sx = p.sx_dev ? *p.sx_dev : p.sx_host;
+        float amax = 0.0f;
+        bool ok = true;
+
+        auto load_meta = [&](int out_tile) {
+            const int n = out_tile * kBM + row;
+            const uint4* src = reinterpret_cast<const uint4*>(p.meta + (size_t)n * p.mrow_words);
+            for (int c = 0; c < p.mrow_words; c += 4) {
+                // rows past the end get a valid "positions 0,1" pattern; their products are discarded
+                uint4 w = (n < p.out) ? __ldg(src + (c >> 2)) : make_uint4(0x44444444u, 0x44444444u, 0x44444444u, 0x44444444u);
+                ptx::tmem_st_32x4(lane_taddr + Cfg::META_COL + c, w.x, w.y, w.z, w.w);
+            }
+            ptx::tmem_st_wait();
+            ptx::tc_fence_before();
+            __syncwarp();
+            if (lane == 0) ptx::mbar_arrive(meta_bar);
+        };
+
+        for (int i = 0; i < tile_count && ok; ++i) {
+            const int tile = tile_begin + i, out_tile = tile / p.n_tok_tiles, buf = i & 1;
+            const int n = out_tile * kBM + row, t0 = (tile % p.n_tok_tiles) * BN;
+            if (SPARSE && i == 0) load_meta(out_tile);
+            bool got = ptx::mbar_wait_bounded(acc_full_bar(buf), (i >> 1) & 1u, abort_flag, kWaitLimit);
+            ok = __all_sync(0xffffffffu, got);
+            if (!ok) { if (lane == 0) raise_timeout(); break; }
+            ptx::tc_fence_after();
+            if (SPARSE && i + 1 < tile_count) {
+                const int next_out_tile = (tile + 1) / p.n_tok_tiles;
+                if (next_out_tile != out_tile) load_meta(next_out_tile);  // MMAs of this output tile are done
+            }
+            const bool n_ok = n < p.out;
+            float c_n = 0.0f, b_n = 0.0f;
+            if (EPI == EPI_F32 && n_ok) {
+                c_n = __fmul_rn(sx, p.sw[n]);
+                b_n = p.bias ? p.bias[n] : 0.0f;
+            }
+#pragma unroll 1
+            for (int c0 = 0; c0 < BN; c0 += 32) {
+                if (t0 + c0 >= p.tokens) break;
+                uint32_t r[32];
+                ptx::tmem_ld_32x32(lane_taddr + buf * BN + c0, r);
+                ptx::tmem_ld_wait();
+                if (n_ok) {
+                    if constexpr (EPI == EPI_F32) {
+                        float* dst = p.Y + (size_t)(t0 + c0) * p.out + n;
+#pragma unroll
+                        for (int j = 0; j < 32; ++j) {
+                            if (t0 + c0 + j < p.tokens) {
+                                const float y = __fmaf_rn((float)(int)r[j], c_n, b_n);
+                                __stcs(dst + (size_t)j * p.out, y);
+                                amax = fmaxf(amax, fabsf(y));
+                            }
+                        }
+                    } else {
+                        int32_t* dst = p.ACC + (size_t)(t0 + c0) * p.out + n;
+#pragma unroll
+                        for (int j = 0; j < 32; ++j)
+                            if (t0 + c0 + j < p.tokens) __stcs(dst + (size_t)j * p.out, (int)r[j]);
+                    }
+                }
+            }
+            ptx::tc_fence_before();
+            __syncwarp();
+            if (lane == 0) ptx::mbar_arrive(acc_empty_bar(buf));
+        }
+        if (EPI == EPI_F32 && p.absmax) {
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, o));
+            if (lane == 0) atomicMax(reinterpret_cast<unsigned*>(p.absmax), __float_as_uint(amax));
+        }
+    }
+
+    ptx::tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        ptx::tc_fence_after();
+        ptx::tmem_dealloc(tmem_base, kTmemCols);
+    }
+}
+
+// ---------------------------------------------------------------------------------------------
+// host side
+// ---------------------------------------------------------------------------------------------
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*,
+                                  CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
+                                  CUtensorMapFloatOOBfill);
+
+static EncodeTiledFn encode_tiled_fn() {
+    static EncodeTiledFn fn = nullptr;
+    static std::once_flag once;
+    std::call_once(once, [] {
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres) == cudaSuccess &&
+            qres == cudaDriverEntryPointSuccess)
+            fn = (EncodeTiledFn)p;
+        (void)cudaGetLastError();
+    });
+    return fn;
+}
+
+// 2-D byte matrix [rows, row_bytes] (pitch = row_bytes), box = [box_rows, box_bytes], swizzled.
+static int make_map(CUtensorMap* map, const void* base, uint64_t rows, uint64_t row_bytes,
+                    uint32_t box_rows, uint32_t box_bytes, CUtensorMapSwizzle swz) {
+    EncodeTiledFn fn = encode_tiled_fn();
+    if (!fn) return record_text_error("cuTensorMapEncodeTiled is not available from the driver");
+    cuuint64_t dims[2] = {row_bytes, rows};
+    cuuint64_t strides[1] = {row_bytes};
+    cuuint32_t box[2] = {box_bytes, box_rows};
+    cuuint32_t estr[2] = {1, 1};
+    CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void*>(base), dims, strides, box, estr,
+                    CU_TENSOR_MAP_INTERLEAVE_NONE, swz, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) return record_text_error("cuTensorMapEncodeTiled failed");
+    return NM_OK;
+}
+
+static int sm_count() {
+    static int cached[64] = {0};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return 148;
+    if (!cached[dev]) {
+        int v = 0;
+        if (cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || v <= 0) v = 148;
+        cached[dev] = v;
+    }
+    return cached[dev];
+}
+
+struct LinearArgs {
+    const int8_t* X; int tokens; const nm_packed_t* W;
+    float sx; const float* sx_dev; const float* sw; const float* bias;
+    float* Y; int32_t* ACC; float* absmax; uint32_t* status; cudaStream_t stream;
+};
+
+template <bool SPARSE, int BN, int EPI>
+static int launch_gemm(const LinearArgs& a) {
+    using Cfg = GemmCfg<SPARSE, BN>;
+    const nm_packed_t& W = *a.W;
+    CUtensorMap tw, tx;
+    int rc = make_map(&tw, W.values, (uint64_t)W.out, (uint64_t)(SPARSE ? W.in / 2 : W.in), kBM, Cfg::A_ROW,
+                      SPARSE ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_128B);
+    if (rc != NM_OK) return rc;
+    rc = make_map(&tx, a.X, (uint64_t)a.tokens, (uint64_t)W.in, BN, 128, CU_TENSOR_MAP_SWIZZLE_128B);
+    if (rc != NM_OK) return rc;
+    GemmParams p{};
+    p.tokens = a.tokens; p.out = W.out; p.in = W.in;
+    p.n_tok_tiles = (a.tokens + BN - 1) / BN;
+    p.n_tiles = p.n_tok_tiles * ((W.out + kBM - 1) / kBM);
+    p.kblocks = W.in / kKB;
+    p.meta = (const uint32_t*)W.meta; p.mrow_words = W.in / 32;
+    p.sw = a.sw; p.bias = a.bias; p.sx_dev = a.sx_dev; p.sx_host = a.sx;
+    p.Y = a.Y; p.ACC = a.ACC; p.absmax = a.absmax; p.status = a.status;
+    auto fn = nm_gemm_kernel<SPARSE, BN, EPI>;
+    NM_CUDA_TRY(cudaFuncSetAttribute((const void*)fn, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::SMEM));
+    const int grid = p.n_tiles < sm_count() ? p.n_tiles : sm_count();
+    fn<<<grid, kGemmThreads, Cfg::SMEM, a.stream>>>(tw, tx, p);
+    NM_CUDA_TRY(cudaGetLastError());
+    return NM_OK;
+}
+
+template <bool SPARSE, int EPI>
+static int pick_bn(const LinearArgs& a) {
+    const int out_tiles = (a.W->out + kBM - 1) / kBM, sms = sm_count();
+    const bool fits192 = !SPARSE || a.W->in / 32 <= GemmCfg<SPARSE, 192>::META_COLS;
+    if (fits192 && (long long)out_tiles * ((a.tokens + 191) / 192) >= sms) return launch_gemm<SPARSE, 192, EPI>(a);
+    if ((long long)out_tiles * ((a.tokens + 127) / 128) >= sms) return launch_gemm<SPARSE, 128, EPI>(a);
+    return launch_gemm<SPARSE, 64, EPI>(a);
+}
+
+static int check_linear(int tokens, int out, int in, int n, int m, int bits) {
+    int rc = check_pattern(out, in, n, m, bits);
+    if (rc != NM_OK) return rc;
+    if (tokens < 0) return NM_ERR_SHAPE;
+    if (in % kKB) return NM_ERR_SHAPE;          // reduction length: whole 128-wide k-blocks
+    if (in > 8192) return NM_ERR_UNSUPPORTED;   // metadata of one output tile must fit in TMEM
+    if (!((n == 2 && m == 4 && bits == 8) || (n == m && bits == 8))) return NM_ERR_UNSUPPORTED;
+    return NM_OK;
+}
+
+static int run_linear(const LinearArgs& a, int epi) {
+    if (!a.W) return NM_ERR_NULL;
+    const nm_packed_t& W = *a.W;
+    int rc = check_linear(a.tokens, W.out, W.in, W.n, W.m, W.bits);
+    if (rc != NM_OK) return rc;
+    const bool sparse = W.n != W.m;
+    if (!a.X || !W.values || (sparse && !W.meta)) return NM_ERR_NULL;
+    if (epi == EPI_F32 && (!a.Y || !a.sw)) return NM_ERR_NULL;
+    if (epi == EPI_ACC && !a.ACC) return NM_ERR_NULL;
+    if (!aligned(a.X, 16) || !aligned(W.values, 16) || (W.meta && !aligned(W.meta, 16))) return NM_ERR_ALIGN;
+    if ((a.Y && !aligned(a.Y, 4)) || (a.ACC && !aligned(a.ACC, 4))) return NM_ERR_ALIGN;
+    if (a.tokens == 0 || W.out == 0) return NM_OK;
+    if (sparse) return epi == EPI_F32 ? pick_bn<true, EPI_F32>(a) : pick_bn<true, EPI_ACC>(a);
+    return epi == EPI_F32 ? pick_bn<false, EPI_F32>(a) : pick_bn<false, EPI_ACC>(a);
+}
+
+}  // namespace nm
+
+extern "C" {
+
+int nm_int_linear_check(int tokens, int out, int in, int n, int m, int bits) {
+    return nm::check_linear(tokens, out, in, n, m, bits);
+}
+
+size_t nm_int_linear_workspace_bytes(int, int, int, int, int, int) { return 0; }
+
+int nm_int_linear(const int8_t* X, int tokens, const nm_packed_t* W, float sx, const float* sw,
+                  const float* bias, float* Y, void*, size_t, uint32_t* status, void* stream) {
+    nm::LinearArgs a{X, tokens, W, sx, nullptr, sw, bias, Y, nullptr, nullptr, status, (cudaStream_t)stream};
+    return nm::run_linear(a, nm::EPI_F32);
+}
+
+int nm_int_linear_dsx(const int8_t* X, int tokens, const nm_packed_t* W, const float* sx_dev,
+                      const float* sw, const float* bias, float* Y, float* absmax_out, void*, size_t,
+                      uint32_t* status, void* stream) {
+    if (!sx_dev) return NM_ERR_NULL;
+    nm::LinearArgs a{X, tokens, W, 0.0f, sx_dev, sw, bias, Y, nullptr, absmax_out, status, (cudaStream_t)stream};
+    return nm::run_linear(a, nm::EPI_F32);
+}
+
+int nm_int_linear_acc(const int8_t* X, int tokens, const nm_packed_t* W, int32_t* ACC, void*, size_t,
+                      uint32_t* status, void* stream) {
+    nm::LinearArgs a{X, tokens, W, 1.0f, nullptr, nullptr, nullptr, nullptr, ACC, nullptr, status, (cudaStream_t)stream};
+    return nm::run_linear(a, nm::EPI_ACC);
+}
+
+}  // extern "C"
