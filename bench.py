@@ -1,0 +1,432 @@
+#!/usr/bin/env python
+"""Benchmark of the N:M low-bit hot path on B200.
+
+One step = one pass of the whole hot path over one batch of synthetic input:
+  (1) projection + quantise + pack (2:4, 8 bit) of the four linear weights of one BERT-large
+      encoder layer (W ~ N(0,0.02) plus ADMM dual U ~ N(0,0.002)), one batched launch;
+  (2) the four integer 2:4 GEMMs of that layer (QKV 1024->3072, out 1024->1024, FFN1 1024->4096,
+      FFN2 4096->1024) at 16384 tokens, int8 activations, fp32 bias + dequantisation epilogue.
+`value` is the dense-equivalent integer throughput of the step's GEMMs (2 * T * K * out summed over
+the four shapes) divided by the whole step time, in TOPS.  Per-kernel figures (GEMM TOPS per shape,
+projection/pack GB/s on the full 24-layer sweep) ride along in `kernels`.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference]
+
+N > 1 (launched under torchrun): every rank runs the same per-GPU workload on its own data, no
+data-path collective (weak scaling); the time is the maximum over ranks.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import tempfile
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np
+
+TOKENS = 16384
+PATTERN = (2, 4, 8)
+NOMINAL_SPARSE_INT8_TOPS = 9000.0   # vendor figure for 2:4 INT8 on one B200 (dense 4500)
+NOMINAL_HBM_GBS = 8000.0
+METRIC = "2:4-sparse INT8 GEMM dense-equivalent TOPS over one hot-path step (pack + 4 GEMMs)"
+WORKLOAD = "BERT-large encoder-layer GEMMs (QKV/out/FFN1/FFN2, hidden 1024) at 16384 tokens, 2:4 int8 weights"
+
+
+def peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        p = json.load(open(path))
+        return {"hbm_gbs": float(p["hbm_gbs"]), "bf16_tflops": float(p["bf16_tflops"]),
+                "bf16_tflops_sustained": float(p.get("bf16_tflops_sustained", p["bf16_tflops"])),
+                "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
+
+
+def gemm_ops(tokens, k, out):
+    return 2.0 * tokens * k * out
+
+
+def gemm_bytes(tokens, k, out, n=2, m=4, bits=8):
+    """Algorithmic HBM bytes of one GEMM launch: X + packed values + metadata + scales/bias + Y."""
+    fb = 2 if m == 4 else 4
+    vals = out * (k // m) * n * bits / 8
+    meta = 0 if n == m else out * (k // m) * n * fb / 8
+    return tokens * k + vals + meta + 8 * out + 4.0 * tokens * out
+
+
+def pack_bytes(out, k, n, m, bits, with_u=True):
+    """Algorithmic HBM bytes of packing one matrix: W (+U) read, values + metadata + scales written."""
+    fb = 2 if m == 4 else 4
+    vals = out * (k // m) * n * bits / 8
+    meta = 0 if n == m else out * (k // m) * n * fb / 8
+    return out * k * 4.0 * (2 if with_u else 1) + vals + meta + 4 * out
+
+
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons while the timed region runs."""
+
+    def __init__(self, index):
+        self.index = index
+        self.proc = None
+        self.path = None
+
+    def start(self):
+        fd, self.path = tempfile.mkstemp(suffix=".csv")
+        os.close(fd)
+        q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+             "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+             "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), f"--query-gpu={q}",
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=open(self.path, "w"), stderr=subprocess.DEVNULL)
+        except OSError:
+            self.proc = None
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.proc is None:
+            return out
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        sm, reasons, mx = [], set(), None
+        for line in open(self.path):
+            f = [x.strip() for x in line.split(",")]
+            if len(f) < 8:
+                continue
+            try:
+                sm.append(float(f[0]))
+                mx = float(f[1])
+            except ValueError:
+                continue
+            for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), f[4:8]):
+                if v.lower().startswith("active"):
+                    reasons.add(name)
+        os.unlink(self.path)
+        if sm:
+            out.update(sm_mhz=float(np.median(sm)), sm_max_mhz=mx, reasons=sorted(reasons), samples=len(sm))
+        return out
+
+
+# ------------------------------------------------------------------------------------------------
+# reference arm: the CPU oracle, as it stands, on a bounded sample of the same workload
+# ------------------------------------------------------------------------------------------------
+def oracle_step(sample_tokens, state):
+    """One bounded step of the oracle: pack the attn_out matrix (1024x1024) and run every GEMM of
+    the layer on `sample_tokens` tokens.  Returns (seconds, dense-equivalent ops)."""
+    import oracle
+    import workloads as wl
+    n, m, bits = PATTERN
+    if "packed" not in state:
+        oracle.set_threads(oracle.max_threads())
+        rng = np.random.default_rng(2)
+        state["packed"], state["X"] = [], []
+        for name, k, out in wl.BERT_LARGE_GEMMS:
+            W = wl.normal(rng, (out, k), wl.W_STD)
+            v, meta, s = oracle.project_pack(W, None, n, m, bits)
+            state["packed"].append((oracle.unpack(v, meta, out, k, n, m, bits), s, wl.normal(rng, (out,), wl.W_STD)))
+            state["X"].append(wl.random_int8(5, (sample_tokens, k)))
+        state["W_pack"], state["U_pack"] = wl.pack_sweep_matrix(3, 1, 1024, 1024)
+    t0 = time.perf_counter()
+    oracle.project_pack(state["W_pack"], state["U_pack"], n, m, bits)
+    ops = 0.0
+    for (D, s, b), X in zip(state["packed"], state["X"]):
+        oracle.int_linear(X, D, 0.03, s, b, want_acc=False)
+        ops += gemm_ops(X.shape[0], D.shape[1], D.shape[0])
+    return time.perf_counter() - t0, ops
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return 0
+    import oracle
+    state = {}
+    sample_tokens = 512
+    for _ in range(max(args.warmup, 1)):
+        oracle_step(sample_tokens, state)
+    secs, ops = 0.0, 0.0
+    for _ in range(args.steps):
+        s, o = oracle_step(sample_tokens, state)
+        secs += s
+        ops += o
+    value = ops / secs / 1e12
+    cores = oracle.max_threads()
+    sample = f"pack of one 1024x1024 matrix + the four BERT-large GEMMs on the first {sample_tokens} tokens per step"
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": "TOPS", "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * secs / args.steps,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "int8",
+            "data": "synthetic", "config": {"workload": WORKLOAD, "sample": sample},
+            "cpu_baseline": {"value": value, "unit": "TOPS", "cores": cores, "kind": "oracle", "sample": sample},
+            "e2e": {"value": value, "unit": "TOPS", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line))
+    return 0
+
+
+def cpu_baseline(budget_s=15.0):
+    """The oracle timed on the host cores on a bounded sample (~budget_s of CPU work)."""
+    import oracle
+    state = {}
+    probe, _ = oracle_step(16, state)          # includes building the inputs' first touch
+    probe, ops = oracle_step(16, state)
+    tokens = int(max(16, min(1024, 16 * budget_s / max(probe, 1e-3))))
+    state = {}
+    oracle_step(tokens, state)
+    secs, ops = oracle_step(tokens, state)
+    return {"value": ops / secs / 1e12, "unit": "TOPS", "cores": oracle.max_threads(), "kind": "oracle",
+            "sample": f"pack of one 1024x1024 matrix + the four BERT-large GEMMs on the first {tokens} tokens "
+                      f"({secs:.1f} s)"}
+
+
+# ------------------------------------------------------------------------------------------------
+# CUDA arm
+# ------------------------------------------------------------------------------------------------
+def run_cuda(args):
+    import torch
+    import torch.distributed as dist
+    import workloads as wl
+    import paper_2206_15014_b200 as nm
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+    n, m, bits = PATTERN
+    pk = peaks()
+
+    # ---- inputs (seeded per rank: independent batches, weak scaling) ---------------------------
+    rng = np.random.default_rng([2, rank])
+    layer = []
+    for name, k, out in wl.BERT_LARGE_GEMMS:
+        W = wl.normal(rng, (out, k), wl.W_STD)
+        U = wl.normal(rng, (out, k), wl.U_STD)
+        b = wl.normal(rng, (out,), wl.W_STD)
+        Xq = wl.random_int8([5, rank, k, out], (TOKENS, k))
+        layer.append((name, k, out, W, U, b, Xq))
+
+    host = []  # pinned host copies for the end-to-end leg
+    devbuf = []
+    for name, k, out, W, U, b, Xq in layer:
+        hW, hU, hX = (torch.from_numpy(a).pin_memory() for a in (W, U, Xq))
+        hY = torch.empty((TOKENS, out), dtype=torch.float32).pin_memory()
+        host.append((hW, hU, hX, hY))
+        vb, mb = nm.nm_packed_sizes(out, k, n, m, bits)
+        d = {"W": hW.to(dev), "U": hU.to(dev), "X": hX.to(dev), "b": torch.from_numpy(b).to(dev),
+             "values": torch.empty(vb, dtype=torch.uint8, device=dev),
+             "meta": torch.empty(mb // 4, dtype=torch.int32, device=dev),
+             "scales": torch.empty(out, dtype=torch.float32, device=dev),
+             "Y": torch.empty((TOKENS, out), dtype=torch.float32, device=dev), "k": k, "out": out, "name": name}
+        d["desc"] = nm.make_packed(out, k, n, m, bits, d["values"], d["meta"])
+        devbuf.append(d)
+    status = torch.zeros(1, dtype=torch.int32, device=dev)
+    jobs = nm.make_pack_jobs([(d["W"], d["U"], n, m, bits, d["values"], d["meta"], d["scales"]) for d in devbuf])
+    ws_bytes = nm.nm_pack_workspace_bytes(len(devbuf))
+    ws = torch.empty(ws_bytes, dtype=torch.uint8, device=dev)
+    sx = 0.03
+
+    ev = lambda: torch.cuda.Event(enable_timing=True)
+    kernel_events = {"pack": []}
+    for d in devbuf:
+        kernel_events[d["name"]] = []
+
+    def step(record=False):
+        if record:
+            e0, e1 = ev(), ev()
+            e0.record()
+        nm.nm_project_pack_batched(jobs, len(devbuf), ws, ws_bytes, status)
+        if record:
+            e1.record()
+            kernel_events["pack"].append((e0, e1))
+        for d in devbuf:
+            if record:
+                e0, e1 = ev(), ev()
+                e0.record()
+            nm.nm_int_linear(d["X"], TOKENS, d["desc"], sx, d["scales"], d["b"], d["Y"], status=status)
+            if record:
+                e1.record()
+                kernel_events[d["name"]].append((e0, e1))
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def max_over_ranks(ms):
+        if world > 1:
+            t = torch.tensor([ms], dtype=torch.float64, device=dev)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            return float(t.item())
+        return ms
+
+    # ---- device-resident timing -----------------------------------------------------------------
+    for _ in range(max(args.warmup, 3)):
+        step()
+    barrier()
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+        time.sleep(0.25)
+    barrier()
+    t0, t1 = ev(), ev()
+    t0.record()
+    for _ in range(args.steps):
+        step(record=True)
+    t1.record()
+    barrier()
+    ms = max_over_ranks(t0.elapsed_time(t1))
+    rc = nm.nm_poll_status(status)
+    if rc != nm.NM_OK:
+        raise RuntimeError("device status: " + nm.nm_strerror(rc))
+    ms_per_step = ms / args.steps
+    ops_step = sum(gemm_ops(TOKENS, d["k"], d["out"]) for d in devbuf)
+    value = world * ops_step / (ms_per_step * 1e-3) / 1e12
+
+    kern = {}
+    for name, pairs in kernel_events.items():
+        kern[name] = float(np.mean([a.elapsed_time(b) for a, b in pairs])) * 1e3  # microseconds
+
+    # ---- end to end: pinned host buffers in, Y out, every step ------------------------------------
+    def e2e_step():
+        for (hW, hU, hX, hY), d in zip(host, devbuf):
+            d["W"].copy_(hW, non_blocking=True)
+            d["U"].copy_(hU, non_blocking=True)
+            d["X"].copy_(hX, non_blocking=True)
+        step()
+        for (hW, hU, hX, hY), d in zip(host, devbuf):
+            hY.copy_(d["Y"], non_blocking=True)
+
+    e2e_steps = max(1, min(args.steps, 5))
+    e2e_step()
+    barrier()
+    t0.record()
+    for _ in range(e2e_steps):
+        e2e_step()
+    t1.record()
+    barrier()
+    e2e_ms = max_over_ranks(t0.elapsed_time(t1)) / e2e_steps
+    h2d = sum(hW.numel() * 4 + hU.numel() * 4 + hX.numel() for hW, hU, hX, hY in host)
+    d2h = sum(hY.numel() * 4 for hW, hU, hX, hY in host)
+    clocks = sampler.stop() if rank == 0 else None
+
+    # ---- projection/pack on the full 24-layer sweep (its own roofline), rank 0 only ---------------
+    pack_info = None
+    if rank == 0 and not args.skip_sweep:
+        pack_info = pack_sweep(nm, torch, dev, status)
+
+    if rank == 0:
+        sparse_peak = 4.0 * pk["bf16_tflops"]
+        per_kernel = {}
+        for d in devbuf:
+            us = kern[d["name"]]
+            ops, byt = gemm_ops(TOKENS, d["k"], d["out"]), gemm_bytes(TOKENS, d["k"], d["out"])
+            per_kernel[d["name"]] = {
+                "us": us, "tops": ops / us / 1e6, "gbs": byt / us / 1e3,
+                "frac_sparse_int8_peak_measured": ops / us / 1e6 / sparse_peak,
+                "frac_sparse_int8_peak_nominal": ops / us / 1e6 / NOMINAL_SPARSE_INT8_TOPS,
+                "frac_hbm_measured": byt / us / 1e3 / pk["hbm_gbs"]}
+        pbytes = sum(pack_bytes(d["out"], d["k"], n, m, bits) for d in devbuf)
+        per_kernel["pack_layer"] = {"us": kern["pack"], "gbs": pbytes / kern["pack"] / 1e3,
+                                    "frac_hbm_measured": pbytes / kern["pack"] / 1e3 / pk["hbm_gbs"]}
+        if pack_info:
+            per_kernel["pack_sweep"] = pack_info
+        # dominant kernel of the step: the FFN1 GEMM launch (longest; bound by the fp32 Y write)
+        dom = per_kernel["ffn1"]
+        roofline = {"kernel": "nm_gemm_kernel<sparse,192> on ffn1 1024->4096", "bound": "hbm",
+                    "achieved": dom["gbs"], "peak": pk["hbm_gbs"], "unit": "GB/s",
+                    "frac": dom["gbs"] / pk["hbm_gbs"], "traffic": None, "peak_source": pk["source"]}
+        f2 = per_kernel["ffn2"]
+        roofline_tensor = {"kernel": "nm_gemm_kernel<sparse,192> on ffn2 4096->1024", "bound": "tensor",
+                           "achieved": f2["tops"], "peak": sparse_peak, "unit": "TOP/s",
+                           "frac": f2["tops"] / sparse_peak,
+                           "peak_note": "4 x measured bf16 burst (nominal int8-sparse : bf16-dense ratio)",
+                           "frac_of_nominal_9000": f2["tops"] / NOMINAL_SPARSE_INT8_TOPS, "traffic": None}
+        line = {"metric": METRIC, "value": value, "unit": "TOPS", "n_gpus": world, "steps": args.steps,
+                "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True,
+                "scaling": "weak", "vs_baseline": None, "dtype": "int8", "data": "synthetic",
+                "config": {"workload": WORKLOAD, "tokens": TOKENS, "pattern": "2:4", "bits": 8,
+                           "l2": "inputs+outputs per step (715 MB) exceed L2; no flush needed"},
+                "clocks": clocks,
+                "e2e": {"value": world * ops_step / (e2e_ms * 1e-3) / 1e12, "unit": "TOPS",
+                        "ms_per_step": e2e_ms, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
+                "gpu_launches": 5 * args.steps,
+                "roofline": roofline, "roofline_tensor": roofline_tensor, "kernels": per_kernel}
+        if pack_info:
+            line["roofline_pack"] = {"kernel": "pack_kernel<2,4,8> on the 24-layer sweep", "bound": "hbm",
+                                     "achieved": pack_info["gbs"], "peak": pk["hbm_gbs"], "unit": "GB/s",
+                                     "frac": pack_info["gbs"] / pk["hbm_gbs"],
+                                     "frac_of_nominal_8000": pack_info["gbs"] / NOMINAL_HBM_GBS, "traffic": None}
+        line["cpu_baseline"] = cpu_baseline() if (world == 1 and not args.skip_cpu) else None
+        print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+    return 0
+
+
+def pack_sweep(nm, torch, dev, status, reps=5):
+    """Projection/pack of all 96 BERT-large encoder weights (302 M parameters, 2.4 GB of fp32 W+U)
+    in one batched launch; returns its time and algorithmic GB/s."""
+    import workloads as wl
+    n, m, bits = PATTERN
+    shapes = wl.pack_sweep_shapes()
+    gen = torch.Generator(device=dev)
+    gen.manual_seed(3)
+    jobs, keep, nbytes = [], [], 0.0
+    for out, k in shapes:
+        W = torch.empty((out, k), dtype=torch.float32, device=dev).normal_(0.0, 0.02, generator=gen)
+        U = torch.empty((out, k), dtype=torch.float32, device=dev).normal_(0.0, 0.002, generator=gen)
+        vb, mb = nm.nm_packed_sizes(out, k, n, m, bits)
+        bufs = (torch.empty(vb, dtype=torch.uint8, device=dev), torch.empty(mb // 4, dtype=torch.int32, device=dev),
+                torch.empty(out, dtype=torch.float32, device=dev))
+        jobs.append((W, U, n, m, bits, *bufs))
+        keep.append((W, U, bufs))
+        nbytes += pack_bytes(out, k, n, m, bits)
+    arr = nm.make_pack_jobs(jobs)
+    ws_bytes = nm.nm_pack_workspace_bytes(len(jobs))
+    ws = torch.empty(ws_bytes, dtype=torch.uint8, device=dev)
+    for _ in range(3):
+        nm.nm_project_pack_batched(arr, len(jobs), ws, ws_bytes, status)
+    torch.cuda.synchronize()
+    times = []
+    for _ in range(reps):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        nm.nm_project_pack_batched(arr, len(jobs), ws, ws_bytes, status)
+        e1.record()
+        torch.cuda.synchronize()
+        times.append(e0.elapsed_time(e1))
+    us = float(np.median(times)) * 1e3
+    return {"us": us, "gbs": nbytes / us / 1e3, "params": int(sum(o * k for o, k in shapes)),
+            "bytes": nbytes, "matrices": len(shapes), "launches": 1}
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
+    ap.add_argument("--skip-cpu", action="store_true", help="leave the CPU-oracle baseline out")
+    ap.add_argument("--skip-sweep", action="store_true", help="leave the 24-layer pack sweep out")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        return run_reference(args)
+    return run_cuda(args)
+
+
+if __name__ == "__main__":
+    sys.exit(main())

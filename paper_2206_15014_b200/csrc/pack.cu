@@ -230,7 +230,7 @@ __global__ void __launch_bounds__(MAXT) pack_kernel(const PackJobDev* __restrict
     {
         constexpr int LB = VBITS / 8;
         uint8_t* dst = job.values + (size_t)row * job.vrow_bytes + (size_t)lane_global * LB;
-        if (full && (job.vrow_bytes % LB) == 0) store_bytes_vec<LB>(dst, vw);
+        if (full && (reinterpret_cast<uintptr_t>(dst) % (LB < 16 ? LB : 16)) == 0) store_bytes_vec<LB>(dst, vw);
         else store_bytes_slow<LB>(dst, vw, nvals / M * N * BITS / 8);
     }
     if constexpr (!kDense) {
@@ -239,12 +239,12 @@ __global__ void __launch_bounds__(MAXT) pack_kernel(const PackJobDev* __restrict
         const unsigned row_bytes = job.mrow_words * 4u;
         uint8_t* dst = reinterpret_cast<uint8_t*>(job.meta + (size_t)row * job.mrow_words) + lane_off;
         const bool last = (lane_first + 32 >= job.in);  // lane holding the end of the row
-        if (full && !last) {
+        if (full && !last && (reinterpret_cast<uintptr_t>(dst) % MB) == 0) {  // aligned vector store
             store_bytes_vec<MB>(dst, mw);
         } else {
             // the last lane also writes the zero padding up to the row's word boundary
             const unsigned wpad[3] = {mw[0], MWORDS > 1 ? mw[MWORDS - 1] : 0u, 0u};
-            store_bytes_slow<MB + 4>(dst, wpad, (int)min(row_bytes - lane_off, (unsigned)(MB + 4)));
+            store_bytes_slow<MB + 4>(dst, wpad, last ? (int)min(row_bytes - lane_off, (unsigned)(MB + 4)) : MB);
         }
     }
 }
