@@ -2,17 +2,20 @@
 //
 // The sparse operand of tcgen05.mma.sp is A, so the kernel computes D = Wq * X^T: a tile is
 // 128 output channels (TMEM lanes) x BN tokens (TMEM columns).  In TMEM one lane therefore holds
-// one output channel, whose scale and bias are per-thread constants in the epilogue, and for a
-// fixed token the 32 lanes of a warp hold 32 consecutive channels = one coalesced 128-byte store
-// into the row-major Y[tokens, out].
+// one output channel, whose scale and bias are per-thread constants in the epilogue.
 //
 // One persistent CTA per SM walks a contiguous range of tiles ordered output-tile-major, so the
 // weight tile (and its metadata) changes at most a few times per CTA.
 //   warp 0      TMA producer: X tile and W tile of every 128-wide k-block into a ring of stages
-//   warp 1      allocates TMEM, issues tcgen05.mma[.sp] (one elected lane), commits to mbarriers
+//   warp 1      allocates TMEM; one lane issues tcgen05.mma[.sp] and commits to mbarriers.  It never
+//               polls an mbarrier itself: a wait in the issuing thread leaves the tensor pipe idle for
+//               its whole latency, so readiness reaches it through hardware named barriers
+//   warp 6      gate: waits on the "stage full" / "accumulator free" / "metadata ready" mbarriers and
+//               relays each k-block to warp 1 with bar.arrive
 //   warps 2-5   copy the index metadata of the current 128 output channels into TMEM
 //               (tcgen05.st, once per output tile, whole K), then run the epilogue of tile i
-//               (tcgen05.ld -> fma -> global) while the MMAs of tile i+1 fill the other accumulator
+//               (tcgen05.ld -> fma -> shared staging -> TMA store) while the MMAs of tile i+1 fill
+//               the other accumulator
 // Every mbarrier wait is bounded; on expiry the CTA raises NM_STATUS_TIMEOUT, drains and exits.
 #include "common.cuh"
 #include "sm100_ptx.cuh"
@@ -24,10 +27,12 @@ namespace nm {
 
 constexpr int kBM = 128;            // output channels per tile (MMA M)
 constexpr int kKB = 128;            // reduction elements per pipeline stage
-constexpr int kGemmThreads = 192;   // 6 warps
+constexpr int kGemmThreads = 224;   // 7 warps
 constexpr int kTmemCols = 512;
 constexpr int kSmemLimit = 232448;  // 227 KB of dynamic shared memory per CTA
 constexpr int kSmemTail = 1024;     // barriers, TMEM slot, abort flag
+constexpr int kStoreStage = 4 * 2 * 4096;  // per epilogue warp two [32 tokens][32 channels] fp32 tiles
+constexpr int kMaxStages = 7;       // the relay cycles through 8 named barriers
 constexpr long long kWaitLimit = 1ll << 31;  // SM clocks (about a second)
 
 enum { EPI_F32 = 0, EPI_ACC = 1 };
@@ -37,6 +42,7 @@ struct GemmParams {
     int n_tok_tiles, n_tiles, kblocks;
     const uint32_t* meta;  // canonical metadata [out, mrow_words] (sparse modes)
     int mrow_words;
+    int tma_store;         // 1: epilogue writes through shared memory + TMA; 0: direct stores
     const float* sw;
     const float* bias;
     const float* sx_dev;
@@ -53,8 +59,9 @@ struct GemmCfg {
     static constexpr int A_BYTES = kBM * A_ROW;
     static constexpr int B_BYTES = BN * 128;
     static constexpr int STAGE = A_BYTES + B_BYTES;
-    static constexpr int STAGES = (kSmemLimit - kSmemTail - 1024) / STAGE;
-    static constexpr int SMEM = STAGES * STAGE + kSmemTail + 1024;
+    static constexpr int FIT = (kSmemLimit - kSmemTail - kStoreStage - 1024) / STAGE;
+    static constexpr int STAGES = FIT < kMaxStages ? FIT : kMaxStages;
+    static constexpr int SMEM = STAGES * STAGE + kStoreStage + kSmemTail + 1024;
     static constexpr int META_COL = 2 * BN;           // first TMEM column of the metadata
     static constexpr int META_COLS = kTmemCols - 2 * BN;
     static_assert(STAGES >= 3, "pipeline too shallow");
@@ -64,12 +71,13 @@ struct GemmCfg {
 template <bool SPARSE, int BN, int EPI>
 __global__ void __launch_bounds__(kGemmThreads, 1)
 nm_gemm_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant__ CUtensorMap tmap_x,
-               const GemmParams p) {
+               const __grid_constant__ CUtensorMap tmap_y, const GemmParams p) {
     using Cfg = GemmCfg<SPARSE, BN>;
     constexpr int S = Cfg::STAGES;
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
-    uint64_t* bars = reinterpret_cast<uint64_t*>(smem + S * Cfg::STAGE);
+    uint8_t* store_stage = smem + S * Cfg::STAGE;
+    uint64_t* bars = reinterpret_cast<uint64_t*>(store_stage + kStoreStage);
     // bars[0..S) full, [S..2S) empty, then acc_full[2], acc_empty[2], meta_ready, drained
     const uint32_t bar0 = ptx::smem_u32(bars);
     auto full_bar = [&](int s) { return bar0 + 8u * s; };
@@ -97,6 +105,7 @@ nm_gemm_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant
         ptx::fence_mbar_init();
         ptx::prefetch_tensormap(&tmap_w);
         ptx::prefetch_tensormap(&tmap_x);
+        if (p.tma_store) ptx::prefetch_tensormap(&tmap_y);
     }
     if (warp == 1) {
         ptx::tmem_alloc(ptx::smem_u32(tmem_slot), kTmemCols);
@@ -138,27 +147,45 @@ nm_gemm_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant
                     ptx::mbar_wait_bounded(full_bar(j % S), (j / S) & 1u, never_flag, kWaitLimit >> 4);
             }
         }
+    } else if (warp == 6) {
+        // ------------------------------ gate: mbarrier waits relayed to the MMA warp ------------
+        // Runs its full trip count even after a timeout (then without waiting), so that the MMA
+        // warp, which blocks on the named barriers, always gets its arrivals.
+        uint32_t it = 0, meta_phase = 0;
+        int prev_out_tile = -1;
+        bool ok = true;
+        auto wait = [&](uint32_t bar, uint32_t parity) {
+            if (lane == 0 && ok && !ptx::mbar_wait_bounded(bar, parity, abort_flag, kWaitLimit)) {
+                raise_timeout();
+                ok = false;
+            }
+        };
+        for (int i = 0; i < tile_count; ++i) {
+            const int tile = tile_begin + i, out_tile = tile / p.n_tok_tiles, buf = i & 1;
+            if (SPARSE && out_tile != prev_out_tile) {
+                wait(meta_bar, meta_phase);
+                meta_phase ^= 1u;
+                prev_out_tile = out_tile;
+            }
+            wait(acc_empty_bar(buf), ((i >> 1) & 1u) ^ 1u);
+            for (int kb = 0; kb < p.kblocks; ++kb, ++it) {
+                wait(full_bar(it % S), (it / S) & 1u);
+                __syncwarp();
+                ptx::named_bar_arrive(1 + (it & 7u), 64);
+            }
+        }
     } else if (warp == 1) {
         // ------------------------------ MMA issuer ---------------------------------------------
-        if (lane == 0) {
-            constexpr uint32_t idesc = ptx::idesc_i8(kBM, BN, SPARSE);
-            uint32_t it = 0, meta_phase = 0;
-            int prev_out_tile = -1;
-            bool ok = true;
-            for (int i = 0; i < tile_count && ok; ++i) {
-                const int tile = tile_begin + i, out_tile = tile / p.n_tok_tiles, buf = i & 1;
-                if (SPARSE && out_tile != prev_out_tile) {
-                    if (!ptx::mbar_wait_bounded(meta_bar, meta_phase, abort_flag, kWaitLimit)) { raise_timeout(); ok = false; break; }
-                    meta_phase ^= 1u;
-                    prev_out_tile = out_tile;
-                }
-                if (!ptx::mbar_wait_bounded(acc_empty_bar(buf), ((i >> 1) & 1u) ^ 1u, abort_flag, kWaitLimit)) { raise_timeout(); ok = false; break; }
-                ptx::tc_fence_after();
-                const uint32_t d_tmem = tmem_base + buf * BN;
-                for (int kb = 0; kb < p.kblocks; ++kb, ++it) {
-                    const int s = it % S;
-                    if (!ptx::mbar_wait_bounded(full_bar(s), (it / S) & 1u, abort_flag, kWaitLimit)) { raise_timeout(); ok = false; break; }
-                    ptx::tc_fence_after();
+        constexpr uint32_t idesc = ptx::idesc_i8(kBM, BN, SPARSE);
+        uint32_t it = 0;
+        for (int i = 0; i < tile_count; ++i) {
+            const int buf = i & 1;
+            const uint32_t d_tmem = tmem_base + buf * BN;
+            for (int kb = 0; kb < p.kblocks; ++kb, ++it) {
+                const int s = it % S;
+                ptx::named_bar_sync(1 + (it & 7u), 64);  // stage s holds k-block kb (and, for kb = 0, the
+                ptx::tc_fence_after();                   // accumulator is free and the metadata in place)
+                if (lane == 0) {
                     const uint32_t a_addr = ptx::smem_u32(smem + s * Cfg::STAGE), b_addr = a_addr + Cfg::A_BYTES;
                     if constexpr (SPARSE) {
 #pragma unroll
@@ -173,10 +200,12 @@ nm_gemm_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant
                                         ptx::smem_desc_kmajor(b_addr + 32 * j, 128, ptx::kSwizzle128), idesc, (kb | j) != 0);
                     }
                     ptx::tc_commit(empty_bar(s));  // stage reusable once these MMAs have read it
+                    if (kb == p.kblocks - 1) ptx::tc_commit(acc_full_bar(buf));
                 }
-                if (ok) ptx::tc_commit(acc_full_bar(buf));
+                __syncwarp();
             }
-            // everything issued has retired before TMEM is released
+        }
+        if (lane == 0) {  // everything issued has retired before TMEM is released
             ptx::tc_commit(drained_bar);
             ptx::mbar_wait_bounded(drained_bar, 0, never_flag, kWaitLimit);
         }
@@ -184,8 +213,10 @@ nm_gemm_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant
         // ------------------------------ metadata + epilogue warps ------------------------------
         const int q = warp & 3, row = q * 32 + lane;
         const uint32_t lane_taddr = tmem_base + ((uint32_t)(q * 32) << 16);
+        float* my_stage = reinterpret_cast<float*>(store_stage + q * 8192);
         const float sx = p.sx_dev ? *p.sx_dev : p.sx_host;
         float amax = 0.0f;
+        uint32_t n_stores = 0;
         bool ok = true;
 
         auto load_meta = [&](int out_tile) {
@@ -204,7 +235,7 @@ nm_gemm_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant
 
         for (int i = 0; i < tile_count && ok; ++i) {
             const int tile = tile_begin + i, out_tile = tile / p.n_tok_tiles, buf = i & 1;
-            const int n = out_tile * kBM + row, t0 = (tile % p.n_tok_tiles) * BN;
+            const int n0 = out_tile * kBM, n = n0 + row, t0 = (tile % p.n_tok_tiles) * BN;
             if (SPARSE && i == 0) load_meta(out_tile);
             bool got = ptx::mbar_wait_bounded(acc_full_bar(buf), (i >> 1) & 1u, abort_flag, kWaitLimit);
             ok = __all_sync(0xffffffffu, got);
@@ -220,35 +251,56 @@ nm_gemm_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant
                 c_n = __fmul_rn(sx, p.sw[n]);
                 b_n = p.bias ? p.bias[n] : 0.0f;
             }
-#pragma unroll 1
-            for (int c0 = 0; c0 < BN; c0 += 32) {
-                if (t0 + c0 >= p.tokens) break;
-                uint32_t r[32];
-                ptx::tmem_ld_32x32(lane_taddr + buf * BN + c0, r);
-                ptx::tmem_ld_wait();
-                if (n_ok) {
-                    if constexpr (EPI == EPI_F32) {
-                        float* dst = p.Y + (size_t)(t0 + c0) * p.out + n;
+            uint32_t r[2][32];
+            ptx::tmem_ld_32x32(lane_taddr + buf * BN, r[0]);
 #pragma unroll
-                        for (int j = 0; j < 32; ++j) {
-                            if (t0 + c0 + j < p.tokens) {
-                                const float y = __fmaf_rn((float)(int)r[j], c_n, b_n);
-                                __stcs(dst + (size_t)j * p.out, y);
-                                amax = fmaxf(amax, fabsf(y));
-                            }
-                        }
+            for (int c = 0; c < BN / 32; ++c) {
+                const int tc0 = t0 + c * 32;
+                if (tc0 < p.tokens) {  // warp-uniform
+                    ptx::tmem_ld_wait();
+                    const bool more = (c + 1 < BN / 32) && (tc0 + 32 < p.tokens);
+                    if (more) {
+                        ptx::tmem_ld_32x32(lane_taddr + buf * BN + (c + 1) * 32, r[(c + 1) & 1]);
                     } else {
-                        int32_t* dst = p.ACC + (size_t)(t0 + c0) * p.out + n;
+                        // the accumulator has been read completely: hand it back to the MMA warp
+                        ptx::tc_fence_before();
+                        __syncwarp();
+                        if (lane == 0) ptx::mbar_arrive(acc_empty_bar(buf));
+                    }
+                    uint32_t o[32];
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) {
+                        if constexpr (EPI == EPI_F32) {
+                            const float y = __fmaf_rn((float)(int)r[c & 1][j], c_n, b_n);
+                            if (n_ok && tc0 + j < p.tokens) amax = fmaxf(amax, fabsf(y));
+                            o[j] = __float_as_uint(y);
+                        } else {
+                            o[j] = r[c & 1][j];
+                        }
+                    }
+                    if (p.tma_store) {
+                        float* sb = my_stage + (n_stores & 1u) * 1024;
+                        if (lane == 0) ptx::bulk_wait_group_read<1>();  // the store issued two chunks ago has read sb
+                        __syncwarp();
+#pragma unroll
+                        for (int j = 0; j < 32; ++j) sb[j * 32 + lane] = __uint_as_float(o[j]);
+                        ptx::fence_proxy_async_smem();
+                        __syncwarp();
+                        if (lane == 0) {
+                            ptx::tma_store_2d(&tmap_y, n0 + q * 32, tc0, ptx::smem_u32(sb));
+                            ptx::bulk_commit_group();
+                        }
+                        ++n_stores;
+                    } else if (n_ok) {
+                        uint32_t* dst = reinterpret_cast<uint32_t*>(EPI == EPI_F32 ? (void*)p.Y : (void*)p.ACC) + (size_t)tc0 * p.out + n;
 #pragma unroll
                         for (int j = 0; j < 32; ++j)
-                            if (t0 + c0 + j < p.tokens) __stcs(dst + (size_t)j * p.out, (int)r[j]);
+                            if (tc0 + j < p.tokens) __stcs(dst + (size_t)j * p.out, o[j]);
                     }
                 }
             }
-            ptx::tc_fence_before();
-            __syncwarp();
-            if (lane == 0) ptx::mbar_arrive(acc_empty_bar(buf));
         }
+        if (lane == 0) ptx::bulk_wait_group<0>();
         if (EPI == EPI_F32 && p.absmax) {
 #pragma unroll
             for (int o = 16; o > 0; o >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, o));
@@ -286,16 +338,17 @@ static EncodeTiledFn encode_tiled_fn() {
     return fn;
 }
 
-// 2-D byte matrix [rows, row_bytes] (pitch = row_bytes), box = [box_rows, box_bytes], swizzled.
-static int make_map(CUtensorMap* map, const void* base, uint64_t rows, uint64_t row_bytes,
-                    uint32_t box_rows, uint32_t box_bytes, CUtensorMapSwizzle swz) {
+// 2-D matrix [rows, row_elems] of `esize`-byte elements (dense pitch), box = [box_rows, box_elems].
+static int make_map(CUtensorMap* map, const void* base, uint64_t rows, uint64_t row_elems,
+                    uint32_t box_rows, uint32_t box_elems, CUtensorMapSwizzle swz,
+                    CUtensorMapDataType dtype = CU_TENSOR_MAP_DATA_TYPE_UINT8, uint32_t esize = 1) {
     EncodeTiledFn fn = encode_tiled_fn();
     if (!fn) return record_text_error("cuTensorMapEncodeTiled is not available from the driver");
-    cuuint64_t dims[2] = {row_bytes, rows};
-    cuuint64_t strides[1] = {row_bytes};
-    cuuint32_t box[2] = {box_bytes, box_rows};
+    cuuint64_t dims[2] = {row_elems, rows};
+    cuuint64_t strides[1] = {row_elems * esize};
+    cuuint32_t box[2] = {box_elems, box_rows};
     cuuint32_t estr[2] = {1, 1};
-    CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void*>(base), dims, strides, box, estr,
+    CUresult r = fn(map, dtype, 2, const_cast<void*>(base), dims, strides, box, estr,
                     CU_TENSOR_MAP_INTERLEAVE_NONE, swz, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                     CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) return record_text_error("cuTensorMapEncodeTiled failed");
@@ -324,13 +377,21 @@ template <bool SPARSE, int BN, int EPI>
 static int launch_gemm(const LinearArgs& a) {
     using Cfg = GemmCfg<SPARSE, BN>;
     const nm_packed_t& W = *a.W;
-    CUtensorMap tw, tx;
+    CUtensorMap tw, tx, ty;
     int rc = make_map(&tw, W.values, (uint64_t)W.out, (uint64_t)(SPARSE ? W.in / 2 : W.in), kBM, Cfg::A_ROW,
                       SPARSE ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_128B);
     if (rc != NM_OK) return rc;
     rc = make_map(&tx, a.X, (uint64_t)a.tokens, (uint64_t)W.in, BN, 128, CU_TENSOR_MAP_SWIZZLE_128B);
     if (rc != NM_OK) return rc;
+    // The epilogue stores through TMA when Y can be described by a tensor map (16-byte aligned
+    // base and row pitch); otherwise the threads store directly.
+    void* ybase = EPI == EPI_F32 ? (void*)a.Y : (void*)a.ACC;
+    const bool tma_store = aligned(ybase, 16) && (W.out % 4) == 0;
+    rc = make_map(&ty, tma_store ? ybase : (const void*)a.X, (uint64_t)a.tokens, (uint64_t)(tma_store ? W.out : W.in / 4), 32, 32,
+                  CU_TENSOR_MAP_SWIZZLE_NONE, EPI == EPI_F32 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_INT32, 4);
+    if (rc != NM_OK) return rc;
     GemmParams p{};
+    p.tma_store = tma_store ? 1 : 0;
     p.tokens = a.tokens; p.out = W.out; p.in = W.in;
     p.n_tok_tiles = (a.tokens + BN - 1) / BN;
     p.n_tiles = p.n_tok_tiles * ((W.out + kBM - 1) / kBM);
@@ -341,7 +402,7 @@ static int launch_gemm(const LinearArgs& a) {
     auto fn = nm_gemm_kernel<SPARSE, BN, EPI>;
     NM_CUDA_TRY(cudaFuncSetAttribute((const void*)fn, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::SMEM));
     const int grid = p.n_tiles < sm_count() ? p.n_tiles : sm_count();
-    fn<<<grid, kGemmThreads, Cfg::SMEM, a.stream>>>(tw, tx, p);
+    fn<<<grid, kGemmThreads, Cfg::SMEM, a.stream>>>(tw, tx, ty, p);
     NM_CUDA_TRY(cudaGetLastError());
     return NM_OK;
 }
