@@ -106,6 +106,32 @@ int nm_project_pack_batched(const nm_pack_job_t *jobs, int njobs, void *ws, size
 size_t nm_pack_workspace_bytes(int njobs);
 
 /*
+ * nm_project_pack_batched for callers that cannot provide scratch memory.  (The paper has no
+ * counterpart: this entry point exists for deployment reasons only.)
+ *
+ * Some hosts of this library must not allocate device memory once they are running: inference
+ * servers that hand the whole GPU to a memory pool at start-up, real-time loops in which a
+ * cudaMalloc (which may synchronise the device and take an unbounded time) is forbidden, and
+ * plug-ins that run inside another framework's stream callbacks where allocation is not allowed.
+ * For them the job table that nm_project_pack_batched keeps in `ws` lives instead in a fixed
+ * device array inside the library image: NM_NOALLOC_MAX_JOBS entries of 64 bytes = 64 KB, present
+ * on every GPU that loads the library until the process exits.  This call performs no cudaMalloc,
+ * cudaFree or other allocating call; inputs and outputs are still the caller's buffers.
+ *
+ *   - njobs > NM_NOALLOC_MAX_JOBS returns NM_ERR_UNSUPPORTED and enqueues nothing.
+ *   - The first call on each device looks up the array's device address; make that first call
+ *     outside any stream capture.
+ *   - All calls on a device share the one table and each call overwrites the entries it uses
+ *     (nothing in it needs clearing).  Two calls whose work overlaps on the GPU -- different
+ *     streams, or different host threads on different streams -- race on it: serialise them
+ *     (same stream, or an event between them).
+ * Results are identical to nm_project_pack_batched on the same jobs.
+ */
+#define NM_NOALLOC_MAX_JOBS 1024
+int nm_project_pack_batched_noalloc(const nm_pack_job_t *jobs, int njobs, uint32_t *status,
+                                    void *stream);
+
+/*
  * Integer N:M linear layer (Sec. 5.3: 8-bit activations, weights of <= 8 bits widened to 8 bits for
  * the multipliers, N:M skipping the pruned half of the products) with the dequantisation of Eq. 4
  * fused in:

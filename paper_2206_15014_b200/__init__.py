@@ -3,7 +3,7 @@
 Every function has the name and the argument order of its C entry point (include/nmsparse.h) and
 takes torch CUDA tensors (used purely as device buffers) or plain integers.  All arithmetic runs in
 the library's CUDA kernels.  There is no CPU fallback: importing this package fails when the
-library has not been built (run ``python -m paper_2206_15014_b200.build``).
+library has not been built (run ``python paper_2206_15014_b200/build.py``).
 """
 from __future__ import annotations
 
@@ -15,7 +15,7 @@ LIB_PATH = os.path.join(_HERE, "libnmsparse.so")
 
 if not os.path.exists(LIB_PATH):
     raise ImportError(
-        f"{LIB_PATH} is missing: build it with `python -m paper_2206_15014_b200.build` "
+        f"{LIB_PATH} is missing: build it with `python paper_2206_15014_b200/build.py` "
         "(there is no fallback path)")
 
 _lib = ctypes.CDLL(LIB_PATH)
@@ -26,6 +26,7 @@ NM_ERR_WORKSPACE, NM_ERR_CUDA, NM_ERR_NONFINITE, NM_ERR_TIMEOUT = -5, -6, -7, -8
 
 EXPORTS = (
     "nm_packed_sizes", "nm_project_pack", "nm_project_pack_batched", "nm_pack_workspace_bytes",
+    "nm_project_pack_batched_noalloc",
     "nm_int_linear", "nm_int_linear_dsx", "nm_int_linear_acc", "nm_int_linear_workspace_bytes",
     "nm_int_linear_check", "nm_absmax", "nm_quantize_act", "nm_poll_status", "nm_strerror",
     "nm_last_cuda_error", "nm_version",
@@ -49,6 +50,7 @@ _vp, _i, _sz, _f = ctypes.c_void_p, ctypes.c_int, ctypes.c_size_t, ctypes.c_floa
 _lib.nm_packed_sizes.argtypes = [_i] * 5 + [ctypes.POINTER(_sz), ctypes.POINTER(_sz)]
 _lib.nm_project_pack.argtypes = [_vp, _vp, _i, _i, _i, _i, _i, _vp, _vp, _vp, _vp, _vp]
 _lib.nm_project_pack_batched.argtypes = [ctypes.POINTER(nm_pack_job_t), _i, _vp, _sz, _vp, _vp]
+_lib.nm_project_pack_batched_noalloc.argtypes = [ctypes.POINTER(nm_pack_job_t), _i, _vp, _vp]
 _lib.nm_pack_workspace_bytes.argtypes = [_i]
 _lib.nm_pack_workspace_bytes.restype = _sz
 _lib.nm_int_linear.argtypes = [_vp, _i, ctypes.POINTER(nm_packed_t), _f, _vp, _vp, _vp, _vp, _sz, _vp, _vp]
@@ -129,6 +131,17 @@ def make_pack_jobs(jobs):
 def nm_project_pack_batched(job_array, njobs, ws, ws_bytes, status=None, stream=None):
     _chk(_lib.nm_project_pack_batched(job_array, njobs, _ptr(ws), ws_bytes, _ptr(status), _stream(stream)),
          "nm_project_pack_batched")
+
+
+NM_NOALLOC_MAX_JOBS = 1024
+
+
+def nm_project_pack_batched_noalloc(job_array, njobs, status=None, stream=None):
+    """Batched projection whose job table sits in a fixed array inside the library (at most
+    NM_NOALLOC_MAX_JOBS jobs): for callers that may not allocate device memory.  Calls that overlap
+    on the GPU share that table and must be serialised by the caller."""
+    _chk(_lib.nm_project_pack_batched_noalloc(job_array, njobs, _ptr(status), _stream(stream)),
+         "nm_project_pack_batched_noalloc")
 
 
 def make_packed(out, in_, n, m, bits, values, meta):

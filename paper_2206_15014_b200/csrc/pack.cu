@@ -9,6 +9,7 @@
 #include "common.cuh"
 #include <cuda_runtime.h>
 #include <vector>
+#include <mutex>
 #include <algorithm>
 
 namespace nm {
@@ -388,3 +389,43 @@ int nm_project_pack_batched(const nm_pack_job_t* jobs, int njobs, void* ws, size
 }
 
 }  // extern "C"
+
+// ---------------------------------------------------------------------------------------------
+// Batched projection without any caller-provided or library-allocated scratch.
+// The job table lives in a fixed device array that is part of the loaded library image.
+// ---------------------------------------------------------------------------------------------
+namespace nm {
+
+constexpr int kNoAllocMaxJobs = 1024;  // 1024 jobs x 64 bytes = 64 KB held on every GPU that loads the library
+static __device__ __align__(256) unsigned char g_noalloc_job_table[kNoAllocMaxJobs * sizeof(PackJobDev)];
+
+// In host code `g_noalloc_job_table` is only a handle; its device address has to be asked for,
+// once per device, with that device current.
+static int noalloc_table_address(void** out) {
+    static void* cached[64] = {nullptr};
+    static std::mutex mu;
+    int dev = 0;
+    NM_CUDA_TRY(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= 64) return record_text_error("device ordinal beyond 63");
+    std::lock_guard<std::mutex> lock(mu);
+    if (!cached[dev]) {
+        void* p = nullptr;
+        NM_CUDA_TRY(cudaGetSymbolAddress(&p, g_noalloc_job_table));
+        cached[dev] = p;
+    }
+    *out = cached[dev];
+    return NM_OK;
+}
+
+}  // namespace nm
+
+extern "C" int nm_project_pack_batched_noalloc(const nm_pack_job_t* jobs, int njobs, uint32_t* status,
+                                               void* stream) {
+    if (njobs < 0) return NM_ERR_SHAPE;
+    if (njobs > nm::kNoAllocMaxJobs) return NM_ERR_UNSUPPORTED;  // beyond NM_NOALLOC_MAX_JOBS
+    if (njobs == 0) return NM_OK;
+    void* table = nullptr;
+    int rc = nm::noalloc_table_address(&table);
+    if (rc != NM_OK) return rc;
+    return nm_project_pack_batched(jobs, njobs, table, sizeof(nm::g_noalloc_job_table), status, stream);
+}
