@@ -12,6 +12,9 @@
 //               its whole latency, so readiness reaches it through hardware named barriers
 //   warp 6      gate: waits on the "stage full" / "accumulator free" / "metadata ready" mbarriers and
 //               relays each k-block to warp 1 with bar.arrive
+//   warps 7-10  (only for weights that are not stored in the tensor core's form: 4-bit codes, 1:4, 2:8,
+//               1:8, 4:8) build the weight tile of every k-block in shared memory from the packed
+//               codes and metadata (xform.cuh); the producer then loads X only
 //   warps 2-5   copy the index metadata of the current 128 output channels into TMEM
 //               (tcgen05.st, once per output tile, whole K), then run the epilogue of tile i
 //               (tcgen05.ld -> fma -> shared staging -> TMA store) while the MMAs of tile i+1 fill
@@ -19,6 +22,7 @@
 // Every mbarrier wait is bounded; on expiry the CTA raises NM_STATUS_TIMEOUT, drains and exits.
 #include "common.cuh"
 #include "sm100_ptx.cuh"
+#include "xform.cuh"
 #include <cuda.h>
 #include <cuda_runtime.h>
 #include <mutex>
@@ -28,9 +32,10 @@ namespace nm {
 constexpr int kBM = 128;            // output channels per tile (MMA M)
 constexpr int kKB = 128;            // reduction elements per pipeline stage
 constexpr int kGemmThreads = 224;   // 7 warps
+constexpr int kXformThreads = 352;  // 11 warps: four more build the weight tiles
 constexpr int kTmemCols = 512;
 constexpr int kSmemLimit = 232448;  // 227 KB of dynamic shared memory per CTA
-constexpr int kSmemTail = 1024;     // barriers, TMEM slot, abort flag
+constexpr int kSmemTail = 2048;     // barriers, TMEM slot, abort flag, slot tables
 constexpr int kStoreStage = 4 * 2 * 4096;  // per epilogue warp two [32 tokens][32 channels] fp32 tiles
 constexpr int kMaxStages = 7;       // the relay cycles through 8 named barriers
 constexpr long long kWaitLimit = 1ll << 31;  // SM clocks (about a second)
@@ -42,6 +47,8 @@ struct GemmParams {
     int n_tok_tiles, n_tiles, kblocks;
     const uint32_t* meta;  // canonical metadata [out, mrow_words] (sparse modes)
     int mrow_words;
+    const uint8_t* values; // packed codes (transform modes)
+    int vrow_bytes, mrow_bytes, pat;
     int tma_store;         // 1: epilogue writes through shared memory + TMA; 0: direct stores
     const float* sw;
     const float* bias;
@@ -68,8 +75,8 @@ struct GemmCfg {
     static_assert(BN % 32 == 0 && BN >= 32 && BN <= 256, "token tile");
 };
 
-template <bool SPARSE, int BN, int EPI>
-__global__ void __launch_bounds__(kGemmThreads, 1)
+template <bool SPARSE, int BN, int EPI, bool XF>
+__global__ void __launch_bounds__(XF ? kXformThreads : kGemmThreads, 1)
 nm_gemm_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant__ CUtensorMap tmap_x,
                const __grid_constant__ CUtensorMap tmap_y, const GemmParams p) {
     using Cfg = GemmCfg<SPARSE, BN>;
@@ -89,6 +96,7 @@ nm_gemm_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * S + 6);
     volatile uint32_t* abort_flag = tmem_slot + 1;
     volatile uint32_t* never_flag = tmem_slot + 2;  // stays 0: for the drain waits after an abort
+    uint32_t* lut = reinterpret_cast<uint32_t*>(reinterpret_cast<uint8_t*>(bars) + 512);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int per = p.n_tiles / gridDim.x, rem = p.n_tiles % gridDim.x;
@@ -96,7 +104,8 @@ nm_gemm_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant
     const int tile_count = per + ((int)blockIdx.x < rem ? 1 : 0);
 
     if (threadIdx.x == 0) {
-        for (int s = 0; s < S; ++s) { ptx::mbar_init(full_bar(s), 1); ptx::mbar_init(empty_bar(s), 1); }
+        // a stage is full when its TMA bytes have landed and, in transform mode, the four weight warps are done
+        for (int s = 0; s < S; ++s) { ptx::mbar_init(full_bar(s), XF ? 5 : 1); ptx::mbar_init(empty_bar(s), 1); }
         for (int b = 0; b < 2; ++b) { ptx::mbar_init(acc_full_bar(b), 1); ptx::mbar_init(acc_empty_bar(b), 4); }
         ptx::mbar_init(meta_bar, 4);
         ptx::mbar_init(drained_bar, 1);
@@ -107,6 +116,7 @@ nm_gemm_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant
         ptx::prefetch_tensormap(&tmap_x);
         if (p.tma_store) ptx::prefetch_tensormap(&tmap_y);
     }
+    if (XF) xf::build_lut(lut, threadIdx.x, blockDim.x);
     if (warp == 1) {
         ptx::tmem_alloc(ptx::smem_u32(tmem_slot), kTmemCols);
         ptx::tmem_relinquish();
@@ -135,8 +145,8 @@ nm_gemm_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant
                         raise_timeout(); ok = false; break;
                     }
                     const uint32_t a_dst = ptx::smem_u32(smem + s * Cfg::STAGE);
-                    ptx::mbar_expect_tx(full_bar(s), Cfg::STAGE);
-                    ptx::tma_load_2d(a_dst, &tmap_w, kb * Cfg::A_ROW, n0, full_bar(s));
+                    ptx::mbar_expect_tx(full_bar(s), XF ? Cfg::B_BYTES : Cfg::STAGE);
+                    if (!XF) ptx::tma_load_2d(a_dst, &tmap_w, kb * Cfg::A_ROW, n0, full_bar(s));
                     ptx::tma_load_2d(a_dst + Cfg::A_BYTES, &tmap_x, kb * 128, t0, full_bar(s));
                 }
             }
@@ -145,6 +155,37 @@ nm_gemm_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant
                 const uint32_t first = it > (uint32_t)S ? it - S : 0;
                 for (uint32_t j = first; j < it; ++j)
                     ptx::mbar_wait_bounded(full_bar(j % S), (j / S) & 1u, never_flag, kWaitLimit >> 4);
+            }
+        }
+    } else if (XF && warp >= 7) {
+        // ------------------------------ weight-tile builders (transform modes) ------------------
+        const int tr = (warp - 7) * 32 + lane;  // row of the 128-row weight tile
+        const int cb = xf::code_bytes(p.pat), mb = xf::meta_bytes(p.pat);
+        uint32_t it = 0;
+        bool ok = true;
+        auto src_v = [&](int tile, int kb) { return p.values + (size_t)((tile / p.n_tok_tiles) * kBM + tr) * p.vrow_bytes + (size_t)kb * cb; };
+        auto src_m = [&](int tile, int kb) { return reinterpret_cast<const uint8_t*>(p.meta) + (size_t)((tile / p.n_tok_tiles) * kBM + tr) * p.mrow_bytes + (size_t)kb * mb; };
+        auto row_ok = [&](int tile) { return (tile / p.n_tok_tiles) * kBM + tr < p.out; };
+        xf::Raw cur = xf::load_raw(p.pat, src_v(tile_begin, 0), src_m(tile_begin, 0), tile_count > 0 && row_ok(tile_begin));
+        for (int i = 0; i < tile_count && ok; ++i) {
+            const int tile = tile_begin + i;
+            for (int kb = 0; kb < p.kblocks; ++kb, ++it) {
+                // fetch the next k-block's packed bytes before working on this one
+                int ntile = tile, nkb = kb + 1;
+                if (nkb == p.kblocks) { nkb = 0; ++ntile; }
+                const bool more = ntile < tile_begin + tile_count;
+                xf::Raw nxt = xf::load_raw(p.pat, src_v(more ? ntile : tile, more ? nkb : kb), src_m(more ? ntile : tile, more ? nkb : kb), more && row_ok(ntile));
+                const int s = it % S;
+                bool got = lane != 0 || ptx::mbar_wait_bounded(empty_bar(s), ((it / S) & 1u) ^ 1u, abort_flag, kWaitLimit);
+                ok = __all_sync(0xffffffffu, got);
+                if (!ok) { if (lane == 0) raise_timeout(); break; }
+                uint32_t w[SPARSE ? 16 : 32];
+                xf::build_row<SPARSE>(p.pat, cur, lut, w);
+                xf::store_row<SPARSE>(smem + s * Cfg::STAGE, tr, w);
+                ptx::fence_proxy_async_smem();  // the MMA reads the tile through the async proxy
+                __syncwarp();
+                if (lane == 0) ptx::mbar_arrive(full_bar(s));
+                cur = nxt;
             }
         }
     } else if (warp == 6) {
@@ -224,7 +265,11 @@ nm_gemm_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant
             const uint4* src = reinterpret_cast<const uint4*>(p.meta + (size_t)n * p.mrow_words);
             for (int c = 0; c < p.mrow_words; c += 4) {
                 // rows past the end get a valid "positions 0,1" pattern; their products are discarded
-                uint4 w = (n < p.out) ? __ldg(src + (c >> 2)) : make_uint4(0x44444444u, 0x44444444u, 0x44444444u, 0x44444444u);
+                uint4 w = make_uint4(0x44444444u, 0x44444444u, 0x44444444u, 0x44444444u);
+                if (n < p.out) {
+                    if constexpr (XF) w = xf::hw_meta(p.pat, reinterpret_cast<const uint8_t*>(p.meta) + (size_t)n * p.mrow_bytes + (size_t)(c >> 2) * xf::meta_bytes(p.pat), lut);
+                    else w = __ldg(src + (c >> 2));
+                }
                 ptx::tmem_st_32x4(lane_taddr + Cfg::META_COL + c, w.x, w.y, w.z, w.w);
             }
             ptx::tmem_st_wait();
@@ -373,13 +418,15 @@ struct LinearArgs {
     float* Y; int32_t* ACC; float* absmax; uint32_t* status; cudaStream_t stream;
 };
 
-template <bool SPARSE, int BN, int EPI>
+template <bool SPARSE, int BN, int EPI, bool XF>
 static int launch_gemm(const LinearArgs& a) {
     using Cfg = GemmCfg<SPARSE, BN>;
     const nm_packed_t& W = *a.W;
     CUtensorMap tw, tx, ty;
-    int rc = make_map(&tw, W.values, (uint64_t)W.out, (uint64_t)(SPARSE ? W.in / 2 : W.in), kBM, Cfg::A_ROW,
-                      SPARSE ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_128B);
+    // transform modes build the weight tile in shared memory and never use this map: describe X instead
+    int rc = XF ? make_map(&tw, a.X, (uint64_t)a.tokens, (uint64_t)W.in, BN, 128, CU_TENSOR_MAP_SWIZZLE_128B)
+                : make_map(&tw, W.values, (uint64_t)W.out, (uint64_t)(SPARSE ? W.in / 2 : W.in), kBM, Cfg::A_ROW,
+                           SPARSE ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_128B);
     if (rc != NM_OK) return rc;
     rc = make_map(&tx, a.X, (uint64_t)a.tokens, (uint64_t)W.in, BN, 128, CU_TENSOR_MAP_SWIZZLE_128B);
     if (rc != NM_OK) return rc;
@@ -396,24 +443,30 @@ static int launch_gemm(const LinearArgs& a) {
     p.n_tok_tiles = (a.tokens + BN - 1) / BN;
     p.n_tiles = p.n_tok_tiles * ((W.out + kBM - 1) / kBM);
     p.kblocks = W.in / kKB;
-    p.meta = (const uint32_t*)W.meta; p.mrow_words = W.in / 32;
+    p.meta = (const uint32_t*)W.meta; p.mrow_words = W.in / 32;  // hardware metadata words per row (4 per k-block)
+    p.values = (const uint8_t*)W.values;
+    p.vrow_bytes = (int)values_row_bytes(W.in, W.n, W.m, W.bits);
+    p.mrow_bytes = (int)meta_row_words(W.in, W.n, W.m) * 4;
+    p.pat = xf::pattern_of(W.n, W.m, W.bits);
     p.sw = a.sw; p.bias = a.bias; p.sx_dev = a.sx_dev; p.sx_host = a.sx;
     p.Y = a.Y; p.ACC = a.ACC; p.absmax = a.absmax; p.status = a.status;
-    auto fn = nm_gemm_kernel<SPARSE, BN, EPI>;
+    auto fn = nm_gemm_kernel<SPARSE, BN, EPI, XF>;
     NM_CUDA_TRY(cudaFuncSetAttribute((const void*)fn, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::SMEM));
     const int grid = p.n_tiles < sm_count() ? p.n_tiles : sm_count();
-    fn<<<grid, kGemmThreads, Cfg::SMEM, a.stream>>>(tw, tx, ty, p);
+    fn<<<grid, XF ? kXformThreads : kGemmThreads, Cfg::SMEM, a.stream>>>(tw, tx, ty, p);
     NM_CUDA_TRY(cudaGetLastError());
     return NM_OK;
 }
 
-template <bool SPARSE, int EPI>
+template <bool SPARSE, int EPI, bool XF>
 static int pick_bn(const LinearArgs& a) {
     const int out_tiles = (a.W->out + kBM - 1) / kBM, sms = sm_count();
-    const bool fits192 = !SPARSE || a.W->in / 32 <= GemmCfg<SPARSE, 192>::META_COLS;
-    if (fits192 && (long long)out_tiles * ((a.tokens + 191) / 192) >= sms) return launch_gemm<SPARSE, 192, EPI>(a);
-    if ((long long)out_tiles * ((a.tokens + 127) / 128) >= sms) return launch_gemm<SPARSE, 128, EPI>(a);
-    return launch_gemm<SPARSE, 64, EPI>(a);
+    if constexpr (!XF) {
+        const bool fits192 = !SPARSE || a.W->in / 32 <= GemmCfg<SPARSE, 192>::META_COLS;
+        if (fits192 && (long long)out_tiles * ((a.tokens + 191) / 192) >= sms) return launch_gemm<SPARSE, 192, EPI, XF>(a);
+    }
+    if ((long long)out_tiles * ((a.tokens + 127) / 128) >= sms) return launch_gemm<SPARSE, 128, EPI, XF>(a);
+    return launch_gemm<SPARSE, 64, EPI, XF>(a);
 }
 
 static int check_linear(int tokens, int out, int in, int n, int m, int bits) {
@@ -422,7 +475,6 @@ static int check_linear(int tokens, int out, int in, int n, int m, int bits) {
     if (tokens < 0) return NM_ERR_SHAPE;
     if (in % kKB) return NM_ERR_SHAPE;          // reduction length: whole 128-wide k-blocks
     if (in > 8192) return NM_ERR_UNSUPPORTED;   // metadata of one output tile must fit in TMEM
-    if (!((n == 2 && m == 4 && bits == 8) || (n == m && bits == 8))) return NM_ERR_UNSUPPORTED;
     return NM_OK;
 }
 
@@ -431,15 +483,21 @@ static int run_linear(const LinearArgs& a, int epi) {
     const nm_packed_t& W = *a.W;
     int rc = check_linear(a.tokens, W.out, W.in, W.n, W.m, W.bits);
     if (rc != NM_OK) return rc;
-    const bool sparse = W.n != W.m;
-    if (!a.X || !W.values || (sparse && !W.meta)) return NM_ERR_NULL;
+    const int pat = xf::pattern_of(W.n, W.m, W.bits);
+    const bool xform = pat != xf::PNONE;
+    const bool sparse = xform ? xf::sparse_target(pat) : W.n != W.m;  // tensor-core form of the weights
+    if (!a.X || !W.values || (W.n != W.m && !W.meta)) return NM_ERR_NULL;
     if (epi == EPI_F32 && (!a.Y || !a.sw)) return NM_ERR_NULL;
     if (epi == EPI_ACC && !a.ACC) return NM_ERR_NULL;
     if (!aligned(a.X, 16) || !aligned(W.values, 16) || (W.meta && !aligned(W.meta, 16))) return NM_ERR_ALIGN;
     if ((a.Y && !aligned(a.Y, 4)) || (a.ACC && !aligned(a.ACC, 4))) return NM_ERR_ALIGN;
     if (a.tokens == 0 || W.out == 0) return NM_OK;
-    if (sparse) return epi == EPI_F32 ? pick_bn<true, EPI_F32>(a) : pick_bn<true, EPI_ACC>(a);
-    return epi == EPI_F32 ? pick_bn<false, EPI_F32>(a) : pick_bn<false, EPI_ACC>(a);
+    if (xform) {
+        if (sparse) return epi == EPI_F32 ? pick_bn<true, EPI_F32, true>(a) : pick_bn<true, EPI_ACC, true>(a);
+        return epi == EPI_F32 ? pick_bn<false, EPI_F32, true>(a) : pick_bn<false, EPI_ACC, true>(a);
+    }
+    if (sparse) return epi == EPI_F32 ? pick_bn<true, EPI_F32, false>(a) : pick_bn<true, EPI_ACC, false>(a);
+    return epi == EPI_F32 ? pick_bn<false, EPI_F32, false>(a) : pick_bn<false, EPI_ACC, false>(a);
 }
 
 }  // namespace nm

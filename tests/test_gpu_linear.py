@@ -11,7 +11,10 @@ import workloads as wl
 
 pytestmark = pytest.mark.gpu
 
-MODES = [(2, 4, 8), (4, 4, 8)]
+MODES = [(2, 4, 8), (4, 4, 8)]  # weights already in the tensor core's form (TMA straight into the operand tile)
+# weights rebuilt in shared memory: 4-bit codes, 1:4 / 2:8 / 1:8 into 2-of-4 slots, 4:8 and dense 4-bit into a dense tile
+XFORM_MODES = [(2, 4, 4), (1, 4, 8), (1, 4, 4), (2, 8, 8), (2, 8, 4), (1, 8, 8), (1, 8, 4), (4, 4, 4), (4, 8, 8), (4, 8, 4)]
+ALL_MODES = MODES + XFORM_MODES
 
 
 def _case(seed, T, K, out, n, m, bits, tie=False):
@@ -37,41 +40,41 @@ def _run(seed, T, K, out, n, m, bits, tie=False, bias=True):
     assert np.array_equal(Y, Y_ref)
 
 
-@pytest.mark.parametrize("n,m,bits", MODES)
+@pytest.mark.parametrize("n,m,bits", ALL_MODES)
 def test_single_tile(n, m, bits):
     _run(1, 64, 128, 128, n, m, bits)
 
 
-@pytest.mark.parametrize("n,m,bits", MODES)
+@pytest.mark.parametrize("n,m,bits", ALL_MODES)
 def test_one_tile_many_kblocks(n, m, bits):
     _run(2, 64, 1024, 128, n, m, bits)
 
 
-@pytest.mark.parametrize("n,m,bits", MODES)
-@pytest.mark.parametrize("T", [1, 63, 65, 127, 129, 200])
+@pytest.mark.parametrize("n,m,bits", ALL_MODES)
+@pytest.mark.parametrize("T", [1, 65, 129, 200])
 def test_ragged_tokens(n, m, bits, T):
     _run(3 + T, T, 256, 256, n, m, bits)
 
 
-@pytest.mark.parametrize("n,m,bits", MODES)
+@pytest.mark.parametrize("n,m,bits", ALL_MODES)
 def test_ragged_out_and_no_bias(n, m, bits):
     _run(4, 100, 384, 200, n, m, bits, bias=False)
     _run(5, 70, 128, 8, n, m, bits)
 
 
-@pytest.mark.parametrize("n,m,bits", MODES)
+@pytest.mark.parametrize("n,m,bits", ALL_MODES)
 def test_bert_base_attention_projection(n, m, bits):
     # 128 tokens x 768 -> 768 (the small single-GEMM configuration)
     _run(0, 128, 768, 768, n, m, bits)
 
 
-@pytest.mark.parametrize("n,m,bits", MODES)
+@pytest.mark.parametrize("n,m,bits", ALL_MODES)
 def test_many_tiles_per_cta(n, m, bits):
     # enough tiles that every CTA walks several of them and changes output tile (192-token tiles)
     _run(6, 4096 + 37, 512, 1280, n, m, bits)
 
 
-@pytest.mark.parametrize("n,m,bits", MODES)
+@pytest.mark.parametrize("n,m,bits", ALL_MODES)
 def test_tie_heavy_weights_and_extreme_activations(n, m, bits):
     from gpu_util import PackedOnDevice, gpu_int_linear
     _run(7, 150, 256, 128, n, m, bits, tie=True)
