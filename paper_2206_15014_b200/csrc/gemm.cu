@@ -31,12 +31,14 @@ namespace nm {
 
 constexpr int kBM = 128;            // output channels per tile (MMA M)
 constexpr int kKB = 128;            // reduction elements per pipeline stage
-constexpr int kGemmThreads = 224;   // 7 warps
-constexpr int kXformThreads = 352;  // 11 warps: four more build the weight tiles
+constexpr int kEpiWarps = 8;        // epilogue warps when the weights come straight from TMA (two per TMEM lane quarter)
+constexpr int kEpiWarpsXf = 4;      // with the four weight-building warps present
+constexpr int kGemmThreads = 32 * (3 + kEpiWarps);        // producer, MMA, epilogue warps, gate
+constexpr int kXformThreads = 32 * (3 + kEpiWarpsXf + 4); // ... plus four warps that build the weight tiles
 constexpr int kTmemCols = 512;
 constexpr int kSmemLimit = 232448;  // 227 KB of dynamic shared memory per CTA
 constexpr int kSmemTail = 2048;     // barriers, TMEM slot, abort flag, slot tables
-constexpr int kStoreStage = 4 * 2 * 4096;  // per epilogue warp two [32 tokens][32 channels] fp32 tiles
+constexpr int kStoreStage = 8 * 4096;  // [32 tokens][32 channels] fp32 staging tiles: two per warp (4 warps) or one (8 warps)
 constexpr int kMaxStages = 7;       // the relay cycles through 8 named barriers
 constexpr long long kWaitLimit = 1ll << 31;  // SM clocks (about a second)
 
@@ -98,6 +100,7 @@ nm_gemm_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant
     volatile uint32_t* never_flag = tmem_slot + 2;  // stays 0: for the drain waits after an abort
     uint32_t* lut = reinterpret_cast<uint32_t*>(reinterpret_cast<uint8_t*>(bars) + 512);
 
+    constexpr int EW = XF ? kEpiWarpsXf : kEpiWarps, kGateWarp = 2 + EW;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int per = p.n_tiles / gridDim.x, rem = p.n_tiles % gridDim.x;
     const int tile_begin = blockIdx.x * per + min((int)blockIdx.x, rem);
@@ -106,7 +109,7 @@ nm_gemm_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant
     if (threadIdx.x == 0) {
         // a stage is full when its TMA bytes have landed and, in transform mode, the four weight warps are done
         for (int s = 0; s < S; ++s) { ptx::mbar_init(full_bar(s), XF ? 5 : 1); ptx::mbar_init(empty_bar(s), 1); }
-        for (int b = 0; b < 2; ++b) { ptx::mbar_init(acc_full_bar(b), 1); ptx::mbar_init(acc_empty_bar(b), 4); }
+        for (int b = 0; b < 2; ++b) { ptx::mbar_init(acc_full_bar(b), 1); ptx::mbar_init(acc_empty_bar(b), XF ? kEpiWarpsXf : kEpiWarps); }
         ptx::mbar_init(meta_bar, 4);
         ptx::mbar_init(drained_bar, 1);
         *abort_flag = 0;
@@ -157,9 +160,9 @@ nm_gemm_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant
                     ptx::mbar_wait_bounded(full_bar(j % S), (j / S) & 1u, never_flag, kWaitLimit >> 4);
             }
         }
-    } else if (XF && warp >= 7) {
+    } else if (XF && warp >= kGateWarp + 1) {
         // ------------------------------ weight-tile builders (transform modes) ------------------
-        const int tr = (warp - 7) * 32 + lane;  // row of the 128-row weight tile
+        const int tr = (warp - (kGateWarp + 1)) * 32 + lane;  // row of the 128-row weight tile
         const int cb = xf::code_bytes(p.pat), mb = xf::meta_bytes(p.pat);
         uint32_t it = 0;
         bool ok = true;
@@ -188,7 +191,7 @@ nm_gemm_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant
                 cur = nxt;
             }
         }
-    } else if (warp == 6) {
+    } else if (warp == kGateWarp) {
         // ------------------------------ gate: mbarrier waits relayed to the MMA warp ------------
         // Runs its full trip count even after a timeout (then without waiting), so that the MMA
         // warp, which blocks on the named barriers, always gets its arrivals.
@@ -252,9 +255,15 @@ nm_gemm_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant
         }
     } else {
         // ------------------------------ metadata + epilogue warps ------------------------------
-        const int q = warp & 3, row = q * 32 + lane;
+        // Warp w may touch TMEM lanes 32 * (w % 4) ... + 31.  With eight warps two share a lane quarter
+        // and take alternate 32-column chunks of the accumulator.
+        constexpr int EWH = EW / 4;               // warps per lane quarter
+        constexpr int NBUF = 8 / EW;              // staging tiles per warp
+        constexpr int CH = BN / 32;               // chunks per accumulator
+        constexpr int CI = (CH + EWH - 1) / EWH;  // chunks per warp
+        const int ew = warp - 2, q = warp & 3, half = ew >> 2, row = q * 32 + lane;
         const uint32_t lane_taddr = tmem_base + ((uint32_t)(q * 32) << 16);
-        float* my_stage = reinterpret_cast<float*>(store_stage + q * 8192);
+        float* my_stage = reinterpret_cast<float*>(store_stage + ew * (NBUF * 4096));
         const float sx = p.sx_dev ? *p.sx_dev : p.sx_host;
         float amax = 0.0f;
         uint32_t n_stores = 0;
@@ -277,16 +286,21 @@ nm_gemm_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant
             __syncwarp();
             if (lane == 0) ptx::mbar_arrive(meta_bar);
         };
+        auto release_acc = [&](int buf) {  // this warp has read all it needs from the accumulator
+            ptx::tc_fence_before();
+            __syncwarp();
+            if (lane == 0) ptx::mbar_arrive(acc_empty_bar(buf));
+        };
 
         for (int i = 0; i < tile_count && ok; ++i) {
             const int tile = tile_begin + i, out_tile = tile / p.n_tok_tiles, buf = i & 1;
             const int n0 = out_tile * kBM, n = n0 + row, t0 = (tile % p.n_tok_tiles) * BN;
-            if (SPARSE && i == 0) load_meta(out_tile);
+            if (SPARSE && i == 0 && half == 0) load_meta(out_tile);
             bool got = ptx::mbar_wait_bounded(acc_full_bar(buf), (i >> 1) & 1u, abort_flag, kWaitLimit);
             ok = __all_sync(0xffffffffu, got);
             if (!ok) { if (lane == 0) raise_timeout(); break; }
             ptx::tc_fence_after();
-            if (SPARSE && i + 1 < tile_count) {
+            if (SPARSE && half == 0 && i + 1 < tile_count) {
                 const int next_out_tile = (tile + 1) / p.n_tok_tiles;
                 if (next_out_tile != out_tile) load_meta(next_out_tile);  // MMAs of this output tile are done
             }
@@ -296,39 +310,35 @@ nm_gemm_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant
                 c_n = __fmul_rn(sx, p.sw[n]);
                 b_n = p.bias ? p.bias[n] : 0.0f;
             }
+            const int nact = min(CH, (p.tokens - t0 + 31) >> 5);  // chunks that hold tokens (warp-uniform)
             uint32_t r[2][32];
-            ptx::tmem_ld_32x32(lane_taddr + buf * BN, r[0]);
+            if (half < nact) ptx::tmem_ld_32x32(lane_taddr + buf * BN + half * 32, r[0]);
+            else release_acc(buf);
 #pragma unroll
-            for (int c = 0; c < BN / 32; ++c) {
-                const int tc0 = t0 + c * 32;
-                if (tc0 < p.tokens) {  // warp-uniform
-                    ptx::tmem_ld_wait();
-                    const bool more = (c + 1 < BN / 32) && (tc0 + 32 < p.tokens);
-                    if (more) {
-                        ptx::tmem_ld_32x32(lane_taddr + buf * BN + (c + 1) * 32, r[(c + 1) & 1]);
-                    } else {
-                        // the accumulator has been read completely: hand it back to the MMA warp
-                        ptx::tc_fence_before();
+            for (int ci = 0; ci < CI; ++ci) {
+                const int c = half + ci * EWH, tc0 = t0 + c * 32;
+                if (c < nact) {
+                    float* sb = my_stage + (NBUF == 2 ? (n_stores & 1u) * 1024 : 0);
+                    if (p.tma_store) {  // the store that last used this staging tile has read it
+                        if (lane == 0) ptx::bulk_wait_group_read<NBUF - 1>();
                         __syncwarp();
-                        if (lane == 0) ptx::mbar_arrive(acc_empty_bar(buf));
                     }
+                    ptx::tmem_ld_wait();
+                    if (c + EWH < nact) ptx::tmem_ld_32x32(lane_taddr + buf * BN + (c + EWH) * 32, r[(ci + 1) & 1]);
+                    else release_acc(buf);
                     uint32_t o[32];
 #pragma unroll
                     for (int j = 0; j < 32; ++j) {
                         if constexpr (EPI == EPI_F32) {
-                            const float y = __fmaf_rn((float)(int)r[c & 1][j], c_n, b_n);
+                            const float y = __fmaf_rn((float)(int)r[ci & 1][j], c_n, b_n);
                             if (n_ok && tc0 + j < p.tokens) amax = fmaxf(amax, fabsf(y));
                             o[j] = __float_as_uint(y);
                         } else {
-                            o[j] = r[c & 1][j];
+                            o[j] = r[ci & 1][j];
                         }
+                        if (p.tma_store) sb[j * 32 + lane] = __uint_as_float(o[j]);
                     }
                     if (p.tma_store) {
-                        float* sb = my_stage + (n_stores & 1u) * 1024;
-                        if (lane == 0) ptx::bulk_wait_group_read<1>();  // the store issued two chunks ago has read sb
-                        __syncwarp();
-#pragma unroll
-                        for (int j = 0; j < 32; ++j) sb[j * 32 + lane] = __uint_as_float(o[j]);
                         ptx::fence_proxy_async_smem();
                         __syncwarp();
                         if (lane == 0) {
