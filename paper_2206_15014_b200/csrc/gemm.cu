@@ -26,6 +26,7 @@
 #include <cuda.h>
 #include <cuda_runtime.h>
 #include <mutex>
+#include <cstdlib>
 
 namespace nm {
 
@@ -372,6 +373,291 @@ nm_gemm_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant
 }
 
 // ---------------------------------------------------------------------------------------------
+// CTA-pair variant (cluster of two, tcgen05 cta_group::2) for weights already in tensor-core form.
+// A pair tile is 256 output channels x BN tokens.  Each CTA stages its own 128 weight rows and HALF of
+// the X tile (BN/2 tokens); one MMA issued by the leader CTA (cluster rank 0) spans both CTAs: every
+// CTA's tensor core accumulates its 128 rows over all BN tokens, taking the other half of X from the
+// peer's shared memory.  Per MAC this moves 0.63x the bytes of the one-CTA kernel through L2 and
+// through each SM's shared-memory port, and the sparse MMA is no longer shared-memory bound.
+// Protocol differences: both producers' TMA bytes are counted on the LEADER's "full" barrier; the
+// leader's commits are multicast to the "empty" / "accumulator full" barriers of both CTAs; the
+// peer's epilogue and metadata warps arrive remotely on the leader's barriers; the pair synchronises
+// as a cluster before the first remote operation and before TMEM is released.
+// ---------------------------------------------------------------------------------------------
+constexpr int kPairThreads = 32 * (3 + kEpiWarps);
+constexpr int kPairMaxStages = 9;   // the relay cycles through 15 named barriers
+
+template <bool SPARSE, int BN>
+struct PairCfg {
+    static constexpr int A_ROW = SPARSE ? 64 : 128;
+    static constexpr int A_BYTES = kBM * A_ROW;
+    static constexpr int B_ROWS = BN / 2;            // tokens staged by each CTA
+    static constexpr int B_BYTES = B_ROWS * 128;
+    static constexpr int STAGE = A_BYTES + B_BYTES;
+    static constexpr int FIT = (kSmemLimit - kSmemTail - kStoreStage - 1024) / STAGE;
+    static constexpr int STAGES = FIT < kPairMaxStages ? FIT : kPairMaxStages;
+    static constexpr int SMEM = STAGES * STAGE + kStoreStage + kSmemTail + 1024;
+    static constexpr int META_COL = 2 * BN;
+    static constexpr int META_COLS = kTmemCols - 2 * BN;
+    static_assert(B_BYTES % 1024 == 0, "X half tile must keep the swizzle alignment");
+    static_assert(BN % 32 == 0 && BN <= 256, "token tile");
+};
+
+template <bool SPARSE, int BN, int EPI>
+__global__ void __launch_bounds__(kPairThreads, 1)
+nm_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant__ CUtensorMap tmap_x,
+                    const __grid_constant__ CUtensorMap tmap_y, const GemmParams p) {
+    using Cfg = PairCfg<SPARSE, BN>;
+    constexpr int S = Cfg::STAGES;
+    constexpr int EW = kEpiWarps, kGateWarp = 2 + EW;
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = reinterpret_cast<uint8_t*>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+    uint8_t* store_stage = smem + S * Cfg::STAGE;
+    uint64_t* bars = reinterpret_cast<uint64_t*>(store_stage + kStoreStage);
+    const uint32_t bar0 = ptx::smem_u32(bars);
+    auto full_bar = [&](int s) { return bar0 + 8u * s; };              // used in the leader
+    auto empty_bar = [&](int s) { return bar0 + 8u * (S + s); };       // both CTAs (multicast commit)
+    auto acc_full_bar = [&](int b) { return bar0 + 8u * (2 * S + b); };   // both CTAs (multicast commit)
+    auto acc_empty_bar = [&](int b) { return bar0 + 8u * (2 * S + 2 + b); };  // leader; arrivals from both
+    const uint32_t meta_bar = bar0 + 8u * (2 * S + 4);                 // leader; arrivals from both
+    const uint32_t drained_bar = bar0 + 8u * (2 * S + 5);
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * S + 6);
+    volatile uint32_t* abort_flag = tmem_slot + 1;
+    volatile uint32_t* never_flag = tmem_slot + 2;
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t rank = ptx::cluster_ctarank();
+    const bool leader = rank == 0;
+    const int n_pairs = gridDim.x >> 1, pair = blockIdx.x >> 1;
+    const int per = p.n_tiles / n_pairs, rem = p.n_tiles % n_pairs;
+    const int tile_begin = pair * per + min(pair, rem);
+    const int tile_count = per + (pair < rem ? 1 : 0);
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < S; ++s) { ptx::mbar_init(full_bar(s), 1); ptx::mbar_init(empty_bar(s), 1); }
+        for (int b = 0; b < 2; ++b) { ptx::mbar_init(acc_full_bar(b), 1); ptx::mbar_init(acc_empty_bar(b), 2 * EW); }
+        ptx::mbar_init(meta_bar, 8);
+        ptx::mbar_init(drained_bar, 1);
+        *abort_flag = 0;
+        *never_flag = 0;
+        ptx::fence_mbar_init();
+        ptx::prefetch_tensormap(&tmap_w);
+        ptx::prefetch_tensormap(&tmap_x);
+        if (p.tma_store) ptx::prefetch_tensormap(&tmap_y);
+    }
+    __syncthreads();
+    ptx::cluster_arrive();   // both CTAs' barriers exist before anything remote touches them
+    ptx::cluster_wait();
+    if (warp == 1) {
+        ptx::tmem_alloc_pair(ptx::smem_u32(tmem_slot), kTmemCols);
+        ptx::tmem_relinquish_pair();
+    }
+    ptx::tc_fence_before();
+    __syncthreads();
+    ptx::tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+
+    auto raise_timeout = [&]() {
+        *abort_flag = 1;
+        if (p.status) atomicOr(p.status, NM_STATUS_TIMEOUT);
+    };
+
+    if (warp == 0) {
+        // ------------------------------ TMA producer (both CTAs) --------------------------------
+        if (lane == 0) {
+            uint32_t it = 0;
+            bool ok = true;
+            for (int i = 0; i < tile_count && ok; ++i) {
+                const int tile = tile_begin + i;
+                const int n0 = (tile / p.n_tok_tiles) * (2 * kBM) + (int)rank * kBM;
+                const int t0 = (tile % p.n_tok_tiles) * BN + (int)rank * Cfg::B_ROWS;
+                for (int kb = 0; kb < p.kblocks; ++kb, ++it) {
+                    const int s = it % S;
+                    if (!ptx::mbar_wait_bounded(empty_bar(s), ((it / S) & 1u) ^ 1u, abort_flag, kWaitLimit)) {
+                        raise_timeout(); ok = false; break;
+                    }
+                    const uint32_t a_dst = ptx::smem_u32(smem + s * Cfg::STAGE);
+                    const uint32_t lead_full = ptx::map_to_cta(full_bar(s), 0);
+                    if (leader) ptx::mbar_expect_tx(full_bar(s), 2 * Cfg::STAGE);  // bytes of both CTAs
+                    ptx::tma_load_2d_pair(a_dst, &tmap_w, kb * Cfg::A_ROW, n0, lead_full);
+                    ptx::tma_load_2d_pair(a_dst + Cfg::A_BYTES, &tmap_x, kb * 128, t0, lead_full);
+                }
+            }
+        }
+    } else if (warp == kGateWarp) {
+        // ------------------------------ gate (leader): mbarrier waits relayed to the MMA warp ------
+        if (leader) {
+            uint32_t it = 0, meta_phase = 0;
+            int prev_out_tile = -1;
+            bool ok = true;
+            auto wait = [&](uint32_t bar, uint32_t parity) {
+                if (lane == 0 && ok && !ptx::mbar_wait_bounded(bar, parity, abort_flag, kWaitLimit)) {
+                    raise_timeout();
+                    ok = false;
+                }
+            };
+            for (int i = 0; i < tile_count; ++i) {
+                const int tile = tile_begin + i, out_tile = tile / p.n_tok_tiles, buf = i & 1;
+                if (SPARSE && out_tile != prev_out_tile) {
+                    wait(meta_bar, meta_phase);
+                    meta_phase ^= 1u;
+                    prev_out_tile = out_tile;
+                }
+                wait(acc_empty_bar(buf), ((i >> 1) & 1u) ^ 1u);
+                for (int kb = 0; kb < p.kblocks; ++kb, ++it) {
+                    wait(full_bar(it % S), (it / S) & 1u);
+                    __syncwarp();
+                    ptx::named_bar_arrive(1 + (it % 15u), 64);
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // ------------------------------ MMA issuer (leader) --------------------------------------
+        if (leader) {
+            constexpr uint32_t idesc = ptx::idesc_i8(2 * kBM, BN, SPARSE);
+            uint32_t it = 0;
+            for (int i = 0; i < tile_count; ++i) {
+                const int buf = i & 1;
+                const uint32_t d_tmem = tmem_base + buf * BN;
+                for (int kb = 0; kb < p.kblocks; ++kb, ++it) {
+                    const int s = it % S;
+                    ptx::named_bar_sync(1 + (it % 15u), 64);
+                    ptx::tc_fence_after();
+                    if (lane == 0) {
+                        const uint32_t a_addr = ptx::smem_u32(smem + s * Cfg::STAGE), b_addr = a_addr + Cfg::A_BYTES;
+                        if constexpr (SPARSE) {
+#pragma unroll
+                            for (int j = 0; j < 2; ++j)
+                                ptx::mma_sp_i8_pair(d_tmem, ptx::smem_desc_kmajor(a_addr + 32 * j, 64, ptx::kSwizzle64),
+                                                    ptx::smem_desc_kmajor(b_addr + 64 * j, 128, ptx::kSwizzle128),
+                                                    tmem_base + Cfg::META_COL + kb * 4 + 2 * j, idesc, (kb | j) != 0);
+                        } else {
+#pragma unroll
+                            for (int j = 0; j < 4; ++j)
+                                ptx::mma_i8_pair(d_tmem, ptx::smem_desc_kmajor(a_addr + 32 * j, 128, ptx::kSwizzle128),
+                                                 ptx::smem_desc_kmajor(b_addr + 32 * j, 128, ptx::kSwizzle128), idesc, (kb | j) != 0);
+                        }
+                        ptx::tc_commit_pair(empty_bar(s), 3);   // both producers may refill the stage
+                        if (kb == p.kblocks - 1) ptx::tc_commit_pair(acc_full_bar(buf), 3);
+                    }
+                    __syncwarp();
+                }
+            }
+            if (lane == 0) {
+                ptx::tc_commit_pair(drained_bar, 1);
+                ptx::mbar_wait_bounded(drained_bar, 0, never_flag, kWaitLimit);
+            }
+        }
+    } else {
+        // ------------------------------ metadata + epilogue warps (both CTAs) ----------------------
+        constexpr int EWH = EW / 4, CH = BN / 32, CI = (CH + EWH - 1) / EWH;
+        const int ew = warp - 2, q = warp & 3, half = ew >> 2, row = q * 32 + lane;
+        const uint32_t lane_taddr = tmem_base + ((uint32_t)(q * 32) << 16);
+        float* my_stage = reinterpret_cast<float*>(store_stage + ew * 4096);
+        const float sx = p.sx_dev ? *p.sx_dev : p.sx_host;
+        const uint32_t lead_meta = ptx::map_to_cta(meta_bar, 0);
+        float amax = 0.0f;
+        bool ok = true;
+
+        auto load_meta = [&](int out_tile) {
+            const int n = out_tile * (2 * kBM) + (int)rank * kBM + row;
+            const uint4* src = reinterpret_cast<const uint4*>(p.meta + (size_t)n * p.mrow_words);
+            for (int c = 0; c < p.mrow_words; c += 4) {
+                uint4 w = (n < p.out) ? __ldg(src + (c >> 2)) : make_uint4(0x44444444u, 0x44444444u, 0x44444444u, 0x44444444u);
+                ptx::tmem_st_32x4(lane_taddr + Cfg::META_COL + c, w.x, w.y, w.z, w.w);
+            }
+            ptx::tmem_st_wait();
+            ptx::tc_fence_before();
+            __syncwarp();
+            if (lane == 0) ptx::mbar_arrive_cluster(lead_meta);
+        };
+        auto release_acc = [&](int buf) {
+            ptx::tc_fence_before();
+            __syncwarp();
+            if (lane == 0) ptx::mbar_arrive_cluster(ptx::map_to_cta(acc_empty_bar(buf), 0));
+        };
+
+        for (int i = 0; i < tile_count && ok; ++i) {
+            const int tile = tile_begin + i, out_tile = tile / p.n_tok_tiles, buf = i & 1;
+            const int n0 = out_tile * (2 * kBM) + (int)rank * kBM, n = n0 + row, t0 = (tile % p.n_tok_tiles) * BN;
+            if (SPARSE && i == 0 && half == 0) load_meta(out_tile);
+            bool got = ptx::mbar_wait_bounded(acc_full_bar(buf), (i >> 1) & 1u, abort_flag, kWaitLimit);
+            ok = __all_sync(0xffffffffu, got);
+            if (!ok) { if (lane == 0) raise_timeout(); break; }
+            ptx::tc_fence_after();
+            if (SPARSE && half == 0 && i + 1 < tile_count) {
+                const int next_out_tile = (tile + 1) / p.n_tok_tiles;
+                if (next_out_tile != out_tile) load_meta(next_out_tile);
+            }
+            const bool n_ok = n < p.out;
+            float c_n = 0.0f, b_n = 0.0f;
+            if (EPI == EPI_F32 && n_ok) {
+                c_n = __fmul_rn(sx, p.sw[n]);
+                b_n = p.bias ? p.bias[n] : 0.0f;
+            }
+            const int nact = min(CH, (p.tokens - t0 + 31) >> 5);
+            uint32_t r[2][32];
+            if (half < nact) ptx::tmem_ld_32x32(lane_taddr + buf * BN + half * 32, r[0]);
+            else release_acc(buf);
+#pragma unroll
+            for (int ci = 0; ci < CI; ++ci) {
+                const int c = half + ci * EWH, tc0 = t0 + c * 32;
+                if (c < nact) {
+                    if (p.tma_store) {
+                        if (lane == 0) ptx::bulk_wait_group_read<0>();
+                        __syncwarp();
+                    }
+                    ptx::tmem_ld_wait();
+                    if (c + EWH < nact) ptx::tmem_ld_32x32(lane_taddr + buf * BN + (c + EWH) * 32, r[(ci + 1) & 1]);
+                    else release_acc(buf);
+                    uint32_t o[32];
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) {
+                        if constexpr (EPI == EPI_F32) {
+                            const float y = __fmaf_rn((float)(int)r[ci & 1][j], c_n, b_n);
+                            if (n_ok && tc0 + j < p.tokens) amax = fmaxf(amax, fabsf(y));
+                            o[j] = __float_as_uint(y);
+                        } else {
+                            o[j] = r[ci & 1][j];
+                        }
+                        if (p.tma_store) my_stage[j * 32 + lane] = __uint_as_float(o[j]);
+                    }
+                    if (p.tma_store) {
+                        ptx::fence_proxy_async_smem();
+                        __syncwarp();
+                        if (lane == 0) {
+                            ptx::tma_store_2d(&tmap_y, n0 + q * 32, tc0, ptx::smem_u32(my_stage));
+                            ptx::bulk_commit_group();
+                        }
+                    } else if (n_ok) {
+                        uint32_t* dst = reinterpret_cast<uint32_t*>(EPI == EPI_F32 ? (void*)p.Y : (void*)p.ACC) + (size_t)tc0 * p.out + n;
+#pragma unroll
+                        for (int j = 0; j < 32; ++j)
+                            if (tc0 + j < p.tokens) __stcs(dst + (size_t)j * p.out, o[j]);
+                    }
+                }
+            }
+        }
+        if (lane == 0) ptx::bulk_wait_group<0>();
+        if (EPI == EPI_F32 && p.absmax) {
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, o));
+            if (lane == 0) atomicMax(reinterpret_cast<unsigned*>(p.absmax), __float_as_uint(amax));
+        }
+    }
+
+    // Neither CTA may release TMEM or exit while the other can still reach into it.
+    ptx::tc_fence_before();
+    __syncthreads();
+    ptx::cluster_arrive();
+    ptx::cluster_wait();
+    if (warp == 1) {
+        ptx::tc_fence_after();
+        ptx::tmem_dealloc_pair(tmem_base, kTmemCols);
+    }
+}
+
+// ---------------------------------------------------------------------------------------------
 // host side
 // ---------------------------------------------------------------------------------------------
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
@@ -468,6 +754,55 @@ static int launch_gemm(const LinearArgs& a) {
     return NM_OK;
 }
 
+template <bool SPARSE, int BN, int EPI>
+static int launch_gemm_pair(const LinearArgs& a) {
+    using Cfg = PairCfg<SPARSE, BN>;
+    const nm_packed_t& W = *a.W;
+    CUtensorMap tw, tx, ty;
+    int rc = make_map(&tw, W.values, (uint64_t)W.out, (uint64_t)(SPARSE ? W.in / 2 : W.in), kBM, Cfg::A_ROW,
+                      SPARSE ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_128B);
+    if (rc != NM_OK) return rc;
+    rc = make_map(&tx, a.X, (uint64_t)a.tokens, (uint64_t)W.in, Cfg::B_ROWS, 128, CU_TENSOR_MAP_SWIZZLE_128B);
+    if (rc != NM_OK) return rc;
+    void* ybase = EPI == EPI_F32 ? (void*)a.Y : (void*)a.ACC;
+    const bool tma_store = aligned(ybase, 16) && (W.out % 4) == 0;
+    rc = make_map(&ty, tma_store ? ybase : (const void*)a.X, (uint64_t)a.tokens, (uint64_t)(tma_store ? W.out : W.in / 4), 32, 32,
+                  CU_TENSOR_MAP_SWIZZLE_NONE, EPI == EPI_F32 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_INT32, 4);
+    if (rc != NM_OK) return rc;
+    GemmParams p{};
+    p.tma_store = tma_store ? 1 : 0;
+    p.tokens = a.tokens; p.out = W.out; p.in = W.in;
+    p.n_tok_tiles = (a.tokens + BN - 1) / BN;
+    p.n_tiles = p.n_tok_tiles * ((W.out + 2 * kBM - 1) / (2 * kBM));
+    p.kblocks = W.in / 128;
+    p.meta = (const uint32_t*)W.meta; p.mrow_words = W.in / 32;
+    p.sw = a.sw; p.bias = a.bias; p.sx_dev = a.sx_dev; p.sx_host = a.sx;
+    p.Y = a.Y; p.ACC = a.ACC; p.absmax = a.absmax; p.status = a.status;
+    auto fn = nm_gemm_pair_kernel<SPARSE, BN, EPI>;
+    NM_CUDA_TRY(cudaFuncSetAttribute((const void*)fn, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::SMEM));
+    const int pairs = p.n_tiles < sm_count() / 2 ? p.n_tiles : sm_count() / 2;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(2 * pairs, 1, 1);
+    cfg.blockDim = dim3(kPairThreads, 1, 1);
+    cfg.dynamicSmemBytes = Cfg::SMEM;
+    cfg.stream = a.stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr; cfg.numAttrs = 1;
+    NM_CUDA_TRY(cudaLaunchKernelEx(&cfg, fn, tw, tx, ty, p));
+    return NM_OK;
+}
+
+// The pair kernel pays off when there is enough work for every SM pair; small problems stay on one CTA.
+template <bool SPARSE, int EPI>
+static bool use_pair(const LinearArgs& a) {
+    if (getenv("NM_NO_PAIR")) return false;
+    const long long tiles = (long long)((a.W->out + 2 * kBM - 1) / (2 * kBM)) * ((a.tokens + 191) / 192);
+    const bool fits = !SPARSE || a.W->in / 32 <= PairCfg<SPARSE, 192>::META_COLS;
+    return fits && tiles >= sm_count() / 2;
+}
+
 template <bool SPARSE, int EPI, bool XF>
 static int pick_bn(const LinearArgs& a) {
     const int out_tiles = (a.W->out + kBM - 1) / kBM, sms = sm_count();
@@ -506,8 +841,12 @@ static int run_linear(const LinearArgs& a, int epi) {
         if (sparse) return epi == EPI_F32 ? pick_bn<true, EPI_F32, true>(a) : pick_bn<true, EPI_ACC, true>(a);
         return epi == EPI_F32 ? pick_bn<false, EPI_F32, true>(a) : pick_bn<false, EPI_ACC, true>(a);
     }
-    if (sparse) return epi == EPI_F32 ? pick_bn<true, EPI_F32, false>(a) : pick_bn<true, EPI_ACC, false>(a);
-    return epi == EPI_F32 ? pick_bn<false, EPI_F32, false>(a) : pick_bn<false, EPI_ACC, false>(a);
+    if (sparse) {
+        if (epi == EPI_F32) return use_pair<true, EPI_F32>(a) ? launch_gemm_pair<true, 192, EPI_F32>(a) : pick_bn<true, EPI_F32, false>(a);
+        return use_pair<true, EPI_ACC>(a) ? launch_gemm_pair<true, 192, EPI_ACC>(a) : pick_bn<true, EPI_ACC, false>(a);
+    }
+    if (epi == EPI_F32) return use_pair<false, EPI_F32>(a) ? launch_gemm_pair<false, 192, EPI_F32>(a) : pick_bn<false, EPI_F32, false>(a);
+    return use_pair<false, EPI_ACC>(a) ? launch_gemm_pair<false, 192, EPI_ACC>(a) : pick_bn<false, EPI_ACC, false>(a);
 }
 
 }  // namespace nm
