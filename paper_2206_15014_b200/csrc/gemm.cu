@@ -389,17 +389,21 @@ constexpr int kPairMaxStages = 9;   // the relay cycles through 15 named barrier
 
 template <bool SPARSE, int BN>
 struct PairCfg {
-    static constexpr int A_ROW = SPARSE ? 64 : 128;
+    // A stage holds 128 stored bytes of every weight row (256 reduction elements when 2:4 compressed,
+    // 128 when dense) and the matching 128-byte-wide slices of X: one TMA operation each, four MMAs.
+    static constexpr int KB = SPARSE ? 256 : 128;
+    static constexpr int A_ROW = 128;
     static constexpr int A_BYTES = kBM * A_ROW;
     static constexpr int B_ROWS = BN / 2;            // tokens staged by each CTA
-    static constexpr int B_BYTES = B_ROWS * 128;
+    static constexpr int B_SUB = B_ROWS * 128;       // one 128-byte-wide slice of the X half tile
+    static constexpr int B_BYTES = B_SUB * (KB / 128);
     static constexpr int STAGE = A_BYTES + B_BYTES;
     static constexpr int FIT = (kSmemLimit - kSmemTail - kStoreStage - 1024) / STAGE;
     static constexpr int STAGES = FIT < kPairMaxStages ? FIT : kPairMaxStages;
     static constexpr int SMEM = STAGES * STAGE + kStoreStage + kSmemTail + 1024;
     static constexpr int META_COL = 2 * BN;
     static constexpr int META_COLS = kTmemCols - 2 * BN;
-    static_assert(B_BYTES % 1024 == 0, "X half tile must keep the swizzle alignment");
+    static_assert(B_SUB % 1024 == 0, "X half tile must keep the swizzle alignment");
     static_assert(BN % 32 == 0 && BN <= 256, "token tile");
 };
 
@@ -480,7 +484,8 @@ nm_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_con
                     const uint32_t lead_full = ptx::map_to_cta(full_bar(s), 0);
                     if (leader) ptx::mbar_expect_tx(full_bar(s), 2 * Cfg::STAGE);  // bytes of both CTAs
                     ptx::tma_load_2d_pair(a_dst, &tmap_w, kb * Cfg::A_ROW, n0, lead_full);
-                    ptx::tma_load_2d_pair(a_dst + Cfg::A_BYTES, &tmap_x, kb * 128, t0, lead_full);
+                    // X is mapped as [k-slice][token][128 bytes]: both slices of the stage in one operation
+                    ptx::tma_load_3d_pair(a_dst + Cfg::A_BYTES, &tmap_x, 0, t0, kb * (Cfg::KB / 128), lead_full);
                 }
             }
         }
@@ -527,10 +532,10 @@ nm_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_con
                         const uint32_t a_addr = ptx::smem_u32(smem + s * Cfg::STAGE), b_addr = a_addr + Cfg::A_BYTES;
                         if constexpr (SPARSE) {
 #pragma unroll
-                            for (int j = 0; j < 2; ++j)
-                                ptx::mma_sp_i8_pair(d_tmem, ptx::smem_desc_kmajor(a_addr + 32 * j, 64, ptx::kSwizzle64),
-                                                    ptx::smem_desc_kmajor(b_addr + 64 * j, 128, ptx::kSwizzle128),
-                                                    tmem_base + Cfg::META_COL + kb * 4 + 2 * j, idesc, (kb | j) != 0);
+                            for (int j = 0; j < 4; ++j)  // 64 reduction elements each: 32 stored bytes of A, 64 of X
+                                ptx::mma_sp_i8_pair(d_tmem, ptx::smem_desc_kmajor(a_addr + 32 * j, 128, ptx::kSwizzle128),
+                                                    ptx::smem_desc_kmajor(b_addr + (j >> 1) * Cfg::B_SUB + 64 * (j & 1), 128, ptx::kSwizzle128),
+                                                    tmem_base + Cfg::META_COL + kb * 8 + 2 * j, idesc, (kb | j) != 0);
                         } else {
 #pragma unroll
                             for (int j = 0; j < 4; ++j)
@@ -696,6 +701,21 @@ static int make_map(CUtensorMap* map, const void* base, uint64_t rows, uint64_t 
     return NM_OK;
 }
 
+// X viewed as [k-slice][token][128 bytes] so that one box covers several 128-byte-wide slices of a token tile.
+static int make_map_x3(CUtensorMap* map, const void* base, uint64_t tokens, uint64_t k_bytes, uint32_t box_rows, uint32_t box_slices) {
+    EncodeTiledFn fn = encode_tiled_fn();
+    if (!fn) return record_text_error("cuTensorMapEncodeTiled is not available from the driver");
+    cuuint64_t dims[3] = {128, tokens, k_bytes / 128};
+    cuuint64_t strides[2] = {k_bytes, 128};
+    cuuint32_t box[3] = {128, box_rows, box_slices};
+    cuuint32_t estr[3] = {1, 1, 1};
+    CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 3, const_cast<void*>(base), dims, strides, box, estr,
+                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) return record_text_error("cuTensorMapEncodeTiled failed for the 3-D view of X");
+    return NM_OK;
+}
+
 static int sm_count() {
     static int cached[64] = {0};
     int dev = 0;
@@ -760,9 +780,9 @@ static int launch_gemm_pair(const LinearArgs& a) {
     const nm_packed_t& W = *a.W;
     CUtensorMap tw, tx, ty;
     int rc = make_map(&tw, W.values, (uint64_t)W.out, (uint64_t)(SPARSE ? W.in / 2 : W.in), kBM, Cfg::A_ROW,
-                      SPARSE ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_128B);
+                      CU_TENSOR_MAP_SWIZZLE_128B);
     if (rc != NM_OK) return rc;
-    rc = make_map(&tx, a.X, (uint64_t)a.tokens, (uint64_t)W.in, Cfg::B_ROWS, 128, CU_TENSOR_MAP_SWIZZLE_128B);
+    rc = make_map_x3(&tx, a.X, (uint64_t)a.tokens, (uint64_t)W.in, Cfg::B_ROWS, Cfg::KB / 128);
     if (rc != NM_OK) return rc;
     void* ybase = EPI == EPI_F32 ? (void*)a.Y : (void*)a.ACC;
     const bool tma_store = aligned(ybase, 16) && (W.out % 4) == 0;
@@ -774,7 +794,7 @@ static int launch_gemm_pair(const LinearArgs& a) {
     p.tokens = a.tokens; p.out = W.out; p.in = W.in;
     p.n_tok_tiles = (a.tokens + BN - 1) / BN;
     p.n_tiles = p.n_tok_tiles * ((W.out + 2 * kBM - 1) / (2 * kBM));
-    p.kblocks = W.in / 128;
+    p.kblocks = (W.in + Cfg::KB - 1) / Cfg::KB;
     p.meta = (const uint32_t*)W.meta; p.mrow_words = W.in / 32;
     p.sw = a.sw; p.bias = a.bias; p.sx_dev = a.sx_dev; p.sx_host = a.sx;
     p.Y = a.Y; p.ACC = a.ACC; p.absmax = a.absmax; p.status = a.status;
