@@ -229,7 +229,11 @@ nm_gemm_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant
             for (int kb = 0; kb < p.kblocks; ++kb, ++it) {
                 const int s = it % S;
                 ptx::named_bar_sync(1 + (it & 7u), 64);  // stage s holds k-block kb (and, for kb = 0, the
-                ptx::tc_fence_after();                   // accumulator is free and the metadata in place)
+                                                         // accumulator is free and the metadata in place)
+                // The tcgen05 fence orders the MMAs after other threads' TMEM accesses (accumulator read
+                // back, metadata stores): needed once per tile.  Executed every stage it drains the MMA
+                // pipe (measured ~585 clk per stage); the staged operands are ordered by the mbarrier.
+                if (kb == 0) ptx::tc_fence_after();
                 if (lane == 0) {
                     const uint32_t a_addr = ptx::smem_u32(smem + s * Cfg::STAGE), b_addr = a_addr + Cfg::A_BYTES;
                     if constexpr (SPARSE) {
@@ -527,7 +531,7 @@ nm_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_con
                 for (int kb = 0; kb < p.kblocks; ++kb, ++it) {
                     const int s = it % S;
                     ptx::named_bar_sync(1 + (it % 15u), 64);
-                    ptx::tc_fence_after();
+                    if (kb == 0) ptx::tc_fence_after();  // once per tile (see the one-CTA kernel)
                     if (lane == 0) {
                         const uint32_t a_addr = ptx::smem_u32(smem + s * Cfg::STAGE), b_addr = a_addr + Cfg::A_BYTES;
                         if constexpr (SPARSE) {

@@ -222,6 +222,15 @@ __device__ __forceinline__ uint64_t smem_desc_kmajor(uint32_t smem_addr, uint32_
     return d;
 }
 
+// The same descriptor with its start-address field moved by `byte_offset` (a multiple of 16 that does not
+// carry out of the 14-bit field): one 32-bit add on the low word.
+__device__ __forceinline__ uint64_t desc_advance(uint64_t desc, uint32_t byte_offset) {
+    uint32_t lo = (uint32_t)desc + (byte_offset >> 4), hi = (uint32_t)(desc >> 32);
+    uint64_t r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "r"(lo), "r"(hi));
+    return r;
+}
+
 // Instruction descriptor for kind::i8: signed 8-bit A and B (both K-major), int32 accumulator.
 __host__ __device__ constexpr uint32_t idesc_i8(int m_rows, int n_cols, bool sparse) {
     return (sparse ? (1u << 2) : 0u)      // A is 2:4 sparse
