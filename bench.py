@@ -380,39 +380,42 @@ def run_cuda(args):
 
 def pack_sweep(nm, torch, dev, status, reps=5):
     """Projection/pack of all 96 BERT-large encoder weights (302 M parameters, 2.4 GB of fp32 W+U)
-    in one batched launch; returns its time and algorithmic GB/s."""
+    in one batched launch, for every (n:m, bits) of the sweep; returns time and algorithmic GB/s of the
+    2:4 / 8-bit variant plus a per-variant table."""
     import workloads as wl
-    n, m, bits = PATTERN
     shapes = wl.pack_sweep_shapes()
     gen = torch.Generator(device=dev)
     gen.manual_seed(3)
-    jobs, keep, nbytes = [], [], 0.0
+    mats = []
     for out, k in shapes:
         W = torch.empty((out, k), dtype=torch.float32, device=dev).normal_(0.0, 0.02, generator=gen)
         U = torch.empty((out, k), dtype=torch.float32, device=dev).normal_(0.0, 0.002, generator=gen)
-        vb, mb = nm.nm_packed_sizes(out, k, n, m, bits)
-        bufs = (torch.empty(vb, dtype=torch.uint8, device=dev), torch.empty(mb // 4, dtype=torch.int32, device=dev),
-                torch.empty(out, dtype=torch.float32, device=dev))
-        jobs.append((W, U, n, m, bits, *bufs))
-        keep.append((W, U, bufs))
-        nbytes += pack_bytes(out, k, n, m, bits)
-    arr = nm.make_pack_jobs(jobs)
-    ws_bytes = nm.nm_pack_workspace_bytes(len(jobs))
+        sizes = [nm.nm_packed_sizes(out, k, n, m, bits) for (n, m, bits) in wl.PACK_SWEEP]
+        vb, mb = max(v for v, _ in sizes), max(x for _, x in sizes)  # buffers large enough for every variant
+        mats.append((W, U, torch.empty(vb, dtype=torch.uint8, device=dev), torch.empty(mb // 4, dtype=torch.int32, device=dev),
+                     torch.empty(out, dtype=torch.float32, device=dev)))
+    ws_bytes = nm.nm_pack_workspace_bytes(len(mats))
     ws = torch.empty(ws_bytes, dtype=torch.uint8, device=dev)
-    for _ in range(3):
-        nm.nm_project_pack_batched(arr, len(jobs), ws, ws_bytes, status)
-    torch.cuda.synchronize()
-    times = []
-    for _ in range(reps):
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        e0.record()
-        nm.nm_project_pack_batched(arr, len(jobs), ws, ws_bytes, status)
-        e1.record()
+    table = {}
+    for (n, m, bits) in wl.PACK_SWEEP:
+        arr = nm.make_pack_jobs([(W, U, n, m, bits, v, mt, sc) for (W, U, v, mt, sc) in mats])
+        nbytes = sum(pack_bytes(o, k, n, m, bits) for o, k in shapes)
+        for _ in range(3):
+            nm.nm_project_pack_batched(arr, len(mats), ws, ws_bytes, status)
         torch.cuda.synchronize()
-        times.append(e0.elapsed_time(e1))
-    us = float(np.median(times)) * 1e3
-    return {"us": us, "gbs": nbytes / us / 1e3, "params": int(sum(o * k for o, k in shapes)),
-            "bytes": nbytes, "matrices": len(shapes), "launches": 1}
+        times = []
+        for _ in range(reps):
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            nm.nm_project_pack_batched(arr, len(mats), ws, ws_bytes, status)
+            e1.record()
+            torch.cuda.synchronize()
+            times.append(e0.elapsed_time(e1))
+        us = float(np.median(times)) * 1e3
+        table[f"{n}:{m}/{bits}b"] = {"us": us, "gbs": nbytes / us / 1e3, "bytes": nbytes}
+    head = table["2:4/8b"]
+    return {"us": head["us"], "gbs": head["gbs"], "params": int(sum(o * k for o, k in shapes)),
+            "bytes": head["bytes"], "matrices": len(shapes), "launches": 1, "variants": table}
 
 
 def main():

@@ -82,7 +82,7 @@ __device__ __forceinline__ void store_bytes_slow(uint8_t* dst, const unsigned* w
 
 // N == M: dense (quantise only, no metadata), processed in groups of 4.
 template <int N, int M, int BITS, int MAXT>
-__global__ void __launch_bounds__(MAXT) pack_kernel(const PackJobDev* __restrict__ jobs, int njobs,
+__global__ void __launch_bounds__(MAXT, MAXT == 128 ? 8 : 1) pack_kernel(const PackJobDev* __restrict__ jobs, int njobs,
                                                     PackJobDev single, uint32_t* status) {
     constexpr bool kDense = (N == M);
     constexpr int G = 32 / M;                          // groups per lane
