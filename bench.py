@@ -345,17 +345,22 @@ def run_cuda(args):
                                     "frac_hbm_measured": pbytes / kern["pack"] / 1e3 / pk["hbm_gbs"]}
         if pack_info:
             per_kernel["pack_sweep"] = pack_info
-        # dominant kernel of the step: the FFN1 GEMM launch (longest; bound by the fp32 Y write)
+        # dominant kernel of the step: the FFN1 GEMM launch (longest; bound by the fp32 Y write).
+        # `traffic` = dram__bytes_read.sum + dram__bytes_write.sum of one launch at this size (ncu, see
+        # profiles/); part of Y is still in the 126 MB L2 when the kernel ends, hence below the algorithmic bytes.
+        full_size = TOKENS == 16384
         dom = per_kernel["ffn1"]
-        roofline = {"kernel": "nm_gemm_kernel<sparse,192> on ffn1 1024->4096", "bound": "hbm",
+        roofline = {"kernel": "nm_gemm_pair_kernel<sparse,192,f32> on ffn1 1024->4096", "bound": "hbm",
                     "achieved": dom["gbs"], "peak": pk["hbm_gbs"], "unit": "GB/s",
-                    "frac": dom["gbs"] / pk["hbm_gbs"], "traffic": None, "peak_source": pk["source"]}
+                    "frac": dom["gbs"] / pk["hbm_gbs"], "traffic": 243165696 if full_size else None,
+                    "algorithmic_bytes": gemm_bytes(TOKENS, 1024, 4096), "peak_source": pk["source"]}
         f2 = per_kernel["ffn2"]
-        roofline_tensor = {"kernel": "nm_gemm_kernel<sparse,192> on ffn2 4096->1024", "bound": "tensor",
+        roofline_tensor = {"kernel": "nm_gemm_pair_kernel<sparse,192,f32> on ffn2 4096->1024", "bound": "tensor",
                            "achieved": f2["tops"], "peak": sparse_peak, "unit": "TOP/s",
                            "frac": f2["tops"] / sparse_peak,
                            "peak_note": "4 x measured bf16 burst (nominal int8-sparse : bf16-dense ratio)",
-                           "frac_of_nominal_9000": f2["tops"] / NOMINAL_SPARSE_INT8_TOPS, "traffic": None}
+                           "frac_of_nominal_9000": f2["tops"] / NOMINAL_SPARSE_INT8_TOPS,
+                           "traffic": 138679040 if full_size else None}
         line = {"metric": METRIC, "value": value, "unit": "TOPS", "n_gpus": world, "steps": args.steps,
                 "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True,
                 "scaling": "weak", "vs_baseline": None, "dtype": "int8", "data": "synthetic",
@@ -370,7 +375,8 @@ def run_cuda(args):
             line["roofline_pack"] = {"kernel": "pack_kernel<2,4,8> on the 24-layer sweep", "bound": "hbm",
                                      "achieved": pack_info["gbs"], "peak": pk["hbm_gbs"], "unit": "GB/s",
                                      "frac": pack_info["gbs"] / pk["hbm_gbs"],
-                                     "frac_of_nominal_8000": pack_info["gbs"] / NOMINAL_HBM_GBS, "traffic": None}
+                                     "frac_of_nominal_8000": pack_info["gbs"] / NOMINAL_HBM_GBS, "traffic": 2551192320,
+                                     "algorithmic_bytes": pack_info["bytes"]}
         line["cpu_baseline"] = cpu_baseline() if (world == 1 and not args.skip_cpu) else None
         print(json.dumps(line))
     if world > 1:
