@@ -77,12 +77,22 @@ __device__ __forceinline__ unsigned keep_mask(const float* a) {
     return mask;
 }
 
+// Integer code of v / s: clamp(rne(fl32(v / s))).  The scale is constant along a row, so the quotient is
+// formed from the correctly rounded reciprocal r = RN(1 / s) with one FMA correction step
+// (q = v * r; q += r * (v - s * q)), which lands within an ulp or two of the IEEE quotient.  That can
+// only change the rounded integer when the quotient sits next to a half-integer: those cases (and
+// anything non-finite, e.g. a subnormal scale whose reciprocal overflows) take the true IEEE division,
+// so the result is the same bit for bit.
 template <int BITS>
-__device__ __forceinline__ unsigned quantise_code(float v, float s) {
+__device__ __forceinline__ unsigned quantise_code(float v, float s, float r) {
     constexpr int hi = (1 << (BITS - 1)) - 1, lo = -(1 << (BITS - 1));
-    int q = __float2int_rn(__fdiv_rn(v, s));  // IEEE division, round half to even
-    q = max(lo, min(hi, q));
-    return (unsigned)q & ((1u << BITS) - 1u);
+    float q = __fmul_rn(v, r);
+    q = __fmaf_rn(__fmaf_rn(-s, q, v), r, q);
+    const float f = q - rintf(q);                      // in [-0.5, 0.5]
+    if (!(fabsf(f) <= 0.49996948f)) q = __fdiv_rn(v, s);  // within 2^-15 of a tie, or not finite
+    int c = __float2int_rn(q);                         // round half to even
+    c = max(lo, min(hi, c));
+    return (unsigned)c & ((1u << BITS) - 1u);
 }
 
 template <int NBYTES>
@@ -189,6 +199,7 @@ __global__ void __launch_bounds__(MAXT, MAXT == 128 ? 8 : 1) pack_kernel(const P
     constexpr float qmax = (float)((1 << (BITS - 1)) - 1);
     const float s = (amax == 0.0f) ? 1.0f : __fdiv_rn(amax, qmax);
     if (row_ok && chunk == 0 && lane == 0) job.scales[row] = s;
+    const float rs = __frcp_rn(s);  // correctly rounded reciprocal, once per row
 
     // ---- this lane's 32 consecutive values ----------------------------------------------------
     float v[32];
@@ -214,7 +225,7 @@ __global__ void __launch_bounds__(MAXT, MAXT == 128 ? 8 : 1) pack_kernel(const P
 #pragma unroll
                 for (int p = 0; p < M; ++p) {
                     const int pos = (g * M + p) * BITS;
-                    vw[pos >> 5] |= quantise_code<BITS>(v[g * M + p], s) << (pos & 31);
+                    vw[pos >> 5] |= quantise_code<BITS>(v[g * M + p], s, rs) << (pos & 31);
                 }
             } else {
                 float a[M];
@@ -243,7 +254,7 @@ __global__ void __launch_bounds__(MAXT, MAXT == 128 ? 8 : 1) pack_kernel(const P
 #pragma unroll
                 for (int c = 0; c < N; ++c) {
                     const int vpos = (g * N + c) * BITS, mpos = (g * N + c) * F;
-                    vw[vpos >> 5] |= quantise_code<BITS>(sel[c], s) << (vpos & 31);
+                    vw[vpos >> 5] |= quantise_code<BITS>(sel[c], s, rs) << (vpos & 31);
                     mw[mpos >> 5] |= selp[c] << (mpos & 31);
                 }
             }
