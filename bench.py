@@ -190,6 +190,22 @@ def cpu_baseline(budget_s=15.0):
                       f"({secs:.1f} s)"}
 
 
+def reduce_max_ms(ms, world, device="cpu"):
+    """Time of the slowest rank (all ranks get it).  One scalar all-reduce; the data path has none."""
+    if world <= 1:
+        return ms
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([ms], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_tops(ops_per_rank_step, world, ms_per_step):
+    """Aggregate throughput of `world` ranks that each do the same per-GPU work (weak scaling)."""
+    return world * ops_per_rank_step / (ms_per_step * 1e-3) / 1e12
+
+
 # ------------------------------------------------------------------------------------------------
 # CUDA arm
 # ------------------------------------------------------------------------------------------------
@@ -268,11 +284,7 @@ def run_cuda(args):
         torch.cuda.synchronize()
 
     def max_over_ranks(ms):
-        if world > 1:
-            t = torch.tensor([ms], dtype=torch.float64, device=dev)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            return float(t.item())
-        return ms
+        return reduce_max_ms(ms, world, dev)
 
     # ---- device-resident timing -----------------------------------------------------------------
     for _ in range(max(args.warmup, 3)):
@@ -295,7 +307,7 @@ def run_cuda(args):
         raise RuntimeError("device status: " + nm.nm_strerror(rc))
     ms_per_step = ms / args.steps
     ops_step = sum(gemm_ops(TOKENS, d["k"], d["out"]) for d in devbuf)
-    value = world * ops_step / (ms_per_step * 1e-3) / 1e12
+    value = whole_job_tops(ops_step, world, ms_per_step)
 
     kern = {}
     for name, pairs in kernel_events.items():
@@ -367,7 +379,7 @@ def run_cuda(args):
                 "config": {"workload": WORKLOAD if TOKENS == 16384 else WORKLOAD + f" (reduced to {TOKENS} tokens)", "tokens": TOKENS, "pattern": "2:4", "bits": 8,
                            "l2": "inputs+outputs per step (715 MB) exceed L2; no flush needed"},
                 "clocks": clocks,
-                "e2e": {"value": world * ops_step / (e2e_ms * 1e-3) / 1e12, "unit": "TOPS",
+                "e2e": {"value": whole_job_tops(ops_step, world, e2e_ms), "unit": "TOPS",
                         "ms_per_step": e2e_ms, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
                 "gpu_launches": 5 * args.steps,
                 "roofline": roofline, "roofline_tensor": roofline_tensor, "kernels": per_kernel}
