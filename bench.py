@@ -211,6 +211,7 @@ def whole_job_tops(ops_per_rank_step, world, ms_per_step):
 # ------------------------------------------------------------------------------------------------
 def run_cuda(args):
     TOKENS = args.tokens
+    PATTERN = (2, 4, args.bits)
     import torch
     import torch.distributed as dist
     import workloads as wl
@@ -346,7 +347,7 @@ def run_cuda(args):
         per_kernel = {}
         for d in devbuf:
             us = kern[d["name"]]
-            ops, byt = gemm_ops(TOKENS, d["k"], d["out"]), gemm_bytes(TOKENS, d["k"], d["out"])
+            ops, byt = gemm_ops(TOKENS, d["k"], d["out"]), gemm_bytes(TOKENS, d["k"], d["out"], n, m, bits)
             per_kernel[d["name"]] = {
                 "us": us, "tops": ops / us / 1e6, "gbs": byt / us / 1e3,
                 "frac_sparse_int8_peak_measured": ops / us / 1e6 / sparse_peak,
@@ -360,7 +361,7 @@ def run_cuda(args):
         # dominant kernel of the step: the FFN1 GEMM launch (longest; bound by the fp32 Y write).
         # `traffic` = dram__bytes_read.sum + dram__bytes_write.sum of one launch at this size (ncu, see
         # profiles/); part of Y is still in the 126 MB L2 when the kernel ends, hence below the algorithmic bytes.
-        full_size = TOKENS == 16384
+        full_size = TOKENS == 16384 and bits == 8
         dom = per_kernel["ffn1"]
         roofline = {"kernel": "nm_gemm_pair_kernel<sparse,192,f32> on ffn1 1024->4096", "bound": "hbm",
                     "achieved": dom["gbs"], "peak": pk["hbm_gbs"], "unit": "GB/s",
@@ -376,7 +377,7 @@ def run_cuda(args):
         line = {"metric": METRIC, "value": value, "unit": "TOPS", "n_gpus": world, "steps": args.steps,
                 "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True,
                 "scaling": "weak", "vs_baseline": None, "dtype": "int8", "data": "synthetic",
-                "config": {"workload": WORKLOAD if TOKENS == 16384 else WORKLOAD + f" (reduced to {TOKENS} tokens)", "tokens": TOKENS, "pattern": "2:4", "bits": 8,
+                "config": {"workload": WORKLOAD if TOKENS == 16384 else WORKLOAD + f" (reduced to {TOKENS} tokens)", "tokens": TOKENS, "pattern": "2:4", "bits": bits,
                            "l2": "inputs+outputs per step (715 MB) exceed L2; no flush needed"},
                 "clocks": clocks,
                 "e2e": {"value": whole_job_tops(ops_step, world, e2e_ms), "unit": "TOPS",
@@ -442,6 +443,7 @@ def main():
     ap.add_argument("--steps", type=int, default=50)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
+    ap.add_argument("--bits", type=int, default=8, choices=[8, 4], help="weight code width of the 2:4 weights (default 8)")
     ap.add_argument("--tokens", type=int, default=TOKENS, help="tokens per GEMM (default: the full workload)")
     ap.add_argument("--skip-cpu", action="store_true", help="leave the CPU-oracle baseline out")
     ap.add_argument("--skip-sweep", action="store_true", help="leave the 24-layer pack sweep out")

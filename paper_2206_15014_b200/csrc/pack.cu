@@ -33,6 +33,39 @@ __device__ __forceinline__ float4 ld_stream(const float4* p) { return __ldcs(p);
 
 // Bit mask of the positions kept in one group: position i is kept iff fewer than N others beat it,
 // where j beats i when |v_j| > |v_i|, or |v_j| == |v_i| and j < i.
+// n = 1, and 2 of 8: the kept values and their positions straight from one or two passes of
+// "largest magnitude, first one on equality" (strict >), positions ascending.
+template <int N, int M>
+__device__ __forceinline__ void select_passes(const float* v, float* sel, unsigned* selp) {
+    float best = fabsf(v[0]), bv = v[0];
+    unsigned bi = 0;
+#pragma unroll
+    for (int j = 1; j < M; ++j) {
+        const float aj = fabsf(v[j]);
+        const bool gt = aj > best;
+        best = gt ? aj : best;
+        bv = gt ? v[j] : bv;
+        bi = gt ? (unsigned)j : bi;
+    }
+    if constexpr (N == 1) {
+        sel[0] = bv; selp[0] = bi;
+    } else {
+        float best2 = -1.0f, bv2 = 0.0f;  // magnitudes are >= 0
+        unsigned bj = 0;
+#pragma unroll
+        for (int j = 0; j < M; ++j) {
+            const float aj = fabsf(v[j]);
+            const bool gt = (aj > best2) && ((unsigned)j != bi);
+            best2 = gt ? aj : best2;
+            bv2 = gt ? v[j] : bv2;
+            bj = gt ? (unsigned)j : bj;
+        }
+        const bool sw = bj < bi;
+        sel[0] = sw ? bv2 : bv; selp[0] = sw ? bj : bi;
+        sel[1] = sw ? bv : bv2; selp[1] = sw ? bi : bj;
+    }
+}
+
 template <int N, int M>
 __device__ __forceinline__ unsigned keep_mask(const float* a) {
     if constexpr (N == 1 || (N == 2 && M == 8)) {  // (2:4 is faster with the 6-compare rank network below)
@@ -228,15 +261,31 @@ __global__ void __launch_bounds__(MAXT, MAXT == 128 ? 8 : 1) pack_kernel(const P
                     vw[pos >> 5] |= quantise_code<BITS>(v[g * M + p], s, rs) << (pos & 31);
                 }
             } else {
-                float a[M];
-#pragma unroll
-                for (int p = 0; p < M; ++p) a[p] = fabsf(v[g * M + p]);
-                const unsigned mask = keep_mask<N, M>(a);
-                // compaction: slot c receives the c-th kept position (ascending)
                 float sel[N];
                 unsigned selp[N];
 #pragma unroll
                 for (int c = 0; c < N; ++c) { sel[c] = 0.0f; selp[c] = 0; }
+                constexpr bool kPasses = (N == 1) || (N == 2 && M == 8);
+                unsigned mask = 0;
+                if constexpr (kPasses) {
+                    select_passes<N, M>(v + g * M, sel, selp);
+                } else {
+                    float a[M];
+#pragma unroll
+                    for (int p = 0; p < M; ++p) a[p] = fabsf(v[g * M + p]);
+                    mask = keep_mask<N, M>(a);
+                }
+                // compaction: slot c receives the c-th kept position (ascending)
+                if constexpr (kPasses) {
+                } else if constexpr (N == 2 && M == 4) {
+                    // two of four: the first kept position is 0, 1 or 2, the second 3, 2 or 1
+                    const float* g4 = v + g * 4;
+                    const bool b0 = mask & 1u, b1 = mask & 2u, b2 = mask & 4u, b3 = mask & 8u;
+                    sel[0] = b0 ? g4[0] : (b1 ? g4[1] : g4[2]);
+                    selp[0] = b0 ? 0u : (b1 ? 1u : 2u);
+                    sel[1] = b3 ? g4[3] : (b2 ? g4[2] : g4[1]);
+                    selp[1] = b3 ? 3u : (b2 ? 2u : 1u);
+                } else {
 #pragma unroll
                 for (int p = 0; p < M; ++p) {
                     const bool kept = (mask >> p) & 1u;
@@ -250,6 +299,7 @@ __global__ void __launch_bounds__(MAXT, MAXT == 128 ? 8 : 1) pack_kernel(const P
                             selp[c] = hit ? (unsigned)p : selp[c];
                         }
                     }
+                }
                 }
 #pragma unroll
                 for (int c = 0; c < N; ++c) {
