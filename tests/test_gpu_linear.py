@@ -121,3 +121,50 @@ def test_linear_is_deterministic():
     a = gpu_int_linear(Xq, packed, sx, b)
     c = gpu_int_linear(Xq, packed, sx, b)
     assert np.array_equal(a[0], c[0]) and np.array_equal(a[1], c[1])
+
+
+@pytest.mark.parametrize("n,m,bits,K", [(2, 4, 8, 8192), (2, 4, 8, 6144), (4, 4, 8, 8192), (2, 4, 4, 6144), (1, 8, 8, 8192)])
+def test_long_reductions(n, m, bits, K):
+    # reductions beyond 4096: the metadata of one output tile only fits next to 128-token accumulators
+    _run(10 + K, 300, K, 256, n, m, bits)
+
+
+def test_largest_accumulators_fit_int32():
+    # K = 8192 with saturated operands: |acc| = 8192 * 128 * 127 < 2^31
+    from gpu_util import PackedOnDevice, gpu_int_linear
+    K, out, T = 8192, 128, 40
+    W = np.ones((out, K), np.float32)
+    v, meta, s = oracle.project_pack(W, None, 4, 4, 8)
+    D = oracle.unpack(v, meta, out, K, 4, 4, 8)
+    Xq = np.full((T, K), -128, np.int8)
+    acc_ref, _ = oracle.int_linear(Xq, D, 1.0, s, None, want_y=False)
+    acc, _ = gpu_int_linear(Xq, PackedOnDevice(v, meta, s, out, K, 4, 4, 8), 1.0, None)
+    assert np.array_equal(acc, acc_ref) and acc.min() == -8192 * 128 * 127
+
+
+def test_linear_argument_errors():
+    import torch
+    import paper_2206_15014_b200 as nm
+    from gpu_util import DEV
+    X = torch.zeros((16, 128), dtype=torch.int8, device=DEV)
+    vals = torch.zeros(128 * 64 + 16, dtype=torch.uint8, device=DEV)
+    meta = torch.zeros(128 * 4, dtype=torch.int32, device=DEV)
+    sw = torch.ones(128, device=DEV)
+    Y = torch.zeros((16, 128), device=DEV)
+    good = nm.make_packed(128, 128, 2, 4, 8, vals, meta)
+    nm.nm_int_linear(X, 16, good, 1.0, sw, None, Y)
+    for call, code in [
+        (lambda: nm.nm_int_linear(None, 16, good, 1.0, sw, None, Y), nm.NM_ERR_NULL),
+        (lambda: nm.nm_int_linear(X, 16, good, 1.0, None, None, Y), nm.NM_ERR_NULL),
+        (lambda: nm.nm_int_linear(X, 16, nm.make_packed(128, 128, 2, 4, 8, vals, None), 1.0, sw, None, Y), nm.NM_ERR_NULL),
+        (lambda: nm.nm_int_linear(X.view(-1)[1:], 15, good, 1.0, sw, None, Y), nm.NM_ERR_ALIGN),
+        (lambda: nm.nm_int_linear(X, 16, nm.make_packed(128, 128, 2, 4, 8, vals[1:], meta), 1.0, sw, None, Y), nm.NM_ERR_ALIGN),
+        (lambda: nm.nm_int_linear(X, 16, nm.make_packed(128, 96, 2, 4, 8, vals, meta), 1.0, sw, None, Y), nm.NM_ERR_SHAPE),
+        (lambda: nm.nm_int_linear(X, -1, good, 1.0, sw, None, Y), nm.NM_ERR_SHAPE),
+        (lambda: nm.nm_int_linear(X, 16, nm.make_packed(128, 128, 2, 4, 6, vals, meta), 1.0, sw, None, Y), nm.NM_ERR_UNSUPPORTED),
+    ]:
+        with pytest.raises(nm.NmError) as e:
+            call()
+        assert e.value.code == code
+    nm.nm_int_linear(X, 0, good, 1.0, sw, None, Y)  # no tokens: nothing to do
+    assert nm.nm_poll_status() == nm.NM_OK
