@@ -10,15 +10,16 @@
 //   warp 1      allocates TMEM; one lane issues tcgen05.mma[.sp] and commits to mbarriers.  It never
 //               polls an mbarrier itself: a wait in the issuing thread leaves the tensor pipe idle for
 //               its whole latency, so readiness reaches it through hardware named barriers
-//   warp 6      gate: waits on the "stage full" / "accumulator free" / "metadata ready" mbarriers and
-//               relays each k-block to warp 1 with bar.arrive
-//   warps 7-10  (only for weights that are not stored in the tensor core's form: 4-bit codes, 1:4, 2:8,
-//               1:8, 4:8) build the weight tile of every k-block in shared memory from the packed
-//               codes and metadata (xform.cuh); the producer then loads X only
-//   warps 2-5   copy the index metadata of the current 128 output channels into TMEM
+//   warps 2-9   copy the index metadata of the current 128 output channels into TMEM
 //               (tcgen05.st, once per output tile, whole K), then run the epilogue of tile i
 //               (tcgen05.ld -> fma -> shared staging -> TMA store) while the MMAs of tile i+1 fill
-//               the other accumulator
+//               the other accumulator; two warps share a TMEM lane quarter and alternate chunks
+//   warp 10     gate: waits on the "stage full" / "accumulator free" / "metadata ready" mbarriers and
+//               relays each k-block to warp 1 with bar.arrive
+//   warps 11-   (only for weights that are not stored in the tensor core's form: 4-bit codes, 1:4, 2:8,
+//               1:8, 4:8) groups of four warps build the weight tile of every k-block in shared
+//               memory from the packed codes and metadata (xform.cuh), the groups taking k-blocks
+//               round-robin; the producer then loads X only
 // Every mbarrier wait is bounded; on expiry the CTA raises NM_STATUS_TIMEOUT, drains and exits.
 #include "common.cuh"
 #include "sm100_ptx.cuh"
@@ -33,9 +34,10 @@ namespace nm {
 constexpr int kBM = 128;            // output channels per tile (MMA M)
 constexpr int kKB = 128;            // reduction elements per pipeline stage
 constexpr int kEpiWarps = 8;        // epilogue warps when the weights come straight from TMA (two per TMEM lane quarter)
-constexpr int kEpiWarpsXf = 4;      // with the four weight-building warps present
+constexpr int kEpiWarpsXf = 8;      // with the weight-building warps present
+constexpr int kBuildGroups = 3;     // groups of four weight-building warps; group g takes k-blocks g, g + groups, ...
 constexpr int kGemmThreads = 32 * (3 + kEpiWarps);        // producer, MMA, epilogue warps, gate
-constexpr int kXformThreads = 32 * (3 + kEpiWarpsXf + 4); // ... plus four warps that build the weight tiles
+constexpr int kXformThreads = 32 * (3 + kEpiWarpsXf + 4 * kBuildGroups); // ... plus the warps that build the weight tiles
 constexpr int kTmemCols = 512;
 constexpr int kSmemLimit = 232448;  // 227 KB of dynamic shared memory per CTA
 constexpr int kSmemTail = 2048;     // barriers, TMEM slot, abort flag, slot tables
@@ -108,7 +110,7 @@ nm_gemm_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant
     const int tile_count = per + ((int)blockIdx.x < rem ? 1 : 0);
 
     if (threadIdx.x == 0) {
-        // a stage is full when its TMA bytes have landed and, in transform mode, the four weight warps are done
+        // a stage is full when its TMA bytes have landed and, in transform mode, the four warps building it are done
         for (int s = 0; s < S; ++s) { ptx::mbar_init(full_bar(s), XF ? 5 : 1); ptx::mbar_init(empty_bar(s), 1); }
         for (int b = 0; b < 2; ++b) { ptx::mbar_init(acc_full_bar(b), 1); ptx::mbar_init(acc_empty_bar(b), XF ? kEpiWarpsXf : kEpiWarps); }
         ptx::mbar_init(meta_bar, 4);
@@ -163,34 +165,55 @@ nm_gemm_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant
         }
     } else if (XF && warp >= kGateWarp + 1) {
         // ------------------------------ weight-tile builders (transform modes) ------------------
-        const int tr = (warp - (kGateWarp + 1)) * 32 + lane;  // row of the 128-row weight tile
+        // One thread builds one row of a k-block.  The work of one k-block is a long dependent chain
+        // (unpack, table lookups, byte permutes, stores, fence), so several groups of four warps
+        // take the k-blocks round-robin: group g builds pipeline steps g, g + G, g + 2G, ...
+        constexpr int G = kBuildGroups;
+        static_assert(S > G, "every group needs a stage of its own in flight");
+        const int bw = warp - (kGateWarp + 1), grp = bw >> 2;
+        const int tr = (bw & 3) * 32 + lane;  // row of the 128-row weight tile
         const int cb = xf::code_bytes(p.pat), mb = xf::meta_bytes(p.pat);
-        uint32_t it = 0;
-        bool ok = true;
-        auto src_v = [&](int tile, int kb) { return p.values + (size_t)((tile / p.n_tok_tiles) * kBM + tr) * p.vrow_bytes + (size_t)kb * cb; };
-        auto src_m = [&](int tile, int kb) { return reinterpret_cast<const uint8_t*>(p.meta) + (size_t)((tile / p.n_tok_tiles) * kBM + tr) * p.mrow_bytes + (size_t)kb * mb; };
-        auto row_ok = [&](int tile) { return (tile / p.n_tok_tiles) * kBM + tr < p.out; };
-        xf::Raw cur = xf::load_raw(p.pat, src_v(tile_begin, 0), src_m(tile_begin, 0), tile_count > 0 && row_ok(tile_begin));
-        for (int i = 0; i < tile_count && ok; ++i) {
-            const int tile = tile_begin + i;
-            for (int kb = 0; kb < p.kblocks; ++kb, ++it) {
-                // fetch the next k-block's packed bytes before working on this one
-                int ntile = tile, nkb = kb + 1;
-                if (nkb == p.kblocks) { nkb = 0; ++ntile; }
-                const bool more = ntile < tile_begin + tile_count;
-                xf::Raw nxt = xf::load_raw(p.pat, src_v(more ? ntile : tile, more ? nkb : kb), src_m(more ? ntile : tile, more ? nkb : kb), more && row_ok(ntile));
-                const int s = it % S;
-                bool got = lane != 0 || ptx::mbar_wait_bounded(empty_bar(s), ((it / S) & 1u) ^ 1u, abort_flag, kWaitLimit);
-                ok = __all_sync(0xffffffffu, got);
-                if (!ok) { if (lane == 0) raise_timeout(); break; }
-                uint32_t w[SPARSE ? 16 : 32];
-                xf::build_row<SPARSE>(p.pat, cur, lut, w);
-                xf::store_row<SPARSE>(smem + s * Cfg::STAGE, tr, w);
-                ptx::fence_proxy_async_smem();  // the MMA reads the tile through the async proxy
-                __syncwarp();
-                if (lane == 0) ptx::mbar_arrive(full_bar(s));
-                cur = nxt;
+        const uint8_t* meta8 = reinterpret_cast<const uint8_t*>(p.meta);
+        // position of a pipeline step: tile index i within this CTA's range, k-block kb; row pointers follow i
+        struct Pos { int i, kb; const uint8_t* v; const uint8_t* m; bool ok; };
+        auto locate = [&](Pos& q) {  // row pointers and validity for tile q.i
+            q.ok = q.i < tile_count;
+            const int n = q.ok ? ((tile_begin + q.i) / p.n_tok_tiles) * kBM + tr : 0;
+            q.ok = q.ok && n < p.out;
+            q.v = p.values + (size_t)n * p.vrow_bytes;
+            q.m = meta8 + (size_t)n * p.mrow_bytes;
+        };
+        auto advance = [&](Pos& q) {  // G pipeline steps further
+            q.kb += G;
+            if (q.kb >= p.kblocks) {
+                do { q.kb -= p.kblocks; ++q.i; } while (q.kb >= p.kblocks);
+                locate(q);
             }
+        };
+        Pos at{0, 0, nullptr, nullptr, false};
+        at.kb = grp;
+        while (at.kb >= p.kblocks) { at.kb -= p.kblocks; ++at.i; }
+        locate(at);
+        int s = grp % S;
+        uint32_t parity = 1u;  // of the empty barrier: the first pass over the ring finds every stage free
+        xf::Raw cur = xf::load_raw(p.pat, at.v + (size_t)at.kb * cb, at.m + (size_t)at.kb * mb, at.ok);
+        while (at.i < tile_count) {
+            // fetch this group's next k-block before working on the current one
+            Pos nx = at;
+            advance(nx);
+            xf::Raw nxt = xf::load_raw(p.pat, nx.v + (size_t)nx.kb * cb, nx.m + (size_t)nx.kb * mb, nx.ok);
+            bool got = lane != 0 || ptx::mbar_wait_bounded(empty_bar(s), parity, abort_flag, kWaitLimit);
+            if (!__all_sync(0xffffffffu, got)) { if (lane == 0) raise_timeout(); break; }
+            uint32_t w[SPARSE ? 16 : 32];
+            xf::build_row<SPARSE>(p.pat, cur, lut, w);
+            xf::store_row<SPARSE>(smem + s * Cfg::STAGE, tr, w);
+            ptx::fence_proxy_async_smem();  // the MMA reads the tile through the async proxy
+            __syncwarp();
+            if (lane == 0) ptx::mbar_arrive(full_bar(s));
+            cur = nxt;
+            at = nx;
+            s += G;
+            if (s >= S) { s -= S; parity ^= 1u; }
         }
     } else if (warp == kGateWarp) {
         // ------------------------------ gate: mbarrier waits relayed to the MMA warp ------------
@@ -316,9 +339,12 @@ nm_gemm_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant
                 b_n = p.bias ? p.bias[n] : 0.0f;
             }
             const int nact = min(CH, (p.tokens - t0 + 31) >> 5);  // chunks that hold tokens (warp-uniform)
-            uint32_t r[2][32];
-            if (half < nact) ptx::tmem_ld_32x32(lane_taddr + buf * BN + half * 32, r[0]);
-            else release_acc(buf);
+            // Accumulator chunks are read one ahead of their conversion (two register buffers); the
+            // transform kernels, short of registers with their extra warps, read each chunk when it is due.
+            constexpr int RB = XF ? 1 : 2;
+            uint32_t r[RB][32];
+            if (half >= nact) release_acc(buf);
+            else if (RB == 2) ptx::tmem_ld_32x32(lane_taddr + buf * BN + half * 32, r[0]);
 #pragma unroll
             for (int ci = 0; ci < CI; ++ci) {
                 const int c = half + ci * EWH, tc0 = t0 + c * 32;
@@ -328,20 +354,24 @@ nm_gemm_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant
                         if (lane == 0) ptx::bulk_wait_group_read<NBUF - 1>();
                         __syncwarp();
                     }
+                    if (RB == 1) ptx::tmem_ld_32x32(lane_taddr + buf * BN + c * 32, r[0]);
                     ptx::tmem_ld_wait();
-                    if (c + EWH < nact) ptx::tmem_ld_32x32(lane_taddr + buf * BN + (c + EWH) * 32, r[(ci + 1) & 1]);
-                    else release_acc(buf);
-                    uint32_t o[32];
+                    if (c + EWH >= nact) release_acc(buf);
+                    else if (RB == 2) ptx::tmem_ld_32x32(lane_taddr + buf * BN + (c + EWH) * 32, r[(ci + 1) & (RB - 1)]);
+                    // direct-store fallback (output rows not 16-byte aligned): lane = channel, j = token
+                    uint32_t* dst = reinterpret_cast<uint32_t*>(EPI == EPI_F32 ? (void*)p.Y : (void*)p.ACC) + (size_t)tc0 * p.out + n;
 #pragma unroll
                     for (int j = 0; j < 32; ++j) {
+                        uint32_t o;
                         if constexpr (EPI == EPI_F32) {
-                            const float y = __fmaf_rn((float)(int)r[ci & 1][j], c_n, b_n);
+                            const float y = __fmaf_rn((float)(int)r[ci & (RB - 1)][j], c_n, b_n);
                             if (n_ok && tc0 + j < p.tokens) amax = fmaxf(amax, fabsf(y));
-                            o[j] = __float_as_uint(y);
+                            o = __float_as_uint(y);
                         } else {
-                            o[j] = r[ci & 1][j];
+                            o = r[ci & (RB - 1)][j];
                         }
-                        if (p.tma_store) sb[j * 32 + lane] = __uint_as_float(o[j]);
+                        if (p.tma_store) sb[j * 32 + lane] = __uint_as_float(o);
+                        else if (n_ok && tc0 + j < p.tokens) __stcs(dst + (size_t)j * p.out, o);
                     }
                     if (p.tma_store) {
                         ptx::fence_proxy_async_smem();
@@ -351,11 +381,6 @@ nm_gemm_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant
                             ptx::bulk_commit_group();
                         }
                         ++n_stores;
-                    } else if (n_ok) {
-                        uint32_t* dst = reinterpret_cast<uint32_t*>(EPI == EPI_F32 ? (void*)p.Y : (void*)p.ACC) + (size_t)tc0 * p.out + n;
-#pragma unroll
-                        for (int j = 0; j < 32; ++j)
-                            if (tc0 + j < p.tokens) __stcs(dst + (size_t)j * p.out, o[j]);
                     }
                 }
             }
