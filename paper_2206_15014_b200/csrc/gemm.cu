@@ -46,6 +46,10 @@ constexpr int kMaxStages = 7;       // the relay cycles through 8 named barriers
 constexpr long long kWaitLimit = 1ll << 31;  // SM clocks (about a second)
 
 enum { EPI_F32 = 0, EPI_ACC = 1 };
+// Where the weight operand comes from: TMA (already in tensor-core form), built per k-block into the
+// stage ring, or built once per output tile into a resident region (reduction length <= kResidentKB k-blocks).
+enum { W_TMA = 0, W_BUILD = 1, W_RESIDENT = 2 };
+constexpr int kResidentKB = 8;
 
 struct GemmParams {
     int tokens, out, in;
@@ -65,32 +69,36 @@ struct GemmParams {
     uint32_t* status;
 };
 
-template <bool SPARSE, int BN>
+template <bool SPARSE, int BN, bool RESIDENT = false>
 struct GemmCfg {
     static constexpr int A_ROW = SPARSE ? 64 : 128;   // bytes of one weight row per stage
     static constexpr int A_BYTES = kBM * A_ROW;
     static constexpr int B_BYTES = BN * 128;
-    static constexpr int STAGE = A_BYTES + B_BYTES;
-    static constexpr int FIT = (kSmemLimit - kSmemTail - kStoreStage - 1024) / STAGE;
+    static constexpr int A_RES = RESIDENT ? kResidentKB * A_BYTES : 0;  // whole-K weight tile kept across token tiles
+    static constexpr int B_OFF = RESIDENT ? 0 : A_BYTES;                // X tile within a stage
+    static constexpr int STAGE = B_OFF + B_BYTES;
+    static constexpr int FIT = (kSmemLimit - kSmemTail - kStoreStage - 1024 - A_RES) / STAGE;
     static constexpr int STAGES = FIT < kMaxStages ? FIT : kMaxStages;
-    static constexpr int SMEM = STAGES * STAGE + kStoreStage + kSmemTail + 1024;
+    static constexpr int SMEM = STAGES * STAGE + A_RES + kStoreStage + kSmemTail + 1024;
     static constexpr int META_COL = 2 * BN;           // first TMEM column of the metadata
     static constexpr int META_COLS = kTmemCols - 2 * BN;
     static_assert(STAGES >= 3, "pipeline too shallow");
     static_assert(BN % 32 == 0 && BN >= 32 && BN <= 256, "token tile");
 };
 
-template <bool SPARSE, int BN, int EPI, bool XF>
-__global__ void __launch_bounds__(XF ? kXformThreads : kGemmThreads, 1)
+template <bool SPARSE, int BN, int EPI, int WSRC>
+__global__ void __launch_bounds__(WSRC != W_TMA ? kXformThreads : kGemmThreads, 1)
 nm_gemm_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant__ CUtensorMap tmap_x,
                const __grid_constant__ CUtensorMap tmap_y, const GemmParams p) {
-    using Cfg = GemmCfg<SPARSE, BN>;
+    constexpr bool XF = WSRC != W_TMA, RES = WSRC == W_RESIDENT;
+    using Cfg = GemmCfg<SPARSE, BN, RES>;
     constexpr int S = Cfg::STAGES;
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
-    uint8_t* store_stage = smem + S * Cfg::STAGE;
+    uint8_t* a_res = smem + S * Cfg::STAGE;  // resident weight tile: kResidentKB k-blocks of A_BYTES
+    uint8_t* store_stage = a_res + Cfg::A_RES;
     uint64_t* bars = reinterpret_cast<uint64_t*>(store_stage + kStoreStage);
-    // bars[0..S) full, [S..2S) empty, then acc_full[2], acc_empty[2], meta_ready, drained
+    // bars[0..S) full, [S..2S) empty, then acc_full[2], acc_empty[2], meta_ready, drained, a_full, a_free
     const uint32_t bar0 = ptx::smem_u32(bars);
     auto full_bar = [&](int s) { return bar0 + 8u * s; };
     auto empty_bar = [&](int s) { return bar0 + 8u * (S + s); };
@@ -98,7 +106,9 @@ nm_gemm_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant
     auto acc_empty_bar = [&](int b) { return bar0 + 8u * (2 * S + 2 + b); };
     const uint32_t meta_bar = bar0 + 8u * (2 * S + 4);
     const uint32_t drained_bar = bar0 + 8u * (2 * S + 5);
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * S + 6);
+    const uint32_t a_full_bar = bar0 + 8u * (2 * S + 6);  // resident weight tile built (all builder warps)
+    const uint32_t a_free_bar = bar0 + 8u * (2 * S + 7);  // ... and no longer read by any MMA
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * S + 8);
     volatile uint32_t* abort_flag = tmem_slot + 1;
     volatile uint32_t* never_flag = tmem_slot + 2;  // stays 0: for the drain waits after an abort
     uint32_t* lut = reinterpret_cast<uint32_t*>(reinterpret_cast<uint8_t*>(bars) + 512);
@@ -111,7 +121,9 @@ nm_gemm_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant
 
     if (threadIdx.x == 0) {
         // a stage is full when its TMA bytes have landed and, in transform mode, the four warps building it are done
-        for (int s = 0; s < S; ++s) { ptx::mbar_init(full_bar(s), XF ? 5 : 1); ptx::mbar_init(empty_bar(s), 1); }
+        for (int s = 0; s < S; ++s) { ptx::mbar_init(full_bar(s), WSRC == W_BUILD ? 5 : 1); ptx::mbar_init(empty_bar(s), 1); }
+        ptx::mbar_init(a_full_bar, 4 * kBuildGroups);
+        ptx::mbar_init(a_free_bar, 1);
         for (int b = 0; b < 2; ++b) { ptx::mbar_init(acc_full_bar(b), 1); ptx::mbar_init(acc_empty_bar(b), XF ? kEpiWarpsXf : kEpiWarps); }
         ptx::mbar_init(meta_bar, 4);
         ptx::mbar_init(drained_bar, 1);
@@ -153,7 +165,7 @@ nm_gemm_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant
                     const uint32_t a_dst = ptx::smem_u32(smem + s * Cfg::STAGE);
                     ptx::mbar_expect_tx(full_bar(s), XF ? Cfg::B_BYTES : Cfg::STAGE);
                     if (!XF) ptx::tma_load_2d(a_dst, &tmap_w, kb * Cfg::A_ROW, n0, full_bar(s));
-                    ptx::tma_load_2d(a_dst + Cfg::A_BYTES, &tmap_x, kb * 128, t0, full_bar(s));
+                    ptx::tma_load_2d(a_dst + Cfg::B_OFF, &tmap_x, kb * 128, t0, full_bar(s));
                 }
             }
             if (!ok) {
@@ -169,11 +181,42 @@ nm_gemm_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant
         // (unpack, table lookups, byte permutes, stores, fence), so several groups of four warps
         // take the k-blocks round-robin: group g builds pipeline steps g, g + G, g + 2G, ...
         constexpr int G = kBuildGroups;
-        static_assert(S > G, "every group needs a stage of its own in flight");
+        static_assert(RES || S > G, "every group needs a stage of its own in flight");
         const int bw = warp - (kGateWarp + 1), grp = bw >> 2;
         const int tr = (bw & 3) * 32 + lane;  // row of the 128-row weight tile
         const int cb = xf::code_bytes(p.pat), mb = xf::meta_bytes(p.pat);
         const uint8_t* meta8 = reinterpret_cast<const uint8_t*>(p.meta);
+        if constexpr (RES) {
+            // Short reductions: the whole-K weight tile of an output tile is built once and stays in
+            // shared memory for all token tiles of that output tile; the ring then carries X only.
+            int prev_out_tile = -1;
+            uint32_t free_parity = 1u;  // nothing reads the region before the first build
+            for (int i = 0; i < tile_count; ++i) {
+                const int out_tile = (tile_begin + i) / p.n_tok_tiles;
+                if (out_tile == prev_out_tile) continue;
+                prev_out_tile = out_tile;
+                const int n = out_tile * kBM + tr;
+                const bool row_ok = n < p.out;
+                const uint8_t* v = p.values + (size_t)(row_ok ? n : 0) * p.vrow_bytes;
+                const uint8_t* m = meta8 + (size_t)(row_ok ? n : 0) * p.mrow_bytes;
+                xf::Raw cur = xf::load_raw(p.pat, v + (size_t)grp * cb, m + (size_t)grp * mb, row_ok && grp < p.kblocks);
+                // the MMAs of the previous output tile have finished reading the region
+                bool got = lane != 0 || ptx::mbar_wait_bounded(a_free_bar, free_parity, abort_flag, kWaitLimit);
+                free_parity ^= 1u;
+                if (!__all_sync(0xffffffffu, got)) { if (lane == 0) raise_timeout(); break; }
+                for (int kb = grp; kb < p.kblocks; kb += G) {
+                    const int nkb = kb + G;
+                    xf::Raw nxt = xf::load_raw(p.pat, v + (size_t)nkb * cb, m + (size_t)nkb * mb, row_ok && nkb < p.kblocks);
+                    uint32_t w[SPARSE ? 16 : 32];
+                    xf::build_row<SPARSE>(p.pat, cur, lut, w);
+                    xf::store_row<SPARSE>(a_res + kb * Cfg::A_BYTES, tr, w);
+                    cur = nxt;
+                }
+                ptx::fence_proxy_async_smem();  // the MMA reads the tile through the async proxy
+                __syncwarp();
+                if (lane == 0) ptx::mbar_arrive(a_full_bar);
+            }
+        } else {
         // position of a pipeline step: tile index i within this CTA's range, k-block kb; row pointers follow i
         struct Pos { int i, kb; const uint8_t* v; const uint8_t* m; bool ok; };
         auto locate = [&](Pos& q) {  // row pointers and validity for tile q.i
@@ -215,11 +258,12 @@ nm_gemm_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant
             s += G;
             if (s >= S) { s -= S; parity ^= 1u; }
         }
+        }
     } else if (warp == kGateWarp) {
         // ------------------------------ gate: mbarrier waits relayed to the MMA warp ------------
         // Runs its full trip count even after a timeout (then without waiting), so that the MMA
         // warp, which blocks on the named barriers, always gets its arrivals.
-        uint32_t it = 0, meta_phase = 0;
+        uint32_t it = 0, meta_phase = 0, a_phase = 0;
         int prev_out_tile = -1;
         bool ok = true;
         auto wait = [&](uint32_t bar, uint32_t parity) {
@@ -230,9 +274,9 @@ nm_gemm_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant
         };
         for (int i = 0; i < tile_count; ++i) {
             const int tile = tile_begin + i, out_tile = tile / p.n_tok_tiles, buf = i & 1;
-            if (SPARSE && out_tile != prev_out_tile) {
-                wait(meta_bar, meta_phase);
-                meta_phase ^= 1u;
+            if (out_tile != prev_out_tile) {
+                if (SPARSE) { wait(meta_bar, meta_phase); meta_phase ^= 1u; }
+                if (RES) { wait(a_full_bar, a_phase); a_phase ^= 1u; }
                 prev_out_tile = out_tile;
             }
             wait(acc_empty_bar(buf), ((i >> 1) & 1u) ^ 1u);
@@ -249,6 +293,7 @@ nm_gemm_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant
         for (int i = 0; i < tile_count; ++i) {
             const int buf = i & 1;
             const uint32_t d_tmem = tmem_base + buf * BN;
+            const bool last_of_out_tile = RES && (tile_begin + i + 1) / p.n_tok_tiles != (tile_begin + i) / p.n_tok_tiles;
             for (int kb = 0; kb < p.kblocks; ++kb, ++it) {
                 const int s = it % S;
                 ptx::named_bar_sync(1 + (it & 7u), 64);  // stage s holds k-block kb (and, for kb = 0, the
@@ -258,7 +303,8 @@ nm_gemm_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant
                 // pipe (measured ~585 clk per stage); the staged operands are ordered by the mbarrier.
                 if (kb == 0) ptx::tc_fence_after();
                 if (lane == 0) {
-                    const uint32_t a_addr = ptx::smem_u32(smem + s * Cfg::STAGE), b_addr = a_addr + Cfg::A_BYTES;
+                    const uint32_t st_addr = ptx::smem_u32(smem + s * Cfg::STAGE), b_addr = st_addr + Cfg::B_OFF;
+                    const uint32_t a_addr = RES ? ptx::smem_u32(a_res + kb * Cfg::A_BYTES) : st_addr;
                     if constexpr (SPARSE) {
 #pragma unroll
                         for (int j = 0; j < 2; ++j)  // 64 logical k each: 32 stored bytes of A, 64 of B
@@ -272,7 +318,10 @@ nm_gemm_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant
                                         ptx::smem_desc_kmajor(b_addr + 32 * j, 128, ptx::kSwizzle128), idesc, (kb | j) != 0);
                     }
                     ptx::tc_commit(empty_bar(s));  // stage reusable once these MMAs have read it
-                    if (kb == p.kblocks - 1) ptx::tc_commit(acc_full_bar(buf));
+                    if (kb == p.kblocks - 1) {
+                        ptx::tc_commit(acc_full_bar(buf));
+                        if (RES && last_of_out_tile) ptx::tc_commit(a_free_bar);  // the builders may overwrite the weight tile
+                    }
                 }
                 __syncwarp();
             }
@@ -763,9 +812,10 @@ struct LinearArgs {
     float* Y; int32_t* ACC; float* absmax; uint32_t* status; cudaStream_t stream;
 };
 
-template <bool SPARSE, int BN, int EPI, bool XF>
+template <bool SPARSE, int BN, int EPI, int WSRC>
 static int launch_gemm(const LinearArgs& a) {
-    using Cfg = GemmCfg<SPARSE, BN>;
+    constexpr bool XF = WSRC != W_TMA;
+    using Cfg = GemmCfg<SPARSE, BN, WSRC == W_RESIDENT>;
     const nm_packed_t& W = *a.W;
     CUtensorMap tw, tx, ty;
     // transform modes build the weight tile in shared memory and never use this map: describe X instead
@@ -795,7 +845,7 @@ static int launch_gemm(const LinearArgs& a) {
     p.pat = xf::pattern_of(W.n, W.m, W.bits);
     p.sw = a.sw; p.bias = a.bias; p.sx_dev = a.sx_dev; p.sx_host = a.sx;
     p.Y = a.Y; p.ACC = a.ACC; p.absmax = a.absmax; p.status = a.status;
-    auto fn = nm_gemm_kernel<SPARSE, BN, EPI, XF>;
+    auto fn = nm_gemm_kernel<SPARSE, BN, EPI, WSRC>;
     NM_CUDA_TRY(cudaFuncSetAttribute((const void*)fn, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::SMEM));
     const int grid = p.n_tiles < sm_count() ? p.n_tiles : sm_count();
     fn<<<grid, XF ? kXformThreads : kGemmThreads, Cfg::SMEM, a.stream>>>(tw, tx, ty, p);
@@ -857,10 +907,17 @@ static int pick_bn(const LinearArgs& a) {
     const int out_tiles = (a.W->out + kBM - 1) / kBM, sms = sm_count();
     if constexpr (!XF) {
         const bool fits192 = !SPARSE || a.W->in / 32 <= GemmCfg<SPARSE, 192>::META_COLS;
-        if (fits192 && (long long)out_tiles * ((a.tokens + 191) / 192) >= sms) return launch_gemm<SPARSE, 192, EPI, XF>(a);
+        if (fits192 && (long long)out_tiles * ((a.tokens + 191) / 192) >= sms) return launch_gemm<SPARSE, 192, EPI, W_TMA>(a);
+        if ((long long)out_tiles * ((a.tokens + 127) / 128) >= sms) return launch_gemm<SPARSE, 128, EPI, W_TMA>(a);
+        return launch_gemm<SPARSE, 64, EPI, W_TMA>(a);
+    } else {
+        // Short reductions with many token tiles per output tile: build each weight tile once and keep it.
+        constexpr int BNR = SPARSE ? 192 : 128;
+        if (a.W->in / kKB <= kResidentKB && (long long)out_tiles * ((a.tokens + BNR - 1) / BNR) >= sms && !getenv("NM_NO_RESIDENT"))
+            return launch_gemm<SPARSE, BNR, EPI, W_RESIDENT>(a);
+        if ((long long)out_tiles * ((a.tokens + 127) / 128) >= sms) return launch_gemm<SPARSE, 128, EPI, W_BUILD>(a);
+        return launch_gemm<SPARSE, 64, EPI, W_BUILD>(a);
     }
-    if ((long long)out_tiles * ((a.tokens + 127) / 128) >= sms) return launch_gemm<SPARSE, 128, EPI, XF>(a);
-    return launch_gemm<SPARSE, 64, EPI, XF>(a);
 }
 
 static int check_linear(int tokens, int out, int in, int n, int m, int bits) {

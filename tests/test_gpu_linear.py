@@ -75,6 +75,15 @@ def test_many_tiles_per_cta(n, m, bits):
 
 
 @pytest.mark.parametrize("n,m,bits", ALL_MODES)
+@pytest.mark.parametrize("T,K,out", [(8192 + 5, 1024, 1100), (6000, 384, 640), (6000, 128, 700)])
+def test_short_reduction_many_token_tiles(n, m, bits, T, K, out):
+    # reduction of at most eight k-blocks and several token tiles per CTA: in the transform modes the
+    # weight tile is built once per output tile, kept in shared memory and rebuilt when a CTA moves on
+    # to the next output tile (8, 3 and 1 k-blocks: more than, as many as, fewer than the builder groups)
+    _run(8, T, K, out, n, m, bits)
+
+
+@pytest.mark.parametrize("n,m,bits", ALL_MODES)
 def test_tie_heavy_weights_and_extreme_activations(n, m, bits):
     from gpu_util import PackedOnDevice, gpu_int_linear
     _run(7, 150, 256, 128, n, m, bits, tie=True)
