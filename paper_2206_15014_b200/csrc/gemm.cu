@@ -915,6 +915,10 @@ static int pick_bn(const LinearArgs& a) {
         constexpr int BNR = SPARSE ? 192 : 128;
         if (a.W->in / kKB <= kResidentKB && (long long)out_tiles * ((a.tokens + BNR - 1) / BNR) >= sms && !getenv("NM_NO_RESIDENT"))
             return launch_gemm<SPARSE, BNR, EPI, W_RESIDENT>(a);
+        if constexpr (SPARSE) {  // wider token tiles: each built weight tile serves more columns
+            if (a.W->in / 32 <= GemmCfg<SPARSE, 192>::META_COLS && (long long)out_tiles * ((a.tokens + 191) / 192) >= sms)
+                return launch_gemm<SPARSE, 192, EPI, W_BUILD>(a);
+        }
         if ((long long)out_tiles * ((a.tokens + 127) / 128) >= sms) return launch_gemm<SPARSE, 128, EPI, W_BUILD>(a);
         return launch_gemm<SPARSE, 64, EPI, W_BUILD>(a);
     }

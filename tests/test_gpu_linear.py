@@ -84,6 +84,13 @@ def test_short_reduction_many_token_tiles(n, m, bits, T, K, out):
 
 
 @pytest.mark.parametrize("n,m,bits", ALL_MODES)
+def test_longer_reduction_many_token_tiles(n, m, bits):
+    # sixteen k-blocks: the transform modes build the weight tile of every k-block into the stage ring
+    # (192-token tiles for the sparse targets), with a ragged last output tile and token tile
+    _run(9, 6000 + 3, 2048, 600, n, m, bits)
+
+
+@pytest.mark.parametrize("n,m,bits", ALL_MODES)
 def test_tie_heavy_weights_and_extreme_activations(n, m, bits):
     from gpu_util import PackedOnDevice, gpu_int_linear
     _run(7, 150, 256, 128, n, m, bits, tie=True)
