@@ -407,22 +407,22 @@ nm_gemm_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant
                     ptx::tmem_ld_wait();
                     if (c + EWH >= nact) release_acc(buf);
                     else if (RB == 2) ptx::tmem_ld_32x32(lane_taddr + buf * BN + (c + EWH) * 32, r[(ci + 1) & (RB - 1)]);
-                    // direct-store fallback (output rows not 16-byte aligned): lane = channel, j = token
-                    uint32_t* dst = reinterpret_cast<uint32_t*>(EPI == EPI_F32 ? (void*)p.Y : (void*)p.ACC) + (size_t)tc0 * p.out + n;
-#pragma unroll
-                    for (int j = 0; j < 32; ++j) {
-                        uint32_t o;
+                    // conversion of accumulator column j of this chunk; jmax = outputs of this lane that exist
+                    const int jmax = n_ok ? min(32, p.tokens - tc0) : 0;
+                    auto conv = [&](int j) -> uint32_t {
                         if constexpr (EPI == EPI_F32) {
                             const float y = __fmaf_rn((float)(int)r[ci & (RB - 1)][j], c_n, b_n);
-                            if (n_ok && tc0 + j < p.tokens) amax = fmaxf(amax, fabsf(y));
-                            o = __float_as_uint(y);
+                            amax = fmaxf(amax, j < jmax ? fabsf(y) : 0.0f);
+                            return __float_as_uint(y);
                         } else {
-                            o = r[ci & (RB - 1)][j];
+                            return r[ci & (RB - 1)][j];
                         }
-                        if (p.tma_store) sb[j * 32 + lane] = __uint_as_float(o);
-                        else if (n_ok && tc0 + j < p.tokens) __stcs(dst + (size_t)j * p.out, o);
-                    }
+                    };
+                    // The two store paths are separate loops: a branch inside the unrolled loop costs a
+                    // pipeline refill per column (measured ~30 clk each), far more than its arithmetic.
                     if (p.tma_store) {
+#pragma unroll
+                        for (int j = 0; j < 32; ++j) sb[j * 32 + lane] = __uint_as_float(conv(j));
                         ptx::fence_proxy_async_smem();
                         __syncwarp();
                         if (lane == 0) {
@@ -430,6 +430,13 @@ nm_gemm_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant
                             ptx::bulk_commit_group();
                         }
                         ++n_stores;
+                    } else {  // output rows not 16-byte aligned: lane = channel, j = token
+                        uint32_t* dst = reinterpret_cast<uint32_t*>(EPI == EPI_F32 ? (void*)p.Y : (void*)p.ACC) + (size_t)tc0 * p.out + n;
+#pragma unroll
+                        for (int j = 0; j < 32; ++j) {
+                            const uint32_t o = conv(j);
+                            if (j < jmax) __stcs(dst + (size_t)j * p.out, o);
+                        }
                     }
                 }
             }
@@ -693,30 +700,32 @@ nm_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_con
                     ptx::tmem_ld_wait();
                     if (c + EWH < nact) ptx::tmem_ld_32x32(lane_taddr + buf * BN + (c + EWH) * 32, r[(ci + 1) & 1]);
                     else release_acc(buf);
-                    uint32_t o[32];
-#pragma unroll
-                    for (int j = 0; j < 32; ++j) {
+                    const int jmax = n_ok ? min(32, p.tokens - tc0) : 0;  // outputs of this lane that exist
+                    auto conv = [&](int j) -> uint32_t {
                         if constexpr (EPI == EPI_F32) {
                             const float y = __fmaf_rn((float)(int)r[ci & 1][j], c_n, b_n);
-                            if (n_ok && tc0 + j < p.tokens) amax = fmaxf(amax, fabsf(y));
-                            o[j] = __float_as_uint(y);
+                            amax = fmaxf(amax, j < jmax ? fabsf(y) : 0.0f);
+                            return __float_as_uint(y);
                         } else {
-                            o[j] = r[ci & 1][j];
+                            return r[ci & 1][j];
                         }
-                        if (p.tma_store) my_stage[j * 32 + lane] = __uint_as_float(o[j]);
-                    }
-                    if (p.tma_store) {
+                    };
+                    if (p.tma_store) {  // separate branch-free loops for the two store paths
+#pragma unroll
+                        for (int j = 0; j < 32; ++j) my_stage[j * 32 + lane] = __uint_as_float(conv(j));
                         ptx::fence_proxy_async_smem();
                         __syncwarp();
                         if (lane == 0) {
                             ptx::tma_store_2d(&tmap_y, n0 + q * 32, tc0, ptx::smem_u32(my_stage));
                             ptx::bulk_commit_group();
                         }
-                    } else if (n_ok) {
+                    } else {
                         uint32_t* dst = reinterpret_cast<uint32_t*>(EPI == EPI_F32 ? (void*)p.Y : (void*)p.ACC) + (size_t)tc0 * p.out + n;
 #pragma unroll
-                        for (int j = 0; j < 32; ++j)
-                            if (tc0 + j < p.tokens) __stcs(dst + (size_t)j * p.out, o[j]);
+                        for (int j = 0; j < 32; ++j) {
+                            const uint32_t o = conv(j);
+                            if (j < jmax) __stcs(dst + (size_t)j * p.out, o);
+                        }
                     }
                 }
             }
