@@ -472,7 +472,9 @@ nm_gemm_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant
 constexpr int kPairThreads = 32 * (3 + kEpiWarps);
 constexpr int kPairMaxStages = 9;   // the relay cycles through 15 named barriers
 
-template <bool SPARSE, int BN>
+constexpr int kPairResStages = 4;   // stages of weights a CTA can keep resident (1024 reduction elements at 2:4)
+
+template <bool SPARSE, int BN, bool RES = false>
 struct PairCfg {
     // A stage holds 128 stored bytes of every weight row (256 reduction elements when 2:4 compressed,
     // 128 when dense) and the matching 128-byte-wide slices of X: one TMA operation each, four MMAs.
@@ -482,26 +484,32 @@ struct PairCfg {
     static constexpr int B_ROWS = BN / 2;            // tokens staged by each CTA
     static constexpr int B_SUB = B_ROWS * 128;       // one 128-byte-wide slice of the X half tile
     static constexpr int B_BYTES = B_SUB * (KB / 128);
-    static constexpr int STAGE = A_BYTES + B_BYTES;
-    static constexpr int FIT = (kSmemLimit - kSmemTail - kStoreStage - 1024) / STAGE;
+    // RES: the whole-K weight rows of the CTA stay in shared memory across the token tiles of an
+    // output tile; the ring then carries X only and holds more of it.
+    static constexpr int A_RES = RES ? kPairResStages * A_BYTES : 0;
+    static constexpr int B_OFF = RES ? 0 : A_BYTES;
+    static constexpr int STAGE = B_OFF + B_BYTES;
+    static constexpr int FIT = (kSmemLimit - kSmemTail - kStoreStage - 1024 - A_RES) / STAGE;
     static constexpr int STAGES = FIT < kPairMaxStages ? FIT : kPairMaxStages;
-    static constexpr int SMEM = STAGES * STAGE + kStoreStage + kSmemTail + 1024;
+    static constexpr int SMEM = STAGES * STAGE + A_RES + kStoreStage + kSmemTail + 1024;
+    static_assert(STAGES >= 3, "pipeline too shallow");
     static constexpr int META_COL = 2 * BN;
     static constexpr int META_COLS = kTmemCols - 2 * BN;
     static_assert(B_SUB % 1024 == 0, "X half tile must keep the swizzle alignment");
     static_assert(BN % 32 == 0 && BN <= 256, "token tile");
 };
 
-template <bool SPARSE, int BN, int EPI>
+template <bool SPARSE, int BN, int EPI, bool RES>
 __global__ void __launch_bounds__(kPairThreads, 1)
 nm_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant__ CUtensorMap tmap_x,
                     const __grid_constant__ CUtensorMap tmap_y, const GemmParams p) {
-    using Cfg = PairCfg<SPARSE, BN>;
+    using Cfg = PairCfg<SPARSE, BN, RES>;
     constexpr int S = Cfg::STAGES;
     constexpr int EW = kEpiWarps, kGateWarp = 2 + EW;
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
-    uint8_t* store_stage = smem + S * Cfg::STAGE;
+    uint8_t* a_res = smem + S * Cfg::STAGE;  // resident weight rows: kPairResStages stages of A_BYTES
+    uint8_t* store_stage = a_res + Cfg::A_RES;
     uint64_t* bars = reinterpret_cast<uint64_t*>(store_stage + kStoreStage);
     const uint32_t bar0 = ptx::smem_u32(bars);
     auto full_bar = [&](int s) { return bar0 + 8u * s; };              // used in the leader
@@ -510,7 +518,9 @@ nm_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_con
     auto acc_empty_bar = [&](int b) { return bar0 + 8u * (2 * S + 2 + b); };  // leader; arrivals from both
     const uint32_t meta_bar = bar0 + 8u * (2 * S + 4);                 // leader; arrivals from both
     const uint32_t drained_bar = bar0 + 8u * (2 * S + 5);
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * S + 6);
+    const uint32_t a_full_bar = bar0 + 8u * (2 * S + 6);               // leader: resident weights of both CTAs landed
+    const uint32_t a_free_bar = bar0 + 8u * (2 * S + 7);               // both CTAs (multicast commit): no MMA reads them any more
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * S + 8);
     volatile uint32_t* abort_flag = tmem_slot + 1;
     volatile uint32_t* never_flag = tmem_slot + 2;
 
@@ -527,6 +537,8 @@ nm_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_con
         for (int b = 0; b < 2; ++b) { ptx::mbar_init(acc_full_bar(b), 1); ptx::mbar_init(acc_empty_bar(b), 2 * EW); }
         ptx::mbar_init(meta_bar, 8);
         ptx::mbar_init(drained_bar, 1);
+        ptx::mbar_init(a_full_bar, 1);
+        ptx::mbar_init(a_free_bar, 1);
         *abort_flag = 0;
         *never_flag = 0;
         ptx::fence_mbar_init();
@@ -554,12 +566,25 @@ nm_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_con
     if (warp == 0) {
         // ------------------------------ TMA producer (both CTAs) --------------------------------
         if (lane == 0) {
-            uint32_t it = 0;
+            uint32_t it = 0, free_parity = 1u;  // nothing reads the resident region before the first load
+            int prev_out_tile = -1;
             bool ok = true;
             for (int i = 0; i < tile_count && ok; ++i) {
                 const int tile = tile_begin + i;
                 const int n0 = (tile / p.n_tok_tiles) * (2 * kBM) + (int)rank * kBM;
                 const int t0 = (tile % p.n_tok_tiles) * BN + (int)rank * Cfg::B_ROWS;
+                if (RES && tile / p.n_tok_tiles != prev_out_tile) {
+                    // new output tile: once the MMAs of the previous one are done, fetch this CTA's weight rows for the whole reduction
+                    prev_out_tile = tile / p.n_tok_tiles;
+                    if (!ptx::mbar_wait_bounded(a_free_bar, free_parity, abort_flag, kWaitLimit)) {
+                        raise_timeout(); ok = false; break;
+                    }
+                    free_parity ^= 1u;
+                    const uint32_t lead_a_full = ptx::map_to_cta(a_full_bar, 0);
+                    if (leader) ptx::mbar_expect_tx(a_full_bar, 2 * p.kblocks * Cfg::A_BYTES);  // bytes of both CTAs
+                    for (int kb = 0; kb < p.kblocks; ++kb)
+                        ptx::tma_load_2d_pair(ptx::smem_u32(a_res + kb * Cfg::A_BYTES), &tmap_w, kb * Cfg::A_ROW, n0, lead_a_full);
+                }
                 for (int kb = 0; kb < p.kblocks; ++kb, ++it) {
                     const int s = it % S;
                     if (!ptx::mbar_wait_bounded(empty_bar(s), ((it / S) & 1u) ^ 1u, abort_flag, kWaitLimit)) {
@@ -568,16 +593,16 @@ nm_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_con
                     const uint32_t a_dst = ptx::smem_u32(smem + s * Cfg::STAGE);
                     const uint32_t lead_full = ptx::map_to_cta(full_bar(s), 0);
                     if (leader) ptx::mbar_expect_tx(full_bar(s), 2 * Cfg::STAGE);  // bytes of both CTAs
-                    ptx::tma_load_2d_pair(a_dst, &tmap_w, kb * Cfg::A_ROW, n0, lead_full);
+                    if (!RES) ptx::tma_load_2d_pair(a_dst, &tmap_w, kb * Cfg::A_ROW, n0, lead_full);
                     // X is mapped as [k-slice][token][128 bytes]: both slices of the stage in one operation
-                    ptx::tma_load_3d_pair(a_dst + Cfg::A_BYTES, &tmap_x, 0, t0, kb * (Cfg::KB / 128), lead_full);
+                    ptx::tma_load_3d_pair(a_dst + Cfg::B_OFF, &tmap_x, 0, t0, kb * (Cfg::KB / 128), lead_full);
                 }
             }
         }
     } else if (warp == kGateWarp) {
         // ------------------------------ gate (leader): mbarrier waits relayed to the MMA warp ------
         if (leader) {
-            uint32_t it = 0, meta_phase = 0;
+            uint32_t it = 0, meta_phase = 0, a_phase = 0;
             int prev_out_tile = -1;
             bool ok = true;
             auto wait = [&](uint32_t bar, uint32_t parity) {
@@ -588,9 +613,9 @@ nm_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_con
             };
             for (int i = 0; i < tile_count; ++i) {
                 const int tile = tile_begin + i, out_tile = tile / p.n_tok_tiles, buf = i & 1;
-                if (SPARSE && out_tile != prev_out_tile) {
-                    wait(meta_bar, meta_phase);
-                    meta_phase ^= 1u;
+                if (out_tile != prev_out_tile) {
+                    if (SPARSE) { wait(meta_bar, meta_phase); meta_phase ^= 1u; }
+                    if (RES) { wait(a_full_bar, a_phase); a_phase ^= 1u; }
                     prev_out_tile = out_tile;
                 }
                 wait(acc_empty_bar(buf), ((i >> 1) & 1u) ^ 1u);
@@ -609,12 +634,14 @@ nm_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_con
             for (int i = 0; i < tile_count; ++i) {
                 const int buf = i & 1;
                 const uint32_t d_tmem = tmem_base + buf * BN;
+                const bool last_of_out_tile = RES && (tile_begin + i + 1) / p.n_tok_tiles != (tile_begin + i) / p.n_tok_tiles;
                 for (int kb = 0; kb < p.kblocks; ++kb, ++it) {
                     const int s = it % S;
                     ptx::named_bar_sync(1 + (it % 15u), 64);
                     if (kb == 0) ptx::tc_fence_after();  // once per tile (see the one-CTA kernel)
                     if (lane == 0) {
-                        const uint32_t a_addr = ptx::smem_u32(smem + s * Cfg::STAGE), b_addr = a_addr + Cfg::A_BYTES;
+                        const uint32_t st_addr = ptx::smem_u32(smem + s * Cfg::STAGE), b_addr = st_addr + Cfg::B_OFF;
+                        const uint32_t a_addr = RES ? ptx::smem_u32(a_res + kb * Cfg::A_BYTES) : st_addr;
                         if constexpr (SPARSE) {
 #pragma unroll
                             for (int j = 0; j < 4; ++j)  // 64 reduction elements each: 32 stored bytes of A, 64 of X
@@ -628,7 +655,10 @@ nm_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_con
                                                  ptx::smem_desc_kmajor(b_addr + 32 * j, 128, ptx::kSwizzle128), idesc, (kb | j) != 0);
                         }
                         ptx::tc_commit_pair(empty_bar(s), 3);   // both producers may refill the stage
-                        if (kb == p.kblocks - 1) ptx::tc_commit_pair(acc_full_bar(buf), 3);
+                        if (kb == p.kblocks - 1) {
+                            ptx::tc_commit_pair(acc_full_bar(buf), 3);
+                            if (last_of_out_tile) ptx::tc_commit_pair(a_free_bar, 3);  // both producers may replace the weights
+                        }
                     }
                     __syncwarp();
                 }
@@ -862,9 +892,9 @@ static int launch_gemm(const LinearArgs& a) {
     return NM_OK;
 }
 
-template <bool SPARSE, int BN, int EPI>
+template <bool SPARSE, int BN, int EPI, bool RES>
 static int launch_gemm_pair(const LinearArgs& a) {
-    using Cfg = PairCfg<SPARSE, BN>;
+    using Cfg = PairCfg<SPARSE, BN, RES>;
     const nm_packed_t& W = *a.W;
     CUtensorMap tw, tx, ty;
     int rc = make_map(&tw, W.values, (uint64_t)W.out, (uint64_t)(SPARSE ? W.in / 2 : W.in), kBM, Cfg::A_ROW,
@@ -886,7 +916,7 @@ static int launch_gemm_pair(const LinearArgs& a) {
     p.meta = (const uint32_t*)W.meta; p.mrow_words = W.in / 32;
     p.sw = a.sw; p.bias = a.bias; p.sx_dev = a.sx_dev; p.sx_host = a.sx;
     p.Y = a.Y; p.ACC = a.ACC; p.absmax = a.absmax; p.status = a.status;
-    auto fn = nm_gemm_pair_kernel<SPARSE, BN, EPI>;
+    auto fn = nm_gemm_pair_kernel<SPARSE, BN, EPI, RES>;
     NM_CUDA_TRY(cudaFuncSetAttribute((const void*)fn, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::SMEM));
     const int pairs = p.n_tiles < sm_count() / 2 ? p.n_tiles : sm_count() / 2;
     cudaLaunchConfig_t cfg = {};
@@ -909,6 +939,16 @@ static bool use_pair(const LinearArgs& a) {
     const long long tiles = (long long)((a.W->out + 2 * kBM - 1) / (2 * kBM)) * ((a.tokens + 191) / 192);
     const bool fits = !SPARSE || a.W->in / 32 <= PairCfg<SPARSE, 192>::META_COLS;
     return fits && tiles >= sm_count() / 2;
+}
+
+// Pair kernel with the weights streamed through the ring, or (2:4, reduction up to 1024) kept resident.
+template <bool SPARSE, int EPI>
+static int pick_pair(const LinearArgs& a) {
+    if constexpr (SPARSE) {
+        if (a.W->in <= kPairResStages * PairCfg<true, 192>::KB && !getenv("NM_NO_RESIDENT"))
+            return launch_gemm_pair<true, 192, EPI, true>(a);
+    }
+    return launch_gemm_pair<SPARSE, 192, EPI, false>(a);
 }
 
 template <bool SPARSE, int EPI, bool XF>
@@ -961,11 +1001,11 @@ static int run_linear(const LinearArgs& a, int epi) {
         return epi == EPI_F32 ? pick_bn<false, EPI_F32, true>(a) : pick_bn<false, EPI_ACC, true>(a);
     }
     if (sparse) {
-        if (epi == EPI_F32) return use_pair<true, EPI_F32>(a) ? launch_gemm_pair<true, 192, EPI_F32>(a) : pick_bn<true, EPI_F32, false>(a);
-        return use_pair<true, EPI_ACC>(a) ? launch_gemm_pair<true, 192, EPI_ACC>(a) : pick_bn<true, EPI_ACC, false>(a);
+        if (epi == EPI_F32) return use_pair<true, EPI_F32>(a) ? pick_pair<true, EPI_F32>(a) : pick_bn<true, EPI_F32, false>(a);
+        return use_pair<true, EPI_ACC>(a) ? pick_pair<true, EPI_ACC>(a) : pick_bn<true, EPI_ACC, false>(a);
     }
-    if (epi == EPI_F32) return use_pair<false, EPI_F32>(a) ? launch_gemm_pair<false, 192, EPI_F32>(a) : pick_bn<false, EPI_F32, false>(a);
-    return use_pair<false, EPI_ACC>(a) ? launch_gemm_pair<false, 192, EPI_ACC>(a) : pick_bn<false, EPI_ACC, false>(a);
+    if (epi == EPI_F32) return use_pair<false, EPI_F32>(a) ? pick_pair<false, EPI_F32>(a) : pick_bn<false, EPI_F32, false>(a);
+    return use_pair<false, EPI_ACC>(a) ? pick_pair<false, EPI_ACC>(a) : pick_bn<false, EPI_ACC, false>(a);
 }
 
 }  // namespace nm
