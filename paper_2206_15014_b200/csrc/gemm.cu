@@ -41,7 +41,7 @@ constexpr int kXformThreads = 32 * (3 + kEpiWarpsXf + 4 * kBuildGroups); // ... 
 constexpr int kTmemCols = 512;
 constexpr int kSmemLimit = 232448;  // 227 KB of dynamic shared memory per CTA
 constexpr int kSmemTail = 2048;     // barriers, TMEM slot, abort flag, slot tables
-constexpr int kStoreStage = 8 * 4096;  // [32 tokens][32 channels] fp32 staging tiles: two per warp (4 warps) or one (8 warps)
+constexpr int kStoreStage = 8 * 4096;  // per epilogue warp two [16 tokens][32 channels] fp32 staging tiles, used alternately
 constexpr int kMaxStages = 7;       // the relay cycles through 8 named barriers
 constexpr long long kWaitLimit = 1ll << 31;  // SM clocks (about a second)
 
@@ -335,14 +335,14 @@ nm_gemm_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant
         // Warp w may touch TMEM lanes 32 * (w % 4) ... + 31.  With eight warps two share a lane quarter
         // and take alternate 32-column chunks of the accumulator.
         constexpr int EWH = EW / 4;               // warps per lane quarter
-        constexpr int NBUF = 8 / EW;              // staging tiles per warp
         constexpr int CH = BN / 32;               // chunks per accumulator
         constexpr int CI = (CH + EWH - 1) / EWH;  // chunks per warp
         const int ew = warp - 2, q = warp & 3, half = ew >> 2, row = q * 32 + lane;
         const uint32_t lane_taddr = tmem_base + ((uint32_t)(q * 32) << 16);
-        float* my_stage = reinterpret_cast<float*>(store_stage + ew * (NBUF * 4096));
+        float* my_stage = reinterpret_cast<float*>(store_stage + ew * 4096);
         const float sx = p.sx_dev ? *p.sx_dev : p.sx_host;
-        float amax = 0.0f;
+        float amax = 0.0f, c_n = 0.0f, b_n = 0.0f;
+        int scaled_out_tile = -1;
         uint32_t n_stores = 0;
         bool ok = true;
 
@@ -382,10 +382,10 @@ nm_gemm_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant
                 if (next_out_tile != out_tile) load_meta(next_out_tile);  // MMAs of this output tile are done
             }
             const bool n_ok = n < p.out;
-            float c_n = 0.0f, b_n = 0.0f;
-            if (EPI == EPI_F32 && n_ok) {
-                c_n = __fmul_rn(sx, p.sw[n]);
-                b_n = p.bias ? p.bias[n] : 0.0f;
+            if (EPI == EPI_F32 && out_tile != scaled_out_tile) {  // channel constants: fetched once per output tile
+                scaled_out_tile = out_tile;
+                c_n = n_ok ? __fmul_rn(sx, p.sw[n]) : 0.0f;
+                b_n = n_ok && p.bias ? p.bias[n] : 0.0f;
             }
             const int nact = min(CH, (p.tokens - t0 + 31) >> 5);  // chunks that hold tokens (warp-uniform)
             // Accumulator chunks are read one ahead of their conversion (two register buffers); the
@@ -398,11 +398,6 @@ nm_gemm_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant
             for (int ci = 0; ci < CI; ++ci) {
                 const int c = half + ci * EWH, tc0 = t0 + c * 32;
                 if (c < nact) {
-                    float* sb = my_stage + (NBUF == 2 ? (n_stores & 1u) * 1024 : 0);
-                    if (p.tma_store) {  // the store that last used this staging tile has read it
-                        if (lane == 0) ptx::bulk_wait_group_read<NBUF - 1>();
-                        __syncwarp();
-                    }
                     if (RB == 1) ptx::tmem_ld_32x32(lane_taddr + buf * BN + c * 32, r[0]);
                     ptx::tmem_ld_wait();
                     if (c + EWH >= nact) release_acc(buf);
@@ -421,15 +416,25 @@ nm_gemm_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant
                     // The two store paths are separate loops: a branch inside the unrolled loop costs a
                     // pipeline refill per column (measured ~30 clk each), far more than its arithmetic.
                     if (p.tma_store) {
+                        // two stores of 16 tokens each, through alternating staging tiles: while one is
+                        // being read by its TMA store the other is filled
 #pragma unroll
-                        for (int j = 0; j < 32; ++j) sb[j * 32 + lane] = __uint_as_float(conv(j));
-                        ptx::fence_proxy_async_smem();
-                        __syncwarp();
-                        if (lane == 0) {
-                            ptx::tma_store_2d(&tmap_y, n0 + q * 32, tc0, ptx::smem_u32(sb));
-                            ptx::bulk_commit_group();
+                        for (int h = 0; h < 2; ++h) {
+                            if (tc0 + 16 * h < p.tokens) {  // warp-uniform
+                                float* sb = my_stage + (n_stores & 1u) * 512;
+                                if (lane == 0) ptx::bulk_wait_group_read<1>();  // the store before the last has read this tile
+                                __syncwarp();
+#pragma unroll
+                                for (int j = 0; j < 16; ++j) sb[j * 32 + lane] = __uint_as_float(conv(16 * h + j));
+                                ptx::fence_proxy_async_smem();
+                                __syncwarp();
+                                if (lane == 0) {
+                                    ptx::tma_store_2d(&tmap_y, n0 + q * 32, tc0 + 16 * h, ptx::smem_u32(sb));
+                                    ptx::bulk_commit_group();
+                                }
+                                ++n_stores;
+                            }
                         }
-                        ++n_stores;
                     } else {  // output rows not 16-byte aligned: lane = channel, j = token
                         uint32_t* dst = reinterpret_cast<uint32_t*>(EPI == EPI_F32 ? (void*)p.Y : (void*)p.ACC) + (size_t)tc0 * p.out + n;
 #pragma unroll
@@ -676,7 +681,9 @@ nm_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_con
         float* my_stage = reinterpret_cast<float*>(store_stage + ew * 4096);
         const float sx = p.sx_dev ? *p.sx_dev : p.sx_host;
         const uint32_t lead_meta = ptx::map_to_cta(meta_bar, 0);
-        float amax = 0.0f;
+        float amax = 0.0f, c_n = 0.0f, b_n = 0.0f;
+        int scaled_out_tile = -1;
+        uint32_t n_stores = 0;
         bool ok = true;
 
         auto load_meta = [&](int out_tile) {
@@ -697,23 +704,24 @@ nm_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_con
             if (lane == 0) ptx::mbar_arrive_cluster(ptx::map_to_cta(acc_empty_bar(buf), 0));
         };
 
-        for (int i = 0; i < tile_count && ok; ++i) {
-            const int tile = tile_begin + i, out_tile = tile / p.n_tok_tiles, buf = i & 1;
-            const int n0 = out_tile * (2 * kBM) + (int)rank * kBM, n = n0 + row, t0 = (tile % p.n_tok_tiles) * BN;
+        // position of the current tile, advanced without divisions
+        int out_tile = tile_begin / p.n_tok_tiles, tok_tile = tile_begin % p.n_tok_tiles;
+        for (int i = 0; i < tile_count && ok; ++i, ++tok_tile) {
+            if (tok_tile == p.n_tok_tiles) { tok_tile = 0; ++out_tile; }
+            const int buf = i & 1;
+            const int n0 = out_tile * (2 * kBM) + (int)rank * kBM, n = n0 + row, t0 = tok_tile * BN;
             if (SPARSE && i == 0 && half == 0) load_meta(out_tile);
             bool got = ptx::mbar_wait_bounded(acc_full_bar(buf), (i >> 1) & 1u, abort_flag, kWaitLimit);
             ok = __all_sync(0xffffffffu, got);
             if (!ok) { if (lane == 0) raise_timeout(); break; }
             ptx::tc_fence_after();
-            if (SPARSE && half == 0 && i + 1 < tile_count) {
-                const int next_out_tile = (tile + 1) / p.n_tok_tiles;
-                if (next_out_tile != out_tile) load_meta(next_out_tile);
-            }
+            // the next tile starts a new output tile: its metadata can go in now, the MMAs of this one are done
+            if (SPARSE && half == 0 && i + 1 < tile_count && tok_tile + 1 == p.n_tok_tiles) load_meta(out_tile + 1);
             const bool n_ok = n < p.out;
-            float c_n = 0.0f, b_n = 0.0f;
-            if (EPI == EPI_F32 && n_ok) {
-                c_n = __fmul_rn(sx, p.sw[n]);
-                b_n = p.bias ? p.bias[n] : 0.0f;
+            if (EPI == EPI_F32 && out_tile != scaled_out_tile) {  // channel constants: fetched once per output tile
+                scaled_out_tile = out_tile;
+                c_n = n_ok ? __fmul_rn(sx, p.sw[n]) : 0.0f;
+                b_n = n_ok && p.bias ? p.bias[n] : 0.0f;
             }
             const int nact = min(CH, (p.tokens - t0 + 31) >> 5);
             uint32_t r[2][32];
@@ -723,10 +731,6 @@ nm_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_con
             for (int ci = 0; ci < CI; ++ci) {
                 const int c = half + ci * EWH, tc0 = t0 + c * 32;
                 if (c < nact) {
-                    if (p.tma_store) {
-                        if (lane == 0) ptx::bulk_wait_group_read<0>();
-                        __syncwarp();
-                    }
                     ptx::tmem_ld_wait();
                     if (c + EWH < nact) ptx::tmem_ld_32x32(lane_taddr + buf * BN + (c + EWH) * 32, r[(ci + 1) & 1]);
                     else release_acc(buf);
@@ -742,12 +746,21 @@ nm_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_con
                     };
                     if (p.tma_store) {  // separate branch-free loops for the two store paths
 #pragma unroll
-                        for (int j = 0; j < 32; ++j) my_stage[j * 32 + lane] = __uint_as_float(conv(j));
-                        ptx::fence_proxy_async_smem();
-                        __syncwarp();
-                        if (lane == 0) {
-                            ptx::tma_store_2d(&tmap_y, n0 + q * 32, tc0, ptx::smem_u32(my_stage));
-                            ptx::bulk_commit_group();
+                        for (int h = 0; h < 2; ++h) {  // 16 tokens per store, alternating staging tiles
+                            if (tc0 + 16 * h < p.tokens) {  // warp-uniform
+                                float* sb = my_stage + (n_stores & 1u) * 512;
+                                if (lane == 0) ptx::bulk_wait_group_read<1>();  // the store before the last has read this tile
+                                __syncwarp();
+#pragma unroll
+                                for (int j = 0; j < 16; ++j) sb[j * 32 + lane] = __uint_as_float(conv(16 * h + j));
+                                ptx::fence_proxy_async_smem();
+                                __syncwarp();
+                                if (lane == 0) {
+                                    ptx::tma_store_2d(&tmap_y, n0 + q * 32, tc0 + 16 * h, ptx::smem_u32(sb));
+                                    ptx::bulk_commit_group();
+                                }
+                                ++n_stores;
+                            }
                         }
                     } else {
                         uint32_t* dst = reinterpret_cast<uint32_t*>(EPI == EPI_F32 ? (void*)p.Y : (void*)p.ACC) + (size_t)tc0 * p.out + n;
@@ -868,7 +881,7 @@ static int launch_gemm(const LinearArgs& a) {
     // base and row pitch); otherwise the threads store directly.
     void* ybase = EPI == EPI_F32 ? (void*)a.Y : (void*)a.ACC;
     const bool tma_store = aligned(ybase, 16) && (W.out % 4) == 0;
-    rc = make_map(&ty, tma_store ? ybase : (const void*)a.X, (uint64_t)a.tokens, (uint64_t)(tma_store ? W.out : W.in / 4), 32, 32,
+    rc = make_map(&ty, tma_store ? ybase : (const void*)a.X, (uint64_t)a.tokens, (uint64_t)(tma_store ? W.out : W.in / 4), 16, 32,
                   CU_TENSOR_MAP_SWIZZLE_NONE, EPI == EPI_F32 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_INT32, 4);
     if (rc != NM_OK) return rc;
     GemmParams p{};
@@ -904,7 +917,7 @@ static int launch_gemm_pair(const LinearArgs& a) {
     if (rc != NM_OK) return rc;
     void* ybase = EPI == EPI_F32 ? (void*)a.Y : (void*)a.ACC;
     const bool tma_store = aligned(ybase, 16) && (W.out % 4) == 0;
-    rc = make_map(&ty, tma_store ? ybase : (const void*)a.X, (uint64_t)a.tokens, (uint64_t)(tma_store ? W.out : W.in / 4), 32, 32,
+    rc = make_map(&ty, tma_store ? ybase : (const void*)a.X, (uint64_t)a.tokens, (uint64_t)(tma_store ? W.out : W.in / 4), 16, 32,
                   CU_TENSOR_MAP_SWIZZLE_NONE, EPI == EPI_F32 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_INT32, 4);
     if (rc != NM_OK) return rc;
     GemmParams p{};
