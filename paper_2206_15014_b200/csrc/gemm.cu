@@ -494,9 +494,13 @@ struct PairCfg {
     static constexpr int A_RES = RES ? kPairResStages * A_BYTES : 0;
     static constexpr int B_OFF = RES ? 0 : A_BYTES;
     static constexpr int STAGE = B_OFF + B_BYTES;
-    static constexpr int FIT = (kSmemLimit - kSmemTail - kStoreStage - 1024 - A_RES) / STAGE;
+    // Epilogue staging: two [16 tokens][32 channels] fp32 tiles per warp where the epilogue sets the pace
+    // (short reductions, RES); one where the main loop does and a fifth stage in the ring is worth more.
+    static constexpr int STORE_BUFS = RES ? 2 : 1;
+    static constexpr int STORE_STAGE = kEpiWarps * STORE_BUFS * 2048;
+    static constexpr int FIT = (kSmemLimit - kSmemTail - STORE_STAGE - 1024 - A_RES) / STAGE;
     static constexpr int STAGES = FIT < kPairMaxStages ? FIT : kPairMaxStages;
-    static constexpr int SMEM = STAGES * STAGE + A_RES + kStoreStage + kSmemTail + 1024;
+    static constexpr int SMEM = STAGES * STAGE + A_RES + STORE_STAGE + kSmemTail + 1024;
     static_assert(STAGES >= 3, "pipeline too shallow");
     static constexpr int META_COL = 2 * BN;
     static constexpr int META_COLS = kTmemCols - 2 * BN;
@@ -515,7 +519,7 @@ nm_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_con
     uint8_t* smem = reinterpret_cast<uint8_t*>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
     uint8_t* a_res = smem + S * Cfg::STAGE;  // resident weight rows: kPairResStages stages of A_BYTES
     uint8_t* store_stage = a_res + Cfg::A_RES;
-    uint64_t* bars = reinterpret_cast<uint64_t*>(store_stage + kStoreStage);
+    uint64_t* bars = reinterpret_cast<uint64_t*>(store_stage + Cfg::STORE_STAGE);
     const uint32_t bar0 = ptx::smem_u32(bars);
     auto full_bar = [&](int s) { return bar0 + 8u * s; };              // used in the leader
     auto empty_bar = [&](int s) { return bar0 + 8u * (S + s); };       // both CTAs (multicast commit)
@@ -678,7 +682,8 @@ nm_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_con
         constexpr int EWH = EW / 4, CH = BN / 32, CI = (CH + EWH - 1) / EWH;
         const int ew = warp - 2, q = warp & 3, half = ew >> 2, row = q * 32 + lane;
         const uint32_t lane_taddr = tmem_base + ((uint32_t)(q * 32) << 16);
-        float* my_stage = reinterpret_cast<float*>(store_stage + ew * 4096);
+        constexpr int NB = Cfg::STORE_BUFS;
+        float* my_stage = reinterpret_cast<float*>(store_stage + ew * (NB * 2048));
         const float sx = p.sx_dev ? *p.sx_dev : p.sx_host;
         const uint32_t lead_meta = ptx::map_to_cta(meta_bar, 0);
         float amax = 0.0f, c_n = 0.0f, b_n = 0.0f;
@@ -748,8 +753,8 @@ nm_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_con
 #pragma unroll
                         for (int h = 0; h < 2; ++h) {  // 16 tokens per store, alternating staging tiles
                             if (tc0 + 16 * h < p.tokens) {  // warp-uniform
-                                float* sb = my_stage + (n_stores & 1u) * 512;
-                                if (lane == 0) ptx::bulk_wait_group_read<1>();  // the store before the last has read this tile
+                                float* sb = my_stage + (NB == 2 ? (n_stores & 1u) * 512 : 0);
+                                if (lane == 0) ptx::bulk_wait_group_read<NB - 1>();  // the store that last used this tile has read it
                                 __syncwarp();
 #pragma unroll
                                 for (int j = 0; j < 16; ++j) sb[j * 32 + lane] = __uint_as_float(conv(16 * h + j));
