@@ -148,5 +148,22 @@ def quantize_act(Y):
     return Xq, np.float32(sx.value)
 
 
+def requantize_static(Y, sy):
+    """Eq. 5 with b = 8 and a given scale: -> int8 like Y."""
+    Y = np.ascontiguousarray(Y, dtype=np.float32)
+    Yq = np.zeros(Y.shape, dtype=np.int8)
+    _chk(lib().oracle_requantize_static(_p(Y), ctypes.c_size_t(Y.size), ctypes.c_float(float(sy)), _p(Yq)),
+         "oracle_requantize_static")
+    return Yq
+
+
+def to_bf16(Y):
+    """fp32 -> bfloat16 bit patterns (uint16 like Y), round to nearest even."""
+    Y = np.ascontiguousarray(Y, dtype=np.float32)
+    out = np.zeros(Y.shape, dtype=np.uint16)
+    _chk(lib().oracle_to_bf16(_p(Y), ctypes.c_size_t(Y.size), _p(out)), "oracle_to_bf16")
+    return out
+
+
 def bits_per_param(n, m, bits, index_bits=-1):
     return float(lib().oracle_bits_per_param(n, m, bits, index_bits))

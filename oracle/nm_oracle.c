@@ -28,6 +28,10 @@
  *   The byte-level packing of values and metadata is this library's own
  *   convention (the paper specifies none): parity unpinned beyond the
  *   pack -> unpack round trip and the 2-index-bits-per-kept-value accounting.
+ *   Narrow forms of the layer's output -- Eq. 5 with a scale fixed ahead of
+ *   time (8-bit activations handed to the next layer, Sec. 4.5) and binary32 ->
+ *   bfloat16 rounding: pinned by closed forms (exact multiples, ties), exact
+ *   rational arithmetic, error bounds and an independent conversion routine.
  */
 #include <math.h>
 #include <stddef.h>
@@ -372,6 +376,39 @@ int oracle_quantize_act(const float *Y, size_t count, int8_t *Xq, float *sx)
     float s = a == 0.0f ? 1.0f : a / 127.0f;
     *sx = s;
     for (size_t i = 0; i < count; ++i) Xq[i] = (int8_t)quantise(Y[i], s, 8);
+    return ORACLE_OK;
+}
+
+/*
+ * Static-scale 8-bit re-quantiser: Eq. 5 with b = 8 and a scale sy fixed ahead of
+ * time instead of taken from the tensor.  It is the form in which an integer
+ * encoder hands the output of one linear layer to the next as 8-bit activations
+ * (Sec. 4.5: all activations kept at 8 bits).
+ */
+int oracle_requantize_static(const float *Y, size_t count, float sy, int8_t *Yq)
+{
+    if (!(sy > 0.0f) || !isfinite(sy)) return ORACLE_ERR_SHAPE;
+    for (size_t i = 0; i < count; ++i) {
+        if (!isfinite(Y[i])) return ORACLE_ERR_NONFINITE;
+        Yq[i] = (int8_t)quantise(Y[i], sy, 8);
+    }
+    return ORACLE_OK;
+}
+
+/*
+ * binary32 -> bfloat16 (the upper 16 bits of the binary32 pattern), rounded to
+ * nearest with ties to even, for finite inputs: the discarded 16 bits decide.
+ */
+int oracle_to_bf16(const float *Y, size_t count, uint16_t *out)
+{
+    for (size_t i = 0; i < count; ++i) {
+        if (!isfinite(Y[i])) return ORACLE_ERR_NONFINITE;
+        uint32_t u;
+        memcpy(&u, &Y[i], sizeof u);
+        uint32_t upper = u >> 16, lower = u & 0xFFFFu;
+        if (lower > 0x8000u || (lower == 0x8000u && (upper & 1u))) upper += 1u;
+        out[i] = (uint16_t)upper;
+    }
     return ORACLE_OK;
 }
 

@@ -412,3 +412,79 @@ def test_table3_ratios_are_self_consistent():
     assert round(fp16 / nm, 1) == sp[0]
     assert round(fp16 / int8, 2) == sp[1]
     assert round(int8 / nm, 2) == sp[2]
+
+
+# ---- narrow-output forms of the linear layer's result (static-scale int8, bfloat16) -------------------
+
+def test_static_requantiser_closed_forms():
+    # exact multiples of a power-of-two scale: the quotient is exact, the code is the clamped multiple
+    sy = np.float32(2.0 ** -3)
+    k = np.arange(-200, 201, dtype=np.int32)
+    q = oracle.requantize_static(k.astype(np.float32) * sy, sy)
+    assert np.array_equal(q, np.clip(k, -128, 127).astype(np.int8))
+    # exact halves go to the even neighbour (Eq. 5's round read as round-half-to-even)
+    halves = (np.arange(-130, 130, dtype=np.float32) + np.float32(0.5)) * sy
+    expect = np.array([int(np.clip(2 * round((j + 0.5) / 2), -128, 127)) for j in range(-130, 130)], dtype=np.int8)
+    assert np.array_equal(oracle.requantize_static(halves, sy), expect)
+    # a scale that is not positive and finite is rejected
+    for bad in (0.0, -1.0, float("inf"), float("nan")):
+        with pytest.raises(RuntimeError):
+            oracle.requantize_static(np.zeros(4, np.float32), bad)
+
+
+def test_static_requantiser_properties_and_exact_arithmetic():
+    rng = np.random.default_rng(11)
+    Y = wl.normal(rng, (4096,), 3.0)
+    sy = np.float32(0.0371)
+    q = oracle.requantize_static(Y, sy).astype(np.int64)
+    inside = np.abs(Y.astype(np.float64)) <= 127.0 * float(sy)
+    # within the representable range the reconstruction error is at most half a step (plus the
+    # rounding of the fp32 quotient: one part in 2^24 of |y|)
+    err = np.abs(Y.astype(np.float64) - float(sy) * q)
+    assert np.all(err[inside] <= 0.5 * float(sy) + np.abs(Y[inside]) * 2.0 ** -23)
+    assert np.all(q[~inside & (Y > 0)] == 127) and np.all(q[~inside & (Y < 0)] <= -127)
+    # monotone in y
+    order = np.argsort(Y, kind="stable")
+    assert np.all(np.diff(q[order]) >= 0)
+    # exact rational arithmetic on the correctly rounded fp32 quotient, element by element
+    for y, c in zip(Y[:300], q[:300]):
+        quo = Fraction(float(np.float32(y) / sy))        # numpy's IEEE binary32 division
+        lo = quo.numerator // quo.denominator
+        frac = quo - lo
+        r = lo + (1 if (frac > Fraction(1, 2) or (frac == Fraction(1, 2) and lo % 2 == 1)) else 0)
+        assert c == max(-128, min(127, r))
+    # with the tensor's own max/127 as the scale it is the dynamic quantiser
+    Xq, sx = oracle.quantize_act(Y)
+    assert np.array_equal(oracle.requantize_static(Y, sx), Xq)
+
+
+def test_bf16_rounding_closed_forms_and_library():
+    import torch
+    one = np.float32(1.0)
+    cases = {
+        1.0: 0x3F80, -2.75: 0xC030, 0.0: 0x0000,
+        float(one + np.float32(2.0 ** -8)): 0x3F80,                          # tie, lower neighbour even
+        float(one + np.float32(3 * 2.0 ** -8)): 0x3F82,                      # tie, upper neighbour even
+        float(one + np.float32(2.0 ** -8) + np.float32(2.0 ** -20)): 0x3F81,  # just above the tie
+        float(one + np.float32(2.0 ** -8) - np.float32(2.0 ** -20)): 0x3F80,  # just below the tie
+        float(np.float32(3.3895313892515355e38)): 0x7F7F,                    # largest finite bfloat16 stays
+    }
+    got = oracle.to_bf16(np.array(list(cases.keys()), dtype=np.float32))
+    assert [int(g) for g in got] == list(cases.values())
+    # values with at most 8 significant bits are reproduced exactly
+    exact = (np.arange(-255, 256, dtype=np.float32) * np.float32(2.0 ** -10))
+    back = (oracle.to_bf16(exact).astype(np.uint32) << 16).view(np.float32)
+    assert np.array_equal(back, exact)
+    # half-ulp error bound, monotonicity, agreement with an independent conversion routine
+    rng = np.random.default_rng(12)
+    Y = np.concatenate([wl.normal(rng, (100000,), 5.0), wl.normal(rng, (1000,), 1e-30), wl.normal(rng, (1000,), 1e30)])
+    b = oracle.to_bf16(Y)
+    back = (b.astype(np.uint32) << 16).view(np.float32).astype(np.float64)
+    normal = np.abs(Y) >= 2.0 ** -126
+    assert np.all(np.abs(back - Y)[normal] <= np.abs(Y[normal].astype(np.float64)) * 2.0 ** -8)
+    order = np.argsort(Y, kind="stable")
+    assert np.all(np.diff(back[order]) >= 0)
+    lib = torch.from_numpy(Y).to(torch.bfloat16).view(torch.int16).numpy().view(np.uint16)
+    assert np.array_equal(b, lib)
+    with pytest.raises(RuntimeError):
+        oracle.to_bf16(np.array([np.inf], np.float32))
