@@ -54,12 +54,12 @@ def gemm_ops(tokens, k, out):
     return 2.0 * tokens * k * out
 
 
-def gemm_bytes(tokens, k, out, n=2, m=4, bits=8):
+def gemm_bytes(tokens, k, out, n=2, m=4, bits=8, ybytes=4):
     """Algorithmic HBM bytes of one GEMM launch: X + packed values + metadata + scales/bias + Y."""
     fb = 2 if m == 4 else 4
     vals = out * (k // m) * n * bits / 8
     meta = 0 if n == m else out * (k // m) * n * fb / 8
-    return tokens * k + vals + meta + 8 * out + 4.0 * tokens * out
+    return tokens * k + vals + meta + 8 * out + float(ybytes) * tokens * out
 
 
 def pack_bytes(out, k, n, m, bits, with_u=True):
@@ -226,6 +226,8 @@ def run_cuda(args):
         dist.init_process_group("nccl", device_id=dev)
     n, m, bits = PATTERN
     pk = peaks()
+    YDTYPE = {"f32": torch.float32, "int8": torch.int8, "bf16": torch.bfloat16}[args.out]
+    YB = {"f32": 4, "int8": 1, "bf16": 2}[args.out]
 
     # ---- inputs (seeded per rank: independent batches, weak scaling) ---------------------------
     rng = np.random.default_rng([2, rank])
@@ -241,14 +243,14 @@ def run_cuda(args):
     devbuf = []
     for name, k, out, W, U, b, Xq in layer:
         hW, hU, hX = (torch.from_numpy(a).pin_memory() for a in (W, U, Xq))
-        hY = torch.empty((TOKENS, out), dtype=torch.float32).pin_memory()
+        hY = torch.empty((TOKENS, out), dtype=YDTYPE).pin_memory()
         host.append((hW, hU, hX, hY))
         vb, mb = nm.nm_packed_sizes(out, k, n, m, bits)
         d = {"W": hW.to(dev), "U": hU.to(dev), "X": hX.to(dev), "b": torch.from_numpy(b).to(dev),
              "values": torch.empty(vb, dtype=torch.uint8, device=dev),
              "meta": torch.empty(mb // 4, dtype=torch.int32, device=dev),
              "scales": torch.empty(out, dtype=torch.float32, device=dev),
-             "Y": torch.empty((TOKENS, out), dtype=torch.float32, device=dev), "k": k, "out": out, "name": name}
+             "Y": torch.empty((TOKENS, out), dtype=YDTYPE, device=dev), "k": k, "out": out, "name": name}
         d["desc"] = nm.make_packed(out, k, n, m, bits, d["values"], d["meta"])
         devbuf.append(d)
     status = torch.zeros(1, dtype=torch.int32, device=dev)
@@ -256,6 +258,7 @@ def run_cuda(args):
     ws_bytes = nm.nm_pack_workspace_bytes(len(devbuf))
     ws = torch.empty(ws_bytes, dtype=torch.uint8, device=dev)
     sx = 0.03
+    SY = 0.05  # static output scale of the int8-output variant (outputs are ~N(0, 0.5): little clamping)
 
     ev = lambda: torch.cuda.Event(enable_timing=True)
     kernel_events = {"pack": []}
@@ -274,7 +277,12 @@ def run_cuda(args):
             if record:
                 e0, e1 = ev(), ev()
                 e0.record()
-            nm.nm_int_linear(d["X"], TOKENS, d["desc"], sx, d["scales"], d["b"], d["Y"], status=status)
+            if args.out == "f32":
+                nm.nm_int_linear(d["X"], TOKENS, d["desc"], sx, d["scales"], d["b"], d["Y"], status=status)
+            elif args.out == "int8":
+                nm.nm_int_linear_q8(d["X"], TOKENS, d["desc"], sx, d["scales"], d["b"], SY, d["Y"], status=status)
+            else:
+                nm.nm_int_linear_bf16(d["X"], TOKENS, d["desc"], sx, d["scales"], d["b"], d["Y"], status=status)
             if record:
                 e1.record()
                 kernel_events[d["name"]].append((e0, e1))
@@ -334,7 +342,7 @@ def run_cuda(args):
     barrier()
     e2e_ms = max_over_ranks(t0.elapsed_time(t1)) / e2e_steps
     h2d = sum(hW.numel() * 4 + hU.numel() * 4 + hX.numel() for hW, hU, hX, hY in host)
-    d2h = sum(hY.numel() * 4 for hW, hU, hX, hY in host)
+    d2h = sum(hY.numel() * YB for hW, hU, hX, hY in host)
     clocks = sampler.stop() if rank == 0 else None
 
     # ---- projection/pack on the full 24-layer sweep (its own roofline), rank 0 only ---------------
@@ -347,7 +355,7 @@ def run_cuda(args):
         per_kernel = {}
         for d in devbuf:
             us = kern[d["name"]]
-            ops, byt = gemm_ops(TOKENS, d["k"], d["out"]), gemm_bytes(TOKENS, d["k"], d["out"], n, m, bits)
+            ops, byt = gemm_ops(TOKENS, d["k"], d["out"]), gemm_bytes(TOKENS, d["k"], d["out"], n, m, bits, YB)
             per_kernel[d["name"]] = {
                 "us": us, "tops": ops / us / 1e6, "gbs": byt / us / 1e3,
                 "frac_sparse_int8_peak_measured": ops / us / 1e6 / sparse_peak,
@@ -361,16 +369,16 @@ def run_cuda(args):
         # dominant kernel of the step: the FFN1 GEMM launch (longest; bound by the fp32 Y write).
         # `traffic` = dram__bytes_read.sum + dram__bytes_write.sum of one launch at this size (ncu, see
         # profiles/); part of Y is still in the 126 MB L2 when the kernel ends, hence below the algorithmic bytes.
-        full_size = TOKENS == 16384 and bits == 8
+        full_size = TOKENS == 16384 and bits == 8 and args.out == "f32"
         dom = per_kernel["ffn1"]
         # kernel variant the library picks at this size: CTA pairs with resident / streamed weights for
         # int8 2:4; for 4-bit codes the one-CTA kernel whose builder warps widen them in shared memory
-        k1 = "nm_gemm_pair_kernel<sparse,192,f32,resident>" if bits == 8 else "nm_gemm_kernel<sparse,192,f32,build-resident>"
-        k2 = "nm_gemm_pair_kernel<sparse,192,f32,streamed>" if bits == 8 else "nm_gemm_kernel<sparse,192,f32,build-per-k-block>"
+        k1 = f"nm_gemm_pair_kernel<sparse,192,{args.out},resident>" if bits == 8 else f"nm_gemm_kernel<sparse,192,{args.out},build-resident>"
+        k2 = f"nm_gemm_pair_kernel<sparse,192,{args.out},streamed>" if bits == 8 else f"nm_gemm_kernel<sparse,192,{args.out},build-per-k-block>"
         roofline = {"kernel": k1 + " on ffn1 1024->4096", "bound": "hbm",
                     "achieved": dom["gbs"], "peak": pk["hbm_gbs"], "unit": "GB/s",
                     "frac": dom["gbs"] / pk["hbm_gbs"], "traffic": 241945088 if full_size else None,
-                    "algorithmic_bytes": gemm_bytes(TOKENS, 1024, 4096), "peak_source": pk["source"]}
+                    "algorithmic_bytes": gemm_bytes(TOKENS, 1024, 4096, n, m, bits, YB), "peak_source": pk["source"]}
         f2 = per_kernel["ffn2"]
         roofline_tensor = {"kernel": k2 + " on ffn2 4096->1024", "bound": "tensor",
                            "achieved": f2["tops"], "peak": sparse_peak, "unit": "TOP/s",
@@ -381,7 +389,7 @@ def run_cuda(args):
         line = {"metric": METRIC, "value": value, "unit": "TOPS", "n_gpus": world, "steps": args.steps,
                 "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True,
                 "scaling": "weak", "vs_baseline": None, "dtype": "int8", "data": "synthetic",
-                "config": {"workload": WORKLOAD if TOKENS == 16384 else WORKLOAD + f" (reduced to {TOKENS} tokens)", "tokens": TOKENS, "pattern": "2:4", "bits": bits,
+                "config": {"workload": WORKLOAD if TOKENS == 16384 else WORKLOAD + f" (reduced to {TOKENS} tokens)", "tokens": TOKENS, "pattern": "2:4", "bits": bits, "out": args.out,
                            "l2": "inputs+outputs per step (715 MB) exceed L2; no flush needed"},
                 "clocks": clocks,
                 "e2e": {"value": whole_job_tops(ops_step, world, e2e_ms), "unit": "TOPS",
@@ -448,6 +456,8 @@ def main():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
     ap.add_argument("--bits", type=int, default=8, choices=[8, 4], help="weight code width of the 2:4 weights (default 8)")
+    ap.add_argument("--out", default="f32", choices=["f32", "int8", "bf16"],
+                    help="element type the GEMMs write: fp32 (the headline), int8 with a static scale, bfloat16")
     ap.add_argument("--tokens", type=int, default=TOKENS, help="tokens per GEMM (default: the full workload)")
     ap.add_argument("--skip-cpu", action="store_true", help="leave the CPU-oracle baseline out")
     ap.add_argument("--skip-sweep", action="store_true", help="leave the 24-layer pack sweep out")

@@ -156,6 +156,27 @@ int nm_int_linear_dsx(const int8_t *X, int tokens, const nm_packed_t *W, const f
                       const float *sw, const float *bias, float *Y, float *absmax_out, void *ws,
                       size_t ws_bytes, uint32_t *status, void *stream);
 
+/*
+ * Narrow outputs of the same layer, for encoders that keep their activations at 8 bits between
+ * layers (Sec. 4.5, Sec. 5.3) or hand them on in bfloat16: y = fma((float)acc, sx * sw[o], bias[o])
+ * is formed as in nm_int_linear and leaves the kernel as
+ *   nm_int_linear_q8:   Yq[t,o] = clamp(rne(y / sy), -128, 127)   (Eq. 5 with b = 8 and the scale sy
+ *                       fixed ahead of time; IEEE fp32 division, round half to even), int8
+ *                       [tokens, out] row-major, directly usable as the next layer's X with sx = sy;
+ *                       sy must be positive and finite (NM_ERR_SHAPE otherwise);
+ *   nm_int_linear_bf16: Y[t,o] = y rounded to bfloat16 (nearest, ties to even), bit patterns as
+ *                       uint16 [tokens, out] row-major; 2-byte aligned.
+ * All other arguments, errors and ownership as for nm_int_linear.  The output goes through the
+ * TMA-store epilogue when its base and row pitch are multiples of 16 bytes (out % 16 == 0 for
+ * int8, out % 8 == 0 for bfloat16), else through plain stores.
+ */
+int nm_int_linear_q8(const int8_t *X, int tokens, const nm_packed_t *W, float sx, const float *sw,
+                     const float *bias, float sy, int8_t *Yq, void *ws, size_t ws_bytes,
+                     uint32_t *status, void *stream);
+int nm_int_linear_bf16(const int8_t *X, int tokens, const nm_packed_t *W, float sx, const float *sw,
+                       const float *bias, uint16_t *Ybf16, void *ws, size_t ws_bytes,
+                       uint32_t *status, void *stream);
+
 /* The raw int32 accumulators acc[t,o] (row-major [tokens, out]) of the same product, no epilogue. */
 int nm_int_linear_acc(const int8_t *X, int tokens, const nm_packed_t *W, int32_t *ACC, void *ws,
                       size_t ws_bytes, uint32_t *status, void *stream);

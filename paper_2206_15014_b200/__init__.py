@@ -27,7 +27,8 @@ NM_ERR_WORKSPACE, NM_ERR_CUDA, NM_ERR_NONFINITE, NM_ERR_TIMEOUT = -5, -6, -7, -8
 EXPORTS = (
     "nm_packed_sizes", "nm_project_pack", "nm_project_pack_batched", "nm_pack_workspace_bytes",
     "nm_project_pack_batched_noalloc",
-    "nm_int_linear", "nm_int_linear_dsx", "nm_int_linear_acc", "nm_int_linear_workspace_bytes",
+    "nm_int_linear", "nm_int_linear_dsx", "nm_int_linear_acc", "nm_int_linear_q8", "nm_int_linear_bf16",
+    "nm_int_linear_workspace_bytes",
     "nm_int_linear_check", "nm_absmax", "nm_quantize_act", "nm_poll_status", "nm_strerror",
     "nm_last_cuda_error", "nm_version",
 )
@@ -56,6 +57,8 @@ _lib.nm_pack_workspace_bytes.restype = _sz
 _lib.nm_int_linear.argtypes = [_vp, _i, ctypes.POINTER(nm_packed_t), _f, _vp, _vp, _vp, _vp, _sz, _vp, _vp]
 _lib.nm_int_linear_dsx.argtypes = [_vp, _i, ctypes.POINTER(nm_packed_t), _vp, _vp, _vp, _vp, _vp, _vp, _sz, _vp, _vp]
 _lib.nm_int_linear_acc.argtypes = [_vp, _i, ctypes.POINTER(nm_packed_t), _vp, _vp, _sz, _vp, _vp]
+_lib.nm_int_linear_q8.argtypes = [_vp, _i, ctypes.POINTER(nm_packed_t), _f, _vp, _vp, _f, _vp, _vp, _sz, _vp, _vp]
+_lib.nm_int_linear_bf16.argtypes = [_vp, _i, ctypes.POINTER(nm_packed_t), _f, _vp, _vp, _vp, _vp, _sz, _vp, _vp]
 _lib.nm_int_linear_workspace_bytes.argtypes = [_i] * 6
 _lib.nm_int_linear_workspace_bytes.restype = _sz
 _lib.nm_int_linear_check.argtypes = [_i] * 6
@@ -171,6 +174,17 @@ def nm_int_linear_dsx(X, tokens, W, sx_dev, sw, bias, Y, absmax_out=None, ws=Non
 def nm_int_linear_acc(X, tokens, W, ACC, ws=None, ws_bytes=0, status=None, stream=None):
     _chk(_lib.nm_int_linear_acc(_ptr(X), tokens, ctypes.byref(W), _ptr(ACC), _ptr(ws), ws_bytes,
                                 _ptr(status), _stream(stream)), "nm_int_linear_acc")
+
+
+def nm_int_linear_q8(X, tokens, W, sx, sw, bias, sy, Yq, ws=None, ws_bytes=0, status=None, stream=None):
+    _chk(_lib.nm_int_linear_q8(_ptr(X), tokens, ctypes.byref(W), float(sx), _ptr(sw), _ptr(bias), float(sy),
+                               _ptr(Yq), _ptr(ws), ws_bytes, _ptr(status), _stream(stream)), "nm_int_linear_q8")
+
+
+def nm_int_linear_bf16(X, tokens, W, sx, sw, bias, Ybf16, ws=None, ws_bytes=0, status=None, stream=None):
+    _chk(_lib.nm_int_linear_bf16(_ptr(X), tokens, ctypes.byref(W), float(sx), _ptr(sw), _ptr(bias),
+                                 _ptr(Ybf16), _ptr(ws), ws_bytes, _ptr(status), _stream(stream)),
+         "nm_int_linear_bf16")
 
 
 def nm_absmax(Y, count, absmax, stream=None):

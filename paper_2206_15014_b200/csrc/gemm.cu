@@ -45,7 +45,35 @@ constexpr int kStoreStage = 8 * 4096;  // per epilogue warp two [16 tokens][32 c
 constexpr int kMaxStages = 7;       // the relay cycles through 8 named barriers
 constexpr long long kWaitLimit = 1ll << 31;  // SM clocks (about a second)
 
-enum { EPI_F32 = 0, EPI_ACC = 1 };
+// What the epilogue writes: y = fma(acc, sx * sw[o], b[o]) as fp32; the raw int32 accumulators; y re-quantised
+// to 8 bits with a scale fixed ahead of time (Eq. 5, b = 8); y rounded to bfloat16.
+enum { EPI_F32 = 0, EPI_ACC = 1, EPI_Q8 = 2, EPI_BF16 = 3 };
+template <int EPI> struct EpiOut { using type = uint32_t; };          // fp32 / int32 move as 32-bit patterns
+template <> struct EpiOut<EPI_Q8> { using type = uint8_t; };
+template <> struct EpiOut<EPI_BF16> { using type = uint16_t; };
+
+// One output element from an accumulator: fp32 value y, then the narrowing the epilogue kind asks for.
+template <int EPI>
+__device__ __forceinline__ typename EpiOut<EPI>::type epi_convert(uint32_t acc, float c_n, float b_n, float sy, float& y_abs) {
+    if constexpr (EPI == EPI_ACC) {
+        y_abs = 0.0f;
+        return acc;
+    } else {
+        const float y = __fmaf_rn((float)(int)acc, c_n, b_n);
+        y_abs = fabsf(y);
+        if constexpr (EPI == EPI_F32) {
+            return __float_as_uint(y);
+        } else if constexpr (EPI == EPI_Q8) {
+            // true IEEE division, round half to even, clamp to [-128, 127]
+            const int q = __float2int_rn(__fdiv_rn(y, sy));
+            return (uint8_t)(int8_t)max(-128, min(127, q));
+        } else {
+            uint16_t h;
+            asm("cvt.rn.bf16.f32 %0, %1;" : "=h"(h) : "f"(y));
+            return h;
+        }
+    }
+}
 // Where the weight operand comes from: TMA (already in tensor-core form), built per k-block into the
 // stage ring, or built once per output tile into a resident region (reduction length <= kResidentKB k-blocks).
 enum { W_TMA = 0, W_BUILD = 1, W_RESIDENT = 2 };
@@ -65,6 +93,8 @@ struct GemmParams {
     float sx_host;
     float* Y;
     int32_t* ACC;
+    void* NARROW;          // int8 (EPI_Q8) or bfloat16 (EPI_BF16) output [tokens, out]
+    float sy;              // static output scale of EPI_Q8
     float* absmax;
     uint32_t* status;
 };
@@ -382,7 +412,7 @@ nm_gemm_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant
                 if (next_out_tile != out_tile) load_meta(next_out_tile);  // MMAs of this output tile are done
             }
             const bool n_ok = n < p.out;
-            if (EPI == EPI_F32 && out_tile != scaled_out_tile) {  // channel constants: fetched once per output tile
+            if (EPI != EPI_ACC && out_tile != scaled_out_tile) {  // channel constants: fetched once per output tile
                 scaled_out_tile = out_tile;
                 c_n = n_ok ? __fmul_rn(sx, p.sw[n]) : 0.0f;
                 b_n = n_ok && p.bias ? p.bias[n] : 0.0f;
@@ -404,14 +434,12 @@ nm_gemm_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant
                     else if (RB == 2) ptx::tmem_ld_32x32(lane_taddr + buf * BN + (c + EWH) * 32, r[(ci + 1) & (RB - 1)]);
                     // conversion of accumulator column j of this chunk; jmax = outputs of this lane that exist
                     const int jmax = n_ok ? min(32, p.tokens - tc0) : 0;
-                    auto conv = [&](int j) -> uint32_t {
-                        if constexpr (EPI == EPI_F32) {
-                            const float y = __fmaf_rn((float)(int)r[ci & (RB - 1)][j], c_n, b_n);
-                            amax = fmaxf(amax, j < jmax ? fabsf(y) : 0.0f);
-                            return __float_as_uint(y);
-                        } else {
-                            return r[ci & (RB - 1)][j];
-                        }
+                    using OT = typename EpiOut<EPI>::type;
+                    auto conv = [&](int j) -> OT {
+                        float y_abs;
+                        const OT o = epi_convert<EPI>(r[ci & (RB - 1)][j], c_n, b_n, p.sy, y_abs);
+                        if constexpr (EPI == EPI_F32) amax = fmaxf(amax, j < jmax ? y_abs : 0.0f);
+                        return o;
                     };
                     // The two store paths are separate loops: a branch inside the unrolled loop costs a
                     // pipeline refill per column (measured ~30 clk each), far more than its arithmetic.
@@ -421,11 +449,11 @@ nm_gemm_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant
 #pragma unroll
                         for (int h = 0; h < 2; ++h) {
                             if (tc0 + 16 * h < p.tokens) {  // warp-uniform
-                                float* sb = my_stage + (n_stores & 1u) * 512;
+                                OT* sb = reinterpret_cast<OT*>(my_stage + (n_stores & 1u) * 512);
                                 if (lane == 0) ptx::bulk_wait_group_read<1>();  // the store before the last has read this tile
                                 __syncwarp();
 #pragma unroll
-                                for (int j = 0; j < 16; ++j) sb[j * 32 + lane] = __uint_as_float(conv(16 * h + j));
+                                for (int j = 0; j < 16; ++j) sb[j * 32 + lane] = conv(16 * h + j);
                                 ptx::fence_proxy_async_smem();
                                 __syncwarp();
                                 if (lane == 0) {
@@ -436,11 +464,11 @@ nm_gemm_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant
                             }
                         }
                     } else {  // output rows not 16-byte aligned: lane = channel, j = token
-                        uint32_t* dst = reinterpret_cast<uint32_t*>(EPI == EPI_F32 ? (void*)p.Y : (void*)p.ACC) + (size_t)tc0 * p.out + n;
+                        OT* dst = reinterpret_cast<OT*>(EPI == EPI_F32 ? (void*)p.Y : EPI == EPI_ACC ? (void*)p.ACC : p.NARROW) + (size_t)tc0 * p.out + n;
 #pragma unroll
                         for (int j = 0; j < 32; ++j) {
-                            const uint32_t o = conv(j);
-                            if (j < jmax) __stcs(dst + (size_t)j * p.out, o);
+                            const OT o = conv(j);
+                            if (j < jmax) dst[(size_t)j * p.out] = o;
                         }
                     }
                 }
@@ -723,7 +751,7 @@ nm_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_con
             // the next tile starts a new output tile: its metadata can go in now, the MMAs of this one are done
             if (SPARSE && half == 0 && i + 1 < tile_count && tok_tile + 1 == p.n_tok_tiles) load_meta(out_tile + 1);
             const bool n_ok = n < p.out;
-            if (EPI == EPI_F32 && out_tile != scaled_out_tile) {  // channel constants: fetched once per output tile
+            if (EPI != EPI_ACC && out_tile != scaled_out_tile) {  // channel constants: fetched once per output tile
                 scaled_out_tile = out_tile;
                 c_n = n_ok ? __fmul_rn(sx, p.sw[n]) : 0.0f;
                 b_n = n_ok && p.bias ? p.bias[n] : 0.0f;
@@ -740,24 +768,22 @@ nm_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_con
                     if (c + EWH < nact) ptx::tmem_ld_32x32(lane_taddr + buf * BN + (c + EWH) * 32, r[(ci + 1) & 1]);
                     else release_acc(buf);
                     const int jmax = n_ok ? min(32, p.tokens - tc0) : 0;  // outputs of this lane that exist
-                    auto conv = [&](int j) -> uint32_t {
-                        if constexpr (EPI == EPI_F32) {
-                            const float y = __fmaf_rn((float)(int)r[ci & 1][j], c_n, b_n);
-                            amax = fmaxf(amax, j < jmax ? fabsf(y) : 0.0f);
-                            return __float_as_uint(y);
-                        } else {
-                            return r[ci & 1][j];
-                        }
+                    using OT = typename EpiOut<EPI>::type;
+                    auto conv = [&](int j) -> OT {
+                        float y_abs;
+                        const OT o = epi_convert<EPI>(r[ci & 1][j], c_n, b_n, p.sy, y_abs);
+                        if constexpr (EPI == EPI_F32) amax = fmaxf(amax, j < jmax ? y_abs : 0.0f);
+                        return o;
                     };
                     if (p.tma_store) {  // separate branch-free loops for the two store paths
 #pragma unroll
                         for (int h = 0; h < 2; ++h) {  // 16 tokens per store, alternating staging tiles
                             if (tc0 + 16 * h < p.tokens) {  // warp-uniform
-                                float* sb = my_stage + (NB == 2 ? (n_stores & 1u) * 512 : 0);
+                                OT* sb = reinterpret_cast<OT*>(my_stage + (NB == 2 ? (n_stores & 1u) * 512 : 0));
                                 if (lane == 0) ptx::bulk_wait_group_read<NB - 1>();  // the store that last used this tile has read it
                                 __syncwarp();
 #pragma unroll
-                                for (int j = 0; j < 16; ++j) sb[j * 32 + lane] = __uint_as_float(conv(16 * h + j));
+                                for (int j = 0; j < 16; ++j) sb[j * 32 + lane] = conv(16 * h + j);
                                 ptx::fence_proxy_async_smem();
                                 __syncwarp();
                                 if (lane == 0) {
@@ -768,11 +794,11 @@ nm_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_con
                             }
                         }
                     } else {
-                        uint32_t* dst = reinterpret_cast<uint32_t*>(EPI == EPI_F32 ? (void*)p.Y : (void*)p.ACC) + (size_t)tc0 * p.out + n;
+                        OT* dst = reinterpret_cast<OT*>(EPI == EPI_F32 ? (void*)p.Y : EPI == EPI_ACC ? (void*)p.ACC : p.NARROW) + (size_t)tc0 * p.out + n;
 #pragma unroll
                         for (int j = 0; j < 32; ++j) {
-                            const uint32_t o = conv(j);
-                            if (j < jmax) __stcs(dst + (size_t)j * p.out, o);
+                            const OT o = conv(j);
+                            if (j < jmax) dst[(size_t)j * p.out] = o;
                         }
                     }
                 }
@@ -867,7 +893,24 @@ struct LinearArgs {
     const int8_t* X; int tokens; const nm_packed_t* W;
     float sx; const float* sx_dev; const float* sw; const float* bias;
     float* Y; int32_t* ACC; float* absmax; uint32_t* status; cudaStream_t stream;
+    void* NARROW = nullptr; float sy = 1.0f;
 };
+
+// Tensor map of the output for the epilogue's TMA stores ([16 tokens][32 channels] boxes).  The epilogue stores
+// through TMA when the output can be described by a tensor map (16-byte aligned base and row pitch);
+// otherwise *tma_store is cleared, the threads store directly and the map describes X as a stand-in.
+template <int EPI>
+static int make_store_map(CUtensorMap* ty, const LinearArgs& a, bool* tma_store) {
+    const nm_packed_t& W = *a.W;
+    constexpr uint32_t es = (uint32_t)sizeof(typename EpiOut<EPI>::type);
+    void* ybase = EPI == EPI_F32 ? (void*)a.Y : EPI == EPI_ACC ? (void*)a.ACC : a.NARROW;
+    *tma_store = aligned(ybase, 16) && ((size_t)W.out * es) % 16 == 0;
+    const CUtensorMapDataType dt = EPI == EPI_F32 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : EPI == EPI_ACC ? CU_TENSOR_MAP_DATA_TYPE_INT32
+                                 : EPI == EPI_Q8 ? CU_TENSOR_MAP_DATA_TYPE_UINT8 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16;
+    if (!*tma_store)
+        return make_map(ty, a.X, (uint64_t)a.tokens, (uint64_t)W.in / 4, 16, 32, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_DATA_TYPE_INT32, 4);
+    return make_map(ty, ybase, (uint64_t)a.tokens, (uint64_t)W.out, 16, 32, CU_TENSOR_MAP_SWIZZLE_NONE, dt, es);
+}
 
 template <bool SPARSE, int BN, int EPI, int WSRC>
 static int launch_gemm(const LinearArgs& a) {
@@ -882,12 +925,8 @@ static int launch_gemm(const LinearArgs& a) {
     if (rc != NM_OK) return rc;
     rc = make_map(&tx, a.X, (uint64_t)a.tokens, (uint64_t)W.in, BN, 128, CU_TENSOR_MAP_SWIZZLE_128B);
     if (rc != NM_OK) return rc;
-    // The epilogue stores through TMA when Y can be described by a tensor map (16-byte aligned
-    // base and row pitch); otherwise the threads store directly.
-    void* ybase = EPI == EPI_F32 ? (void*)a.Y : (void*)a.ACC;
-    const bool tma_store = aligned(ybase, 16) && (W.out % 4) == 0;
-    rc = make_map(&ty, tma_store ? ybase : (const void*)a.X, (uint64_t)a.tokens, (uint64_t)(tma_store ? W.out : W.in / 4), 16, 32,
-                  CU_TENSOR_MAP_SWIZZLE_NONE, EPI == EPI_F32 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_INT32, 4);
+    bool tma_store = false;
+    rc = make_store_map<EPI>(&ty, a, &tma_store);
     if (rc != NM_OK) return rc;
     GemmParams p{};
     p.tma_store = tma_store ? 1 : 0;
@@ -901,7 +940,7 @@ static int launch_gemm(const LinearArgs& a) {
     p.mrow_bytes = (int)meta_row_words(W.in, W.n, W.m) * 4;
     p.pat = xf::pattern_of(W.n, W.m, W.bits);
     p.sw = a.sw; p.bias = a.bias; p.sx_dev = a.sx_dev; p.sx_host = a.sx;
-    p.Y = a.Y; p.ACC = a.ACC; p.absmax = a.absmax; p.status = a.status;
+    p.Y = a.Y; p.ACC = a.ACC; p.NARROW = a.NARROW; p.sy = a.sy; p.absmax = a.absmax; p.status = a.status;
     auto fn = nm_gemm_kernel<SPARSE, BN, EPI, WSRC>;
     NM_CUDA_TRY(cudaFuncSetAttribute((const void*)fn, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::SMEM));
     const int grid = p.n_tiles < sm_count() ? p.n_tiles : sm_count();
@@ -920,10 +959,8 @@ static int launch_gemm_pair(const LinearArgs& a) {
     if (rc != NM_OK) return rc;
     rc = make_map_x3(&tx, a.X, (uint64_t)a.tokens, (uint64_t)W.in, Cfg::B_ROWS, Cfg::KB / 128);
     if (rc != NM_OK) return rc;
-    void* ybase = EPI == EPI_F32 ? (void*)a.Y : (void*)a.ACC;
-    const bool tma_store = aligned(ybase, 16) && (W.out % 4) == 0;
-    rc = make_map(&ty, tma_store ? ybase : (const void*)a.X, (uint64_t)a.tokens, (uint64_t)(tma_store ? W.out : W.in / 4), 16, 32,
-                  CU_TENSOR_MAP_SWIZZLE_NONE, EPI == EPI_F32 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_INT32, 4);
+    bool tma_store = false;
+    rc = make_store_map<EPI>(&ty, a, &tma_store);
     if (rc != NM_OK) return rc;
     GemmParams p{};
     p.tma_store = tma_store ? 1 : 0;
@@ -933,7 +970,7 @@ static int launch_gemm_pair(const LinearArgs& a) {
     p.kblocks = (W.in + Cfg::KB - 1) / Cfg::KB;
     p.meta = (const uint32_t*)W.meta; p.mrow_words = W.in / 32;
     p.sw = a.sw; p.bias = a.bias; p.sx_dev = a.sx_dev; p.sx_host = a.sx;
-    p.Y = a.Y; p.ACC = a.ACC; p.absmax = a.absmax; p.status = a.status;
+    p.Y = a.Y; p.ACC = a.ACC; p.NARROW = a.NARROW; p.sy = a.sy; p.absmax = a.absmax; p.status = a.status;
     auto fn = nm_gemm_pair_kernel<SPARSE, BN, EPI, RES>;
     NM_CUDA_TRY(cudaFuncSetAttribute((const void*)fn, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::SMEM));
     const int pairs = p.n_tiles < sm_count() / 2 ? p.n_tiles : sm_count() / 2;
@@ -1000,6 +1037,13 @@ static int check_linear(int tokens, int out, int in, int n, int m, int bits) {
     return NM_OK;
 }
 
+template <int EPI>
+static int run_linear_epi(const LinearArgs& a, bool xform, bool sparse) {
+    if (xform) return sparse ? pick_bn<true, EPI, true>(a) : pick_bn<false, EPI, true>(a);
+    if (sparse) return use_pair<true, EPI>(a) ? pick_pair<true, EPI>(a) : pick_bn<true, EPI, false>(a);
+    return use_pair<false, EPI>(a) ? pick_pair<false, EPI>(a) : pick_bn<false, EPI, false>(a);
+}
+
 static int run_linear(const LinearArgs& a, int epi) {
     if (!a.W) return NM_ERR_NULL;
     const nm_packed_t& W = *a.W;
@@ -1009,21 +1053,21 @@ static int run_linear(const LinearArgs& a, int epi) {
     const bool xform = pat != xf::PNONE;
     const bool sparse = xform ? xf::sparse_target(pat) : W.n != W.m;  // tensor-core form of the weights
     if (!a.X || !W.values || (W.n != W.m && !W.meta)) return NM_ERR_NULL;
-    if (epi == EPI_F32 && (!a.Y || !a.sw)) return NM_ERR_NULL;
+    if (epi != EPI_ACC && !a.sw) return NM_ERR_NULL;
+    if (epi == EPI_F32 && !a.Y) return NM_ERR_NULL;
     if (epi == EPI_ACC && !a.ACC) return NM_ERR_NULL;
+    if ((epi == EPI_Q8 || epi == EPI_BF16) && !a.NARROW) return NM_ERR_NULL;
+    if (epi == EPI_Q8 && !(a.sy > 0.0f && a.sy <= 3.402823466e38f)) return NM_ERR_SHAPE;  // positive and finite
     if (!aligned(a.X, 16) || !aligned(W.values, 16) || (W.meta && !aligned(W.meta, 16))) return NM_ERR_ALIGN;
     if ((a.Y && !aligned(a.Y, 4)) || (a.ACC && !aligned(a.ACC, 4))) return NM_ERR_ALIGN;
+    if (epi == EPI_BF16 && !aligned(a.NARROW, 2)) return NM_ERR_ALIGN;
     if (a.tokens == 0 || W.out == 0) return NM_OK;
-    if (xform) {
-        if (sparse) return epi == EPI_F32 ? pick_bn<true, EPI_F32, true>(a) : pick_bn<true, EPI_ACC, true>(a);
-        return epi == EPI_F32 ? pick_bn<false, EPI_F32, true>(a) : pick_bn<false, EPI_ACC, true>(a);
+    switch (epi) {
+        case EPI_F32: return run_linear_epi<EPI_F32>(a, xform, sparse);
+        case EPI_ACC: return run_linear_epi<EPI_ACC>(a, xform, sparse);
+        case EPI_Q8: return run_linear_epi<EPI_Q8>(a, xform, sparse);
+        default: return run_linear_epi<EPI_BF16>(a, xform, sparse);
     }
-    if (sparse) {
-        if (epi == EPI_F32) return use_pair<true, EPI_F32>(a) ? pick_pair<true, EPI_F32>(a) : pick_bn<true, EPI_F32, false>(a);
-        return use_pair<true, EPI_ACC>(a) ? pick_pair<true, EPI_ACC>(a) : pick_bn<true, EPI_ACC, false>(a);
-    }
-    if (epi == EPI_F32) return use_pair<false, EPI_F32>(a) ? pick_pair<false, EPI_F32>(a) : pick_bn<false, EPI_F32, false>(a);
-    return use_pair<false, EPI_ACC>(a) ? pick_pair<false, EPI_ACC>(a) : pick_bn<false, EPI_ACC, false>(a);
 }
 
 }  // namespace nm
@@ -1048,6 +1092,20 @@ int nm_int_linear_dsx(const int8_t* X, int tokens, const nm_packed_t* W, const f
     if (!sx_dev) return NM_ERR_NULL;
     nm::LinearArgs a{X, tokens, W, 0.0f, sx_dev, sw, bias, Y, nullptr, absmax_out, status, (cudaStream_t)stream};
     return nm::run_linear(a, nm::EPI_F32);
+}
+
+int nm_int_linear_q8(const int8_t* X, int tokens, const nm_packed_t* W, float sx, const float* sw,
+                     const float* bias, float sy, int8_t* Yq, void*, size_t, uint32_t* status, void* stream) {
+    nm::LinearArgs a{X, tokens, W, sx, nullptr, sw, bias, nullptr, nullptr, nullptr, status, (cudaStream_t)stream};
+    a.NARROW = Yq; a.sy = sy;
+    return nm::run_linear(a, nm::EPI_Q8);
+}
+
+int nm_int_linear_bf16(const int8_t* X, int tokens, const nm_packed_t* W, float sx, const float* sw,
+                       const float* bias, uint16_t* Ybf16, void*, size_t, uint32_t* status, void* stream) {
+    nm::LinearArgs a{X, tokens, W, sx, nullptr, sw, bias, nullptr, nullptr, nullptr, status, (cudaStream_t)stream};
+    a.NARROW = Ybf16;
+    return nm::run_linear(a, nm::EPI_BF16);
 }
 
 int nm_int_linear_acc(const int8_t* X, int tokens, const nm_packed_t* W, int32_t* ACC, void*, size_t,

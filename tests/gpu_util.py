@@ -69,3 +69,29 @@ def assert_close(Y, Y_ref):
     tol = 1e-6 + 1e-5 * np.abs(Y_ref.astype(np.float64))
     bad = err > tol
     assert not bad.any(), f"{bad.sum()} of {bad.size} outside 1e-5 rel / 1e-6 abs; max err {err.max()}"
+
+
+def gpu_int_linear_q8(Xq, packed, sx, bias, sy):
+    """Static-scale int8 output of the layer; one guard row past the last token must stay untouched."""
+    T = Xq.shape[0]
+    status = torch.zeros(1, dtype=torch.int32, device=DEV)
+    Yq = torch.full((T + 1, packed.out), 99, dtype=torch.int8, device=DEV)
+    nm.nm_int_linear_q8(to_dev(Xq), T, packed.desc, float(sx), packed.scales, to_dev(bias), float(sy), Yq, status=status)
+    rc = nm.nm_poll_status(status)
+    assert rc == nm.NM_OK, nm.nm_strerror(rc)
+    h = Yq.cpu().numpy()
+    assert (h[T] == 99).all(), "Yq written past the last token"
+    return h[:T]
+
+
+def gpu_int_linear_bf16(Xq, packed, sx, bias):
+    """bfloat16 output of the layer as uint16 bit patterns."""
+    T = Xq.shape[0]
+    status = torch.zeros(1, dtype=torch.int32, device=DEV)
+    Yb = torch.full((T + 1, packed.out), 0x7FC1, dtype=torch.int16, device=DEV)
+    nm.nm_int_linear_bf16(to_dev(Xq), T, packed.desc, float(sx), packed.scales, to_dev(bias), Yb, status=status)
+    rc = nm.nm_poll_status(status)
+    assert rc == nm.NM_OK, nm.nm_strerror(rc)
+    h = Yb.cpu().numpy().view(np.uint16)
+    assert (h[T] == 0x7FC1).all(), "Y written past the last token"
+    return h[:T]
