@@ -163,7 +163,7 @@ int nm_int_linear_dsx(const int8_t *X, int tokens, const nm_packed_t *W, const f
  *   nm_int_linear_q8:   Yq[t,o] = clamp(rne(y / sy), -128, 127)   (Eq. 5 with b = 8 and the scale sy
  *                       fixed ahead of time; IEEE fp32 division, round half to even), int8
  *                       [tokens, out] row-major, directly usable as the next layer's X with sx = sy;
- *                       sy must be positive and finite (NM_ERR_SHAPE otherwise);
+ *                       sy must be a positive, normal, finite float (NM_ERR_SHAPE otherwise);
  *   nm_int_linear_bf16: Y[t,o] = y rounded to bfloat16 (nearest, ties to even), bit patterns as
  *                       uint16 [tokens, out] row-major; 2-byte aligned.
  * All other arguments, errors and ownership as for nm_int_linear.  The output goes through the

@@ -51,10 +51,30 @@ enum { EPI_F32 = 0, EPI_ACC = 1, EPI_Q8 = 2, EPI_BF16 = 3 };
 template <int EPI> struct EpiOut { using type = uint32_t; };          // fp32 / int32 move as 32-bit patterns
 template <> struct EpiOut<EPI_Q8> { using type = uint8_t; };
 template <> struct EpiOut<EPI_BF16> { using type = uint16_t; };
+// Narrow outputs leave through [16 tokens][128 channels] tiles that the four warps of a TMEM-lane-quarter
+// group fill together (rows of 128 / 256 bytes instead of 32 / 64): named barriers kNarrowFree + half and
+// kNarrowFull + half order the fills against the one warp that issues the TMA store, kNarrowAgree + half
+// makes the group take a timed-out wait together so that nobody is left alone on a barrier.
+// EPI_Q8 without a branch per value: code from the reciprocal rsy = RN(1 / sy).  A value for which only the
+// exact division decides (within 2^-15 of a rounding tie: 6 in 100000) is remembered in (y_tie, j_tie) and
+// counted; the caller repairs it afterwards with one exact division.
+__device__ __forceinline__ uint8_t epi_convert_q8_fast(uint32_t acc, float c_n, float b_n, float rsy, int j,
+                                                       float& y_tie, int& j_tie, int& n_tie) {
+    const float y = __fmaf_rn((float)(int)acc, c_n, b_n);
+    bool near_tie = false;
+    const int code = quantise8_fast(y, rsy, near_tie);
+    y_tie = near_tie ? y : y_tie;
+    j_tie = near_tie ? j : j_tie;
+    n_tie += near_tie ? 1 : 0;
+    return (uint8_t)(int8_t)code;
+}
+
+template <int EPI> constexpr bool kNarrow = EPI == EPI_Q8 || EPI == EPI_BF16;
+constexpr uint32_t kNarrowFree = 9, kNarrowFull = 11, kNarrowAgree = 13;
 
 // One output element from an accumulator: fp32 value y, then the narrowing the epilogue kind asks for.
 template <int EPI>
-__device__ __forceinline__ typename EpiOut<EPI>::type epi_convert(uint32_t acc, float c_n, float b_n, float sy, float& y_abs) {
+__device__ __forceinline__ typename EpiOut<EPI>::type epi_convert(uint32_t acc, float c_n, float b_n, float sy, float rsy, float& y_abs) {
     if constexpr (EPI == EPI_ACC) {
         y_abs = 0.0f;
         return acc;
@@ -64,9 +84,9 @@ __device__ __forceinline__ typename EpiOut<EPI>::type epi_convert(uint32_t acc, 
         if constexpr (EPI == EPI_F32) {
             return __float_as_uint(y);
         } else if constexpr (EPI == EPI_Q8) {
-            // true IEEE division, round half to even, clamp to [-128, 127]
-            const int q = __float2int_rn(__fdiv_rn(y, sy));
-            return (uint8_t)(int8_t)max(-128, min(127, q));
+            // the IEEE quotient y / sy rounded half to even and clamped to [-128, 127]
+            (void)rsy;
+            return (uint8_t)(int8_t)quantise8_exact(y, sy);
         } else {
             uint16_t h;
             asm("cvt.rn.bf16.f32 %0, %1;" : "=h"(h) : "f"(y));
@@ -372,6 +392,7 @@ nm_gemm_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant
         float* my_stage = reinterpret_cast<float*>(store_stage + ew * 4096);
         const float sx = p.sx_dev ? *p.sx_dev : p.sx_host;
         float amax = 0.0f, c_n = 0.0f, b_n = 0.0f;
+        const float rsy = EPI == EPI_Q8 ? __frcp_rn(p.sy) : 0.0f;
         int scaled_out_tile = -1;
         uint32_t n_stores = 0;
         bool ok = true;
@@ -405,7 +426,9 @@ nm_gemm_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant
             if (SPARSE && i == 0 && half == 0) load_meta(out_tile);
             bool got = ptx::mbar_wait_bounded(acc_full_bar(buf), (i >> 1) & 1u, abort_flag, kWaitLimit);
             ok = __all_sync(0xffffffffu, got);
-            if (!ok) { if (lane == 0) raise_timeout(); break; }
+            if (!ok && lane == 0) raise_timeout();
+            if constexpr (kNarrow<EPI>) ok = ptx::named_bar_and(kNarrowAgree + half, 128, ok);  // the group stops together
+            if (!ok) break;
             ptx::tc_fence_after();
             if (SPARSE && half == 0 && i + 1 < tile_count) {
                 const int next_out_tile = (tile + 1) / p.n_tok_tiles;
@@ -437,7 +460,7 @@ nm_gemm_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant
                     using OT = typename EpiOut<EPI>::type;
                     auto conv = [&](int j) -> OT {
                         float y_abs;
-                        const OT o = epi_convert<EPI>(r[ci & (RB - 1)][j], c_n, b_n, p.sy, y_abs);
+                        const OT o = epi_convert<EPI>(r[ci & (RB - 1)][j], c_n, b_n, p.sy, rsy, y_abs);
                         if constexpr (EPI == EPI_F32) amax = fmaxf(amax, j < jmax ? y_abs : 0.0f);
                         return o;
                     };
@@ -448,7 +471,37 @@ nm_gemm_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant
                         // being read by its TMA store the other is filled
 #pragma unroll
                         for (int h = 0; h < 2; ++h) {
-                            if (tc0 + 16 * h < p.tokens) {  // warp-uniform
+                            if (tc0 + 16 * h >= p.tokens) continue;  // warp-uniform (and the same in all warps of a group)
+                            if constexpr (kNarrow<EPI>) {
+                                OT* sb = reinterpret_cast<OT*>(store_stage) + (half * 2 + (n_stores & 1u)) * (16 * 128);
+                                if (q == 0 && lane == 0) ptx::bulk_wait_group_read<1>();  // the store before the last has read this tile
+                                ptx::named_bar_sync(kNarrowFree + half, 128);
+                                if constexpr (EPI == EPI_Q8) {
+                                    float y_tie = 0.0f;
+                                    int j_tie = 0, n_tie = 0;
+#pragma unroll
+                                    for (int j = 0; j < 16; ++j)
+                                        sb[j * 128 + q * 32 + lane] = epi_convert_q8_fast(r[ci & (RB - 1)][16 * h + j], c_n, b_n, rsy, j, y_tie, j_tie, n_tie);
+                                    if (__any_sync(0xffffffffu, n_tie != 0)) {  // rare (3 % of these tiles): repair with the exact division
+                                        if (n_tie == 1) {
+                                            sb[j_tie * 128 + q * 32 + lane] = (uint8_t)(int8_t)quantise8_exact(y_tie, p.sy);
+                                        } else if (n_tie > 1) {
+#pragma unroll
+                                            for (int j = 0; j < 16; ++j) sb[j * 128 + q * 32 + lane] = conv(16 * h + j);
+                                        }
+                                    }
+                                } else {
+#pragma unroll
+                                    for (int j = 0; j < 16; ++j) sb[j * 128 + q * 32 + lane] = conv(16 * h + j);
+                                }
+                                ptx::fence_proxy_async_smem();
+                                ptx::named_bar_sync(kNarrowFull + half, 128);
+                                if (q == 0 && lane == 0) {
+                                    ptx::tma_store_2d(&tmap_y, n0, tc0 + 16 * h, ptx::smem_u32(sb));
+                                    ptx::bulk_commit_group();
+                                }
+                                ++n_stores;
+                            } else {
                                 OT* sb = reinterpret_cast<OT*>(my_stage + (n_stores & 1u) * 512);
                                 if (lane == 0) ptx::bulk_wait_group_read<1>();  // the store before the last has read this tile
                                 __syncwarp();
@@ -503,7 +556,7 @@ nm_gemm_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant
 // as a cluster before the first remote operation and before TMEM is released.
 // ---------------------------------------------------------------------------------------------
 constexpr int kPairThreads = 32 * (3 + kEpiWarps);
-constexpr int kPairMaxStages = 9;   // the relay cycles through 15 named barriers
+constexpr int kPairMaxStages = 7;   // the relay cycles through 8 named barriers (ids 1-8; 9-14 serve the narrow-output epilogue)
 
 constexpr int kPairResStages = 4;   // stages of weights a CTA can keep resident (1024 reduction elements at 2:4)
 
@@ -659,7 +712,7 @@ nm_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_con
                 for (int kb = 0; kb < p.kblocks; ++kb, ++it) {
                     wait(full_bar(it % S), (it / S) & 1u);
                     __syncwarp();
-                    ptx::named_bar_arrive(1 + (it % 15u), 64);
+                    ptx::named_bar_arrive(1 + (it & 7u), 64);
                 }
             }
         }
@@ -674,7 +727,7 @@ nm_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_con
                 const bool last_of_out_tile = RES && (tile_begin + i + 1) / p.n_tok_tiles != (tile_begin + i) / p.n_tok_tiles;
                 for (int kb = 0; kb < p.kblocks; ++kb, ++it) {
                     const int s = it % S;
-                    ptx::named_bar_sync(1 + (it % 15u), 64);
+                    ptx::named_bar_sync(1 + (it & 7u), 64);
                     if (kb == 0) ptx::tc_fence_after();  // once per tile (see the one-CTA kernel)
                     if (lane == 0) {
                         const uint32_t st_addr = ptx::smem_u32(smem + s * Cfg::STAGE), b_addr = st_addr + Cfg::B_OFF;
@@ -715,6 +768,7 @@ nm_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_con
         const float sx = p.sx_dev ? *p.sx_dev : p.sx_host;
         const uint32_t lead_meta = ptx::map_to_cta(meta_bar, 0);
         float amax = 0.0f, c_n = 0.0f, b_n = 0.0f;
+        const float rsy = EPI == EPI_Q8 ? __frcp_rn(p.sy) : 0.0f;
         int scaled_out_tile = -1;
         uint32_t n_stores = 0;
         bool ok = true;
@@ -746,7 +800,9 @@ nm_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_con
             if (SPARSE && i == 0 && half == 0) load_meta(out_tile);
             bool got = ptx::mbar_wait_bounded(acc_full_bar(buf), (i >> 1) & 1u, abort_flag, kWaitLimit);
             ok = __all_sync(0xffffffffu, got);
-            if (!ok) { if (lane == 0) raise_timeout(); break; }
+            if (!ok && lane == 0) raise_timeout();
+            if constexpr (kNarrow<EPI>) ok = ptx::named_bar_and(kNarrowAgree + half, 128, ok);  // the group stops together
+            if (!ok) break;
             ptx::tc_fence_after();
             // the next tile starts a new output tile: its metadata can go in now, the MMAs of this one are done
             if (SPARSE && half == 0 && i + 1 < tile_count && tok_tile + 1 == p.n_tok_tiles) load_meta(out_tile + 1);
@@ -771,14 +827,44 @@ nm_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_con
                     using OT = typename EpiOut<EPI>::type;
                     auto conv = [&](int j) -> OT {
                         float y_abs;
-                        const OT o = epi_convert<EPI>(r[ci & 1][j], c_n, b_n, p.sy, y_abs);
+                        const OT o = epi_convert<EPI>(r[ci & 1][j], c_n, b_n, p.sy, rsy, y_abs);
                         if constexpr (EPI == EPI_F32) amax = fmaxf(amax, j < jmax ? y_abs : 0.0f);
                         return o;
                     };
                     if (p.tma_store) {  // separate branch-free loops for the two store paths
 #pragma unroll
                         for (int h = 0; h < 2; ++h) {  // 16 tokens per store, alternating staging tiles
-                            if (tc0 + 16 * h < p.tokens) {  // warp-uniform
+                            if (tc0 + 16 * h >= p.tokens) continue;  // warp-uniform (and the same in all warps of a group)
+                            if constexpr (kNarrow<EPI>) {  // one [16 tokens][128 channels] tile per four warps
+                                OT* sb = reinterpret_cast<OT*>(store_stage) + (half * 2 + (n_stores & 1u)) * (16 * 128);
+                                if (q == 0 && lane == 0) ptx::bulk_wait_group_read<1>();  // the store before the last has read this tile
+                                ptx::named_bar_sync(kNarrowFree + half, 128);
+                                if constexpr (EPI == EPI_Q8) {
+                                    float y_tie = 0.0f;
+                                    int j_tie = 0, n_tie = 0;
+#pragma unroll
+                                    for (int j = 0; j < 16; ++j)
+                                        sb[j * 128 + q * 32 + lane] = epi_convert_q8_fast(r[ci & 1][16 * h + j], c_n, b_n, rsy, j, y_tie, j_tie, n_tie);
+                                    if (__any_sync(0xffffffffu, n_tie != 0)) {  // rare (3 % of these tiles): repair with the exact division
+                                        if (n_tie == 1) {
+                                            sb[j_tie * 128 + q * 32 + lane] = (uint8_t)(int8_t)quantise8_exact(y_tie, p.sy);
+                                        } else if (n_tie > 1) {
+#pragma unroll
+                                            for (int j = 0; j < 16; ++j) sb[j * 128 + q * 32 + lane] = conv(16 * h + j);
+                                        }
+                                    }
+                                } else {
+#pragma unroll
+                                    for (int j = 0; j < 16; ++j) sb[j * 128 + q * 32 + lane] = conv(16 * h + j);
+                                }
+                                ptx::fence_proxy_async_smem();
+                                ptx::named_bar_sync(kNarrowFull + half, 128);
+                                if (q == 0 && lane == 0) {
+                                    ptx::tma_store_2d(&tmap_y, n0, tc0 + 16 * h, ptx::smem_u32(sb));
+                                    ptx::bulk_commit_group();
+                                }
+                                ++n_stores;
+                            } else {
                                 OT* sb = reinterpret_cast<OT*>(my_stage + (NB == 2 ? (n_stores & 1u) * 512 : 0));
                                 if (lane == 0) ptx::bulk_wait_group_read<NB - 1>();  // the store that last used this tile has read it
                                 __syncwarp();
@@ -909,7 +995,7 @@ static int make_store_map(CUtensorMap* ty, const LinearArgs& a, bool* tma_store)
                                  : EPI == EPI_Q8 ? CU_TENSOR_MAP_DATA_TYPE_UINT8 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16;
     if (!*tma_store)
         return make_map(ty, a.X, (uint64_t)a.tokens, (uint64_t)W.in / 4, 16, 32, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_DATA_TYPE_INT32, 4);
-    return make_map(ty, ybase, (uint64_t)a.tokens, (uint64_t)W.out, 16, 32, CU_TENSOR_MAP_SWIZZLE_NONE, dt, es);
+    return make_map(ty, ybase, (uint64_t)a.tokens, (uint64_t)W.out, 16, kNarrow<EPI> ? 128 : 32, CU_TENSOR_MAP_SWIZZLE_NONE, dt, es);
 }
 
 template <bool SPARSE, int BN, int EPI, int WSRC>
@@ -1057,7 +1143,7 @@ static int run_linear(const LinearArgs& a, int epi) {
     if (epi == EPI_F32 && !a.Y) return NM_ERR_NULL;
     if (epi == EPI_ACC && !a.ACC) return NM_ERR_NULL;
     if ((epi == EPI_Q8 || epi == EPI_BF16) && !a.NARROW) return NM_ERR_NULL;
-    if (epi == EPI_Q8 && !(a.sy > 0.0f && a.sy <= 3.402823466e38f)) return NM_ERR_SHAPE;  // positive and finite
+    if (epi == EPI_Q8 && !(a.sy >= 1.17549435e-38f && a.sy <= 3.402823466e38f)) return NM_ERR_SHAPE;  // positive, normal, finite
     if (!aligned(a.X, 16) || !aligned(W.values, 16) || (W.meta && !aligned(W.meta, 16))) return NM_ERR_ALIGN;
     if ((a.Y && !aligned(a.Y, 4)) || (a.ACC && !aligned(a.ACC, 4))) return NM_ERR_ALIGN;
     if (epi == EPI_BF16 && !aligned(a.NARROW, 2)) return NM_ERR_ALIGN;

@@ -110,22 +110,10 @@ __device__ __forceinline__ unsigned keep_mask(const float* a) {
     return mask;
 }
 
-// Integer code of v / s: clamp(rne(fl32(v / s))).  The scale is constant along a row, so the quotient is
-// formed from the correctly rounded reciprocal r = RN(1 / s) with one FMA correction step
-// (q = v * r; q += r * (v - s * q)), which lands within an ulp or two of the IEEE quotient.  That can
-// only change the rounded integer when the quotient sits next to a half-integer: those cases (and
-// anything non-finite, e.g. a subnormal scale whose reciprocal overflows) take the true IEEE division,
-// so the result is the same bit for bit.
+// Integer code of v / s as an unsigned BITS-wide field (quantise_rn: common.cuh).
 template <int BITS>
 __device__ __forceinline__ unsigned quantise_code(float v, float s, float r) {
-    constexpr int hi = (1 << (BITS - 1)) - 1, lo = -(1 << (BITS - 1));
-    float q = __fmul_rn(v, r);
-    q = __fmaf_rn(__fmaf_rn(-s, q, v), r, q);
-    const float f = q - rintf(q);                      // in [-0.5, 0.5]
-    if (!(fabsf(f) <= 0.49996948f)) q = __fdiv_rn(v, s);  // within 2^-15 of a tie, or not finite
-    int c = __float2int_rn(q);                         // round half to even
-    c = max(lo, min(hi, c));
-    return (unsigned)c & ((1u << BITS) - 1u);
+    return (unsigned)quantise_rn<BITS>(v, s, r) & ((1u << BITS) - 1u);
 }
 
 template <int NBYTES>

@@ -83,6 +83,18 @@ __device__ __forceinline__ void named_bar_arrive(uint32_t id, uint32_t threads) 
     asm volatile("bar.arrive %0, %1;" ::"r"(id), "r"(threads) : "memory");
 }
 
+// Named barrier that also ANDs a predicate over its `threads` participants: everyone gets the same answer.
+__device__ __forceinline__ bool named_bar_and(uint32_t id, uint32_t threads, bool pred) {
+    uint32_t out;
+    asm volatile(
+        "{\n.reg .pred p, q;\n"
+        "setp.ne.u32 q, %3, 0;\n"
+        "bar.red.and.pred p, %1, %2, q;\n"
+        "selp.u32 %0, 1, 0, p;\n}\n"
+        : "=r"(out) : "r"(id), "r"(threads), "r"((uint32_t)pred) : "memory");
+    return out != 0;
+}
+
 // Makes generic-proxy writes to shared memory visible to the async proxy (TMA, tcgen05.mma).
 __device__ __forceinline__ void fence_proxy_async_smem() {
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
