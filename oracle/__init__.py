@@ -112,6 +112,18 @@ def fake_quant(Z, bits, scales):
     return Zq
 
 
+def admm_step(W, U, n, m, bits, want_u=True):
+    """-> (Z f32 like W, U_next f32 | None, scales f32 [out]): joint projection as dense fp32 + dual update."""
+    W = np.ascontiguousarray(W, dtype=np.float32)
+    U = None if U is None else np.ascontiguousarray(U, dtype=np.float32)
+    Z = np.zeros_like(W)
+    Un = np.zeros_like(W) if want_u else None
+    s = np.zeros(W.shape[0], dtype=np.float32)
+    _chk(lib().oracle_admm_step(_p(W), _p(U), W.shape[0], W.shape[1], n, m, bits, _p(Z), _p(Un), _p(s)),
+         "oracle_admm_step")
+    return Z, Un, s
+
+
 def int_linear(X, Wq, sx, sw, bias, want_acc=True, want_y=True):
     """X int8 [T, in], Wq int8 dense [out, in] -> (acc int32 [T, out] | None, Y f32 [T, out] | None)."""
     X = np.ascontiguousarray(X, dtype=np.int8)

@@ -28,6 +28,11 @@
  *   The byte-level packing of values and metadata is this library's own
  *   convention (the paper specifies none): parity unpinned beyond the
  *   pack -> unpack round trip and the 2-index-bits-per-kept-value accounting.
+ *   One ADMM step with dense outputs (joint projection Z as fp32, dual update
+ *   U + W - Z; the paper prints the projection, Eq. 3, the dual update is the
+ *   standard scaled form): pinned as the composition of the pieces above, against
+ *   the packed path, numpy's own fp32 subtraction, the constraint on Z, the
+ *   half-step bound on the dual and the fixed point Z(Z) = Z.
  *   Narrow forms of the layer's output -- Eq. 5 with a scale fixed ahead of
  *   time (8-bit activations handed to the next layer, Sec. 4.5) and binary32 ->
  *   bfloat16 rounding: pinned by closed forms (exact multiples, ties), exact
@@ -288,6 +293,46 @@ int oracle_fake_quant(const float *Z, int out, int in, int bits, const float *sc
             Zq[i] = scales[r] * (float)quantise(Z[i], scales[r], bits);
         }
     return ORACLE_OK;
+}
+
+/*
+ * One ADMM projection step for the joint constraint (Eq. 3 with the sparsity and
+ * quantisation projections solved in sequence, Sec. 3.3.1 last paragraph), dense
+ * outputs:
+ *   V = W + U;  s_r = ADMM-Max scale of row r of V;
+ *   Z = s_r * clamp(round(Pi_S(V) / s_r))     (Eq. 5 then Eq. 4, zero where pruned)
+ *   U_next = V - Z                             (scaled-form dual update U + W - Z)
+ * With U == NULL and U_next == NULL this is the forward pass of the STE
+ * fake-quantiser on a weight that is also N:M-projected (Sec. 3.3.2).
+ * scales (nullable) receives s_r.
+ */
+int oracle_admm_step(const float *W, const float *U, int out, int in, int n, int m, int bits,
+                     float *Z, float *U_next, float *scales)
+{
+    if (n < 1 || n > m || m > 64 || in % m || bits < 2 || bits > 8) return ORACLE_ERR_SHAPE;
+    float *v = (float *)malloc((size_t)in * sizeof(float));
+    if (!v) return ORACLE_ERR_SHAPE;
+    int status = ORACLE_OK;
+    for (int r = 0; r < out; ++r) {
+        size_t base = (size_t)r * in;
+        for (int k = 0; k < in; ++k) v[k] = U ? W[base + k] + U[base + k] : W[base + k];
+        if (!row_finite(v, in)) { status = ORACLE_ERR_NONFINITE; break; }
+        float s = row_scale(v, in, bits);
+        if (scales) scales[r] = s;
+        for (int g = 0; g < in / m; ++g) {
+            int keep[64];
+            for (int i = 0; i < m; ++i) Z[base + (size_t)g * m + i] = 0.0f;
+            group_support(v + (size_t)g * m, n, m, keep);
+            for (int i = 0; i < n; ++i) {
+                size_t k = (size_t)g * m + keep[i];
+                Z[base + k] = s * (float)quantise(v[k], s, bits);
+            }
+        }
+        if (U_next)
+            for (int k = 0; k < in; ++k) U_next[base + k] = v[k] - Z[base + k];
+    }
+    free(v);
+    return status;
 }
 
 /*

@@ -488,3 +488,47 @@ def test_bf16_rounding_closed_forms_and_library():
     assert np.array_equal(b, lib)
     with pytest.raises(RuntimeError):
         oracle.to_bf16(np.array([np.inf], np.float32))
+
+
+# ---- one ADMM projection step with dense outputs (joint projection + dual update) -------------------
+
+@pytest.mark.parametrize("n,m,bits", [(2, 4, 8), (2, 4, 4), (1, 4, 8), (2, 8, 4), (4, 8, 8), (4, 4, 8)])
+def test_admm_step_is_the_composition_of_the_pinned_pieces(n, m, bits):
+    rng = np.random.default_rng(31)
+    W, U = wl.normal(rng, (24, 96), 0.02), wl.normal(rng, (24, 96), 0.002)
+    Z, Un, s = oracle.admm_step(W, U, n, m, bits)
+    V = (W + U).astype(np.float32)
+    # scale, sparsity projection and fake-quantiser, each pinned on its own above
+    assert np.array_equal(s, oracle.row_scales(V, bits))
+    assert np.array_equal(Z, oracle.fake_quant(oracle.project_dense(W, U, n, m), bits, s))
+    # the same weights through the packed path: Z = s * unpack(project_pack)
+    v, meta, s2 = oracle.project_pack(W, U, n, m, bits)
+    D = oracle.unpack(v, meta, 24, 96, n, m, bits)
+    assert np.array_equal(s2, s) and np.array_equal(Z, (s[:, None] * D.astype(np.float32)).astype(np.float32))
+    # dual update U + W - Z, written here with numpy's own fp32 arithmetic
+    assert np.array_equal(Un, (V - Z).astype(np.float32))
+    # the constraint holds for Z: at most n nonzeros per group, integer multiples of the row scale within range
+    assert ((Z.reshape(24, -1, m) != 0).sum(axis=2) <= n).all()
+    codes = Z.astype(np.float64) / s[:, None].astype(np.float64)
+    assert np.all(np.abs(codes - np.rint(codes)) < 1e-4) and np.abs(np.rint(codes)).max() <= 2 ** (bits - 1) - 1
+    # what is left in the dual: the whole value where pruned, at most half a step (+ rounding) where kept
+    kept = Z != 0
+    assert np.array_equal(Un[~kept & (np.abs(V) > s[:, None] / 2)], V[~kept & (np.abs(V) > s[:, None] / 2)])
+    assert np.all(np.abs(Un[kept]) <= (0.5 * s[:, None] * (1 + 2.0 ** -20) + np.abs(V) * 2.0 ** -23)[kept])
+
+
+def test_admm_step_fixed_point_and_ste_form():
+    rng = np.random.default_rng(32)
+    W = wl.normal(rng, (16, 64), 0.02)
+    Z, Un, s = oracle.admm_step(W, None, 2, 4, 8)
+    # STE forward form: no dual in, none out; same Z
+    Z2, none, _ = oracle.admm_step(W, None, 2, 4, 8, want_u=False)
+    assert none is None and np.array_equal(Z, Z2)
+    # a weight that already meets the constraint stays put: Z(Z) has the same codes and the dual stays ~0
+    Zz, Uz, sz = oracle.admm_step(Z, None, 2, 4, 8)
+    assert np.array_equal(np.rint(Zz / sz[:, None]), np.rint(Z / s[:, None]))
+    assert np.all(np.abs(Uz) <= np.abs(Z) * 2.0 ** -22)
+    # W = Z + U_next up to the rounding of the subtraction
+    assert np.all(np.abs((Z.astype(np.float64) + Un.astype(np.float64)) - W.astype(np.float64)) <= np.abs(W) * 2.0 ** -23 + 1e-12)
+    with pytest.raises(RuntimeError):
+        oracle.admm_step(np.array([[np.inf, 0, 0, 0]], np.float32), None, 2, 4, 8)
