@@ -96,6 +96,23 @@ int nm_project_pack(const float *W, const float *U, int out, int in, int n, int 
                     void *values, void *meta, float *scales, uint32_t *status, void *stream);
 
 /*
+ * One ADMM projection step with dense outputs (Eq. 3 for the joint constraint: the sparsity and the
+ * quantisation projection solved in sequence, Sec. 3.3.1), also the forward pass of the STE
+ * fake-quantiser (Sec. 3.3.2) when U and U_next are NULL:
+ *   V = W + U (U NULL = 0);  s[r] = ADMM-Max scale of row r of V;
+ *   Z[r,k]      = s[r] * code[r,k] where (r,k) is kept, 0 where it is pruned   (Eq. 5 then Eq. 4)
+ *   U_next[r,k] = V[r,k] - Z[r,k]                  (scaled-form dual update U + W - Z; NULL = not wanted)
+ * with exactly the support, scales and codes nm_project_pack produces.  Z, U_next: device fp32
+ * [out, in] row-major, 16-byte aligned, caller-owned; U_next may alias U, Z may not alias W or U.
+ * values / meta / scales: the packed outputs of nm_project_pack, each may be NULL when not wanted.
+ * One pass over HBM: W and U read once, every output written once.  Shapes, errors and the
+ * NM_STATUS_NONFINITE bit as for nm_project_pack.
+ */
+int nm_admm_project(const float *W, const float *U, int out, int in, int n, int m, int bits, float *Z,
+                    float *U_next, void *values, void *meta, float *scales, uint32_t *status,
+                    void *stream);
+
+/*
  * The same for a list of matrices with as few launches as their (n, m, bits) allow (one when all
  * jobs share them).  `jobs` is a host array; `ws` is device scratch of at least
  * nm_pack_workspace_bytes(njobs) bytes, 16-byte aligned, which must stay untouched until the

@@ -26,7 +26,7 @@ NM_ERR_WORKSPACE, NM_ERR_CUDA, NM_ERR_NONFINITE, NM_ERR_TIMEOUT = -5, -6, -7, -8
 
 EXPORTS = (
     "nm_packed_sizes", "nm_project_pack", "nm_project_pack_batched", "nm_pack_workspace_bytes",
-    "nm_project_pack_batched_noalloc",
+    "nm_project_pack_batched_noalloc", "nm_admm_project",
     "nm_int_linear", "nm_int_linear_dsx", "nm_int_linear_acc", "nm_int_linear_q8", "nm_int_linear_bf16",
     "nm_int_linear_workspace_bytes",
     "nm_int_linear_check", "nm_absmax", "nm_quantize_act", "nm_poll_status", "nm_strerror",
@@ -52,6 +52,7 @@ _lib.nm_packed_sizes.argtypes = [_i] * 5 + [ctypes.POINTER(_sz), ctypes.POINTER(
 _lib.nm_project_pack.argtypes = [_vp, _vp, _i, _i, _i, _i, _i, _vp, _vp, _vp, _vp, _vp]
 _lib.nm_project_pack_batched.argtypes = [ctypes.POINTER(nm_pack_job_t), _i, _vp, _sz, _vp, _vp]
 _lib.nm_project_pack_batched_noalloc.argtypes = [ctypes.POINTER(nm_pack_job_t), _i, _vp, _vp]
+_lib.nm_admm_project.argtypes = [_vp, _vp, _i, _i, _i, _i, _i, _vp, _vp, _vp, _vp, _vp, _vp, _vp]
 _lib.nm_pack_workspace_bytes.argtypes = [_i]
 _lib.nm_pack_workspace_bytes.restype = _sz
 _lib.nm_int_linear.argtypes = [_vp, _i, ctypes.POINTER(nm_packed_t), _f, _vp, _vp, _vp, _vp, _sz, _vp, _vp]
@@ -149,6 +150,12 @@ def nm_project_pack_batched_noalloc(job_array, njobs, status=None, stream=None):
 
 def make_packed(out, in_, n, m, bits, values, meta):
     return nm_packed_t(out, in_, n, m, bits, values.data_ptr(), meta.data_ptr() if meta is not None else None)
+
+
+def nm_admm_project(W, U, out, in_, n, m, bits, Z, U_next=None, values=None, meta=None, scales=None,
+                    status=None, stream=None):
+    _chk(_lib.nm_admm_project(_ptr(W), _ptr(U), out, in_, n, m, bits, _ptr(Z), _ptr(U_next), _ptr(values),
+                              _ptr(meta), _ptr(scales), _ptr(status), _stream(stream)), "nm_admm_project")
 
 
 def nm_int_linear_workspace_bytes(tokens, out, in_, n, m, bits):

@@ -137,9 +137,14 @@ __device__ __forceinline__ void store_bytes_slow(uint8_t* dst, const unsigned* w
 }
 
 // N == M: dense (quantise only, no metadata), processed in groups of 4.
-template <int N, int M, int BITS, int MAXT>
-__global__ void __launch_bounds__(MAXT, MAXT == 128 ? 8 : 1) pack_kernel(const PackJobDev* __restrict__ jobs, int njobs,
-                                                    PackJobDev single, uint32_t* status) {
+// DENSE_OUT: the ADMM step / STE forward form.  Besides (or instead of: values, meta and scales may then be
+// null) the packed outputs the kernel writes Z = s * code as dense fp32, zero where pruned, and, when
+// U_next is not null, the dual update U_next = (W + U) - Z.  Both go back through the shared-memory
+// tile so that the stores are as coalesced as the loads.
+template <int N, int M, int BITS, int MAXT, bool DENSE_OUT = false>
+__global__ void __launch_bounds__(MAXT, MAXT == 128 ? (DENSE_OUT ? 4 : 8) : 1) pack_kernel(const PackJobDev* __restrict__ jobs, int njobs,
+                                                    PackJobDev single, uint32_t* status, float* __restrict__ Zout,
+                                                    float* __restrict__ Unext) {
     constexpr bool kDense = (N == M);
     constexpr int G = 32 / M;                          // groups per lane
     constexpr int F = (M == 4) ? 2 : 4;                // metadata field width
@@ -219,7 +224,7 @@ __global__ void __launch_bounds__(MAXT, MAXT == 128 ? 8 : 1) pack_kernel(const P
     // ---- ADMM-Max scale ---------------------------------------------------------------------
     constexpr float qmax = (float)((1 << (BITS - 1)) - 1);
     const float s = (amax == 0.0f) ? 1.0f : __fdiv_rn(amax, qmax);
-    if (row_ok && chunk == 0 && lane == 0) job.scales[row] = s;
+    if (row_ok && chunk == 0 && lane == 0 && (!DENSE_OUT || job.scales)) job.scales[row] = s;
     const float rs = __frcp_rn(s);  // correctly rounded reciprocal, once per row
 
     // ---- this lane's 32 consecutive values ----------------------------------------------------
@@ -231,7 +236,12 @@ __global__ void __launch_bounds__(MAXT, MAXT == 128 ? 8 : 1) pack_kernel(const P
     }
     const int lane_first = chunk * 1024 + lane * 32;             // first column of this lane
     const int nvals = max(0, min(32, job.in - lane_first));      // columns inside the row
-    if (!row_ok || nvals == 0) return;
+    if (!DENSE_OUT && (!row_ok || nvals == 0)) return;
+    float z[DENSE_OUT ? 32 : 1];  // dequantised projection of this lane's values (DENSE_OUT)
+    if constexpr (DENSE_OUT) {
+#pragma unroll
+        for (int i = 0; i < 32; ++i) z[i] = 0.0f;
+    }
 
     unsigned vw[VWORDS], mw[MWORDS];
 #pragma unroll
@@ -246,7 +256,9 @@ __global__ void __launch_bounds__(MAXT, MAXT == 128 ? 8 : 1) pack_kernel(const P
 #pragma unroll
                 for (int p = 0; p < M; ++p) {
                     const int pos = (g * M + p) * BITS;
-                    vw[pos >> 5] |= quantise_code<BITS>(v[g * M + p], s, rs) << (pos & 31);
+                    const int code = quantise_rn<BITS>(v[g * M + p], s, rs);
+                    vw[pos >> 5] |= ((unsigned)code & ((1u << BITS) - 1u)) << (pos & 31);
+                    if constexpr (DENSE_OUT) z[g * M + p] = __fmul_rn(s, (float)code);
                 }
             } else {
                 float sel[N];
@@ -292,23 +304,55 @@ __global__ void __launch_bounds__(MAXT, MAXT == 128 ? 8 : 1) pack_kernel(const P
 #pragma unroll
                 for (int c = 0; c < N; ++c) {
                     const int vpos = (g * N + c) * BITS, mpos = (g * N + c) * F;
-                    vw[vpos >> 5] |= quantise_code<BITS>(sel[c], s, rs) << (vpos & 31);
+                    const int code = quantise_rn<BITS>(sel[c], s, rs);
+                    vw[vpos >> 5] |= ((unsigned)code & ((1u << BITS) - 1u)) << (vpos & 31);
                     mw[mpos >> 5] |= selp[c] << (mpos & 31);
+                    if constexpr (DENSE_OUT) {
+                        const float zc = __fmul_rn(s, (float)code);
+#pragma unroll
+                        for (int p = 0; p < M; ++p) z[g * M + p] = (selp[c] == (unsigned)p) ? zc : z[g * M + p];
+                    }
                 }
             }
         }
     }
 
+    // ---- dense outputs (ADMM step): back through the tile, then coalesced 16-byte stores --------
+    if constexpr (DENSE_OUT) {
+        auto write_back = [&](const float* x, float* dst_base) {
+#pragma unroll
+            for (int jj = 0; jj < 8; ++jj)
+                mytile[lane * 8 + (jj ^ (lane & 7))] = make_float4(x[jj * 4], x[jj * 4 + 1], x[jj * 4 + 2], x[jj * 4 + 3]);
+            __syncwarp();
+            float4* D4 = reinterpret_cast<float4*>(dst_base) + (row_ok ? row * in4 : 0);
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+                const int fl = j * 32 + lane, owner = fl >> 3, jj = fl & 7, f = chunk * 256 + fl;
+                const float4 t = mytile[owner * 8 + (jj ^ (owner & 7))];
+                if (row_ok && f < in4) __stcs(D4 + f, t);
+            }
+            __syncwarp();
+        };
+        write_back(z, Zout);
+        if (Unext) {
+#pragma unroll
+            for (int i = 0; i < 32; ++i) v[i] = __fsub_rn(v[i], z[i]);  // (W + U) - Z
+            write_back(v, Unext);
+        }
+        if (!row_ok || nvals == 0) return;
+    }
+
     // ---- stores -----------------------------------------------------------------------------
     const int lane_global = chunk * 32 + lane;
     const bool full = (nvals == 32);
-    {
+    if (!DENSE_OUT || job.values) {
         constexpr int LB = VBITS / 8;
         uint8_t* dst = job.values + (size_t)row * job.vrow_bytes + (size_t)lane_global * LB;
         if (full && (reinterpret_cast<uintptr_t>(dst) % (LB < 16 ? LB : 16)) == 0) store_bytes_vec<LB>(dst, vw);
         else store_bytes_slow<LB>(dst, vw, nvals / M * N * BITS / 8);
     }
     if constexpr (!kDense) {
+        if (DENSE_OUT && !job.meta) return;
         constexpr int MB = MBITS / 8;
         const unsigned lane_off = (unsigned)lane_global * MB;
         const unsigned row_bytes = job.mrow_words * 4u;
@@ -327,21 +371,22 @@ __global__ void __launch_bounds__(MAXT, MAXT == 128 ? 8 : 1) pack_kernel(const P
 // ---------------------------------------------------------------------------------------------
 // host side
 // ---------------------------------------------------------------------------------------------
-using PackFn = void (*)(const PackJobDev*, int, PackJobDev, uint32_t*);
+using PackFn = void (*)(const PackJobDev*, int, PackJobDev, uint32_t*, float*, float*);
 
-template <int N, int M>
+template <int N, int M, bool DENSE_OUT>
 static PackFn pick_bits(int bits, int warps) {
     if (warps <= kPackMinWarps)
-        return bits == 8 ? (PackFn)pack_kernel<N, M, 8, 128> : (PackFn)pack_kernel<N, M, 4, 128>;
-    return bits == 8 ? (PackFn)pack_kernel<N, M, 8, 1024> : (PackFn)pack_kernel<N, M, 4, 1024>;
+        return bits == 8 ? (PackFn)pack_kernel<N, M, 8, 128, DENSE_OUT> : (PackFn)pack_kernel<N, M, 4, 128, DENSE_OUT>;
+    return bits == 8 ? (PackFn)pack_kernel<N, M, 8, 1024, DENSE_OUT> : (PackFn)pack_kernel<N, M, 4, 1024, DENSE_OUT>;
 }
 
+template <bool DENSE_OUT = false>
 static PackFn pick_kernel(int n, int m, int bits, int warps) {
-    if (n == m) return pick_bits<4, 4>(bits, warps);
-    if (m == 4) return n == 1 ? pick_bits<1, 4>(bits, warps) : pick_bits<2, 4>(bits, warps);
-    if (n == 1) return pick_bits<1, 8>(bits, warps);
-    if (n == 2) return pick_bits<2, 8>(bits, warps);
-    return pick_bits<4, 8>(bits, warps);
+    if (n == m) return pick_bits<4, 4, DENSE_OUT>(bits, warps);
+    if (m == 4) return n == 1 ? pick_bits<1, 4, DENSE_OUT>(bits, warps) : pick_bits<2, 4, DENSE_OUT>(bits, warps);
+    if (n == 1) return pick_bits<1, 8, DENSE_OUT>(bits, warps);
+    if (n == 2) return pick_bits<2, 8, DENSE_OUT>(bits, warps);
+    return pick_bits<4, 8, DENSE_OUT>(bits, warps);
 }
 
 static int validate_job(const nm_pack_job_t& j) {
@@ -374,11 +419,12 @@ static PackJobDev to_dev(const nm_pack_job_t& j) {
 }
 
 static int launch(PackFn fn, const PackJobDev* jobs_dev, int njobs, const PackJobDev& single,
-                  unsigned blocks, int warps, uint32_t* status, cudaStream_t stream) {
+                  unsigned blocks, int warps, uint32_t* status, cudaStream_t stream,
+                  float* Z = nullptr, float* U_next = nullptr) {
     size_t smem = (size_t)warps * (256 * sizeof(float4) + sizeof(float));
     if (smem > 48 * 1024)
         NM_CUDA_TRY(cudaFuncSetAttribute((const void*)fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    fn<<<blocks, warps * 32, smem, stream>>>(jobs_dev, njobs, single, status);
+    fn<<<blocks, warps * 32, smem, stream>>>(jobs_dev, njobs, single, status, Z, U_next);
     NM_CUDA_TRY(cudaGetLastError());
     return NM_OK;
 }
@@ -398,6 +444,26 @@ int nm_project_pack(const float* W, const float* U, int out, int in, int n, int 
     int rows_per_block = warps >> d.wpr_log2;
     unsigned blocks = (unsigned)((out + rows_per_block - 1) / rows_per_block);
     return nm::launch(nm::pick_kernel(n, m, bits, warps), nullptr, 0, d, blocks, warps, status, (cudaStream_t)stream);
+}
+
+int nm_admm_project(const float* W, const float* U, int out, int in, int n, int m, int bits, float* Z,
+                    float* U_next, void* values, void* meta, float* scales, uint32_t* status, void* stream) {
+    int rc = nm::check_pattern(out, in, n, m, bits);
+    if (rc != NM_OK) return rc;
+    if (!W || !Z) return NM_ERR_NULL;
+    if (in % 4) return NM_ERR_SHAPE;
+    if (in > 32768) return NM_ERR_UNSUPPORTED;
+    if (!nm::aligned(W, 16) || (U && !nm::aligned(U, 16)) || !nm::aligned(Z, 16) || (U_next && !nm::aligned(U_next, 16)) ||
+        (values && !nm::aligned(values, 16)) || (meta && !nm::aligned(meta, 4)) || (scales && !nm::aligned(scales, 4)))
+        return NM_ERR_ALIGN;
+    if (out == 0 || in == 0) return NM_OK;
+    nm_pack_job_t j{W, U, out, in, n, m, bits, values, meta, scales};
+    nm::PackJobDev d = nm::to_dev(j);
+    int warps = std::max(nm::kPackMinWarps, 1 << d.wpr_log2);
+    int rows_per_block = warps >> d.wpr_log2;
+    unsigned blocks = (unsigned)((out + rows_per_block - 1) / rows_per_block);
+    return nm::launch(nm::pick_kernel<true>(n, m, bits, warps), nullptr, 0, d, blocks, warps, status,
+                      (cudaStream_t)stream, Z, U_next);
 }
 
 size_t nm_pack_workspace_bytes(int njobs) {

@@ -1,0 +1,111 @@
+"""GPU parity: one ADMM projection step with dense outputs (nm_admm_project) against the CPU oracle.
+
+Z (dequantised joint projection), U_next (dual update) and the optional packed outputs are compared bit
+for bit: both sides round the same operations (fp32 add, IEEE division and round-half-even inside the
+quantiser, one multiply s * code, one subtract).
+"""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import workloads as wl
+
+pytestmark = pytest.mark.gpu
+
+PATTERNS = [(1, 4), (2, 4), (1, 8), (2, 8), (4, 8), (4, 4)]
+
+
+def _gpu_admm(W, U, n, m, bits, want_u=True, want_packed=True):
+    import paper_2206_15014_b200 as nm
+    from gpu_util import to_dev, DEV
+    out, k = W.shape
+    Wd, Ud = to_dev(W), to_dev(U)
+    Z = torch.full((out + 1, k), float("nan"), dtype=torch.float32, device=DEV)       # one guard row
+    Un = torch.full((out + 1, k), float("nan"), dtype=torch.float32, device=DEV) if want_u else None
+    status = torch.zeros(1, dtype=torch.int32, device=DEV)
+    vb, mb = nm.nm_packed_sizes(out, k, n, m, bits)
+    values = torch.zeros(vb, dtype=torch.uint8, device=DEV) if want_packed else None
+    meta = torch.zeros(max(mb // 4, 1), dtype=torch.int32, device=DEV) if want_packed else None
+    scales = torch.zeros(out, dtype=torch.float32, device=DEV) if want_packed else None
+    nm.nm_admm_project(Wd, Ud, out, k, n, m, bits, Z, Un, values, meta if n != m else None, scales, status=status)
+    rc = nm.nm_poll_status(status)
+    Zh = Z.cpu().numpy()
+    assert np.isnan(Zh[out]).all(), "Z written past the last row"
+    Unh = None
+    if want_u:
+        Unh = Un.cpu().numpy()
+        assert np.isnan(Unh[out]).all(), "U_next written past the last row"
+        Unh = Unh[:out]
+    packed = None
+    if want_packed:
+        packed = (values.cpu().numpy(), meta.cpu().numpy().view(np.uint32)[: mb // 4], scales.cpu().numpy())
+    return Zh[:out], Unh, packed, rc
+
+
+def _check(W, U, n, m, bits):
+    Z, Un, packed, rc = _gpu_admm(W, U, n, m, bits)
+    assert rc == 0
+    Zr, Unr, sr = oracle.admm_step(W, U, n, m, bits)
+    assert np.array_equal(Z, Zr), f"Z differs in {(Z != Zr).sum()} of {Z.size}"
+    assert np.array_equal(Un, Unr), f"U_next differs in {(Un != Unr).sum()} of {Un.size}"
+    v_ref, meta_ref, s_ref = oracle.project_pack(W, U, n, m, bits)
+    assert np.array_equal(packed[2], s_ref) and np.array_equal(packed[0], np.asarray(v_ref).reshape(-1))
+    if n != m:
+        assert np.array_equal(packed[1], np.asarray(meta_ref).reshape(-1))
+
+
+@pytest.mark.parametrize("n,m", PATTERNS)
+@pytest.mark.parametrize("bits", [8, 4])
+def test_admm_step_bert_rows(n, m, bits):
+    oracle.set_threads(oracle.max_threads())
+    for seed, (out, k) in enumerate([(260, 1024), (70, 4096), (133, 768), (37, 3072)]):
+        W, U = wl.pack_sweep_matrix(3, seed, out, k)
+        _check(W, U, n, m, bits)
+
+
+@pytest.mark.parametrize("n,m", PATTERNS)
+@pytest.mark.parametrize("bits", [8, 4])
+def test_admm_step_ragged_ties_and_wide_rows(n, m, bits):
+    for seed, (out, k) in enumerate([(5, 8), (3, 40), (9, 1032), (6, 2072), (2, 8200), (2, 16384 + 64)]):
+        if (k // m * n * bits) % 8:
+            k *= 2
+        _check(wl.with_outliers(210 + seed, out, k), wl.tie_heavy(220 + seed, out, k, levels=1), n, m, bits)
+        _check(wl.tie_heavy(200 + seed, out, k), None, n, m, bits)
+
+
+def test_ste_forward_form_and_optional_outputs():
+    # no dual in, none out, no packed outputs: the fake-quantised, N:M-projected weight alone
+    W = wl.normal(np.random.default_rng(230), (300, 1024), 0.02)
+    Z, Un, packed, rc = _gpu_admm(W, None, 2, 4, 8, want_u=False, want_packed=False)
+    assert rc == 0 and Un is None and packed is None
+    Zr, _, _ = oracle.admm_step(W, None, 2, 4, 8, want_u=False)
+    assert np.array_equal(Z, Zr)
+    # fixed point: projecting Z again reproduces it (same codes; the scale may move by an ulp) and leaves ~0 in the dual
+    Z2, U2, _, _ = _gpu_admm(Z, None, 2, 4, 8)
+    Z2r, U2r, _ = oracle.admm_step(Z, None, 2, 4, 8)
+    assert np.array_equal(Z2, Z2r) and np.array_equal(U2, U2r)
+    assert np.all(np.abs(U2) <= np.abs(Z) * 2.0 ** -22)
+
+
+def test_admm_step_in_place_dual_and_errors():
+    import paper_2206_15014_b200 as nm
+    from gpu_util import to_dev, DEV
+    W, U = wl.pack_sweep_matrix(3, 7, 128, 1024)
+    Wd, Ud = to_dev(W), to_dev(U)
+    Z = torch.empty((128, 1024), dtype=torch.float32, device=DEV)
+    nm.nm_admm_project(Wd, Ud, 128, 1024, 2, 4, 8, Z, Ud)        # U_next written over U
+    torch.cuda.synchronize()
+    Zr, Unr, _ = oracle.admm_step(W, U, 2, 4, 8)
+    assert np.array_equal(Z.cpu().numpy(), Zr) and np.array_equal(Ud.cpu().numpy(), Unr)
+    with pytest.raises(nm.NmError):
+        nm.nm_admm_project(Wd, None, 128, 1024, 2, 4, 8, None)       # Z is required
+    with pytest.raises(nm.NmError):
+        nm.nm_admm_project(Wd, None, 128, 1022, 2, 4, 8, Z)          # in % m != 0
+    with pytest.raises(nm.NmError):
+        nm.nm_admm_project(Wd, None, 128, 1024, 3, 4, 8, Z)          # unsupported pattern
+    # non-finite input raises the status bit
+    Wbad = W.copy(); Wbad[5, 17] = np.inf
+    status = torch.zeros(1, dtype=torch.int32, device=DEV)
+    nm.nm_admm_project(to_dev(Wbad), None, 128, 1024, 2, 4, 8, Z, status=status)
+    assert nm.nm_poll_status(status) == nm.NM_ERR_NONFINITE
