@@ -227,6 +227,26 @@ const char *nm_strerror(int code);
 /* Text of the last CUDA error this thread met inside the library (static storage, "" if none). */
 const char *nm_last_cuda_error(void);
 
+/*
+ * Cost model behind the paper's size and FLOP columns (Table 1, Table 4; Sec. 4: a compression
+ * scheme is scored without running it).  Host-only arithmetic.
+ *   nm_bits_per_param: stored bits per dense parameter of an n:m sparse b-bit matrix = n/m * (bits +
+ *     index_bits); dense (n == m): bits.  index_bits < 0 selects this library's metadata field (2 for
+ *     m = 4, 4 for m = 8); the paper's tables use 2 at m = 4; 0 gives the headline ratios that ignore
+ *     metadata.  Returns -1 for an invalid pattern.
+ *   nm_encoder_cost: one encoder whose six linear components (Q, K, V, attention output, FFN1, FFN2,
+ *     in this order; relative sizes 1, 1, 1, 1, 4, 4) each have their own (n, m, bits):
+ *     *compression = 1 - stored bits / (32 bits per parameter), *mac_reduction = fraction of the dense
+ *     multiply-accumulates saved (one half for every component that runs on the 2-of-4 sparse path:
+ *     1:4, 2:4, 1:8, 2:8; nothing for dense and 4:8).  Either output may be NULL.
+ */
+typedef struct {
+    int32_t n, m, bits;
+} nm_component_cfg_t;
+double nm_bits_per_param(int n, int m, int bits, int index_bits);
+int nm_encoder_cost(const nm_component_cfg_t *cfg /* [6], host */, int index_bits, double *compression,
+                    double *mac_reduction);
+
 /* Library version, major * 100 + minor. */
 int nm_version(void);
 

@@ -30,7 +30,7 @@ EXPORTS = (
     "nm_int_linear", "nm_int_linear_dsx", "nm_int_linear_acc", "nm_int_linear_q8", "nm_int_linear_bf16",
     "nm_int_linear_workspace_bytes",
     "nm_int_linear_check", "nm_absmax", "nm_quantize_act", "nm_poll_status", "nm_strerror",
-    "nm_last_cuda_error", "nm_version",
+    "nm_last_cuda_error", "nm_version", "nm_bits_per_param", "nm_encoder_cost",
 )
 
 
@@ -66,6 +66,8 @@ _lib.nm_int_linear_check.argtypes = [_i] * 6
 _lib.nm_absmax.argtypes = [_vp, _sz, _vp, _vp]
 _lib.nm_quantize_act.argtypes = [_vp, _sz, _vp, _vp, _vp, _vp]
 _lib.nm_poll_status.argtypes = [_vp, _vp]
+_lib.nm_bits_per_param.argtypes = [_i] * 4
+_lib.nm_bits_per_param.restype = ctypes.c_double
 _lib.nm_strerror.argtypes = [_i]
 _lib.nm_strerror.restype = ctypes.c_char_p
 _lib.nm_last_cuda_error.restype = ctypes.c_char_p
@@ -192,6 +194,22 @@ def nm_int_linear_bf16(X, tokens, W, sx, sw, bias, Ybf16, ws=None, ws_bytes=0, s
     _chk(_lib.nm_int_linear_bf16(_ptr(X), tokens, ctypes.byref(W), float(sx), _ptr(sw), _ptr(bias),
                                  _ptr(Ybf16), _ptr(ws), ws_bytes, _ptr(status), _stream(stream)),
          "nm_int_linear_bf16")
+
+
+class nm_component_cfg_t(ctypes.Structure):
+    _fields_ = [("n", ctypes.c_int32), ("m", ctypes.c_int32), ("bits", ctypes.c_int32)]
+
+
+def nm_bits_per_param(n, m, bits, index_bits=-1):
+    return float(_lib.nm_bits_per_param(n, m, bits, index_bits))
+
+
+def nm_encoder_cost(cfg, index_bits=-1):
+    """cfg: six (n, m, bits) for Q, K, V, attention output, FFN1, FFN2 -> (compression, mac_reduction)."""
+    arr = (nm_component_cfg_t * 6)(*[nm_component_cfg_t(*c) for c in cfg])
+    comp, red = ctypes.c_double(), ctypes.c_double()
+    _chk(_lib.nm_encoder_cost(arr, index_bits, ctypes.byref(comp), ctypes.byref(red)), "nm_encoder_cost")
+    return comp.value, red.value
 
 
 def nm_absmax(Y, count, absmax, stream=None):

@@ -75,6 +75,32 @@ const char* nm_strerror(int code) {
 
 const char* nm_last_cuda_error(void) { return nm::g_last_error; }
 
-int nm_version(void) { return 100; }
+double nm_bits_per_param(int n, int m, int bits, int index_bits) {
+    if (n < 1 || m < 1 || n > m || bits < 1) return -1.0;
+    if (n == m) return (double)bits;  // dense: no index metadata
+    const int ib = index_bits < 0 ? nm::meta_field_bits(m) : index_bits;
+    return (double)n * (double)(bits + ib) / (double)m;
+}
+
+int nm_encoder_cost(const nm_component_cfg_t* cfg, int index_bits, double* compression, double* mac_reduction) {
+    if (!cfg) return NM_ERR_NULL;
+    // Q, K, V and the attention output are hidden x hidden, the two feed-forward matrices 4 x that
+    static const int units[6] = {1, 1, 1, 1, 4, 4};
+    double bits = 0.0, saved = 0.0;
+    for (int i = 0; i < 6; ++i) {
+        const double b = nm_bits_per_param(cfg[i].n, cfg[i].m, cfg[i].bits, index_bits);
+        if (b < 0.0) return NM_ERR_SHAPE;
+        bits += units[i] * b;
+        // a pattern that always fits the 2-of-4 hardware form (at most two kept values in any aligned chunk of
+        // four: 1:4, 2:4, 1:8, 2:8) executes half of the dense multiply-accumulates
+        const bool sparse_path = cfg[i].n != cfg[i].m && cfg[i].n <= 2 && (cfg[i].m == 4 || cfg[i].m == 8);
+        if (sparse_path) saved += 0.5 * units[i];
+    }
+    if (compression) *compression = 1.0 - bits / (12.0 * 32.0);
+    if (mac_reduction) *mac_reduction = saved / 12.0;
+    return NM_OK;
+}
+
+int nm_version(void) { return 101; }
 
 }  // extern "C"

@@ -39,3 +39,32 @@ def test_host_only_entry_points():
     for code in range(-8, 1):
         assert nm.nm_strerror(code) != "unknown nmsparse code"
     assert nm.nm_int_linear_check(4096, 768, 768, 2, 4, 8) == nm.NM_OK
+
+
+def test_cost_model_reproduces_the_paper_tables():
+    # the library's own cost model against the size / FLOP columns the paper prints (Table 1, Table 4
+    # and the headline ratios), read from the golden file
+    entry.build()
+    import paper_2206_15014_b200 as nm
+    rows = [ln.split() for ln in open(os.path.join(ROOT, "tests", "golden", "paper_tables.txt")) if ln.strip() and not ln.startswith("#")]
+    cfg_of = {"Q4": (4, 4, 4), "Q8": (4, 4, 8), "S4": (2, 4, 4), "S8": (2, 4, 8)}
+    seen = 0
+    for r in rows:
+        if r[0] != "table4":
+            continue
+        comp, red = nm.nm_encoder_cost([cfg_of[c] for c in r[2:8]], index_bits=2)
+        assert round(100 * comp, 1) == float(r[8]), r
+        if r[9] != "-":
+            assert round(100 * red, 1) == float(r[9]), r
+        seen += 1
+    assert seen >= 8
+    head = {r[1]: float(r[2]) for r in rows if r[0] == "headline"}
+    assert 100 * (1 - nm.nm_bits_per_param(2, 4, 4, 0) / 32) == head["sparse_q4"]
+    assert 100 * (1 - nm.nm_bits_per_param(4, 4, 4) / 32) == head["dense_q4"]
+    # stored sizes agree with the model at this library's field widths
+    for n, m, bits in [(2, 4, 8), (1, 4, 4), (2, 8, 8), (1, 8, 4), (4, 8, 8), (4, 4, 4)]:
+        vb, mb = nm.nm_packed_sizes(768, 3072, n, m, bits)
+        assert (vb + mb) * 8 == 768 * 3072 * nm.nm_bits_per_param(n, m, bits)
+    assert nm.nm_bits_per_param(3, 2, 8) == -1.0
+    # 1:4 and 2:8 run on the 2-of-4 path, 4:8 does not
+    assert nm.nm_encoder_cost([(1, 4, 8)] * 6)[1] == 0.5 and nm.nm_encoder_cost([(4, 8, 8)] * 6)[1] == 0.0
