@@ -113,6 +113,26 @@ int nm_admm_project(const float *W, const float *U, int out, int in, int n, int 
                     void *stream);
 
 /*
+ * The same for many matrices with one launch per group of jobs that share (n, m, bits) and block
+ * size.  `jobs`: host array of host structs holding device pointers, with the meaning of
+ * nm_admm_project's arguments; `ws`: device scratch of at least nm_admm_workspace_bytes(njobs)
+ * bytes, 16-byte aligned, caller-owned, reusable once the stream has passed the call.
+ */
+typedef struct nm_admm_job_t {
+    const float *W;
+    const float *U; /* NULL: project W alone */
+    int32_t out, in, n, m, bits;
+    float *Z;
+    float *U_next; /* NULL: not wanted; may be U */
+    void *values;  /* packed outputs: each NULL when not wanted */
+    void *meta;
+    float *scales;
+} nm_admm_job_t;
+size_t nm_admm_workspace_bytes(int njobs);
+int nm_admm_project_batched(const nm_admm_job_t *jobs, int njobs, void *ws, size_t ws_bytes,
+                            uint32_t *status, void *stream);
+
+/*
  * The same for a list of matrices with as few launches as their (n, m, bits) allow (one when all
  * jobs share them).  `jobs` is a host array; `ws` is device scratch of at least
  * nm_pack_workspace_bytes(njobs) bytes, 16-byte aligned, which must stay untouched until the

@@ -26,7 +26,7 @@ NM_ERR_WORKSPACE, NM_ERR_CUDA, NM_ERR_NONFINITE, NM_ERR_TIMEOUT = -5, -6, -7, -8
 
 EXPORTS = (
     "nm_packed_sizes", "nm_project_pack", "nm_project_pack_batched", "nm_pack_workspace_bytes",
-    "nm_project_pack_batched_noalloc", "nm_admm_project",
+    "nm_project_pack_batched_noalloc", "nm_admm_project", "nm_admm_project_batched", "nm_admm_workspace_bytes",
     "nm_int_linear", "nm_int_linear_dsx", "nm_int_linear_acc", "nm_int_linear_q8", "nm_int_linear_bf16",
     "nm_int_linear_workspace_bytes",
     "nm_int_linear_check", "nm_absmax", "nm_quantize_act", "nm_poll_status", "nm_strerror",
@@ -47,12 +47,22 @@ class nm_pack_job_t(ctypes.Structure):
                 ("scales", ctypes.c_void_p)]
 
 
+class nm_admm_job_t(ctypes.Structure):
+    _fields_ = [("W", ctypes.c_void_p), ("U", ctypes.c_void_p), ("out", ctypes.c_int32),
+                ("in_", ctypes.c_int32), ("n", ctypes.c_int32), ("m", ctypes.c_int32),
+                ("bits", ctypes.c_int32), ("Z", ctypes.c_void_p), ("U_next", ctypes.c_void_p),
+                ("values", ctypes.c_void_p), ("meta", ctypes.c_void_p), ("scales", ctypes.c_void_p)]
+
+
 _vp, _i, _sz, _f = ctypes.c_void_p, ctypes.c_int, ctypes.c_size_t, ctypes.c_float
 _lib.nm_packed_sizes.argtypes = [_i] * 5 + [ctypes.POINTER(_sz), ctypes.POINTER(_sz)]
 _lib.nm_project_pack.argtypes = [_vp, _vp, _i, _i, _i, _i, _i, _vp, _vp, _vp, _vp, _vp]
 _lib.nm_project_pack_batched.argtypes = [ctypes.POINTER(nm_pack_job_t), _i, _vp, _sz, _vp, _vp]
 _lib.nm_project_pack_batched_noalloc.argtypes = [ctypes.POINTER(nm_pack_job_t), _i, _vp, _vp]
+_lib.nm_admm_project_batched.argtypes = [ctypes.POINTER(nm_admm_job_t), _i, _vp, _sz, _vp, _vp]
 _lib.nm_admm_project.argtypes = [_vp, _vp, _i, _i, _i, _i, _i, _vp, _vp, _vp, _vp, _vp, _vp, _vp]
+_lib.nm_admm_workspace_bytes.argtypes = [_i]
+_lib.nm_admm_workspace_bytes.restype = _sz
 _lib.nm_pack_workspace_bytes.argtypes = [_i]
 _lib.nm_pack_workspace_bytes.restype = _sz
 _lib.nm_int_linear.argtypes = [_vp, _i, ctypes.POINTER(nm_packed_t), _f, _vp, _vp, _vp, _vp, _sz, _vp, _vp]
@@ -158,6 +168,24 @@ def nm_admm_project(W, U, out, in_, n, m, bits, Z, U_next=None, values=None, met
                     status=None, stream=None):
     _chk(_lib.nm_admm_project(_ptr(W), _ptr(U), out, in_, n, m, bits, _ptr(Z), _ptr(U_next), _ptr(values),
                               _ptr(meta), _ptr(scales), _ptr(status), _stream(stream)), "nm_admm_project")
+
+
+def nm_admm_workspace_bytes(njobs):
+    return int(_lib.nm_admm_workspace_bytes(njobs))
+
+
+def make_admm_jobs(jobs):
+    """jobs: iterable of (W, U, n, m, bits, Z, U_next, values, meta, scales) tensors / None -> ctypes array."""
+    dp = lambda t: None if t is None else t.data_ptr()
+    arr = (nm_admm_job_t * len(jobs))()
+    for i, (W, U, n, m, bits, Z, Un, v, mt, sc) in enumerate(jobs):
+        arr[i] = nm_admm_job_t(dp(W), dp(U), W.shape[0], W.shape[1], n, m, bits, dp(Z), dp(Un), dp(v), dp(mt), dp(sc))
+    return arr
+
+
+def nm_admm_project_batched(jobs, njobs, ws, ws_bytes, status=None, stream=None):
+    _chk(_lib.nm_admm_project_batched(jobs, njobs, _ptr(ws), ws_bytes, _ptr(status), _stream(stream)),
+         "nm_admm_project_batched")
 
 
 def nm_int_linear_workspace_bytes(tokens, out, in_, n, m, bits):

@@ -27,6 +27,12 @@ struct PackJobDev {
     unsigned mrow_words;  // words of one row of metadata
 };
 
+// Dense outputs of one job of a batched ADMM step (parallel to the PackJobDev table).
+struct DenseOutDev {
+    float* Z;
+    float* U_next;
+};
+
 static constexpr int kPackMinWarps = 4;
 
 __device__ __forceinline__ float4 ld_stream(const float4* p) { return __ldcs(p); }
@@ -144,7 +150,7 @@ __device__ __forceinline__ void store_bytes_slow(uint8_t* dst, const unsigned* w
 template <int N, int M, int BITS, int MAXT, bool DENSE_OUT = false>
 __global__ void __launch_bounds__(MAXT, MAXT == 128 ? (DENSE_OUT ? 4 : 8) : 1) pack_kernel(const PackJobDev* __restrict__ jobs, int njobs,
                                                     PackJobDev single, uint32_t* status, float* __restrict__ Zout,
-                                                    float* __restrict__ Unext) {
+                                                    float* __restrict__ Unext, const DenseOutDev* __restrict__ dense_jobs) {
     constexpr bool kDense = (N == M);
     constexpr int G = 32 / M;                          // groups per lane
     constexpr int F = (M == 4) ? 2 : 4;                // metadata field width
@@ -165,6 +171,7 @@ __global__ void __launch_bounds__(MAXT, MAXT == 128 ? (DENSE_OUT ? 4 : 8) : 1) p
             if (jobs[mid].unit_begin <= blockIdx.x) lo = mid; else hi = mid - 1;
         }
         job = jobs[lo];
+        if constexpr (DENSE_OUT) { Zout = dense_jobs[lo].Z; Unext = dense_jobs[lo].U_next; }
     } else {
         job = single;
     }
@@ -371,7 +378,7 @@ __global__ void __launch_bounds__(MAXT, MAXT == 128 ? (DENSE_OUT ? 4 : 8) : 1) p
 // ---------------------------------------------------------------------------------------------
 // host side
 // ---------------------------------------------------------------------------------------------
-using PackFn = void (*)(const PackJobDev*, int, PackJobDev, uint32_t*, float*, float*);
+using PackFn = void (*)(const PackJobDev*, int, PackJobDev, uint32_t*, float*, float*, const DenseOutDev*);
 
 template <int N, int M, bool DENSE_OUT>
 static PackFn pick_bits(int bits, int warps) {
@@ -420,12 +427,83 @@ static PackJobDev to_dev(const nm_pack_job_t& j) {
 
 static int launch(PackFn fn, const PackJobDev* jobs_dev, int njobs, const PackJobDev& single,
                   unsigned blocks, int warps, uint32_t* status, cudaStream_t stream,
-                  float* Z = nullptr, float* U_next = nullptr) {
+                  float* Z = nullptr, float* U_next = nullptr, const DenseOutDev* dense_jobs = nullptr) {
     size_t smem = (size_t)warps * (256 * sizeof(float4) + sizeof(float));
     if (smem > 48 * 1024)
         NM_CUDA_TRY(cudaFuncSetAttribute((const void*)fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    fn<<<blocks, warps * 32, smem, stream>>>(jobs_dev, njobs, single, status, Z, U_next);
+    fn<<<blocks, warps * 32, smem, stream>>>(jobs_dev, njobs, single, status, Z, U_next, dense_jobs);
     NM_CUDA_TRY(cudaGetLastError());
+    return NM_OK;
+}
+
+// Shared by the batched entry points: groups the jobs that can share one launch (same pattern, code width
+// and block size), writes the device job table(s) into `ws` and launches one kernel per group.
+template <bool DENSE_OUT>
+static int launch_batched(const nm_pack_job_t* jobs, const DenseOutDev* dense, int njobs, void* ws,
+                          uint32_t* status, cudaStream_t s) {
+    // Group jobs that can share one launch: same (n == m ? dense : n, m), bits and block size.
+    struct Key { int n, m, bits, warps; };
+    std::vector<Key> keys;
+    std::vector<std::vector<int>> groups;
+    for (int i = 0; i < njobs; ++i) {
+        const nm_pack_job_t& j = jobs[i];
+        if (j.out == 0 || j.in == 0) continue;
+        Key k{j.n == j.m ? 4 : j.n, j.n == j.m ? 4 : j.m, j.bits,
+              std::max(nm::kPackMinWarps, 1 << nm::wpr_log2_of(j.in))};
+        size_t g = 0;
+        for (; g < keys.size(); ++g)
+            if (keys[g].n == k.n && keys[g].m == k.m && keys[g].bits == k.bits && keys[g].warps == k.warps) break;
+        if (g == keys.size()) { keys.push_back(k); groups.emplace_back(); }
+        groups[g].push_back(i);
+    }
+    std::vector<nm::PackJobDev> table;
+    std::vector<DenseOutDev> dense_table;  // same order as `table`
+    table.reserve(njobs);
+    std::vector<unsigned> group_blocks(keys.size());
+    std::vector<size_t> group_first(keys.size());
+    for (size_t g = 0; g < keys.size(); ++g) {
+        unsigned blocks = 0;
+        group_first[g] = table.size();
+        for (int i : groups[g]) {
+            nm::PackJobDev d = nm::to_dev(jobs[i]);
+            int rows_per_block = keys[g].warps >> d.wpr_log2;
+            d.unit_begin = blocks;
+            unsigned long long nb = ((unsigned long long)d.out + rows_per_block - 1) / rows_per_block;
+            if (blocks + nb > 0x7fffffffull) return NM_ERR_UNSUPPORTED;
+            blocks += (unsigned)nb;
+            table.push_back(d);
+            if (DENSE_OUT) dense_table.push_back(dense[i]);
+        }
+        group_blocks[g] = blocks;
+    }
+    // Pageable-source async copies are staged before the call returns, so `table` may go away.
+    NM_CUDA_TRY(cudaMemcpyAsync(ws, table.data(), table.size() * sizeof(nm::PackJobDev),
+                                cudaMemcpyHostToDevice, s));
+    // the dense-output table follows the job table (njobs entries were reserved for each)
+    DenseOutDev* dense_dev = reinterpret_cast<DenseOutDev*>(reinterpret_cast<PackJobDev*>(ws) + njobs);
+    if (DENSE_OUT)
+        NM_CUDA_TRY(cudaMemcpyAsync(dense_dev, dense_table.data(), dense_table.size() * sizeof(DenseOutDev),
+                                    cudaMemcpyHostToDevice, s));
+    for (size_t g = 0; g < keys.size(); ++g) {
+        const nm::PackJobDev* dev = reinterpret_cast<const nm::PackJobDev*>(ws) + group_first[g];
+        int rc = nm::launch(nm::pick_kernel<DENSE_OUT>(keys[g].n, keys[g].m, keys[g].bits, keys[g].warps), dev,
+                            (int)groups[g].size(), nm::PackJobDev{}, group_blocks[g], keys[g].warps,
+                            status, s, nullptr, nullptr, DENSE_OUT ? dense_dev + group_first[g] : nullptr);
+        if (rc != NM_OK) return rc;
+    }
+    return NM_OK;
+}
+
+static int validate_admm(const float* W, const float* U, int out, int in, int n, int m, int bits, const float* Z,
+                         const float* U_next, const void* values, const void* meta, const float* scales) {
+    int rc = check_pattern(out, in, n, m, bits);
+    if (rc != NM_OK) return rc;
+    if (!W || !Z) return NM_ERR_NULL;
+    if (in % 4) return NM_ERR_SHAPE;
+    if (in > 32768) return NM_ERR_UNSUPPORTED;
+    if (!aligned(W, 16) || (U && !aligned(U, 16)) || !aligned(Z, 16) || (U_next && !aligned(U_next, 16)) ||
+        (values && !aligned(values, 16)) || (meta && !aligned(meta, 4)) || (scales && !aligned(scales, 4)))
+        return NM_ERR_ALIGN;
     return NM_OK;
 }
 
@@ -448,14 +526,8 @@ int nm_project_pack(const float* W, const float* U, int out, int in, int n, int 
 
 int nm_admm_project(const float* W, const float* U, int out, int in, int n, int m, int bits, float* Z,
                     float* U_next, void* values, void* meta, float* scales, uint32_t* status, void* stream) {
-    int rc = nm::check_pattern(out, in, n, m, bits);
+    int rc = nm::validate_admm(W, U, out, in, n, m, bits, Z, U_next, values, meta, scales);
     if (rc != NM_OK) return rc;
-    if (!W || !Z) return NM_ERR_NULL;
-    if (in % 4) return NM_ERR_SHAPE;
-    if (in > 32768) return NM_ERR_UNSUPPORTED;
-    if (!nm::aligned(W, 16) || (U && !nm::aligned(U, 16)) || !nm::aligned(Z, 16) || (U_next && !nm::aligned(U_next, 16)) ||
-        (values && !nm::aligned(values, 16)) || (meta && !nm::aligned(meta, 4)) || (scales && !nm::aligned(scales, 4)))
-        return NM_ERR_ALIGN;
     if (out == 0 || in == 0) return NM_OK;
     nm_pack_job_t j{W, U, out, in, n, m, bits, values, meta, scales};
     nm::PackJobDev d = nm::to_dev(j);
@@ -481,51 +553,30 @@ int nm_project_pack_batched(const nm_pack_job_t* jobs, int njobs, void* ws, size
         int rc = nm::validate_job(jobs[i]);
         if (rc != NM_OK) return rc;
     }
-    // Group jobs that can share one launch: same (n == m ? dense : n, m), bits and block size.
-    struct Key { int n, m, bits, warps; };
-    std::vector<Key> keys;
-    std::vector<std::vector<int>> groups;
+    return nm::launch_batched<false>(jobs, nullptr, njobs, ws, status, (cudaStream_t)stream);
+}
+
+size_t nm_admm_workspace_bytes(int njobs) {
+    return njobs <= 0 ? 0 : (size_t)njobs * (sizeof(nm::PackJobDev) + sizeof(nm::DenseOutDev));
+}
+
+int nm_admm_project_batched(const nm_admm_job_t* jobs, int njobs, void* ws, size_t ws_bytes,
+                            uint32_t* status, void* stream) {
+    if (njobs < 0) return NM_ERR_SHAPE;
+    if (njobs == 0) return NM_OK;
+    if (!jobs) return NM_ERR_NULL;
+    if (!ws || ws_bytes < nm_admm_workspace_bytes(njobs)) return NM_ERR_WORKSPACE;
+    if (!nm::aligned(ws, 16)) return NM_ERR_ALIGN;
+    std::vector<nm_pack_job_t> pj(njobs);
+    std::vector<nm::DenseOutDev> dj(njobs);
     for (int i = 0; i < njobs; ++i) {
-        const nm_pack_job_t& j = jobs[i];
-        if (j.out == 0 || j.in == 0) continue;
-        Key k{j.n == j.m ? 4 : j.n, j.n == j.m ? 4 : j.m, j.bits,
-              std::max(nm::kPackMinWarps, 1 << nm::wpr_log2_of(j.in))};
-        size_t g = 0;
-        for (; g < keys.size(); ++g)
-            if (keys[g].n == k.n && keys[g].m == k.m && keys[g].bits == k.bits && keys[g].warps == k.warps) break;
-        if (g == keys.size()) { keys.push_back(k); groups.emplace_back(); }
-        groups[g].push_back(i);
-    }
-    std::vector<nm::PackJobDev> table;
-    table.reserve(njobs);
-    std::vector<unsigned> group_blocks(keys.size());
-    std::vector<size_t> group_first(keys.size());
-    for (size_t g = 0; g < keys.size(); ++g) {
-        unsigned blocks = 0;
-        group_first[g] = table.size();
-        for (int i : groups[g]) {
-            nm::PackJobDev d = nm::to_dev(jobs[i]);
-            int rows_per_block = keys[g].warps >> d.wpr_log2;
-            d.unit_begin = blocks;
-            unsigned long long nb = ((unsigned long long)d.out + rows_per_block - 1) / rows_per_block;
-            if (blocks + nb > 0x7fffffffull) return NM_ERR_UNSUPPORTED;
-            blocks += (unsigned)nb;
-            table.push_back(d);
-        }
-        group_blocks[g] = blocks;
-    }
-    cudaStream_t s = (cudaStream_t)stream;
-    // Pageable-source async copies are staged before the call returns, so `table` may go away.
-    NM_CUDA_TRY(cudaMemcpyAsync(ws, table.data(), table.size() * sizeof(nm::PackJobDev),
-                                cudaMemcpyHostToDevice, s));
-    for (size_t g = 0; g < keys.size(); ++g) {
-        const nm::PackJobDev* dev = reinterpret_cast<const nm::PackJobDev*>(ws) + group_first[g];
-        int rc = nm::launch(nm::pick_kernel(keys[g].n, keys[g].m, keys[g].bits, keys[g].warps), dev,
-                            (int)groups[g].size(), nm::PackJobDev{}, group_blocks[g], keys[g].warps,
-                            status, s);
+        const nm_admm_job_t& a = jobs[i];
+        int rc = nm::validate_admm(a.W, a.U, a.out, a.in, a.n, a.m, a.bits, a.Z, a.U_next, a.values, a.meta, a.scales);
         if (rc != NM_OK) return rc;
+        pj[i] = nm_pack_job_t{a.W, a.U, a.out, a.in, a.n, a.m, a.bits, a.values, a.meta, a.scales};
+        dj[i] = nm::DenseOutDev{a.Z, a.U_next};
     }
-    return NM_OK;
+    return nm::launch_batched<true>(pj.data(), dj.data(), njobs, ws, status, (cudaStream_t)stream);
 }
 
 }  // extern "C"

@@ -109,3 +109,41 @@ def test_admm_step_in_place_dual_and_errors():
     status = torch.zeros(1, dtype=torch.int32, device=DEV)
     nm.nm_admm_project(to_dev(Wbad), None, 128, 1024, 2, 4, 8, Z, status=status)
     assert nm.nm_poll_status(status) == nm.NM_ERR_NONFINITE
+
+
+def test_batched_admm_step_over_a_heterogeneous_layer():
+    # the four matrices of a BERT-large layer, each with its own pattern and code width, in one call
+    import paper_2206_15014_b200 as nm
+    from gpu_util import to_dev, DEV
+    cfgs = [(2, 4, 8), (1, 4, 4), (4, 8, 8), (4, 4, 4)]
+    shapes = [(3072, 1024), (1024, 1024), (4096, 1024), (1024, 4096)]
+    oracle.set_threads(oracle.max_threads())
+    jobs, keep, refs = [], [], []
+    for idx, ((out, k), (n, m, bits)) in enumerate(zip(shapes, cfgs)):
+        W, U = wl.pack_sweep_matrix(3, 40 + idx, out, k)
+        vb, mb = nm.nm_packed_sizes(out, k, n, m, bits)
+        Wd, Ud = to_dev(W), to_dev(U)
+        Z = torch.full((out, k), float("nan"), dtype=torch.float32, device=DEV)
+        Un = torch.full((out, k), float("nan"), dtype=torch.float32, device=DEV)
+        v = torch.zeros(vb, dtype=torch.uint8, device=DEV)
+        mt = torch.zeros(max(mb // 4, 1), dtype=torch.int32, device=DEV) if n != m else None
+        sc = torch.zeros(out, dtype=torch.float32, device=DEV)
+        # the third job asks for the dense outputs only
+        jobs.append((Wd, Ud, n, m, bits, Z, Un, None if idx == 2 else v, None if idx == 2 else mt, None if idx == 2 else sc))
+        keep.append((Z, Un, v, mt, sc))
+        refs.append((oracle.admm_step(W, U, n, m, bits), oracle.project_pack(W, U, n, m, bits)))
+    arr = nm.make_admm_jobs(jobs)
+    ws_bytes = nm.nm_admm_workspace_bytes(len(jobs))
+    ws = torch.empty(ws_bytes, dtype=torch.uint8, device=DEV)
+    status = torch.zeros(1, dtype=torch.int32, device=DEV)
+    nm.nm_admm_project_batched(arr, len(jobs), ws, ws_bytes, status)
+    assert nm.nm_poll_status(status) == nm.NM_OK
+    for idx, ((Z, Un, v, mt, sc), ((Zr, Unr, sr), (vr, mr, s2))) in enumerate(zip(keep, refs)):
+        assert np.array_equal(Z.cpu().numpy(), Zr) and np.array_equal(Un.cpu().numpy(), Unr), idx
+        if idx != 2:
+            assert np.array_equal(sc.cpu().numpy(), sr)
+            assert np.array_equal(v.cpu().numpy(), np.asarray(vr).reshape(-1))
+            if mt is not None:
+                assert np.array_equal(mt.cpu().numpy().view(np.uint32), np.asarray(mr).reshape(-1))
+    with pytest.raises(nm.NmError):
+        nm.nm_admm_project_batched(arr, len(jobs), ws, ws_bytes - 1, status)   # workspace too small
