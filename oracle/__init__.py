@@ -87,6 +87,20 @@ def unpack(values, meta, out, inn, n, m, bits):
     return Wq
 
 
+def project_pack_grouped(W, U, n, m, bits, group_rows):
+    """As project_pack with one scale per group of `group_rows` output channels (<= 0: whole matrix)."""
+    W = np.ascontiguousarray(W, dtype=np.float32)
+    U = None if U is None else np.ascontiguousarray(U, dtype=np.float32)
+    out, inn = W.shape
+    vb, mb = packed_sizes(out, inn, n, m, bits)
+    values = np.zeros((out, vb // max(out, 1)), dtype=np.uint8)
+    meta = np.zeros((out, mb // 4 // max(out, 1)), dtype=np.uint32)
+    scales = np.zeros(out, dtype=np.float32)
+    _chk(lib().oracle_project_pack_grouped(_p(W), _p(U), out, inn, n, m, bits, int(group_rows), _p(values),
+                                           _p(meta) if mb else None, _p(scales)), "oracle_project_pack_grouped")
+    return values, meta, scales
+
+
 def project_dense(W, U, n, m):
     W = np.ascontiguousarray(W, dtype=np.float32)
     U = None if U is None else np.ascontiguousarray(U, dtype=np.float32)

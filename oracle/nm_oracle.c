@@ -171,8 +171,8 @@ static int row_finite(const float *v, int in)
  * quantisation constraint, scale from ADMM-Max.  V = W + U is the Z-update's
  * argument (Eq. 3); U may be NULL.
  */
-int oracle_project_pack(const float *W, const float *U, int out, int in, int n, int m, int bits,
-                        uint8_t *values, uint32_t *meta, float *scales)
+static int project_pack_impl(const float *W, const float *U, int out, int in, int n, int m, int bits,
+                             const float *given_scales, uint8_t *values, uint32_t *meta, float *scales)
 {
     if (!shape_ok(out, in, n, m, bits)) return ORACLE_ERR_SHAPE;
     const size_t vrb = values_row_bytes(in, n, m, bits);
@@ -190,7 +190,7 @@ int oracle_project_pack(const float *W, const float *U, int out, int in, int n, 
 #pragma omp atomic write
             status = ORACLE_ERR_NONFINITE;
         }
-        float s = row_scale(v, in, bits);
+        float s = given_scales ? given_scales[r] : row_scale(v, in, bits);
         scales[r] = s;
         uint8_t *vrow = values + (size_t)r * vrb;
         uint32_t *mrow = meta ? meta + (size_t)r * mrw : NULL;
@@ -217,6 +217,45 @@ int oracle_project_pack(const float *W, const float *U, int out, int in, int n, 
         free(v);
     }
     return status;
+}
+
+int oracle_project_pack(const float *W, const float *U, int out, int in, int n, int m, int bits,
+                        uint8_t *values, uint32_t *meta, float *scales)
+{
+    return project_pack_impl(W, U, out, in, n, m, bits, NULL, values, meta, scales);
+}
+
+/*
+ * Group-wise quantisation (Sec. 3.3, "subsets of neurons within a single weight
+ * matrix are quantized using different scales"; whole neurons always share a
+ * scale): rows r with the same r / group_rows share one ADMM-Max scale, the
+ * largest magnitude of W + U over those rows divided by the largest integer
+ * (group_rows <= 0: one scale for the whole matrix; the last group may be
+ * short).  scales[r] receives the scale of row r's group.  Everything else is
+ * oracle_project_pack.
+ */
+int oracle_project_pack_grouped(const float *W, const float *U, int out, int in, int n, int m,
+                                int bits, int group_rows, uint8_t *values, uint32_t *meta,
+                                float *scales)
+{
+    if (!shape_ok(out, in, n, m, bits)) return ORACLE_ERR_SHAPE;
+    const int G = group_rows <= 0 ? (out > 0 ? out : 1) : group_rows;
+    const float qmax = (float)((1 << (bits - 1)) - 1);
+    float *gs = (float *)malloc(sizeof(float) * (size_t)(out > 0 ? out : 1));
+    for (int g0 = 0; g0 < out; g0 += G) {
+        float a = 0.0f;
+        for (int r = g0; r < out && r < g0 + G; ++r)
+            for (int k = 0; k < in; ++k) {
+                float w = W[(size_t)r * in + k];
+                float t = fabsf(U ? w + U[(size_t)r * in + k] : w);
+                if (t > a) a = t;
+            }
+        float sg = a == 0.0f ? 1.0f : a / qmax;
+        for (int r = g0; r < out && r < g0 + G; ++r) gs[r] = sg;
+    }
+    int rc = project_pack_impl(W, U, out, in, n, m, bits, gs, values, meta, scales);
+    free(gs);
+    return rc;
 }
 
 /* Inverse of the packing: dense integer codes [out, in], zero where pruned. */

@@ -532,3 +532,36 @@ def test_admm_step_fixed_point_and_ste_form():
     assert np.all(np.abs((Z.astype(np.float64) + Un.astype(np.float64)) - W.astype(np.float64)) <= np.abs(W) * 2.0 ** -23 + 1e-12)
     with pytest.raises(RuntimeError):
         oracle.admm_step(np.array([[np.inf, 0, 0, 0]], np.float32), None, 2, 4, 8)
+
+
+# ---- group-wise scales (several output channels share one scale) ----------------------------------------
+
+@pytest.mark.parametrize("n,m,bits", [(2, 4, 8), (2, 4, 4), (1, 8, 8), (4, 4, 4)])
+def test_grouped_scales_reduce_to_the_per_channel_and_whole_matrix_cases(n, m, bits):
+    rng = np.random.default_rng(41)
+    W, U = wl.normal(rng, (70, 64), 0.02), wl.normal(rng, (70, 64), 0.002)
+    V = (W + U).astype(np.float32)
+    base = oracle.project_pack(W, U, n, m, bits)
+    g1 = oracle.project_pack_grouped(W, U, n, m, bits, 1)
+    assert all(np.array_equal(a, b) for a, b in zip(base, g1))          # groups of one channel: the per-channel case
+    qmax = np.float32(2 ** (bits - 1) - 1)
+    for G in (32, 64, 0, 1000):
+        v, meta, s = oracle.project_pack_grouped(W, U, n, m, bits, G)
+        rows = 70 if G <= 0 else G
+        # one scale per group: the largest row scale of the group (same max, same single division)
+        for g0 in range(0, 70, rows):
+            grp = slice(g0, min(70, g0 + rows))
+            assert np.all(s[grp] == base[2][grp].max())
+            assert s[g0] == np.abs(V[grp]).max() / qmax
+        # support and metadata do not depend on the scale; the codes are Eq. 5 with the group's scale
+        assert np.array_equal(meta, base[1])
+        D = oracle.unpack(v, meta, 70, 64, n, m, bits)
+        Zs = oracle.project_dense(W, U, n, m)
+        assert np.array_equal((s[:, None] * D.astype(np.float32)).astype(np.float32), oracle.fake_quant(Zs, bits, s))
+        # the group's largest element still maps to +-qmax, nothing exceeds it
+        assert np.abs(D).max() == int(qmax)
+    # a row that is small next to its group's maximum loses resolution: fewer distinct codes than with its own scale
+    W2 = W.copy(); W2[0] *= 50
+    own = oracle.unpack(*oracle.project_pack(W2, None, n, m, bits)[:2], 70, 64, n, m, bits)
+    shared = oracle.unpack(*oracle.project_pack_grouped(W2, None, n, m, bits, 32)[:2], 70, 64, n, m, bits)
+    assert np.abs(shared[1]).max() < np.abs(own[1]).max()
