@@ -113,6 +113,23 @@ int nm_admm_project(const float *W, const float *U, int out, int in, int n, int 
                     void *stream);
 
 /*
+ * Group-wise quantisation (Sec. 3.3: several neurons of a weight matrix may share one scale, whole
+ * neurons always do; the paper's experiments use 32 per scale): output channels r with the same
+ * r / group_rows share the ADMM-Max scale max |W + U| over those rows / (2^(bits-1) - 1); group_rows
+ * <= 0 means one scale for the whole matrix; the last group may be short.  scales[r] (required: it
+ * is also the scratch of the group maxima) receives the scale of row r's group, so that it can be
+ * handed to nm_int_linear unchanged.  Otherwise as nm_project_pack / nm_admm_project.  Two passes
+ * over W and U (the maxima, then the projection); for matrices that fit in L2 the second pass is
+ * served from there.
+ */
+int nm_project_pack_grouped(const float *W, const float *U, int out, int in, int n, int m, int bits,
+                            int group_rows, void *values, void *meta, float *scales,
+                            uint32_t *status, void *stream);
+int nm_admm_project_grouped(const float *W, const float *U, int out, int in, int n, int m, int bits,
+                            int group_rows, float *Z, float *U_next, void *values, void *meta,
+                            float *scales, uint32_t *status, void *stream);
+
+/*
  * The same for many matrices with one launch per group of jobs that share (n, m, bits) and block
  * size.  `jobs`: host array of host structs holding device pointers, with the meaning of
  * nm_admm_project's arguments; `ws`: device scratch of at least nm_admm_workspace_bytes(njobs)

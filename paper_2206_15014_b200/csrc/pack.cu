@@ -150,7 +150,8 @@ __device__ __forceinline__ void store_bytes_slow(uint8_t* dst, const unsigned* w
 template <int N, int M, int BITS, int MAXT, bool DENSE_OUT = false>
 __global__ void __launch_bounds__(MAXT, MAXT == 128 ? (DENSE_OUT ? 4 : 8) : 1) pack_kernel(const PackJobDev* __restrict__ jobs, int njobs,
                                                     PackJobDev single, uint32_t* status, float* __restrict__ Zout,
-                                                    float* __restrict__ Unext, const DenseOutDev* __restrict__ dense_jobs) {
+                                                    float* __restrict__ Unext, const DenseOutDev* __restrict__ dense_jobs,
+                                                    const float* given_scales) {
     constexpr bool kDense = (N == M);
     constexpr int G = 32 / M;                          // groups per lane
     constexpr int F = (M == 4) ? 2 : 4;                // metadata field width
@@ -230,7 +231,8 @@ __global__ void __launch_bounds__(MAXT, MAXT == 128 ? (DENSE_OUT ? 4 : 8) : 1) p
 
     // ---- ADMM-Max scale ---------------------------------------------------------------------
     constexpr float qmax = (float)((1 << (BITS - 1)) - 1);
-    const float s = (amax == 0.0f) ? 1.0f : __fdiv_rn(amax, qmax);
+    // group-wise quantisation hands the scale in (one per row, equal within a group of rows)
+    const float s = given_scales ? given_scales[row_ok ? row : 0] : ((amax == 0.0f) ? 1.0f : __fdiv_rn(amax, qmax));
     if (row_ok && chunk == 0 && lane == 0 && (!DENSE_OUT || job.scales)) job.scales[row] = s;
     const float rs = __frcp_rn(s);  // correctly rounded reciprocal, once per row
 
@@ -376,9 +378,59 @@ __global__ void __launch_bounds__(MAXT, MAXT == 128 ? (DENSE_OUT ? 4 : 8) : 1) p
 }
 
 // ---------------------------------------------------------------------------------------------
+// Group-wise scales: rows r with the same r / group_rows share one ADMM-Max scale.  A first pass folds
+// max |W + U| of every row into the first entry of its group in `scales` (non-negative floats order like
+// their bit patterns, so an unsigned atomicMax does it); a second turns each group's maximum into the
+// scale and writes it to all rows of the group (one thread per group: reads before it writes).
+// ---------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(128) group_absmax_kernel(const float* __restrict__ W, const float* __restrict__ U,
+                                                           int out, int in, int group_rows, float* scales) {
+    const int row = blockIdx.x * 4 + (threadIdx.x >> 5), lane = threadIdx.x & 31;
+    if (row >= out) return;
+    const int in4 = in >> 2;
+    const float4* W4 = reinterpret_cast<const float4*>(W) + (size_t)row * in4;
+    const float4* U4 = U ? reinterpret_cast<const float4*>(U) + (size_t)row * in4 : nullptr;
+    float a = 0.0f;
+    for (int f = lane; f < in4; f += 32) {
+        float4 v = __ldg(W4 + f);  // read again by the projection pass: keep it cached
+        if (U4) {
+            const float4 u = __ldg(U4 + f);
+            v.x = __fadd_rn(v.x, u.x); v.y = __fadd_rn(v.y, u.y); v.z = __fadd_rn(v.z, u.z); v.w = __fadd_rn(v.w, u.w);
+        }
+        a = fmaxf(a, fmaxf(fmaxf(fabsf(v.x), fabsf(v.y)), fmaxf(fabsf(v.z), fabsf(v.w))));
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) a = fmaxf(a, __shfl_xor_sync(0xffffffffu, a, o));
+    if (lane == 0) atomicMax(reinterpret_cast<unsigned*>(scales) + (size_t)(row / group_rows) * group_rows, __float_as_uint(a));
+}
+
+__global__ void __launch_bounds__(128) group_scale_kernel(int out, int group_rows, int bits, float* scales) {
+    const long long g = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    const long long first = g * group_rows;
+    if (first >= out) return;
+    const float a = scales[first];
+    const float qmax = (float)((1 << (bits - 1)) - 1);
+    const float s = (a == 0.0f) ? 1.0f : __fdiv_rn(a, qmax);
+    const long long last = min((long long)out, first + group_rows);
+    for (long long r = first; r < last; ++r) scales[r] = s;
+}
+
+static int launch_group_scales(const float* W, const float* U, int out, int in, int bits, int group_rows,
+                               float* scales, cudaStream_t stream) {
+    const int G = group_rows <= 0 ? out : (group_rows > out ? out : group_rows);
+    NM_CUDA_TRY(cudaMemsetAsync(scales, 0, (size_t)out * sizeof(float), stream));
+    group_absmax_kernel<<<(out + 3) / 4, 128, 0, stream>>>(W, U, out, in, G, scales);
+    NM_CUDA_TRY(cudaGetLastError());
+    const int ngroups = (out + G - 1) / G;
+    group_scale_kernel<<<(ngroups + 127) / 128, 128, 0, stream>>>(out, G, bits, scales);
+    NM_CUDA_TRY(cudaGetLastError());
+    return NM_OK;
+}
+
+// ---------------------------------------------------------------------------------------------
 // host side
 // ---------------------------------------------------------------------------------------------
-using PackFn = void (*)(const PackJobDev*, int, PackJobDev, uint32_t*, float*, float*, const DenseOutDev*);
+using PackFn = void (*)(const PackJobDev*, int, PackJobDev, uint32_t*, float*, float*, const DenseOutDev*, const float*);
 
 template <int N, int M, bool DENSE_OUT>
 static PackFn pick_bits(int bits, int warps) {
@@ -427,11 +479,12 @@ static PackJobDev to_dev(const nm_pack_job_t& j) {
 
 static int launch(PackFn fn, const PackJobDev* jobs_dev, int njobs, const PackJobDev& single,
                   unsigned blocks, int warps, uint32_t* status, cudaStream_t stream,
-                  float* Z = nullptr, float* U_next = nullptr, const DenseOutDev* dense_jobs = nullptr) {
+                  float* Z = nullptr, float* U_next = nullptr, const DenseOutDev* dense_jobs = nullptr,
+                  const float* given_scales = nullptr) {
     size_t smem = (size_t)warps * (256 * sizeof(float4) + sizeof(float));
     if (smem > 48 * 1024)
         NM_CUDA_TRY(cudaFuncSetAttribute((const void*)fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    fn<<<blocks, warps * 32, smem, stream>>>(jobs_dev, njobs, single, status, Z, U_next, dense_jobs);
+    fn<<<blocks, warps * 32, smem, stream>>>(jobs_dev, njobs, single, status, Z, U_next, dense_jobs, given_scales);
     NM_CUDA_TRY(cudaGetLastError());
     return NM_OK;
 }
@@ -536,6 +589,41 @@ int nm_admm_project(const float* W, const float* U, int out, int in, int n, int 
     unsigned blocks = (unsigned)((out + rows_per_block - 1) / rows_per_block);
     return nm::launch(nm::pick_kernel<true>(n, m, bits, warps), nullptr, 0, d, blocks, warps, status,
                       (cudaStream_t)stream, Z, U_next);
+}
+
+int nm_project_pack_grouped(const float* W, const float* U, int out, int in, int n, int m, int bits,
+                            int group_rows, void* values, void* meta, float* scales, uint32_t* status,
+                            void* stream) {
+    nm_pack_job_t j{W, U, out, in, n, m, bits, values, meta, scales};
+    int rc = nm::validate_job(j);
+    if (rc != NM_OK) return rc;
+    if (out == 0 || in == 0) return NM_OK;
+    rc = nm::launch_group_scales(W, U, out, in, bits, group_rows, scales, (cudaStream_t)stream);
+    if (rc != NM_OK) return rc;
+    nm::PackJobDev d = nm::to_dev(j);
+    int warps = std::max(nm::kPackMinWarps, 1 << d.wpr_log2);
+    int rows_per_block = warps >> d.wpr_log2;
+    unsigned blocks = (unsigned)((out + rows_per_block - 1) / rows_per_block);
+    return nm::launch(nm::pick_kernel(n, m, bits, warps), nullptr, 0, d, blocks, warps, status, (cudaStream_t)stream,
+                      nullptr, nullptr, nullptr, scales);
+}
+
+int nm_admm_project_grouped(const float* W, const float* U, int out, int in, int n, int m, int bits,
+                            int group_rows, float* Z, float* U_next, void* values, void* meta, float* scales,
+                            uint32_t* status, void* stream) {
+    int rc = nm::validate_admm(W, U, out, in, n, m, bits, Z, U_next, values, meta, scales);
+    if (rc != NM_OK) return rc;
+    if (!scales) return NM_ERR_NULL;  // also the scratch of the group maxima
+    if (out == 0 || in == 0) return NM_OK;
+    rc = nm::launch_group_scales(W, U, out, in, bits, group_rows, scales, (cudaStream_t)stream);
+    if (rc != NM_OK) return rc;
+    nm_pack_job_t j{W, U, out, in, n, m, bits, values, meta, scales};
+    nm::PackJobDev d = nm::to_dev(j);
+    int warps = std::max(nm::kPackMinWarps, 1 << d.wpr_log2);
+    int rows_per_block = warps >> d.wpr_log2;
+    unsigned blocks = (unsigned)((out + rows_per_block - 1) / rows_per_block);
+    return nm::launch(nm::pick_kernel<true>(n, m, bits, warps), nullptr, 0, d, blocks, warps, status,
+                      (cudaStream_t)stream, Z, U_next, nullptr, scales);
 }
 
 size_t nm_pack_workspace_bytes(int njobs) {

@@ -147,3 +147,40 @@ def test_batched_admm_step_over_a_heterogeneous_layer():
                 assert np.array_equal(mt.cpu().numpy().view(np.uint32), np.asarray(mr).reshape(-1))
     with pytest.raises(nm.NmError):
         nm.nm_admm_project_batched(arr, len(jobs), ws, ws_bytes - 1, status)   # workspace too small
+
+
+@pytest.mark.parametrize("n,m,bits", [(2, 4, 8), (2, 4, 4), (1, 8, 8), (4, 8, 4), (4, 4, 8)])
+@pytest.mark.parametrize("G", [1, 32, 64, 0, 100000])
+def test_grouped_scales_pack_and_admm(n, m, bits, G):
+    # several output channels per scale: packed outputs, Z and U_next against the oracle, bit for bit
+    import paper_2206_15014_b200 as nm
+    from gpu_util import to_dev, DEV
+    oracle.set_threads(oracle.max_threads())
+    for idx, (out, k) in enumerate([(300, 1024), (70, 4096), (45, 1032)]):
+        if (k // m * n * bits) % 8:
+            k *= 2
+        W, U = wl.pack_sweep_matrix(3, 60 + idx, out, k)
+        W[3] *= 20  # one channel far larger than the rest of its group
+        vr, mr, sr = oracle.project_pack_grouped(W, U, n, m, bits, G)
+        D = oracle.unpack(vr, mr, out, k, n, m, bits)
+        Zr = (sr[:, None] * D.astype(np.float32)).astype(np.float32)
+        Unr = ((W + U).astype(np.float32) - Zr).astype(np.float32)
+        vb, mb = nm.nm_packed_sizes(out, k, n, m, bits)
+        Wd, Ud = to_dev(W), to_dev(U)
+        v = torch.zeros(vb, dtype=torch.uint8, device=DEV)
+        mt = torch.zeros(max(mb // 4, 1), dtype=torch.int32, device=DEV) if n != m else None
+        sc = torch.full((out,), -1.0, dtype=torch.float32, device=DEV)
+        status = torch.zeros(1, dtype=torch.int32, device=DEV)
+        nm.nm_project_pack_grouped(Wd, Ud, out, k, n, m, bits, G, v, mt, sc, status)
+        assert nm.nm_poll_status(status) == nm.NM_OK
+        assert np.array_equal(sc.cpu().numpy(), sr), (out, k)
+        assert np.array_equal(v.cpu().numpy(), np.asarray(vr).reshape(-1))
+        if mt is not None:
+            assert np.array_equal(mt.cpu().numpy().view(np.uint32)[: mb // 4], np.asarray(mr).reshape(-1))
+        Z = torch.empty((out, k), dtype=torch.float32, device=DEV)
+        Un = torch.empty((out, k), dtype=torch.float32, device=DEV)
+        sc2 = torch.zeros(out, dtype=torch.float32, device=DEV)
+        nm.nm_admm_project_grouped(Wd, Ud, out, k, n, m, bits, G, Z, Un, None, None, sc2, status)
+        assert nm.nm_poll_status(status) == nm.NM_OK
+        assert np.array_equal(sc2.cpu().numpy(), sr)
+        assert np.array_equal(Z.cpu().numpy(), Zr) and np.array_equal(Un.cpu().numpy(), Unr)
