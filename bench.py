@@ -449,6 +449,24 @@ def pack_sweep(nm, torch, dev, status, reps=5):
             times.append(e0.elapsed_time(e1))
         us = float(np.median(times)) * 1e3
         table[f"{n}:{m}/{bits}b"] = {"us": us, "gbs": nbytes / us / 1e3, "bytes": nbytes}
+    # group-wise scales (32 output channels per scale, the paper's default), one call per matrix: two passes over
+    # W and U, the second served from L2; GB/s on the same algorithmic bytes as the per-channel pack
+    def grouped_pass():
+        for (W, U, v, mt, sc) in mats:
+            nm.nm_project_pack_grouped(W, U, W.shape[0], W.shape[1], 2, 4, 8, 32, v, mt, sc, status)
+    grouped_pass()
+    torch.cuda.synchronize()
+    times = []
+    for _ in range(reps):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        grouped_pass()
+        e1.record()
+        torch.cuda.synchronize()
+        times.append(e0.elapsed_time(e1))
+    grouped_us = float(np.median(times)) * 1e3
+    grouped = {"us": grouped_us, "gbs": table["2:4/8b"]["bytes"] / grouped_us / 1e3, "bytes": table["2:4/8b"]["bytes"],
+               "launches": 3 * len(mats), "group_rows": 32}
     # ADMM step with dense outputs over the same 96 matrices (one batched call): W and U read, Z and
     # U_next (in place over U, so it runs last) written, 16 bytes per parameter; 2:4 / 8-bit, no packed outputs
     Zs = [torch.empty_like(W) for (W, U, v, mt, sc) in mats]
@@ -472,6 +490,7 @@ def pack_sweep(nm, torch, dev, status, reps=5):
     head = table["2:4/8b"]
     return {"us": head["us"], "gbs": head["gbs"], "params": int(sum(o * k for o, k in shapes)),
             "bytes": head["bytes"], "matrices": len(shapes), "launches": 1, "variants": table,
+            "grouped_2:4/8b": grouped,
             "admm_step_2:4/8b": {"us": admm_us, "gbs": admm_bytes / admm_us / 1e3, "bytes": admm_bytes, "launches": 1}}
 
 
