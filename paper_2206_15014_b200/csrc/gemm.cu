@@ -558,6 +558,14 @@ nm_gemm_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant
 constexpr int kPairThreads = 32 * (3 + kEpiWarps);
 constexpr int kPairMaxStages = 7;   // the relay cycles through 8 named barriers (ids 1-8; 9-14 serve the narrow-output epilogue)
 
+// Tile ranges of the CTA pairs, computed on the host: start[p] .. start[p + 1] is pair p's range.  A pair
+// whose range crosses into a new output tile stalls there (weights and metadata are replaced once
+// the MMAs of the old one have drained), so such a range is made shorter by that cost.
+constexpr int kMaxPairs = 128;
+struct PairSchedule {
+    int start[kMaxPairs + 1];
+};
+
 constexpr int kPairResStages = 4;   // stages of weights a CTA can keep resident (1024 reduction elements at 2:4)
 
 template <bool SPARSE, int BN, bool RES = false>
@@ -592,7 +600,8 @@ struct PairCfg {
 template <bool SPARSE, int BN, int EPI, bool RES>
 __global__ void __launch_bounds__(kPairThreads, 1)
 nm_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant__ CUtensorMap tmap_x,
-                    const __grid_constant__ CUtensorMap tmap_y, const GemmParams p) {
+                    const __grid_constant__ CUtensorMap tmap_y, const GemmParams p,
+                    const __grid_constant__ PairSchedule sched) {
     using Cfg = PairCfg<SPARSE, BN, RES>;
     constexpr int S = Cfg::STAGES;
     constexpr int EW = kEpiWarps, kGateWarp = 2 + EW;
@@ -617,10 +626,9 @@ nm_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_con
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t rank = ptx::cluster_ctarank();
     const bool leader = rank == 0;
-    const int n_pairs = gridDim.x >> 1, pair = blockIdx.x >> 1;
-    const int per = p.n_tiles / n_pairs, rem = p.n_tiles % n_pairs;
-    const int tile_begin = pair * per + min(pair, rem);
-    const int tile_count = per + (pair < rem ? 1 : 0);
+    const int pair = blockIdx.x >> 1;
+    const int tile_begin = sched.start[pair];
+    const int tile_count = sched.start[pair + 1] - tile_begin;
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < S; ++s) { ptx::mbar_init(full_bar(s), 1); ptx::mbar_init(empty_bar(s), 1); }
@@ -1059,7 +1067,26 @@ static int launch_gemm_pair(const LinearArgs& a) {
     p.Y = a.Y; p.ACC = a.ACC; p.NARROW = a.NARROW; p.sy = a.sy; p.absmax = a.absmax; p.status = a.status;
     auto fn = nm_gemm_pair_kernel<SPARSE, BN, EPI, RES>;
     NM_CUDA_TRY(cudaFuncSetAttribute((const void*)fn, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::SMEM));
-    const int pairs = p.n_tiles < sm_count() / 2 ? p.n_tiles : sm_count() / 2;
+    int pairs = p.n_tiles < sm_count() / 2 ? p.n_tiles : sm_count() / 2;
+    if (pairs > kMaxPairs) pairs = kMaxPairs;
+    // Contiguous tile ranges of about equal cost: a tile costs 1, entering a new output tile inside a range
+    // costs `crossing` tiles (weights resident: ~1, the reload waits for the MMAs to drain; streamed: metadata only).
+    PairSchedule sched;
+    {
+        const double crossing = RES ? 1.0 : 0.2;
+        auto cost = [&](int t) { return 1.0 + ((t > 0 && t % p.n_tok_tiles == 0) ? crossing : 0.0); };
+        double total = 0.0;
+        for (int t = 0; t < p.n_tiles; ++t) total += cost(t);
+        int t = 0;
+        double before = 0.0;  // cost of the tiles before t
+        for (int q = 0; q < pairs; ++q) {
+            const double threshold = q * total / pairs;
+            while (t < p.n_tiles - (pairs - q) && before + 0.5 * cost(t) < threshold) before += cost(t++);
+            if (q > 0 && t <= sched.start[q - 1]) before += cost(t++);  // every pair gets at least one tile
+            sched.start[q] = t;
+        }
+        sched.start[pairs] = p.n_tiles;
+    }
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(2 * pairs, 1, 1);
     cfg.blockDim = dim3(kPairThreads, 1, 1);
@@ -1069,7 +1096,7 @@ static int launch_gemm_pair(const LinearArgs& a) {
     attr[0].id = cudaLaunchAttributeClusterDimension;
     attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
     cfg.attrs = attr; cfg.numAttrs = 1;
-    NM_CUDA_TRY(cudaLaunchKernelEx(&cfg, fn, tw, tx, ty, p));
+    NM_CUDA_TRY(cudaLaunchKernelEx(&cfg, fn, tw, tx, ty, p, sched));
     return NM_OK;
 }
 
