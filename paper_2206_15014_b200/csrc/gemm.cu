@@ -102,6 +102,7 @@ constexpr int kResidentKB = 8;
 struct GemmParams {
     int tokens, out, in;
     int n_tok_tiles, n_tiles, kblocks;
+    int n_out_tiles, band;  // pair kernel: tiles are ordered band by band (see tile_coord)
     const uint32_t* meta;  // canonical metadata [out, mrow_words] (sparse modes)
     int mrow_words;
     const uint8_t* values; // packed codes (transform modes)
@@ -118,6 +119,20 @@ struct GemmParams {
     float* absmax;
     uint32_t* status;
 };
+
+// Order of the tiles of the pair kernel.  Token tiles are cut into bands of `band` tiles; inside a band the
+// tiles run output-tile-major.  With band = n_tok_tiles this is the plain output-tile-major order (one
+// long run per output tile: weights and metadata change rarely).  A band of about one pair's share
+// makes neighbouring pairs work on the SAME token tiles of different output tiles at the same time, so
+// that X is fetched from DRAM once and found in L2 by the others.
+struct TileCoord { int o, t; };
+__host__ __device__ inline TileCoord tile_coord(int tile, int n_tok_tiles, int n_out_tiles, int band) {
+    const int per_band = band * n_out_tiles;
+    const int b = tile / per_band, r = tile - b * per_band;
+    const int rest = n_tok_tiles - b * band, tb = band < rest ? band : rest;  // the last band may be short
+    const int o = r / tb;
+    return TileCoord{o, b * band + (r - o * tb)};
+}
 
 template <bool SPARSE, int BN, bool RESIDENT = false>
 struct GemmCfg {
@@ -669,11 +684,12 @@ nm_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_con
             bool ok = true;
             for (int i = 0; i < tile_count && ok; ++i) {
                 const int tile = tile_begin + i;
-                const int n0 = (tile / p.n_tok_tiles) * (2 * kBM) + (int)rank * kBM;
-                const int t0 = (tile % p.n_tok_tiles) * BN + (int)rank * Cfg::B_ROWS;
-                if (RES && tile / p.n_tok_tiles != prev_out_tile) {
+                const TileCoord tc = tile_coord(tile, p.n_tok_tiles, p.n_out_tiles, p.band);
+                const int n0 = tc.o * (2 * kBM) + (int)rank * kBM;
+                const int t0 = tc.t * BN + (int)rank * Cfg::B_ROWS;
+                if (RES && tc.o != prev_out_tile) {
                     // new output tile: once the MMAs of the previous one are done, fetch this CTA's weight rows for the whole reduction
-                    prev_out_tile = tile / p.n_tok_tiles;
+                    prev_out_tile = tc.o;
                     if (!ptx::mbar_wait_bounded(a_free_bar, free_parity, abort_flag, kWaitLimit)) {
                         raise_timeout(); ok = false; break;
                     }
@@ -710,7 +726,7 @@ nm_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_con
                 }
             };
             for (int i = 0; i < tile_count; ++i) {
-                const int tile = tile_begin + i, out_tile = tile / p.n_tok_tiles, buf = i & 1;
+                const int tile = tile_begin + i, out_tile = tile_coord(tile, p.n_tok_tiles, p.n_out_tiles, p.band).o, buf = i & 1;
                 if (out_tile != prev_out_tile) {
                     if (SPARSE) { wait(meta_bar, meta_phase); meta_phase ^= 1u; }
                     if (RES) { wait(a_full_bar, a_phase); a_phase ^= 1u; }
@@ -732,7 +748,8 @@ nm_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_con
             for (int i = 0; i < tile_count; ++i) {
                 const int buf = i & 1;
                 const uint32_t d_tmem = tmem_base + buf * BN;
-                const bool last_of_out_tile = RES && (tile_begin + i + 1) / p.n_tok_tiles != (tile_begin + i) / p.n_tok_tiles;
+                const bool last_of_out_tile = RES && (tile_begin + i + 1 >= p.n_tiles ||
+                    tile_coord(tile_begin + i + 1, p.n_tok_tiles, p.n_out_tiles, p.band).o != tile_coord(tile_begin + i, p.n_tok_tiles, p.n_out_tiles, p.band).o);
                 for (int kb = 0; kb < p.kblocks; ++kb, ++it) {
                     const int s = it % S;
                     ptx::named_bar_sync(1 + (it & 7u), 64);
@@ -799,11 +816,9 @@ nm_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_con
             if (lane == 0) ptx::mbar_arrive_cluster(ptx::map_to_cta(acc_empty_bar(buf), 0));
         };
 
-        // position of the current tile, advanced without divisions
-        int out_tile = tile_begin / p.n_tok_tiles, tok_tile = tile_begin % p.n_tok_tiles;
-        for (int i = 0; i < tile_count && ok; ++i, ++tok_tile) {
-            if (tok_tile == p.n_tok_tiles) { tok_tile = 0; ++out_tile; }
-            const int buf = i & 1;
+        for (int i = 0; i < tile_count && ok; ++i) {
+            const TileCoord tc = tile_coord(tile_begin + i, p.n_tok_tiles, p.n_out_tiles, p.band);
+            const int out_tile = tc.o, tok_tile = tc.t, buf = i & 1;
             const int n0 = out_tile * (2 * kBM) + (int)rank * kBM, n = n0 + row, t0 = tok_tile * BN;
             if (SPARSE && i == 0 && half == 0) load_meta(out_tile);
             bool got = ptx::mbar_wait_bounded(acc_full_bar(buf), (i >> 1) & 1u, abort_flag, kWaitLimit);
@@ -813,7 +828,10 @@ nm_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_con
             if (!ok) break;
             ptx::tc_fence_after();
             // the next tile starts a new output tile: its metadata can go in now, the MMAs of this one are done
-            if (SPARSE && half == 0 && i + 1 < tile_count && tok_tile + 1 == p.n_tok_tiles) load_meta(out_tile + 1);
+            if (SPARSE && half == 0 && i + 1 < tile_count) {
+                const int next_out_tile = tile_coord(tile_begin + i + 1, p.n_tok_tiles, p.n_out_tiles, p.band).o;
+                if (next_out_tile != out_tile) load_meta(next_out_tile);
+            }
             const bool n_ok = n < p.out;
             if (EPI != EPI_ACC && out_tile != scaled_out_tile) {  // channel constants: fetched once per output tile
                 scaled_out_tile = out_tile;
@@ -1060,7 +1078,8 @@ static int launch_gemm_pair(const LinearArgs& a) {
     p.tma_store = tma_store ? 1 : 0;
     p.tokens = a.tokens; p.out = W.out; p.in = W.in;
     p.n_tok_tiles = (a.tokens + BN - 1) / BN;
-    p.n_tiles = p.n_tok_tiles * ((W.out + 2 * kBM - 1) / (2 * kBM));
+    p.n_out_tiles = (W.out + 2 * kBM - 1) / (2 * kBM);
+    p.n_tiles = p.n_tok_tiles * p.n_out_tiles;
     p.kblocks = (W.in + Cfg::KB - 1) / Cfg::KB;
     p.meta = (const uint32_t*)W.meta; p.mrow_words = W.in / 32;
     p.sw = a.sw; p.bias = a.bias; p.sx_dev = a.sx_dev; p.sx_host = a.sx;
@@ -1071,10 +1090,19 @@ static int launch_gemm_pair(const LinearArgs& a) {
     if (pairs > kMaxPairs) pairs = kMaxPairs;
     // Contiguous tile ranges of about equal cost: a tile costs 1, entering a new output tile inside a range
     // costs `crossing` tiles (weights resident: ~1, the reload waits for the MMAs to drain; streamed: metadata only).
+    // Streamed weights: a change of output tile only costs the metadata, so the tiles are banded by about
+    // one pair's share and neighbouring pairs share X tiles in L2.  Resident weights: long runs.
+    p.band = p.n_tok_tiles;
+    if (!RES) {
+        int b = (p.n_tiles + pairs / 2) / pairs;
+        if (const char* e = getenv("NM_BAND")) b = atoi(e);
+        p.band = b < 1 ? 1 : (b > p.n_tok_tiles ? p.n_tok_tiles : b);
+    }
     PairSchedule sched;
     {
         const double crossing = RES ? 1.0 : 0.2;
-        auto cost = [&](int t) { return 1.0 + ((t > 0 && t % p.n_tok_tiles == 0) ? crossing : 0.0); };
+        auto out_of = [&](int t) { return tile_coord(t, p.n_tok_tiles, p.n_out_tiles, p.band).o; };
+        auto cost = [&](int t) { return 1.0 + ((t > 0 && out_of(t) != out_of(t - 1)) ? crossing : 0.0); };
         double total = 0.0;
         for (int t = 0; t < p.n_tiles; ++t) total += cost(t);
         int t = 0;
