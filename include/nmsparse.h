@@ -128,6 +128,11 @@ int nm_project_pack_grouped(const float *W, const float *U, int out, int in, int
 int nm_admm_project_grouped(const float *W, const float *U, int out, int in, int n, int m, int bits,
                             int group_rows, float *Z, float *U_next, void *values, void *meta,
                             float *scales, uint32_t *status, void *stream);
+/* nm_project_pack_grouped for many matrices (jobs, ws as for nm_project_pack_batched; one group_rows for all):
+ * per group of jobs that share (n, m, bits) and block size one launch folds the row maxima, one
+ * finishes the scales and one projects and packs. */
+int nm_project_pack_grouped_batched(const nm_pack_job_t *jobs, int njobs, int group_rows, void *ws,
+                                    size_t ws_bytes, uint32_t *status, void *stream);
 
 /*
  * The same for many matrices with one launch per group of jobs that share (n, m, bits) and block

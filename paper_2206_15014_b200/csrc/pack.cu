@@ -34,6 +34,9 @@ struct DenseOutDev {
 };
 
 static constexpr int kPackMinWarps = 4;
+// group_mode of pack_kernel: scale per row from the row itself; only fold the row maxima per group into
+// `scales`; take the scales found in `scales`.
+enum { kGroupNone = 0, kGroupMaxPass = 1, kGroupScalesGiven = 2 };
 
 __device__ __forceinline__ float4 ld_stream(const float4* p) { return __ldcs(p); }
 
@@ -151,7 +154,7 @@ template <int N, int M, int BITS, int MAXT, bool DENSE_OUT = false>
 __global__ void __launch_bounds__(MAXT, MAXT == 128 ? (DENSE_OUT ? 4 : 8) : 1) pack_kernel(const PackJobDev* __restrict__ jobs, int njobs,
                                                     PackJobDev single, uint32_t* status, float* __restrict__ Zout,
                                                     float* __restrict__ Unext, const DenseOutDev* __restrict__ dense_jobs,
-                                                    const float* given_scales) {
+                                                    int group_mode, int group_rows) {
     constexpr bool kDense = (N == M);
     constexpr int G = 32 / M;                          // groups per lane
     constexpr int F = (M == 4) ? 2 : 4;                // metadata field width
@@ -229,10 +232,20 @@ __global__ void __launch_bounds__(MAXT, MAXT == 128 ? (DENSE_OUT ? 4 : 8) : 1) p
         __syncwarp();
     }
 
+    // ---- group-wise scales, first pass: fold this row's maximum into the first entry of its group -----
+    if (group_mode == kGroupMaxPass) {
+        if (row_ok && chunk == 0 && lane == 0) {
+            const int G = (group_rows <= 0 || group_rows > job.out) ? job.out : group_rows;
+            atomicMax(reinterpret_cast<unsigned*>(job.scales) + (size_t)(row / G) * G, __float_as_uint(amax));
+        }
+        return;
+    }
+
     // ---- ADMM-Max scale ---------------------------------------------------------------------
     constexpr float qmax = (float)((1 << (BITS - 1)) - 1);
     // group-wise quantisation hands the scale in (one per row, equal within a group of rows)
-    const float s = given_scales ? given_scales[row_ok ? row : 0] : ((amax == 0.0f) ? 1.0f : __fdiv_rn(amax, qmax));
+    const float s = group_mode == kGroupScalesGiven ? job.scales[row_ok ? row : 0]
+                                                    : ((amax == 0.0f) ? 1.0f : __fdiv_rn(amax, qmax));
     if (row_ok && chunk == 0 && lane == 0 && (!DENSE_OUT || job.scales)) job.scales[row] = s;
     const float rs = __frcp_rn(s);  // correctly rounded reciprocal, once per row
 
@@ -415,6 +428,25 @@ __global__ void __launch_bounds__(128) group_scale_kernel(int out, int group_row
     for (long long r = first; r < last; ++r) scales[r] = s;
 }
 
+// Batched form over a job table: block j serves job j.  phase 0 clears the scales (the maxima are folded
+// in by the pack kernel's kGroupMaxPass), phase 1 turns each group's maximum into the scale of its rows.
+__global__ void __launch_bounds__(256) group_prepare_kernel(const PackJobDev* __restrict__ jobs, int group_rows,
+                                                            int bits, int phase) {
+    const PackJobDev job = jobs[blockIdx.x];
+    if (phase == 0) {
+        for (int r = threadIdx.x; r < job.out; r += blockDim.x) job.scales[r] = 0.0f;
+        return;
+    }
+    const int G = (group_rows <= 0 || group_rows > job.out) ? job.out : group_rows;
+    const float qmax = (float)((1 << (bits - 1)) - 1);
+    for (long long first = (long long)threadIdx.x * G; first < job.out; first += (long long)blockDim.x * G) {
+        const float a = job.scales[first];
+        const float s = (a == 0.0f) ? 1.0f : __fdiv_rn(a, qmax);
+        const long long last = min((long long)job.out, first + G);
+        for (long long r = first; r < last; ++r) job.scales[r] = s;
+    }
+}
+
 static int launch_group_scales(const float* W, const float* U, int out, int in, int bits, int group_rows,
                                float* scales, cudaStream_t stream) {
     const int G = group_rows <= 0 ? out : (group_rows > out ? out : group_rows);
@@ -430,7 +462,7 @@ static int launch_group_scales(const float* W, const float* U, int out, int in, 
 // ---------------------------------------------------------------------------------------------
 // host side
 // ---------------------------------------------------------------------------------------------
-using PackFn = void (*)(const PackJobDev*, int, PackJobDev, uint32_t*, float*, float*, const DenseOutDev*, const float*);
+using PackFn = void (*)(const PackJobDev*, int, PackJobDev, uint32_t*, float*, float*, const DenseOutDev*, int, int);
 
 template <int N, int M, bool DENSE_OUT>
 static PackFn pick_bits(int bits, int warps) {
@@ -480,11 +512,11 @@ static PackJobDev to_dev(const nm_pack_job_t& j) {
 static int launch(PackFn fn, const PackJobDev* jobs_dev, int njobs, const PackJobDev& single,
                   unsigned blocks, int warps, uint32_t* status, cudaStream_t stream,
                   float* Z = nullptr, float* U_next = nullptr, const DenseOutDev* dense_jobs = nullptr,
-                  const float* given_scales = nullptr) {
+                  int group_mode = kGroupNone, int group_rows = 0) {
     size_t smem = (size_t)warps * (256 * sizeof(float4) + sizeof(float));
     if (smem > 48 * 1024)
         NM_CUDA_TRY(cudaFuncSetAttribute((const void*)fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    fn<<<blocks, warps * 32, smem, stream>>>(jobs_dev, njobs, single, status, Z, U_next, dense_jobs, given_scales);
+    fn<<<blocks, warps * 32, smem, stream>>>(jobs_dev, njobs, single, status, Z, U_next, dense_jobs, group_mode, group_rows);
     NM_CUDA_TRY(cudaGetLastError());
     return NM_OK;
 }
@@ -493,7 +525,7 @@ static int launch(PackFn fn, const PackJobDev* jobs_dev, int njobs, const PackJo
 // and block size), writes the device job table(s) into `ws` and launches one kernel per group.
 template <bool DENSE_OUT>
 static int launch_batched(const nm_pack_job_t* jobs, const DenseOutDev* dense, int njobs, void* ws,
-                          uint32_t* status, cudaStream_t s) {
+                          uint32_t* status, cudaStream_t s, bool grouped = false, int group_rows = 0) {
     // Group jobs that can share one launch: same (n == m ? dense : n, m), bits and block size.
     struct Key { int n, m, bits, warps; };
     std::vector<Key> keys;
@@ -537,11 +569,26 @@ static int launch_batched(const nm_pack_job_t* jobs, const DenseOutDev* dense, i
     if (DENSE_OUT)
         NM_CUDA_TRY(cudaMemcpyAsync(dense_dev, dense_table.data(), dense_table.size() * sizeof(DenseOutDev),
                                     cudaMemcpyHostToDevice, s));
+    if (grouped) {
+        // group-wise scales: clear, fold the row maxima per group (a first pass of the same kernel), finish
+        for (size_t g = 0; g < keys.size(); ++g) {
+            const nm::PackJobDev* dev = reinterpret_cast<const nm::PackJobDev*>(ws) + group_first[g];
+            group_prepare_kernel<<<(unsigned)groups[g].size(), 256, 0, s>>>(dev, group_rows, keys[g].bits, 0);
+            NM_CUDA_TRY(cudaGetLastError());
+            int rc = nm::launch(nm::pick_kernel<DENSE_OUT>(keys[g].n, keys[g].m, keys[g].bits, keys[g].warps), dev,
+                                (int)groups[g].size(), nm::PackJobDev{}, group_blocks[g], keys[g].warps, status, s,
+                                nullptr, nullptr, DENSE_OUT ? dense_dev + group_first[g] : nullptr, kGroupMaxPass, group_rows);
+            if (rc != NM_OK) return rc;
+            group_prepare_kernel<<<(unsigned)groups[g].size(), 256, 0, s>>>(dev, group_rows, keys[g].bits, 1);
+            NM_CUDA_TRY(cudaGetLastError());
+        }
+    }
     for (size_t g = 0; g < keys.size(); ++g) {
         const nm::PackJobDev* dev = reinterpret_cast<const nm::PackJobDev*>(ws) + group_first[g];
         int rc = nm::launch(nm::pick_kernel<DENSE_OUT>(keys[g].n, keys[g].m, keys[g].bits, keys[g].warps), dev,
                             (int)groups[g].size(), nm::PackJobDev{}, group_blocks[g], keys[g].warps,
-                            status, s, nullptr, nullptr, DENSE_OUT ? dense_dev + group_first[g] : nullptr);
+                            status, s, nullptr, nullptr, DENSE_OUT ? dense_dev + group_first[g] : nullptr,
+                            grouped ? kGroupScalesGiven : kGroupNone, group_rows);
         if (rc != NM_OK) return rc;
     }
     return NM_OK;
@@ -605,7 +652,7 @@ int nm_project_pack_grouped(const float* W, const float* U, int out, int in, int
     int rows_per_block = warps >> d.wpr_log2;
     unsigned blocks = (unsigned)((out + rows_per_block - 1) / rows_per_block);
     return nm::launch(nm::pick_kernel(n, m, bits, warps), nullptr, 0, d, blocks, warps, status, (cudaStream_t)stream,
-                      nullptr, nullptr, nullptr, scales);
+                      nullptr, nullptr, nullptr, nm::kGroupScalesGiven, group_rows);
 }
 
 int nm_admm_project_grouped(const float* W, const float* U, int out, int in, int n, int m, int bits,
@@ -623,7 +670,7 @@ int nm_admm_project_grouped(const float* W, const float* U, int out, int in, int
     int rows_per_block = warps >> d.wpr_log2;
     unsigned blocks = (unsigned)((out + rows_per_block - 1) / rows_per_block);
     return nm::launch(nm::pick_kernel<true>(n, m, bits, warps), nullptr, 0, d, blocks, warps, status,
-                      (cudaStream_t)stream, Z, U_next, nullptr, scales);
+                      (cudaStream_t)stream, Z, U_next, nullptr, nm::kGroupScalesGiven, group_rows);
 }
 
 size_t nm_pack_workspace_bytes(int njobs) {
@@ -642,6 +689,20 @@ int nm_project_pack_batched(const nm_pack_job_t* jobs, int njobs, void* ws, size
         if (rc != NM_OK) return rc;
     }
     return nm::launch_batched<false>(jobs, nullptr, njobs, ws, status, (cudaStream_t)stream);
+}
+
+int nm_project_pack_grouped_batched(const nm_pack_job_t* jobs, int njobs, int group_rows, void* ws,
+                                    size_t ws_bytes, uint32_t* status, void* stream) {
+    if (njobs < 0) return NM_ERR_SHAPE;
+    if (njobs == 0) return NM_OK;
+    if (!jobs) return NM_ERR_NULL;
+    if (!ws || ws_bytes < nm_pack_workspace_bytes(njobs)) return NM_ERR_WORKSPACE;
+    if (!nm::aligned(ws, 16)) return NM_ERR_ALIGN;
+    for (int i = 0; i < njobs; ++i) {
+        int rc = nm::validate_job(jobs[i]);
+        if (rc != NM_OK) return rc;
+    }
+    return nm::launch_batched<false>(jobs, nullptr, njobs, ws, status, (cudaStream_t)stream, true, group_rows);
 }
 
 size_t nm_admm_workspace_bytes(int njobs) {

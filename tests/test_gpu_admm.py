@@ -184,3 +184,35 @@ def test_grouped_scales_pack_and_admm(n, m, bits, G):
         assert nm.nm_poll_status(status) == nm.NM_OK
         assert np.array_equal(sc2.cpu().numpy(), sr)
         assert np.array_equal(Z.cpu().numpy(), Zr) and np.array_equal(Un.cpu().numpy(), Unr)
+
+
+@pytest.mark.parametrize("G", [32, 0])
+def test_grouped_scales_batched_over_a_heterogeneous_layer(G):
+    import paper_2206_15014_b200 as nm
+    from gpu_util import to_dev, DEV
+    cfgs = [(2, 4, 8), (1, 4, 4), (4, 8, 8), (4, 4, 4), (2, 4, 8)]
+    shapes = [(3072, 1024), (1000, 1024), (4096, 1024), (1024, 4096), (50, 8192)]
+    oracle.set_threads(oracle.max_threads())
+    jobs, keep, refs = [], [], []
+    for idx, ((out, k), (n, m, bits)) in enumerate(zip(shapes, cfgs)):
+        W, U = wl.pack_sweep_matrix(3, 80 + idx, out, k)
+        W[out // 2] *= 30
+        vb, mb = nm.nm_packed_sizes(out, k, n, m, bits)
+        v = torch.zeros(vb, dtype=torch.uint8, device=DEV)
+        mt = torch.zeros(max(mb // 4, 1), dtype=torch.int32, device=DEV) if n != m else None
+        sc = torch.full((out,), -3.0, dtype=torch.float32, device=DEV)
+        jobs.append((to_dev(W), to_dev(U), n, m, bits, v, mt, sc))
+        keep.append((v, mt, sc, mb))
+        refs.append(oracle.project_pack_grouped(W, U, n, m, bits, G))
+    arr = nm.make_pack_jobs(jobs)
+    ws_bytes = nm.nm_pack_workspace_bytes(len(jobs))
+    ws = torch.empty(ws_bytes, dtype=torch.uint8, device=DEV)
+    status = torch.zeros(1, dtype=torch.int32, device=DEV)
+    for _ in range(2):  # a second call must not see the first one's scales as maxima
+        nm.nm_project_pack_grouped_batched(arr, len(jobs), G, ws, ws_bytes, status)
+    assert nm.nm_poll_status(status) == nm.NM_OK
+    for idx, ((v, mt, sc, mb), (vr, mr, sr)) in enumerate(zip(keep, refs)):
+        assert np.array_equal(sc.cpu().numpy(), sr), idx
+        assert np.array_equal(v.cpu().numpy(), np.asarray(vr).reshape(-1)), idx
+        if mt is not None:
+            assert np.array_equal(mt.cpu().numpy().view(np.uint32)[: mb // 4], np.asarray(mr).reshape(-1)), idx
