@@ -242,6 +242,19 @@ int nm_int_linear_acc(const int8_t *X, int tokens, const nm_packed_t *W, int32_t
 
 size_t nm_int_linear_workspace_bytes(int tokens, int out, int in, int n, int m, int bits);
 
+/*
+ * Host-only: how the CTA-pair kernel of nm_int_linear walks an [n_out_tiles x n_tok_tiles] grid of tiles
+ * with `pairs` CTA pairs (for inspection and tests; it launches nothing).  The tiles are numbered band
+ * by band of token tiles, output-tile-major inside a band; pair p works on tiles start[p] ..
+ * start[p + 1] - 1 of that numbering, ranges of about equal cost.  resident != 0: weights kept in shared
+ * memory (one long run per output tile); else bands of about one pair's share, or of band_request > 0
+ * token tiles.  start: [pairs + 1]; tile_out / tile_tok (nullable): [n_out_tiles * n_tok_tiles], the
+ * output tile and token tile of every tile number.  Returns the band size (>= 1) or a negative error
+ * (pairs must not exceed the number of tiles nor 128).
+ */
+int nm_pair_tile_plan(int n_tok_tiles, int n_out_tiles, int pairs, int resident, int band_request,
+                      int *start, int *tile_out, int *tile_tok);
+
 /* Host-only validation of a linear-layer problem: NM_OK or the error nm_int_linear would return. */
 int nm_int_linear_check(int tokens, int out, int in, int n, int m, int bits);
 

@@ -31,7 +31,7 @@ EXPORTS = (
     "nm_int_linear", "nm_int_linear_dsx", "nm_int_linear_acc", "nm_int_linear_q8", "nm_int_linear_bf16",
     "nm_int_linear_workspace_bytes",
     "nm_int_linear_check", "nm_absmax", "nm_quantize_act", "nm_poll_status", "nm_strerror",
-    "nm_last_cuda_error", "nm_version", "nm_bits_per_param", "nm_encoder_cost",
+    "nm_last_cuda_error", "nm_version", "nm_bits_per_param", "nm_encoder_cost", "nm_pair_tile_plan",
 )
 
 
@@ -247,6 +247,16 @@ def nm_int_linear_bf16(X, tokens, W, sx, sw, bias, Ybf16, ws=None, ws_bytes=0, s
 
 class nm_component_cfg_t(ctypes.Structure):
     _fields_ = [("n", ctypes.c_int32), ("m", ctypes.c_int32), ("bits", ctypes.c_int32)]
+
+
+def nm_pair_tile_plan(n_tok_tiles, n_out_tiles, pairs, resident, band_request=0):
+    """-> (band, start list [pairs + 1], tile_out list, tile_tok list): the pair kernel's tile walk (host only)."""
+    n = n_tok_tiles * n_out_tiles
+    start = (ctypes.c_int * (pairs + 1))()
+    to, tt = (ctypes.c_int * max(n, 1))(), (ctypes.c_int * max(n, 1))()
+    band = _lib.nm_pair_tile_plan(n_tok_tiles, n_out_tiles, pairs, int(bool(resident)), band_request, start, to, tt)
+    _chk(min(band, 0), "nm_pair_tile_plan")
+    return band, list(start), list(to)[:n], list(tt)[:n]
 
 
 def nm_bits_per_param(n, m, bits, index_bits=-1):

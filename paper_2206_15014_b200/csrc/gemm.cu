@@ -1061,6 +1061,34 @@ static int launch_gemm(const LinearArgs& a) {
     return NM_OK;
 }
 
+// Tile plan of the pair kernel: the band size of the tile order (returned) and start[0..pairs], the contiguous
+// range of every pair.  Resident weights: one long run per output tile (band = all token tiles).  Streamed
+// weights: bands of about one pair's share, unless `band_request` > 0 asks for another size.  The ranges
+// have about equal cost, a tile costing 1 and an output-tile change inside a range `crossing` tiles.
+static int plan_pair_tiles(int n_tok_tiles, int n_out_tiles, int pairs, bool resident, int band_request, int* start) {
+    const int n_tiles = n_tok_tiles * n_out_tiles;
+    int band = n_tok_tiles;
+    if (!resident) {
+        const int b = band_request > 0 ? band_request : (n_tiles + pairs / 2) / pairs;
+        band = b < 1 ? 1 : (b > n_tok_tiles ? n_tok_tiles : b);
+    }
+    const double crossing = resident ? 1.0 : 0.2;
+    auto out_of = [&](int t) { return tile_coord(t, n_tok_tiles, n_out_tiles, band).o; };
+    auto cost = [&](int t) { return 1.0 + ((t > 0 && out_of(t) != out_of(t - 1)) ? crossing : 0.0); };
+    double total = 0.0;
+    for (int t = 0; t < n_tiles; ++t) total += cost(t);
+    int t = 0;
+    double before = 0.0;  // cost of the tiles before t
+    for (int q = 0; q < pairs; ++q) {
+        const double threshold = q * total / pairs;
+        while (t < n_tiles - (pairs - q) && before + 0.5 * cost(t) < threshold) before += cost(t++);
+        if (q > 0 && t <= start[q - 1]) before += cost(t++);  // every pair gets at least one tile
+        start[q] = t;
+    }
+    start[pairs] = n_tiles;
+    return band;
+}
+
 template <bool SPARSE, int BN, int EPI, bool RES>
 static int launch_gemm_pair(const LinearArgs& a) {
     using Cfg = PairCfg<SPARSE, BN, RES>;
@@ -1092,29 +1120,8 @@ static int launch_gemm_pair(const LinearArgs& a) {
     // costs `crossing` tiles (weights resident: ~1, the reload waits for the MMAs to drain; streamed: metadata only).
     // Streamed weights: a change of output tile only costs the metadata, so the tiles are banded by about
     // one pair's share and neighbouring pairs share X tiles in L2.  Resident weights: long runs.
-    p.band = p.n_tok_tiles;
-    if (!RES) {
-        int b = (p.n_tiles + pairs / 2) / pairs;
-        if (const char* e = getenv("NM_BAND")) b = atoi(e);
-        p.band = b < 1 ? 1 : (b > p.n_tok_tiles ? p.n_tok_tiles : b);
-    }
     PairSchedule sched;
-    {
-        const double crossing = RES ? 1.0 : 0.2;
-        auto out_of = [&](int t) { return tile_coord(t, p.n_tok_tiles, p.n_out_tiles, p.band).o; };
-        auto cost = [&](int t) { return 1.0 + ((t > 0 && out_of(t) != out_of(t - 1)) ? crossing : 0.0); };
-        double total = 0.0;
-        for (int t = 0; t < p.n_tiles; ++t) total += cost(t);
-        int t = 0;
-        double before = 0.0;  // cost of the tiles before t
-        for (int q = 0; q < pairs; ++q) {
-            const double threshold = q * total / pairs;
-            while (t < p.n_tiles - (pairs - q) && before + 0.5 * cost(t) < threshold) before += cost(t++);
-            if (q > 0 && t <= sched.start[q - 1]) before += cost(t++);  // every pair gets at least one tile
-            sched.start[q] = t;
-        }
-        sched.start[pairs] = p.n_tiles;
-    }
+    p.band = plan_pair_tiles(p.n_tok_tiles, p.n_out_tiles, pairs, RES, getenv("NM_BAND") ? atoi(getenv("NM_BAND")) : 0, sched.start);
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(2 * pairs, 1, 1);
     cfg.blockDim = dim3(kPairThreads, 1, 1);
@@ -1214,6 +1221,21 @@ static int run_linear(const LinearArgs& a, int epi) {
 }  // namespace nm
 
 extern "C" {
+
+int nm_pair_tile_plan(int n_tok_tiles, int n_out_tiles, int pairs, int resident, int band_request, int* start,
+                      int* tile_out, int* tile_tok) {
+    if (!start) return NM_ERR_NULL;
+    if (n_tok_tiles < 1 || n_out_tiles < 1 || pairs < 1 || pairs > nm::kMaxPairs ||
+        (long long)n_tok_tiles * n_out_tiles > 0x7fffffffll || pairs > n_tok_tiles * n_out_tiles)
+        return NM_ERR_SHAPE;
+    const int band = nm::plan_pair_tiles(n_tok_tiles, n_out_tiles, pairs, resident != 0, band_request, start);
+    for (int t = 0; t < n_tok_tiles * n_out_tiles; ++t) {
+        const nm::TileCoord c = nm::tile_coord(t, n_tok_tiles, n_out_tiles, band);
+        if (tile_out) tile_out[t] = c.o;
+        if (tile_tok) tile_tok[t] = c.t;
+    }
+    return band;
+}
 
 int nm_int_linear_check(int tokens, int out, int in, int n, int m, int bits) {
     return nm::check_linear(tokens, out, in, n, m, bits);

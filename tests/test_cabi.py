@@ -68,3 +68,30 @@ def test_cost_model_reproduces_the_paper_tables():
     assert nm.nm_bits_per_param(3, 2, 8) == -1.0
     # 1:4 and 2:8 run on the 2-of-4 path, 4:8 does not
     assert nm.nm_encoder_cost([(1, 4, 8)] * 6)[1] == 0.5 and nm.nm_encoder_cost([(4, 8, 8)] * 6)[1] == 0.0
+
+
+def test_pair_tile_plan_covers_every_tile_once_in_balanced_ranges():
+    entry.build()
+    import pytest
+    import paper_2206_15014_b200 as nm
+    for n_tok, n_out, pairs, resident, req in [(86, 16, 74, True, 0), (86, 12, 74, True, 0), (86, 4, 74, False, 0),
+                                               (86, 4, 74, False, 1), (86, 4, 74, False, 9), (10, 8, 74, False, 0),
+                                               (7, 3, 21, True, 0), (1, 1, 1, False, 0), (33, 5, 64, False, 200)]:
+        band, start, to, tt = nm.nm_pair_tile_plan(n_tok, n_out, pairs, resident, req)
+        n = n_tok * n_out
+        assert 1 <= band <= n_tok and (band == n_tok if resident else True)
+        # the numbering is a bijection onto the grid, band by band, output-tile-major inside a band
+        assert sorted(zip(to, tt)) == [(o, t) for o in range(n_out) for t in range(n_tok)]
+        for t in range(1, n):
+            same_band = tt[t] // band == tt[t - 1] // band
+            assert (to[t], tt[t]) > (to[t - 1], tt[t - 1]) if same_band else tt[t] // band == tt[t - 1] // band + 1
+        # contiguous, non-empty ranges that cover everything
+        assert start[0] == 0 and start[-1] == n and all(b > a for a, b in zip(start, start[1:]))
+        # equal cost up to one tile and one crossing
+        crossing = 1.0 if resident else 0.2
+        costs = [(b - a) + crossing * sum(1 for t in range(a + 1, b) if to[t] != to[t - 1]) for a, b in zip(start, start[1:])]
+        assert max(costs) - min(costs) <= 1.0 + 2 * crossing + 1e-9, (n_tok, n_out, pairs, costs)
+    for bad in [(0, 4, 2), (4, 4, 17), (4, 4, 200)]:
+        start = (ctypes.c_int * 300)()
+        lib = ctypes.CDLL(nm.LIB_PATH)
+        assert lib.nm_pair_tile_plan(bad[0], bad[1], bad[2], 0, 0, start, None, None) < 0
