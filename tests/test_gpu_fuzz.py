@@ -56,3 +56,49 @@ def test_random_shape(seed):
     if seed % 3 == 0:
         sy = np.float32(max(np.abs(Y_ref).max(), 1e-3)) / np.float32(100.0)
         assert np.array_equal(gpu_int_linear_q8(Xq, packed, sx, b, sy), oracle.requantize_static(Y_ref, sy)), tag
+
+
+PACK_PATTERNS = [(1, 4), (2, 4), (1, 8), (2, 8), (4, 8), (4, 4)]
+
+
+@pytest.mark.parametrize("seed", range(40))
+def test_random_projection(seed):
+    # projection / pack, the ADMM step and group-wise scales on random shapes: row lengths from one group to
+    # several warps per row (not multiples of 1024), a handful to thousands of rows, with and without the dual
+    import torch
+    import paper_2206_15014_b200 as nm
+    from gpu_util import to_dev, DEV
+    rng = np.random.default_rng(2000 + seed)
+    n, m = PACK_PATTERNS[int(rng.integers(0, len(PACK_PATTERNS)))]
+    bits = int(rng.choice([8, 4]))
+    k = 8 * int(rng.integers(1, 1300 if seed % 4 else 40))               # 8 .. 10392, multiples of 8
+    while (k // m * n * bits) % 8:
+        k += 8
+    out = int(rng.integers(1, 3000 if k < 3000 else 300))
+    G = int(rng.choice([1, 7, 32, 64, 0]))
+    W = wl.tie_heavy(3000 + seed, out, k) if seed % 5 == 0 else wl.normal(rng, (out, k), 0.02)
+    U = None if seed % 3 == 0 else wl.normal(rng, (out, k), 0.002)
+    oracle.set_threads(oracle.max_threads())
+    tag = f"out={out} in={k} {n}:{m}/{bits}b G={G}"
+    vb, mb = nm.nm_packed_sizes(out, k, n, m, bits)
+    Wd, Ud = to_dev(W), to_dev(U)
+    status = torch.zeros(1, dtype=torch.int32, device=DEV)
+    # ADMM step with every output
+    Z = torch.empty((out, k), dtype=torch.float32, device=DEV)
+    Un = torch.empty((out, k), dtype=torch.float32, device=DEV)
+    v = torch.zeros(vb, dtype=torch.uint8, device=DEV)
+    mt = torch.zeros(max(mb // 4, 1), dtype=torch.int32, device=DEV) if n != m else None
+    sc = torch.zeros(out, dtype=torch.float32, device=DEV)
+    nm.nm_admm_project(Wd, Ud, out, k, n, m, bits, Z, Un, v, mt, sc, status)
+    assert nm.nm_poll_status(status) == nm.NM_OK
+    Zr, Unr, sr = oracle.admm_step(W, U, n, m, bits)
+    vr, mr, _ = oracle.project_pack(W, U, n, m, bits)
+    assert np.array_equal(Z.cpu().numpy(), Zr) and np.array_equal(Un.cpu().numpy(), Unr), tag
+    assert np.array_equal(sc.cpu().numpy(), sr) and np.array_equal(v.cpu().numpy(), np.asarray(vr).reshape(-1)), tag
+    if mt is not None:
+        assert np.array_equal(mt.cpu().numpy().view(np.uint32)[: mb // 4], np.asarray(mr).reshape(-1)), tag
+    # group-wise scales
+    nm.nm_project_pack_grouped(Wd, Ud, out, k, n, m, bits, G, v, mt, sc, status)
+    assert nm.nm_poll_status(status) == nm.NM_OK
+    vg, mg, sg = oracle.project_pack_grouped(W, U, n, m, bits, G)
+    assert np.array_equal(sc.cpu().numpy(), sg) and np.array_equal(v.cpu().numpy(), np.asarray(vg).reshape(-1)), tag
