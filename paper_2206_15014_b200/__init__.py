@@ -28,6 +28,7 @@ EXPORTS = (
     "nm_packed_sizes", "nm_project_pack", "nm_project_pack_batched", "nm_pack_workspace_bytes",
     "nm_project_pack_batched_noalloc", "nm_admm_project", "nm_admm_project_batched", "nm_admm_workspace_bytes",
     "nm_project_pack_grouped", "nm_admm_project_grouped", "nm_project_pack_grouped_batched",
+    "nm_admm_project_grouped_batched",
     "nm_int_linear", "nm_int_linear_dsx", "nm_int_linear_acc", "nm_int_linear_q8", "nm_int_linear_bf16",
     "nm_int_linear_workspace_bytes",
     "nm_int_linear_check", "nm_absmax", "nm_quantize_act", "nm_poll_status", "nm_strerror",
@@ -60,6 +61,7 @@ _lib.nm_packed_sizes.argtypes = [_i] * 5 + [ctypes.POINTER(_sz), ctypes.POINTER(
 _lib.nm_project_pack.argtypes = [_vp, _vp, _i, _i, _i, _i, _i, _vp, _vp, _vp, _vp, _vp]
 _lib.nm_project_pack_batched.argtypes = [ctypes.POINTER(nm_pack_job_t), _i, _vp, _sz, _vp, _vp]
 _lib.nm_project_pack_batched_noalloc.argtypes = [ctypes.POINTER(nm_pack_job_t), _i, _vp, _vp]
+_lib.nm_admm_project_grouped_batched.argtypes = [ctypes.POINTER(nm_admm_job_t), _i, _i, _vp, _sz, _vp, _vp]
 _lib.nm_project_pack_grouped_batched.argtypes = [ctypes.POINTER(nm_pack_job_t), _i, _i, _vp, _sz, _vp, _vp]
 _lib.nm_project_pack_grouped.argtypes = [_vp, _vp, _i, _i, _i, _i, _i, _i, _vp, _vp, _vp, _vp, _vp]
 _lib.nm_admm_project_grouped.argtypes = [_vp, _vp, _i, _i, _i, _i, _i, _i, _vp, _vp, _vp, _vp, _vp, _vp, _vp]
@@ -182,6 +184,11 @@ def nm_project_pack_grouped(W, U, out, in_, n, m, bits, group_rows, values, meta
 def nm_project_pack_grouped_batched(jobs, njobs, group_rows, ws, ws_bytes, status=None, stream=None):
     _chk(_lib.nm_project_pack_grouped_batched(jobs, njobs, group_rows, _ptr(ws), ws_bytes, _ptr(status),
                                               _stream(stream)), "nm_project_pack_grouped_batched")
+
+
+def nm_admm_project_grouped_batched(jobs, njobs, group_rows, ws, ws_bytes, status=None, stream=None):
+    _chk(_lib.nm_admm_project_grouped_batched(jobs, njobs, group_rows, _ptr(ws), ws_bytes, _ptr(status),
+                                              _stream(stream)), "nm_admm_project_grouped_batched")
 
 
 def nm_admm_project_grouped(W, U, out, in_, n, m, bits, group_rows, Z, U_next, values, meta, scales,

@@ -95,3 +95,14 @@ def test_pair_tile_plan_covers_every_tile_once_in_balanced_ranges():
         start = (ctypes.c_int * 300)()
         lib = ctypes.CDLL(nm.LIB_PATH)
         assert lib.nm_pair_tile_plan(bad[0], bad[1], bad[2], 0, 0, start, None, None) < 0
+
+
+def test_header_is_plain_c():
+    # the boundary is a C ABI: the header must compile as C99 on its own, with warnings as errors
+    import subprocess
+    import tempfile
+    with tempfile.TemporaryDirectory() as d:
+        src = os.path.join(d, "t.c")
+        open(src, "w").write('#include "nmsparse.h"\nint main(void) { return nm_version() > 0 ? 0 : 1; }\n')
+        subprocess.check_call(["gcc", "-std=c99", "-Wall", "-Wextra", "-Werror", "-pedantic", "-I", os.path.join(ROOT, "include"),
+                               "-c", src, "-o", os.path.join(d, "t.o")])

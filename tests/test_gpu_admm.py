@@ -216,3 +216,33 @@ def test_grouped_scales_batched_over_a_heterogeneous_layer(G):
         assert np.array_equal(v.cpu().numpy(), np.asarray(vr).reshape(-1)), idx
         if mt is not None:
             assert np.array_equal(mt.cpu().numpy().view(np.uint32)[: mb // 4], np.asarray(mr).reshape(-1)), idx
+
+
+def test_grouped_admm_step_batched():
+    import paper_2206_15014_b200 as nm
+    from gpu_util import to_dev, DEV
+    cfgs = [(2, 4, 8), (1, 4, 4), (4, 4, 8)]
+    shapes = [(1000, 1024), (300, 4096), (2048, 1024)]
+    G = 32
+    oracle.set_threads(oracle.max_threads())
+    jobs, keep, refs = [], [], []
+    for idx, ((out, k), (n, m, bits)) in enumerate(zip(shapes, cfgs)):
+        W, U = wl.pack_sweep_matrix(3, 90 + idx, out, k)
+        W[7] *= 25
+        Z = torch.empty((out, k), dtype=torch.float32, device=DEV)
+        Un = torch.empty((out, k), dtype=torch.float32, device=DEV)
+        sc = torch.zeros(out, dtype=torch.float32, device=DEV)
+        jobs.append((to_dev(W), to_dev(U), n, m, bits, Z, Un, None, None, sc))
+        keep.append((Z, Un, sc))
+        vr, mr, sr = oracle.project_pack_grouped(W, U, n, m, bits, G)
+        Zr = (sr[:, None] * oracle.unpack(vr, mr, out, k, n, m, bits).astype(np.float32)).astype(np.float32)
+        refs.append((Zr, ((W + U).astype(np.float32) - Zr).astype(np.float32), sr))
+    arr = nm.make_admm_jobs(jobs)
+    ws_bytes = nm.nm_admm_workspace_bytes(len(jobs))
+    ws = torch.empty(ws_bytes, dtype=torch.uint8, device=DEV)
+    status = torch.zeros(1, dtype=torch.int32, device=DEV)
+    nm.nm_admm_project_grouped_batched(arr, len(jobs), G, ws, ws_bytes, status)
+    assert nm.nm_poll_status(status) == nm.NM_OK
+    for idx, ((Z, Un, sc), (Zr, Unr, sr)) in enumerate(zip(keep, refs)):
+        assert np.array_equal(sc.cpu().numpy(), sr), idx
+        assert np.array_equal(Z.cpu().numpy(), Zr) and np.array_equal(Un.cpu().numpy(), Unr), idx
