@@ -468,6 +468,10 @@ template <int N, int M, bool DENSE_OUT>
 static PackFn pick_bits(int bits, int warps) {
     if (warps <= kPackMinWarps)
         return bits == 8 ? (PackFn)pack_kernel<N, M, 8, 128, DENSE_OUT> : (PackFn)pack_kernel<N, M, 4, 128, DENSE_OUT>;
+    if constexpr (DENSE_OUT) {  // the dense outputs need ~128 registers: blocks of at most 512 threads get them
+        if (warps <= 16)
+            return bits == 8 ? (PackFn)pack_kernel<N, M, 8, 512, true> : (PackFn)pack_kernel<N, M, 4, 512, true>;
+    }
     return bits == 8 ? (PackFn)pack_kernel<N, M, 8, 1024, DENSE_OUT> : (PackFn)pack_kernel<N, M, 4, 1024, DENSE_OUT>;
 }
 
