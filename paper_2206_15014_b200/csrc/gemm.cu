@@ -27,6 +27,7 @@
 #include <cuda.h>
 #include <cuda_runtime.h>
 #include <mutex>
+#include <algorithm>
 #include <cstdlib>
 
 namespace nm {
@@ -1089,6 +1090,25 @@ static int plan_pair_tiles(int n_tok_tiles, int n_out_tiles, int pairs, bool res
     return band;
 }
 
+// The plan costs a pass over all tiles on the host; layers are launched again and again with the same shape, so
+// the last few plans are kept.
+static int cached_pair_plan(int n_tok_tiles, int n_out_tiles, int pairs, bool resident, int band_request, PairSchedule& out) {
+    struct Entry { int key[5]; int band; PairSchedule sched; bool used; };
+    static Entry cache[8];
+    static unsigned next = 0;
+    static std::mutex mu;
+    const int key[5] = {n_tok_tiles, n_out_tiles, pairs, resident ? 1 : 0, band_request};
+    std::lock_guard<std::mutex> lock(mu);
+    for (Entry& e : cache)
+        if (e.used && std::equal(key, key + 5, e.key)) { out = e.sched; return e.band; }
+    Entry& e = cache[next++ % 8];
+    std::copy(key, key + 5, e.key);
+    e.band = plan_pair_tiles(n_tok_tiles, n_out_tiles, pairs, resident, band_request, e.sched.start);
+    e.used = true;
+    out = e.sched;
+    return e.band;
+}
+
 template <bool SPARSE, int BN, int EPI, bool RES>
 static int launch_gemm_pair(const LinearArgs& a) {
     using Cfg = PairCfg<SPARSE, BN, RES>;
@@ -1121,7 +1141,7 @@ static int launch_gemm_pair(const LinearArgs& a) {
     // Streamed weights: a change of output tile only costs the metadata, so the tiles are banded by about
     // one pair's share and neighbouring pairs share X tiles in L2.  Resident weights: long runs.
     PairSchedule sched;
-    p.band = plan_pair_tiles(p.n_tok_tiles, p.n_out_tiles, pairs, RES, getenv("NM_BAND") ? atoi(getenv("NM_BAND")) : 0, sched.start);
+    p.band = cached_pair_plan(p.n_tok_tiles, p.n_out_tiles, pairs, RES, getenv("NM_BAND") ? atoi(getenv("NM_BAND")) : 0, sched);
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(2 * pairs, 1, 1);
     cfg.blockDim = dim3(kPairThreads, 1, 1);
