@@ -440,8 +440,7 @@ nm_gemm_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant
             const int tile = tile_begin + i, out_tile = tile / p.n_tok_tiles, buf = i & 1;
             const int n0 = out_tile * kBM, n = n0 + row, t0 = (tile % p.n_tok_tiles) * BN;
             if (SPARSE && i == 0 && half == 0) load_meta(out_tile);
-            // one lane polls, sleeping between polls: the wait spans a whole tile of MMAs
-            bool got = lane != 0 || ptx::mbar_wait_bounded(acc_full_bar(buf), (i >> 1) & 1u, abort_flag, kWaitLimit, true);
+            bool got = ptx::mbar_wait_bounded(acc_full_bar(buf), (i >> 1) & 1u, abort_flag, kWaitLimit);
             ok = __all_sync(0xffffffffu, got);
             if (!ok && lane == 0) raise_timeout();
             if constexpr (kNarrow<EPI>) ok = ptx::named_bar_and(kNarrowAgree + half, 128, ok);  // the group stops together
@@ -823,8 +822,7 @@ nm_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_con
             const int out_tile = tc.o, tok_tile = tc.t, buf = i & 1;
             const int n0 = out_tile * (2 * kBM) + (int)rank * kBM, n = n0 + row, t0 = tok_tile * BN;
             if (SPARSE && i == 0 && half == 0) load_meta(out_tile);
-            // one lane polls, sleeping between polls: the wait spans a whole tile of MMAs
-            bool got = lane != 0 || ptx::mbar_wait_bounded(acc_full_bar(buf), (i >> 1) & 1u, abort_flag, kWaitLimit, true);
+            bool got = ptx::mbar_wait_bounded(acc_full_bar(buf), (i >> 1) & 1u, abort_flag, kWaitLimit);
             ok = __all_sync(0xffffffffu, got);
             if (!ok && lane == 0) raise_timeout();
             if constexpr (kNarrow<EPI>) ok = ptx::named_bar_and(kNarrowAgree + half, 128, ok);  // the group stops together

@@ -36,17 +36,14 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
 
 // Waits for the phase with the given parity; gives up after `limit_cycles` SM clocks or as soon
 // as *abort_flag (shared memory) is set.  Returns false when it gave up.
-// `relaxed`: for waits that last long and whose end is not urgent (an epilogue warp waiting for a whole tile
-// of MMAs): sleep between polls instead of spinning, which leaves issue slots and power to the other warps.
 __device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity,
                                                   volatile uint32_t* abort_flag,
-                                                  long long limit_cycles, bool relaxed = false) {
+                                                  long long limit_cycles) {
     if (mbar_try_wait(bar, parity)) return true;
     const long long t0 = clock64();
     uint32_t spins = 0;
     while (true) {
         if (mbar_try_wait(bar, parity)) return true;
-        if (relaxed) __nanosleep(200);
         if ((++spins & 63u) == 0) {
             if (*abort_flag) return false;
             if (clock64() - t0 > limit_cycles) return false;
