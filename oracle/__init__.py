@@ -101,6 +101,62 @@ def project_pack_grouped(W, U, n, m, bits, group_rows):
     return values, meta, scales
 
 
+def dist_search(W, U, n, m, bits, ncand):
+    """ADMM-Dist candidate sweep -> (E f64 [out, ncand], S f32 [out, ncand], scales f32 [out], cand i32 [out])."""
+    W = np.ascontiguousarray(W, dtype=np.float32)
+    U = None if U is None else np.ascontiguousarray(U, dtype=np.float32)
+    out, inn = W.shape
+    E = np.zeros((out, ncand), dtype=np.float64)
+    S = np.zeros((out, ncand), dtype=np.float32)
+    scales = np.zeros(out, dtype=np.float32)
+    cand = np.zeros(out, dtype=np.int32)
+    _chk(lib().oracle_dist_search(_p(W), _p(U), out, inn, n, m, bits, int(ncand), _p(E), _p(S), _p(scales),
+                                  _p(cand)), "oracle_dist_search")
+    return E, S, scales, cand
+
+
+def _packed_out(out, inn, n, m, bits):
+    vb, mb = packed_sizes(out, inn, n, m, bits)
+    return (np.zeros((out, vb // max(out, 1)), dtype=np.uint8),
+            np.zeros((out, mb // 4 // max(out, 1)), dtype=np.uint32), np.zeros(out, dtype=np.float32), mb)
+
+
+def project_pack_scaled(W, U, n, m, bits, given_scales):
+    """As project_pack with the per-channel scales handed in."""
+    W = np.ascontiguousarray(W, dtype=np.float32)
+    U = None if U is None else np.ascontiguousarray(U, dtype=np.float32)
+    given = np.ascontiguousarray(given_scales, dtype=np.float32)
+    out, inn = W.shape
+    assert given.shape == (out,)
+    values, meta, scales, mb = _packed_out(out, inn, n, m, bits)
+    _chk(lib().oracle_project_pack_scaled(_p(W), _p(U), out, inn, n, m, bits, _p(given), _p(values),
+                                          _p(meta) if mb else None, _p(scales)), "oracle_project_pack_scaled")
+    return values, meta, scales
+
+
+def project_pack_dist(W, U, n, m, bits, ncand):
+    """As project_pack with the ADMM-Dist scale (candidate sweep of dist_search)."""
+    W = np.ascontiguousarray(W, dtype=np.float32)
+    U = None if U is None else np.ascontiguousarray(U, dtype=np.float32)
+    out, inn = W.shape
+    values, meta, scales, mb = _packed_out(out, inn, n, m, bits)
+    _chk(lib().oracle_project_pack_dist(_p(W), _p(U), out, inn, n, m, bits, int(ncand), _p(values),
+                                        _p(meta) if mb else None, _p(scales)), "oracle_project_pack_dist")
+    return values, meta, scales
+
+
+def admm_step_dist(W, U, n, m, bits, ncand, want_u=True):
+    """admm_step with the ADMM-Dist scale."""
+    W = np.ascontiguousarray(W, dtype=np.float32)
+    U = None if U is None else np.ascontiguousarray(U, dtype=np.float32)
+    Z = np.zeros_like(W)
+    Un = np.zeros_like(W) if want_u else None
+    s = np.zeros(W.shape[0], dtype=np.float32)
+    _chk(lib().oracle_admm_step_dist(_p(W), _p(U), W.shape[0], W.shape[1], n, m, bits, int(ncand), _p(Z),
+                                     _p(Un), _p(s)), "oracle_admm_step_dist")
+    return Z, Un, s
+
+
 def project_dense(W, U, n, m):
     W = np.ascontiguousarray(W, dtype=np.float32)
     U = None if U is None else np.ascontiguousarray(U, dtype=np.float32)

@@ -37,6 +37,12 @@
  *   time (8-bit activations handed to the next layer, Sec. 4.5) and binary32 ->
  *   bfloat16 rounding: pinned by closed forms (exact multiples, ties), exact
  *   rational arithmetic, error bounds and an independent conversion routine.
+ *   ADMM-Dist scale (Sec. 3.3.1, "Minimize Quantization Distance"; the paper
+ *   names the objective and gives no search procedure, so the candidate sweep
+ *   is this library's reading): pinned by its one-candidate case (= ADMM-Max),
+ *   by exact rational arithmetic over every candidate on small rows, by the
+ *   distance recomputed from the packed output with the pinned unpack and
+ *   projection routines, and by invariance under powers of two.
  */
 #include <math.h>
 #include <stddef.h>
@@ -258,6 +264,99 @@ int oracle_project_pack_grouped(const float *W, const float *U, int out, int in,
     return rc;
 }
 
+/*
+ * ADMM-Dist (Sec. 3.3.1, "Minimize Quantization Distance"): the scale of an
+ * output channel is the one that minimises the squared Euclidean distance
+ * between the channel and its quantised form.  With the sparsity constraint the
+ * sparsity projection comes first (Sec. 3.3.1, last paragraph), so the distance
+ * is taken over the kept entries: pruned entries are zero on both sides.
+ *
+ * The paper gives no procedure for the minimisation.  Reading taken here: a
+ * sweep over `ncand` candidate scales (1 <= ncand <= 32)
+ *     s_j = fl32(s_max * c_j),  c_j = (64 - j) / 64,  j = 0 .. ncand-1,
+ * where s_max is the ADMM-Max scale of the channel (so j = 0 is ADMM-Max and the
+ * candidates shrink the representable range down to about half of it).  For
+ * every candidate
+ *     E_j = sum over kept k of (v_k - s_j * q_jk)^2,  q_jk = Eq. 5 at scale s_j,
+ * evaluated in double from the fp32 v_k and s_j (the product s_j * q is exact in
+ * double), summed in index order.  The smallest E_j wins, the lowest j on
+ * equality.  An all-zero channel has s_max = 1 and E_j = 0 for all j: j = 0.
+ *
+ * E (nullable) receives E_j as [out][ncand]; S (nullable) the candidate scales
+ * [out][ncand]; scales (nullable) the chosen scale; cand (nullable) the chosen j.
+ */
+int oracle_dist_search(const float *W, const float *U, int out, int in, int n, int m, int bits,
+                       int ncand, double *E, float *S, float *scales, int32_t *cand)
+{
+    if (!shape_ok(out, in, n, m, bits)) return ORACLE_ERR_SHAPE;
+    if (ncand < 1 || ncand > 32) return ORACLE_ERR_SHAPE;
+    int status = ORACLE_OK;
+#pragma omp parallel for schedule(static) num_threads(g_threads)
+    for (int r = 0; r < out; ++r) {
+        float *v = (float *)malloc(sizeof(float) * (size_t)(in > 0 ? in : 1));
+        int *kept = (int *)malloc(sizeof(int) * (size_t)(in > 0 ? in : 1));
+        for (int k = 0; k < in; ++k) {
+            float w = W[(size_t)r * in + k];
+            v[k] = U ? w + U[(size_t)r * in + k] : w;
+        }
+        if (!row_finite(v, in)) {
+#pragma omp atomic write
+            status = ORACLE_ERR_NONFINITE;
+        }
+        size_t nk = 0;
+        for (int g = 0; g < in / m; ++g) {
+            int keep[64];
+            group_support(v + (size_t)g * m, n, m, keep);
+            for (int i = 0; i < n; ++i) kept[nk++] = g * m + keep[i];
+        }
+        const float smax = row_scale(v, in, bits);
+        int best = 0;
+        double best_e = 0.0;
+        float best_s = smax;
+        for (int j = 0; j < ncand; ++j) {
+            const float cj = (float)(64 - j) / 64.0f; /* exact */
+            const float sj = smax * cj;
+            double e = 0.0;
+            for (size_t i = 0; i < nk; ++i) {
+                const float x = v[kept[i]];
+                const int q = quantise(x, sj, bits);
+                const double d = (double)x - (double)sj * (double)q;
+                e += d * d;
+            }
+            if (E) E[(size_t)r * ncand + j] = e;
+            if (S) S[(size_t)r * ncand + j] = sj;
+            if (j == 0 || e < best_e) { best = j; best_e = e; best_s = sj; }
+        }
+        if (scales) scales[r] = best_s;
+        if (cand) cand[r] = best;
+        free(kept);
+        free(v);
+    }
+    return status;
+}
+
+/* The joint projection with scales handed in (one per output channel). */
+int oracle_project_pack_scaled(const float *W, const float *U, int out, int in, int n, int m,
+                               int bits, const float *given_scales, uint8_t *values,
+                               uint32_t *meta, float *scales)
+{
+    return project_pack_impl(W, U, out, in, n, m, bits, given_scales, values, meta, scales);
+}
+
+/* Joint projection with the ADMM-Dist scale: sparsify, search the scale, quantise, pack. */
+int oracle_project_pack_dist(const float *W, const float *U, int out, int in, int n, int m,
+                             int bits, int ncand, uint8_t *values, uint32_t *meta, float *scales)
+{
+    float *gs = (float *)malloc(sizeof(float) * (size_t)(out > 0 ? out : 1));
+    int rc = oracle_dist_search(W, U, out, in, n, m, bits, ncand, NULL, NULL, gs, NULL);
+    if (rc == ORACLE_OK || rc == ORACLE_ERR_NONFINITE) {
+        int rc2 = project_pack_impl(W, U, out, in, n, m, bits, gs, values, meta, scales);
+        if (rc == ORACLE_OK) rc = rc2;
+    }
+    free(gs);
+    return rc;
+}
+
 /* Inverse of the packing: dense integer codes [out, in], zero where pruned. */
 int oracle_unpack(const uint8_t *values, const uint32_t *meta, int out, int in, int n, int m,
                   int bits, int8_t *Wq)
@@ -345,8 +444,8 @@ int oracle_fake_quant(const float *Z, int out, int in, int bits, const float *sc
  * fake-quantiser on a weight that is also N:M-projected (Sec. 3.3.2).
  * scales (nullable) receives s_r.
  */
-int oracle_admm_step(const float *W, const float *U, int out, int in, int n, int m, int bits,
-                     float *Z, float *U_next, float *scales)
+static int admm_step_impl(const float *W, const float *U, int out, int in, int n, int m, int bits,
+                          const float *given_scales, float *Z, float *U_next, float *scales)
 {
     if (n < 1 || n > m || m > 64 || in % m || bits < 2 || bits > 8) return ORACLE_ERR_SHAPE;
     float *v = (float *)malloc((size_t)in * sizeof(float));
@@ -356,7 +455,7 @@ int oracle_admm_step(const float *W, const float *U, int out, int in, int n, int
         size_t base = (size_t)r * in;
         for (int k = 0; k < in; ++k) v[k] = U ? W[base + k] + U[base + k] : W[base + k];
         if (!row_finite(v, in)) { status = ORACLE_ERR_NONFINITE; break; }
-        float s = row_scale(v, in, bits);
+        float s = given_scales ? given_scales[r] : row_scale(v, in, bits);
         if (scales) scales[r] = s;
         for (int g = 0; g < in / m; ++g) {
             int keep[64];
@@ -372,6 +471,24 @@ int oracle_admm_step(const float *W, const float *U, int out, int in, int n, int
     }
     free(v);
     return status;
+}
+
+int oracle_admm_step(const float *W, const float *U, int out, int in, int n, int m, int bits,
+                     float *Z, float *U_next, float *scales)
+{
+    return admm_step_impl(W, U, out, in, n, m, bits, NULL, Z, U_next, scales);
+}
+
+/* The same step with the ADMM-Dist scale (oracle_dist_search) in place of ADMM-Max. */
+int oracle_admm_step_dist(const float *W, const float *U, int out, int in, int n, int m, int bits,
+                          int ncand, float *Z, float *U_next, float *scales)
+{
+    if (!shape_ok(out, in, n, m, bits)) return ORACLE_ERR_SHAPE;
+    float *gs = (float *)malloc(sizeof(float) * (size_t)(out > 0 ? out : 1));
+    int rc = oracle_dist_search(W, U, out, in, n, m, bits, ncand, NULL, NULL, gs, NULL);
+    if (rc == ORACLE_OK) rc = admm_step_impl(W, U, out, in, n, m, bits, gs, Z, U_next, scales);
+    free(gs);
+    return rc;
 }
 
 /*

@@ -565,3 +565,120 @@ def test_grouped_scales_reduce_to_the_per_channel_and_whole_matrix_cases(n, m, b
     own = oracle.unpack(*oracle.project_pack(W2, None, n, m, bits)[:2], 70, 64, n, m, bits)
     shared = oracle.unpack(*oracle.project_pack_grouped(W2, None, n, m, bits, 32)[:2], 70, 64, n, m, bits)
     assert np.abs(shared[1]).max() < np.abs(own[1]).max()
+
+
+# ---- ADMM-Dist: the scale that minimises the quantisation distance (Sec. 3.3.1) ---------------------------
+
+def _dist_inputs(kind, seed, out, k):
+    rng = np.random.default_rng(seed)
+    if kind == "normal":
+        return wl.normal(rng, (out, k), 0.02), wl.normal(rng, (out, k), 0.002)
+    if kind == "ties":
+        return wl.tie_heavy(seed, out, k), None
+    return wl.with_outliers(seed, out, k), None
+
+
+@pytest.mark.parametrize("n,m,bits", [(2, 4, 8), (2, 4, 4), (1, 4, 4), (2, 8, 8), (4, 8, 4), (4, 4, 4)])
+def test_dist_one_candidate_is_admm_max(n, m, bits):
+    W, U = _dist_inputs("normal", 51, 20, 64)
+    a, b = oracle.project_pack_dist(W, U, n, m, bits, 1), oracle.project_pack(W, U, n, m, bits)
+    assert all(np.array_equal(x, y) for x, y in zip(a, b))
+    E, S, s, c = oracle.dist_search(W, U, n, m, bits, 7)
+    assert np.array_equal(S[:, 0], b[2]) and (c < 7).all() and (c >= 0).all()
+
+
+@pytest.mark.parametrize("kind", ["normal", "ties", "outliers"])
+@pytest.mark.parametrize("n,m,bits", [(2, 4, 8), (2, 4, 4), (1, 4, 8), (2, 8, 4), (4, 8, 8), (4, 4, 4)])
+def test_dist_search_against_exact_rational_arithmetic(kind, n, m, bits):
+    """Every candidate's distance recomputed without rounding: numpy's fp32 division and rint give the codes,
+    fractions give the sum; the sparsity projection comes from the separately pinned dense routine."""
+    out, k, ncand = 6, 32, 32
+    W, U = _dist_inputs(kind, 52, out, k)
+    E, S, s, c = oracle.dist_search(W, U, n, m, bits, ncand)
+    P = oracle.project_dense(W, U, n, m)                     # zero where pruned
+    V = W if U is None else (W + U).astype(np.float32)
+    qmax = np.float32(2 ** (bits - 1) - 1)
+    lo, hi = -(2 ** (bits - 1)), 2 ** (bits - 1) - 1
+    for r in range(out):
+        a = np.abs(V[r]).max()
+        smax = np.float32(1.0) if a == 0 else np.float32(a) / qmax
+        exact = []
+        for j in range(ncand):
+            sj = np.float32(smax * np.float32((64 - j) / 64.0))
+            assert S[r, j] == sj
+            q = np.clip(np.rint(P[r] / sj), lo, hi).astype(np.int64)     # fp32 quotient, half to even
+            e = sum((Fraction(float(x)) - Fraction(float(sj)) * int(qq)) ** 2 for x, qq in zip(P[r], q))
+            exact.append(e)
+            assert abs(float(e) - E[r, j]) <= 1e-12 * float(e) + 1e-300
+        best = min(range(ncand), key=lambda j: (exact[j], j))             # lowest j on equality
+        runner = min(exact[j] for j in range(ncand) if j != best)
+        if runner == exact[best] or float(runner - exact[best]) > 1e-12 * float(exact[best]):
+            assert c[r] == best
+        assert exact[c[r]] <= exact[best] * (1 + Fraction(1, 10 ** 12))
+        assert s[r] == S[r, c[r]]
+
+
+@pytest.mark.parametrize("n,m,bits", [(2, 4, 8), (2, 4, 4), (1, 8, 4), (4, 8, 4)])
+def test_dist_error_is_the_distance_of_the_packed_output(n, m, bits):
+    out, k, ncand = 40, 256, 32
+    W, U = _dist_inputs("normal", 53, out, k)
+    E, S, s, c = oracle.dist_search(W, U, n, m, bits, ncand)
+    P = oracle.project_dense(W, U, n, m).astype(np.float64)
+    for packed, col in ((oracle.project_pack_dist(W, U, n, m, bits, ncand), c),
+                        (oracle.project_pack(W, U, n, m, bits), np.zeros(out, np.int64))):
+        v, meta, sc = packed
+        D = oracle.unpack(v, meta, out, k, n, m, bits).astype(np.float64)
+        dist = ((sc.astype(np.float64)[:, None] * D - P) ** 2).sum(axis=1)
+        assert np.allclose(dist, E[np.arange(out), col], rtol=1e-11, atol=0)
+    # never worse than ADMM-Max, and the minimum over the sweep
+    assert (E[np.arange(out), c] <= E[:, 0]).all() and np.array_equal(E[np.arange(out), c], E.min(axis=1))
+    assert np.array_equal(c, E.argmin(axis=1))                # numpy's argmin: first minimum
+    # the metadata (support) does not depend on the scale
+    assert np.array_equal(oracle.project_pack_dist(W, U, n, m, bits, ncand)[1], oracle.project_pack(W, U, n, m, bits)[1])
+    # handing the chosen scales in gives the same bytes
+    a, b = oracle.project_pack_dist(W, U, n, m, bits, ncand), oracle.project_pack_scaled(W, U, n, m, bits, s)
+    assert all(np.array_equal(x, y) for x, y in zip(a, b))
+
+
+def test_dist_pays_at_four_bits_and_not_at_eight():
+    """Gaussian rows of 1024: with 7 levels a side the best scale clips the tail (c well below 1); with 127 the
+    row maximum (about 3.2 sigma) is already near the best range."""
+    W, _ = _dist_inputs("normal", 54, 48, 1024)
+    E4, _, _, c4 = oracle.dist_search(W, None, 2, 4, 4, 32)
+    E8, _, _, c8 = oracle.dist_search(W, None, 2, 4, 8, 32)
+    assert (c4 >= 4).mean() > 0.9 and (E4[np.arange(48), c4] < 0.9 * E4[:, 0]).mean() > 0.9
+    assert (c8 <= 3).all() and (E8[np.arange(48), c8] > 0.75 * E8[:, 0]).all()
+    assert c4.max() < 31                                        # the sweep's range contains the minimum
+
+
+def test_dist_power_of_two_invariance_zero_rows_and_arguments():
+    W, U = _dist_inputs("outliers", 55, 12, 64)                 # has an all-zero row and zero groups
+    base = oracle.project_pack_dist(W, None, 2, 4, 4, 32)
+    E, S, s, c = oracle.dist_search(W, None, 2, 4, 4, 32)
+    z = 12 // 2
+    assert c[z] == 0 and s[z] == 1.0 and (E[z] == 0).all() and not base[0][z].any()
+    for p in (-20, 7):
+        f = np.float32(2.0 ** p)
+        v, meta, sc = oracle.project_pack_dist(W * f, None, 2, 4, 4, 32)
+        nz = np.arange(12) != z
+        assert np.array_equal(v, base[0]) and np.array_equal(meta, base[1]) and np.array_equal(sc[nz], base[2][nz] * f)
+    for bad in (0, 33):
+        with pytest.raises(RuntimeError):
+            oracle.dist_search(W, None, 2, 4, 4, bad)
+    # clipping reaches the most negative code, which ADMM-Max never produces
+    Wn = np.zeros((1, 64), np.float32); Wn[0, ::2] = 0.01; Wn[0, 0] = -0.05; Wn[0, 2] = 0.05
+    v, meta, sc = oracle.project_pack_dist(Wn, None, 2, 4, 4, 32)
+    D = oracle.unpack(v, meta, 1, 64, 2, 4, 4)
+    assert sc[0] < np.float32(0.05) / 7 and D.min() == -8 and D.max() == 7
+
+
+@pytest.mark.parametrize("n,m,bits", [(2, 4, 4), (1, 4, 8), (4, 4, 4)])
+def test_admm_step_dist_is_the_composition(n, m, bits):
+    W, U = _dist_inputs("normal", 56, 16, 128)
+    Z, Un, s = oracle.admm_step_dist(W, U, n, m, bits, 32)
+    v, meta, s2 = oracle.project_pack_dist(W, U, n, m, bits, 32)
+    D = oracle.unpack(v, meta, 16, 128, n, m, bits)
+    V = (W + U).astype(np.float32)
+    assert np.array_equal(s, s2) and np.array_equal(Z, (s[:, None] * D.astype(np.float32)).astype(np.float32))
+    assert np.array_equal(Un, (V - Z).astype(np.float32))
+    assert np.array_equal(Z, oracle.fake_quant(oracle.project_dense(W, U, n, m), bits, s))
