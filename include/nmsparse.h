@@ -158,6 +158,37 @@ int nm_admm_project_grouped_batched(const nm_admm_job_t *jobs, int njobs, int gr
                                     size_t ws_bytes, uint32_t *status, void *stream);
 
 /*
+ * ADMM-Dist scale (Sec. 3.3.1, "Minimize Quantization Distance"): per output channel the scale that
+ * minimises the squared Euclidean distance between the channel and its quantised form.  With N:M
+ * sparsity the sparsity projection comes first (Sec. 3.3.1, last paragraph), so the distance runs
+ * over the kept entries of V = W + U.  The paper states the objective and no procedure; this
+ * library sweeps `ncand` candidates (1 .. NM_DIST_MAX_CANDIDATES)
+ *     s_j = fl32(s_max * (64 - j) / 64),  j = 0 .. ncand-1,  s_max = the ADMM-Max scale of the row,
+ * evaluates E_j = sum over kept k of (v_k - s_j * code_jk)^2 in double (code_jk = Eq. 5 at scale
+ * s_j), and takes the smallest E_j, the lowest j among equal ones.  ncand = 1 is ADMM-Max.
+ *   nm_dist_scales        scales[out] <- the chosen scale; cand[out] (device int32, nullable) <- j.
+ *   nm_project_pack_dist  the search, then nm_project_pack with that scale (codes beyond the
+ *                         shrunken range clamp to -2^(bits-1) / 2^(bits-1)-1 as Eq. 5 says).
+ *   nm_admm_project_dist  the search, then nm_admm_project with that scale; `scales` is required.
+ *   nm_project_pack_dist_batched  many matrices (jobs, ws as for nm_project_pack_batched): per
+ *                         group of jobs that share (n, m, bits) and block size one launch searches
+ *                         and one projects and packs.
+ * Two passes over W and U (the second is served from L2 for matrices that fit there).  The search
+ * is bound by arithmetic, not by memory.  Pointers, shapes, errors and the NM_STATUS_NONFINITE bit
+ * as for nm_project_pack; ncand out of range returns NM_ERR_SHAPE.  Which of two candidates whose
+ * distances agree to the last few bits of a double wins depends on the order of the summation.
+ */
+#define NM_DIST_MAX_CANDIDATES 32
+int nm_dist_scales(const float *W, const float *U, int out, int in, int n, int m, int bits, int ncand,
+                   float *scales, int32_t *cand, uint32_t *status, void *stream);
+int nm_project_pack_dist(const float *W, const float *U, int out, int in, int n, int m, int bits,
+                         int ncand, void *values, void *meta, float *scales, uint32_t *status,
+                         void *stream);
+int nm_admm_project_dist(const float *W, const float *U, int out, int in, int n, int m, int bits,
+                         int ncand, float *Z, float *U_next, void *values, void *meta, float *scales,
+                         uint32_t *status, void *stream);
+
+/*
  * The same for a list of matrices with as few launches as their (n, m, bits) allow (one when all
  * jobs share them).  `jobs` is a host array; `ws` is device scratch of at least
  * nm_pack_workspace_bytes(njobs) bytes, 16-byte aligned, which must stay untouched until the
@@ -166,6 +197,8 @@ int nm_admm_project_grouped_batched(const nm_admm_job_t *jobs, int njobs, int gr
 int nm_project_pack_batched(const nm_pack_job_t *jobs, int njobs, void *ws, size_t ws_bytes,
                             uint32_t *status, void *stream);
 size_t nm_pack_workspace_bytes(int njobs);
+int nm_project_pack_dist_batched(const nm_pack_job_t *jobs, int njobs, int ncand, void *ws,
+                                 size_t ws_bytes, uint32_t *status, void *stream);
 
 /*
  * nm_project_pack_batched for callers that cannot provide scratch memory.  (The paper has no

@@ -29,6 +29,7 @@ EXPORTS = (
     "nm_project_pack_batched_noalloc", "nm_admm_project", "nm_admm_project_batched", "nm_admm_workspace_bytes",
     "nm_project_pack_grouped", "nm_admm_project_grouped", "nm_project_pack_grouped_batched",
     "nm_admm_project_grouped_batched",
+    "nm_dist_scales", "nm_project_pack_dist", "nm_admm_project_dist", "nm_project_pack_dist_batched",
     "nm_int_linear", "nm_int_linear_dsx", "nm_int_linear_acc", "nm_int_linear_q8", "nm_int_linear_bf16",
     "nm_int_linear_workspace_bytes",
     "nm_int_linear_check", "nm_absmax", "nm_quantize_act", "nm_poll_status", "nm_strerror",
@@ -65,6 +66,10 @@ _lib.nm_admm_project_grouped_batched.argtypes = [ctypes.POINTER(nm_admm_job_t), 
 _lib.nm_project_pack_grouped_batched.argtypes = [ctypes.POINTER(nm_pack_job_t), _i, _i, _vp, _sz, _vp, _vp]
 _lib.nm_project_pack_grouped.argtypes = [_vp, _vp, _i, _i, _i, _i, _i, _i, _vp, _vp, _vp, _vp, _vp]
 _lib.nm_admm_project_grouped.argtypes = [_vp, _vp, _i, _i, _i, _i, _i, _i, _vp, _vp, _vp, _vp, _vp, _vp, _vp]
+_lib.nm_dist_scales.argtypes = [_vp, _vp, _i, _i, _i, _i, _i, _i, _vp, _vp, _vp, _vp]
+_lib.nm_project_pack_dist.argtypes = [_vp, _vp, _i, _i, _i, _i, _i, _i, _vp, _vp, _vp, _vp, _vp]
+_lib.nm_admm_project_dist.argtypes = [_vp, _vp, _i, _i, _i, _i, _i, _i, _vp, _vp, _vp, _vp, _vp, _vp, _vp]
+_lib.nm_project_pack_dist_batched.argtypes = [ctypes.POINTER(nm_pack_job_t), _i, _i, _vp, _sz, _vp, _vp]
 _lib.nm_admm_project_batched.argtypes = [ctypes.POINTER(nm_admm_job_t), _i, _vp, _sz, _vp, _vp]
 _lib.nm_admm_project.argtypes = [_vp, _vp, _i, _i, _i, _i, _i, _vp, _vp, _vp, _vp, _vp, _vp, _vp]
 _lib.nm_admm_workspace_bytes.argtypes = [_i]
@@ -174,6 +179,30 @@ def nm_admm_project(W, U, out, in_, n, m, bits, Z, U_next=None, values=None, met
                     status=None, stream=None):
     _chk(_lib.nm_admm_project(_ptr(W), _ptr(U), out, in_, n, m, bits, _ptr(Z), _ptr(U_next), _ptr(values),
                               _ptr(meta), _ptr(scales), _ptr(status), _stream(stream)), "nm_admm_project")
+
+
+NM_DIST_MAX_CANDIDATES = 32
+
+
+def nm_dist_scales(W, U, out, in_, n, m, bits, ncand, scales, cand=None, status=None, stream=None):
+    _chk(_lib.nm_dist_scales(_ptr(W), _ptr(U), out, in_, n, m, bits, ncand, _ptr(scales), _ptr(cand), _ptr(status),
+                             _stream(stream)), "nm_dist_scales")
+
+
+def nm_project_pack_dist(W, U, out, in_, n, m, bits, ncand, values, meta, scales, status=None, stream=None):
+    _chk(_lib.nm_project_pack_dist(_ptr(W), _ptr(U), out, in_, n, m, bits, ncand, _ptr(values), _ptr(meta),
+                                   _ptr(scales), _ptr(status), _stream(stream)), "nm_project_pack_dist")
+
+
+def nm_admm_project_dist(W, U, out, in_, n, m, bits, ncand, Z, U_next, values, meta, scales, status=None,
+                         stream=None):
+    _chk(_lib.nm_admm_project_dist(_ptr(W), _ptr(U), out, in_, n, m, bits, ncand, _ptr(Z), _ptr(U_next), _ptr(values),
+                                   _ptr(meta), _ptr(scales), _ptr(status), _stream(stream)), "nm_admm_project_dist")
+
+
+def nm_project_pack_dist_batched(jobs, njobs, ncand, ws, ws_bytes, status=None, stream=None):
+    _chk(_lib.nm_project_pack_dist_batched(jobs, njobs, ncand, _ptr(ws), ws_bytes, _ptr(status), _stream(stream)),
+         "nm_project_pack_dist_batched")
 
 
 def nm_project_pack_grouped(W, U, out, in_, n, m, bits, group_rows, values, meta, scales, status=None, stream=None):

@@ -460,6 +460,200 @@ static int launch_group_scales(const float* W, const float* U, int out, int in, 
 }
 
 // ---------------------------------------------------------------------------------------------
+// ADMM-Dist scale (Sec. 3.3.1, "Minimize Quantization Distance"): per output channel the scale that
+// minimises the squared distance between the N:M-projected channel and its quantised form, searched
+// over the candidates s_j = fl32(s_max * (64 - j) / 64), j = 0 .. ncand-1 (s_max = the ADMM-Max scale;
+// lowest j on equal distance).  The kernel writes the winning scale to `scales`; the projection /
+// packing kernel then runs with the scales handed in.
+//
+// Same decomposition as pack_kernel: a warp owns 1024 consecutive weights, a lane 32 consecutive ones,
+// of which it keeps G*N in registers (as fp32 for the quantiser, as fp64 for the distance).  Per
+// candidate and kept value: the code from the reciprocal product (true division when the quotient is
+// within 2^-15 of a rounding tie or the scale is outside the range where the reciprocal is accurate),
+// turned into a double through the 2^52 trick, then d = v - s*code and E += d*d as two fp64 FMAs (the
+// product s*code is exact in double).  E is summed per lane, over the lanes by a butterfly, over the
+// warps of a row through shared memory: a fixed order, so the result is deterministic.  The work is
+// bound by instruction issue (about 15 instructions per candidate and kept value), not by HBM.
+// ---------------------------------------------------------------------------------------------
+template <int N, int M>
+__device__ __forceinline__ void kept_values(const float* v, float* sel) {
+    if constexpr (N == M) {
+#pragma unroll
+        for (int p = 0; p < M; ++p) sel[p] = v[p];
+    } else if constexpr ((N == 1) || (N == 2 && M == 8)) {
+        unsigned selp[N];
+        select_passes<N, M>(v, sel, selp);
+    } else {
+        float a[M];
+#pragma unroll
+        for (int p = 0; p < M; ++p) a[p] = fabsf(v[p]);
+        const unsigned mask = keep_mask<N, M>(a);
+        if constexpr (N == 2 && M == 4) {
+            const bool b0 = mask & 1u, b1 = mask & 2u, b2 = mask & 4u, b3 = mask & 8u;
+            sel[0] = b0 ? v[0] : (b1 ? v[1] : v[2]);
+            sel[1] = b3 ? v[3] : (b2 ? v[2] : v[1]);
+        } else {
+#pragma unroll
+            for (int c = 0; c < N; ++c) sel[c] = 0.0f;
+#pragma unroll
+            for (int p = 0; p < M; ++p) {
+                const bool kept = (mask >> p) & 1u;
+                const int before = __popc(mask & ((1u << p) - 1u));
+#pragma unroll
+                for (int c = 0; c < N; ++c)
+                    if (c <= p && (M - p) >= (N - c)) sel[c] = (kept && before == c) ? v[p] : sel[c];
+            }
+        }
+    }
+}
+
+template <int N, int M, int BITS, int MAXT>
+__global__ void __launch_bounds__(MAXT, MAXT == 128 ? 4 : 1) dist_scale_kernel(const PackJobDev* __restrict__ jobs, int njobs,
+                                                                              PackJobDev single, uint32_t* status, int ncand,
+                                                                              int32_t* __restrict__ cand_out) {
+    constexpr int G = 32 / M;
+    constexpr int KN = G * N;  // kept values per lane
+    extern __shared__ float4 tile[];  // [warps][256] float4, [warps][32] doubles, [warps] floats
+    const int warps = blockDim.x >> 5;
+    double* red_e = reinterpret_cast<double*>(tile + warps * 256);
+    float* red = reinterpret_cast<float*>(red_e + warps * 32);
+
+    PackJobDev job;
+    if (jobs) {
+        int lo = 0, hi = njobs - 1;  // last job whose unit_begin <= blockIdx.x
+        while (lo < hi) {
+            int mid = (lo + hi + 1) >> 1;
+            if (jobs[mid].unit_begin <= blockIdx.x) lo = mid; else hi = mid - 1;
+        }
+        job = jobs[lo];
+    } else {
+        job = single;
+    }
+    const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+    const int wpr = 1 << job.wpr_log2;
+    const int row_in_block = w >> job.wpr_log2, chunk = w & (wpr - 1);
+    const int rows_per_block = warps >> job.wpr_log2;
+    const long long row = (long long)(blockIdx.x - job.unit_begin) * rows_per_block + row_in_block;
+    const bool row_ok = row < job.out;
+    const int in4 = job.in >> 2;
+
+    // ---- V = W + U (coalesced; kept in cache for the projection pass that follows), |max|, transpose ----
+    float4* mytile = tile + w * 256;
+    float amax = 0.0f, poison = 0.0f;
+    {
+        const float4* W4 = reinterpret_cast<const float4*>(job.W) + (row_ok ? row * in4 : 0);
+        const float4* U4 = job.U ? reinterpret_cast<const float4*>(job.U) + (row_ok ? row * in4 : 0) : nullptr;
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            const int f = chunk * 256 + j * 32 + lane;
+            float4 t = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (row_ok && f < in4) {
+                t = __ldg(W4 + f);
+                if (U4) {
+                    const float4 u = __ldg(U4 + f);
+                    t.x = __fadd_rn(t.x, u.x); t.y = __fadd_rn(t.y, u.y);
+                    t.z = __fadd_rn(t.z, u.z); t.w = __fadd_rn(t.w, u.w);
+                }
+            }
+            amax = fmaxf(amax, fmaxf(fmaxf(fabsf(t.x), fabsf(t.y)), fmaxf(fabsf(t.z), fabsf(t.w))));
+            poison = __fmaf_rn(t.x, 0.0f, poison); poison = __fmaf_rn(t.y, 0.0f, poison);
+            poison = __fmaf_rn(t.z, 0.0f, poison); poison = __fmaf_rn(t.w, 0.0f, poison);
+            const int fl = j * 32 + lane, owner = fl >> 3, jj = fl & 7;
+            mytile[owner * 8 + (jj ^ (owner & 7))] = t;
+        }
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, o));
+    const bool bad = __any_sync(0xffffffffu, poison != poison) || !(amax <= 3.402823466e+38f);
+    if (bad && lane == 0 && status) atomicOr(status, NM_STATUS_NONFINITE);
+    if (wpr > 1) {
+        if (lane == 0) red[w] = amax;
+        __syncthreads();
+        for (int c = 0; c < wpr; ++c) amax = fmaxf(amax, red[row_in_block * wpr + c]);
+    } else {
+        __syncwarp();
+    }
+
+    // ---- this lane's kept values (columns beyond the row were loaded as zeros: they add nothing) --------
+    float x[KN];
+    double xd[KN];
+    {
+        float v[32];
+#pragma unroll
+        for (int jj = 0; jj < 8; ++jj) {
+            const float4 t = mytile[lane * 8 + (jj ^ (lane & 7))];
+            v[jj * 4 + 0] = t.x; v[jj * 4 + 1] = t.y; v[jj * 4 + 2] = t.z; v[jj * 4 + 3] = t.w;
+        }
+#pragma unroll
+        for (int g = 0; g < G; ++g) kept_values<N, M>(v + g * M, x + g * N);
+#pragma unroll
+        for (int i = 0; i < KN; ++i) xd[i] = (double)x[i];
+    }
+
+    constexpr float qmax = (float)((1 << (BITS - 1)) - 1);
+    constexpr float kLo = -(float)(1 << (BITS - 1)) - 0.49f, kHi = qmax + 0.49f;
+    constexpr float kMagic = 12582912.0f;             // 1.5 * 2^23 = 0x4B400000
+    constexpr double kMagicD = 4503601774854144.0;    // 2^52 + 2^31
+    const float smax = (amax == 0.0f) ? 1.0f : __fdiv_rn(amax, qmax);
+    double mine = __longlong_as_double(0x7ff0000000000000ll);  // lane j ends up with candidate j's distance
+    for (int j = 0; j < ncand; ++j) {
+        const float sj = __fmul_rn(smax, (float)(64 - j) * 0.015625f);
+        const float rj = __frcp_rn(sj);
+        const double nsd = -(double)sj;
+        // outside [2^-126, 2^125] the reciprocal is subnormal, infinite or the product loses bits
+        const bool fast_ok = (sj >= 1.17549435e-38f) && (sj <= 4.25e37f);
+        unsigned lo[KN];
+        bool near_tie = !fast_ok;
+#pragma unroll
+        for (int i = 0; i < KN; ++i) {
+            const float qc = fminf(fmaxf(__fmul_rn(x[i], rj), kLo), kHi);
+            const float t = __fadd_rn(qc, kMagic);
+            const float f = __fsub_rn(qc, __fsub_rn(t, kMagic));
+            near_tie |= !(fabsf(f) <= 0.49996948f);
+            lo[i] = (unsigned)__float_as_int(t) + 0x34C00000u;  // (code) ^ 0x80000000
+        }
+        if (near_tie) {
+#pragma unroll
+            for (int i = 0; i < KN; ++i) {
+                const float qc = fminf(fmaxf(__fdiv_rn(x[i], sj), kLo), kHi);
+                lo[i] = (unsigned)__float_as_int(__fadd_rn(qc, kMagic)) + 0x34C00000u;
+            }
+        }
+        double e0 = 0.0, e1 = 0.0;
+#pragma unroll
+        for (int i = 0; i < KN; ++i) {
+            const double qd = __hiloint2double(0x43300000, (int)lo[i]) - kMagicD;  // the code as a double
+            const double d = fma(nsd, qd, xd[i]);
+            if (i & 1) e1 = fma(d, d, e1); else e0 = fma(d, d, e0);
+        }
+        double e = e0 + e1;
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) e += __shfl_xor_sync(0xffffffffu, e, o);
+        if (lane == j) mine = e;
+    }
+    if (wpr > 1) {
+        red_e[w * 32 + lane] = mine;
+        __syncthreads();
+        mine = 0.0;
+        for (int c = 0; c < wpr; ++c) mine += red_e[(row_in_block * wpr + c) * 32 + lane];
+    }
+    int bj = lane;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        const double oe = __shfl_xor_sync(0xffffffffu, mine, o);
+        const int oj = __shfl_xor_sync(0xffffffffu, bj, o);
+        const bool take = (oe < mine) || (oe == mine && oj < bj);
+        mine = take ? oe : mine;
+        bj = take ? oj : bj;
+    }
+    if (bj >= ncand) bj = 0;  // only when every distance is NaN or infinite (non-finite input, flagged above)
+    if (row_ok && chunk == 0 && lane == 0) {
+        job.scales[row] = __fmul_rn(smax, (float)(64 - bj) * 0.015625f);
+        if (cand_out) cand_out[row] = bj;
+    }
+}
+
+// ---------------------------------------------------------------------------------------------
 // host side
 // ---------------------------------------------------------------------------------------------
 using PackFn = void (*)(const PackJobDev*, int, PackJobDev, uint32_t*, float*, float*, const DenseOutDev*, int, int);
@@ -525,11 +719,50 @@ static int launch(PackFn fn, const PackJobDev* jobs_dev, int njobs, const PackJo
     return NM_OK;
 }
 
+using DistFn = void (*)(const PackJobDev*, int, PackJobDev, uint32_t*, int, int32_t*);
+
+template <int N, int M>
+static DistFn pick_dist_bits(int bits, int warps) {
+    if (warps <= kPackMinWarps)
+        return bits == 8 ? (DistFn)dist_scale_kernel<N, M, 8, 128> : (DistFn)dist_scale_kernel<N, M, 4, 128>;
+    if (warps <= 16)  // the kept values as fp32 and fp64 need up to ~128 registers
+        return bits == 8 ? (DistFn)dist_scale_kernel<N, M, 8, 512> : (DistFn)dist_scale_kernel<N, M, 4, 512>;
+    return bits == 8 ? (DistFn)dist_scale_kernel<N, M, 8, 1024> : (DistFn)dist_scale_kernel<N, M, 4, 1024>;
+}
+
+static DistFn pick_dist(int n, int m, int bits, int warps) {
+    if (n == m) return pick_dist_bits<4, 4>(bits, warps);
+    if (m == 4) return n == 1 ? pick_dist_bits<1, 4>(bits, warps) : pick_dist_bits<2, 4>(bits, warps);
+    if (n == 1) return pick_dist_bits<1, 8>(bits, warps);
+    if (n == 2) return pick_dist_bits<2, 8>(bits, warps);
+    return pick_dist_bits<4, 8>(bits, warps);
+}
+
+static int launch_dist(DistFn fn, const PackJobDev* jobs_dev, int njobs, const PackJobDev& single, unsigned blocks,
+                       int warps, uint32_t* status, cudaStream_t stream, int ncand, int32_t* cand) {
+    size_t smem = (size_t)warps * (256 * sizeof(float4) + 32 * sizeof(double) + sizeof(float));
+    if (smem > 48 * 1024)
+        NM_CUDA_TRY(cudaFuncSetAttribute((const void*)fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    fn<<<blocks, warps * 32, smem, stream>>>(jobs_dev, njobs, single, status, ncand, cand);
+    NM_CUDA_TRY(cudaGetLastError());
+    return NM_OK;
+}
+
+// One matrix: the ADMM-Dist scales into job.scales (and the winning candidate numbers into `cand`).
+static int launch_dist_single(const nm_pack_job_t& j, int ncand, int32_t* cand, uint32_t* status, cudaStream_t stream) {
+    PackJobDev d = to_dev(j);
+    const int warps = std::max(kPackMinWarps, 1 << d.wpr_log2);
+    const int rows_per_block = warps >> d.wpr_log2;
+    const unsigned blocks = (unsigned)((j.out + rows_per_block - 1) / rows_per_block);
+    return launch_dist(pick_dist(j.n, j.m, j.bits, warps), nullptr, 0, d, blocks, warps, status, stream, ncand, cand);
+}
+
 // Shared by the batched entry points: groups the jobs that can share one launch (same pattern, code width
 // and block size), writes the device job table(s) into `ws` and launches one kernel per group.
 template <bool DENSE_OUT>
 static int launch_batched(const nm_pack_job_t* jobs, const DenseOutDev* dense, int njobs, void* ws,
-                          uint32_t* status, cudaStream_t s, bool grouped = false, int group_rows = 0) {
+                          uint32_t* status, cudaStream_t s, bool grouped = false, int group_rows = 0,
+                          int dist_ncand = 0) {
     // Group jobs that can share one launch: same (n == m ? dense : n, m), bits and block size.
     struct Key { int n, m, bits, warps; };
     std::vector<Key> keys;
@@ -587,12 +820,22 @@ static int launch_batched(const nm_pack_job_t* jobs, const DenseOutDev* dense, i
             NM_CUDA_TRY(cudaGetLastError());
         }
     }
+    if (dist_ncand > 0) {
+        // ADMM-Dist: the scale search writes every job's scales, the projection below takes them
+        for (size_t g = 0; g < keys.size(); ++g) {
+            const nm::PackJobDev* dev = reinterpret_cast<const nm::PackJobDev*>(ws) + group_first[g];
+            int rc = nm::launch_dist(nm::pick_dist(keys[g].n, keys[g].m, keys[g].bits, keys[g].warps), dev,
+                                     (int)groups[g].size(), nm::PackJobDev{}, group_blocks[g], keys[g].warps, status, s,
+                                     dist_ncand, nullptr);
+            if (rc != NM_OK) return rc;
+        }
+    }
     for (size_t g = 0; g < keys.size(); ++g) {
         const nm::PackJobDev* dev = reinterpret_cast<const nm::PackJobDev*>(ws) + group_first[g];
         int rc = nm::launch(nm::pick_kernel<DENSE_OUT>(keys[g].n, keys[g].m, keys[g].bits, keys[g].warps), dev,
                             (int)groups[g].size(), nm::PackJobDev{}, group_blocks[g], keys[g].warps,
                             status, s, nullptr, nullptr, DENSE_OUT ? dense_dev + group_first[g] : nullptr,
-                            grouped ? kGroupScalesGiven : kGroupNone, group_rows);
+                            (grouped || dist_ncand > 0) ? kGroupScalesGiven : kGroupNone, group_rows);
         if (rc != NM_OK) return rc;
     }
     return NM_OK;
@@ -675,6 +918,72 @@ int nm_admm_project_grouped(const float* W, const float* U, int out, int in, int
     unsigned blocks = (unsigned)((out + rows_per_block - 1) / rows_per_block);
     return nm::launch(nm::pick_kernel<true>(n, m, bits, warps), nullptr, 0, d, blocks, warps, status,
                       (cudaStream_t)stream, Z, U_next, nullptr, nm::kGroupScalesGiven, group_rows);
+}
+
+int nm_dist_scales(const float* W, const float* U, int out, int in, int n, int m, int bits, int ncand,
+                   float* scales, int32_t* cand, uint32_t* status, void* stream) {
+    int rc = nm::check_pattern(out, in, n, m, bits);
+    if (rc != NM_OK) return rc;
+    if (ncand < 1 || ncand > NM_DIST_MAX_CANDIDATES) return NM_ERR_SHAPE;
+    if (!W || !scales) return NM_ERR_NULL;
+    if (in % 4) return NM_ERR_SHAPE;
+    if (in > 32768) return NM_ERR_UNSUPPORTED;
+    if (!nm::aligned(W, 16) || (U && !nm::aligned(U, 16)) || !nm::aligned(scales, 4) || (cand && !nm::aligned(cand, 4)))
+        return NM_ERR_ALIGN;
+    if (out == 0 || in == 0) return NM_OK;
+    nm_pack_job_t j{W, U, out, in, n, m, bits, nullptr, nullptr, scales};
+    return nm::launch_dist_single(j, ncand, cand, status, (cudaStream_t)stream);
+}
+
+int nm_project_pack_dist(const float* W, const float* U, int out, int in, int n, int m, int bits, int ncand,
+                         void* values, void* meta, float* scales, uint32_t* status, void* stream) {
+    nm_pack_job_t j{W, U, out, in, n, m, bits, values, meta, scales};
+    int rc = nm::validate_job(j);
+    if (rc != NM_OK) return rc;
+    if (ncand < 1 || ncand > NM_DIST_MAX_CANDIDATES) return NM_ERR_SHAPE;
+    if (out == 0 || in == 0) return NM_OK;
+    rc = nm::launch_dist_single(j, ncand, nullptr, status, (cudaStream_t)stream);
+    if (rc != NM_OK) return rc;
+    nm::PackJobDev d = nm::to_dev(j);
+    int warps = std::max(nm::kPackMinWarps, 1 << d.wpr_log2);
+    int rows_per_block = warps >> d.wpr_log2;
+    unsigned blocks = (unsigned)((out + rows_per_block - 1) / rows_per_block);
+    return nm::launch(nm::pick_kernel(n, m, bits, warps), nullptr, 0, d, blocks, warps, status, (cudaStream_t)stream,
+                      nullptr, nullptr, nullptr, nm::kGroupScalesGiven, 0);
+}
+
+int nm_admm_project_dist(const float* W, const float* U, int out, int in, int n, int m, int bits, int ncand,
+                         float* Z, float* U_next, void* values, void* meta, float* scales, uint32_t* status,
+                         void* stream) {
+    int rc = nm::validate_admm(W, U, out, in, n, m, bits, Z, U_next, values, meta, scales);
+    if (rc != NM_OK) return rc;
+    if (!scales) return NM_ERR_NULL;  // the search hands its result to the projection through it
+    if (ncand < 1 || ncand > NM_DIST_MAX_CANDIDATES) return NM_ERR_SHAPE;
+    if (out == 0 || in == 0) return NM_OK;
+    nm_pack_job_t j{W, U, out, in, n, m, bits, values, meta, scales};
+    rc = nm::launch_dist_single(j, ncand, nullptr, status, (cudaStream_t)stream);
+    if (rc != NM_OK) return rc;
+    nm::PackJobDev d = nm::to_dev(j);
+    int warps = std::max(nm::kPackMinWarps, 1 << d.wpr_log2);
+    int rows_per_block = warps >> d.wpr_log2;
+    unsigned blocks = (unsigned)((out + rows_per_block - 1) / rows_per_block);
+    return nm::launch(nm::pick_kernel<true>(n, m, bits, warps), nullptr, 0, d, blocks, warps, status,
+                      (cudaStream_t)stream, Z, U_next, nullptr, nm::kGroupScalesGiven, 0);
+}
+
+int nm_project_pack_dist_batched(const nm_pack_job_t* jobs, int njobs, int ncand, void* ws, size_t ws_bytes,
+                                 uint32_t* status, void* stream) {
+    if (njobs < 0) return NM_ERR_SHAPE;
+    if (ncand < 1 || ncand > NM_DIST_MAX_CANDIDATES) return NM_ERR_SHAPE;
+    if (njobs == 0) return NM_OK;
+    if (!jobs) return NM_ERR_NULL;
+    if (!ws || ws_bytes < nm_pack_workspace_bytes(njobs)) return NM_ERR_WORKSPACE;
+    if (!nm::aligned(ws, 16)) return NM_ERR_ALIGN;
+    for (int i = 0; i < njobs; ++i) {
+        int rc = nm::validate_job(jobs[i]);
+        if (rc != NM_OK) return rc;
+    }
+    return nm::launch_batched<false>(jobs, nullptr, njobs, ws, status, (cudaStream_t)stream, false, 0, ncand);
 }
 
 size_t nm_pack_workspace_bytes(int njobs) {
