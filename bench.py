@@ -484,6 +484,28 @@ def pack_sweep(nm, torch, dev, status, reps=5):
     grouped_us = float(np.median(times)) * 1e3
     grouped = {"us": grouped_us, "gbs": table["2:4/8b"]["bytes"] / grouped_us / 1e3, "bytes": table["2:4/8b"]["bytes"],
                "launches": 4, "group_rows": 32}
+    # ADMM-Dist scale search (32 candidate scales per output channel) followed by the projection at the chosen
+    # scale, 2:4 with 4-bit and 8-bit codes, one batched call (2 launches).  The search is bound by instruction
+    # issue, not by memory: reported as time and as candidate evaluations (kept value x candidate) per second.
+    dist = {}
+    kept = sum(o * k for o, k in shapes) // 2
+    for bits in (4, 8):
+        dist_jobs = nm.make_pack_jobs([(W, U, 2, 4, bits, v, mt, sc) for (W, U, v, mt, sc) in mats])
+        def dist_pass():
+            nm.nm_project_pack_dist_batched(dist_jobs, len(mats), 32, ws, ws_bytes, status)
+        dist_pass()
+        torch.cuda.synchronize()
+        times = []
+        for _ in range(reps):
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            dist_pass()
+            e1.record()
+            torch.cuda.synchronize()
+            times.append(e0.elapsed_time(e1))
+        us = float(np.median(times)) * 1e3
+        dist[f"2:4/{bits}b"] = {"us": us, "search_us": us - table[f"2:4/{bits}b"]["us"], "candidates": 32, "launches": 2,
+                                "evals_per_s": kept * 32 / (us - table[f"2:4/{bits}b"]["us"]) * 1e6}
     # ADMM step with dense outputs over the same 96 matrices (one batched call): W and U read, Z and
     # U_next (in place over U, so it runs last) written, 16 bytes per parameter; 2:4 / 8-bit, no packed outputs
     Zs = [torch.empty_like(W) for (W, U, v, mt, sc) in mats]
@@ -507,8 +529,42 @@ def pack_sweep(nm, torch, dev, status, reps=5):
     head = table["2:4/8b"]
     return {"us": head["us"], "gbs": head["gbs"], "params": int(sum(o * k for o, k in shapes)),
             "bytes": head["bytes"], "matrices": len(shapes), "launches": 1, "variants": table,
-            "grouped_2:4/8b": grouped,
+            "grouped_2:4/8b": grouped, "admm_dist": dist,
             "admm_step_2:4/8b": {"us": admm_us, "gbs": admm_bytes / admm_us / 1e3, "bytes": admm_bytes, "launches": 1}}
+
+
+def dist_case(bits):
+    """A small ADMM-Dist case for profiler captures: eight 4096x1024 matrices (268 MB of W and U, larger than
+    L2), 2:4, 32 candidates, one batched call = one search launch + one projection launch.  Prints its time."""
+    import torch
+    import paper_2206_15014_b200 as nm
+    dev = torch.device("cuda:0")
+    gen = torch.Generator(device=dev)
+    gen.manual_seed(3)
+    mats = []
+    for _ in range(8):
+        out, k = 4096, 1024
+        W = torch.empty((out, k), dtype=torch.float32, device=dev).normal_(0.0, 0.02, generator=gen)
+        U = torch.empty((out, k), dtype=torch.float32, device=dev).normal_(0.0, 0.002, generator=gen)
+        vb, mb = nm.nm_packed_sizes(out, k, 2, 4, bits)
+        mats.append((W, U, 2, 4, bits, torch.empty(vb, dtype=torch.uint8, device=dev),
+                     torch.empty(mb // 4, dtype=torch.int32, device=dev), torch.empty(out, dtype=torch.float32, device=dev)))
+    ws_bytes = nm.nm_pack_workspace_bytes(len(mats))
+    ws = torch.empty(ws_bytes, dtype=torch.uint8, device=dev)
+    status = torch.zeros(1, dtype=torch.int32, device=dev)
+    jobs = nm.make_pack_jobs(mats)
+    for _ in range(3):
+        nm.nm_project_pack_dist_batched(jobs, len(mats), 32, ws, ws_bytes, status)
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    nm.nm_project_pack_dist_batched(jobs, len(mats), 32, ws, ws_bytes, status)
+    e1.record()
+    torch.cuda.synchronize()
+    rc = nm.nm_poll_status(status)
+    print(json.dumps({"case": "admm_dist 8 x [4096,1024] 2:4", "bits": bits, "candidates": 32,
+                      "us": e0.elapsed_time(e1) * 1e3, "status": rc}))
+    return 0 if rc == 0 else 1
 
 
 def main():
@@ -523,7 +579,11 @@ def main():
     ap.add_argument("--tokens", type=int, default=TOKENS, help="tokens per GEMM (default: the full workload)")
     ap.add_argument("--skip-cpu", action="store_true", help="leave the CPU-oracle baseline out")
     ap.add_argument("--skip-sweep", action="store_true", help="leave the 24-layer pack sweep out")
+    ap.add_argument("--dist-case", type=int, default=0, choices=[0, 4, 8],
+                    help="run only a small ADMM-Dist case with this code width (for profiler captures) and exit")
     args = ap.parse_args()
+    if args.dist_case:
+        return dist_case(args.dist_case)
     if args.impl == "reference":
         return run_reference(args)
     return run_cuda(args)

@@ -470,7 +470,7 @@ static int launch_group_scales(const float* W, const float* U, int out, int in, 
 // of which it keeps G*N in registers (as fp32 for the quantiser, as fp64 for the distance).  Per
 // candidate and kept value: the code from the reciprocal product (true division when the quotient is
 // within 2^-15 of a rounding tie or the scale is outside the range where the reciprocal is accurate),
-// turned into a double through the 2^52 trick, then d = v - s*code and E += d*d as two fp64 FMAs (the
+// converted to a double, then d = v - s*code and E += d*d as two fp64 FMAs (the
 // product s*code is exact in double).  E is summed per lane, over the lanes by a butterfly, over the
 // warps of a row through shared memory: a fixed order, so the result is deterministic.  The work is
 // bound by instruction issue (about 15 instructions per candidate and kept value), not by HBM.
@@ -508,7 +508,7 @@ __device__ __forceinline__ void kept_values(const float* v, float* sel) {
 }
 
 template <int N, int M, int BITS, int MAXT>
-__global__ void __launch_bounds__(MAXT, MAXT == 128 ? 4 : 1) dist_scale_kernel(const PackJobDev* __restrict__ jobs, int njobs,
+__global__ void __launch_bounds__(MAXT, MAXT == 128 ? (32 / M * N > 16 ? 4 : 5) : 1) dist_scale_kernel(const PackJobDev* __restrict__ jobs, int njobs,
                                                                               PackJobDev single, uint32_t* status, int ncand,
                                                                               int32_t* __restrict__ cand_out) {
     constexpr int G = 32 / M;
@@ -593,7 +593,6 @@ __global__ void __launch_bounds__(MAXT, MAXT == 128 ? 4 : 1) dist_scale_kernel(c
     constexpr float qmax = (float)((1 << (BITS - 1)) - 1);
     constexpr float kLo = -(float)(1 << (BITS - 1)) - 0.49f, kHi = qmax + 0.49f;
     constexpr float kMagic = 12582912.0f;             // 1.5 * 2^23 = 0x4B400000
-    constexpr double kMagicD = 4503601774854144.0;    // 2^52 + 2^31
     const float smax = (amax == 0.0f) ? 1.0f : __fdiv_rn(amax, qmax);
     double mine = __longlong_as_double(0x7ff0000000000000ll);  // lane j ends up with candidate j's distance
     for (int j = 0; j < ncand; ++j) {
@@ -602,29 +601,27 @@ __global__ void __launch_bounds__(MAXT, MAXT == 128 ? 4 : 1) dist_scale_kernel(c
         const double nsd = -(double)sj;
         // outside [2^-126, 2^125] the reciprocal is subnormal, infinite or the product loses bits
         const bool fast_ok = (sj >= 1.17549435e-38f) && (sj <= 4.25e37f);
-        unsigned lo[KN];
+        // fast pass: code from the reciprocal product; the rounded quotient (an integer-valued float) goes to
+        // the fp64 pipe through one conversion
         bool near_tie = !fast_ok;
-#pragma unroll
-        for (int i = 0; i < KN; ++i) {
-            const float qc = fminf(fmaxf(__fmul_rn(x[i], rj), kLo), kHi);
-            const float t = __fadd_rn(qc, kMagic);
-            const float f = __fsub_rn(qc, __fsub_rn(t, kMagic));
-            near_tie |= !(fabsf(f) <= 0.49996948f);
-            lo[i] = (unsigned)__float_as_int(t) + 0x34C00000u;  // (code) ^ 0x80000000
-        }
-        if (near_tie) {
-#pragma unroll
-            for (int i = 0; i < KN; ++i) {
-                const float qc = fminf(fmaxf(__fdiv_rn(x[i], sj), kLo), kHi);
-                lo[i] = (unsigned)__float_as_int(__fadd_rn(qc, kMagic)) + 0x34C00000u;
-            }
-        }
         double e0 = 0.0, e1 = 0.0;
 #pragma unroll
         for (int i = 0; i < KN; ++i) {
-            const double qd = __hiloint2double(0x43300000, (int)lo[i]) - kMagicD;  // the code as a double
-            const double d = fma(nsd, qd, xd[i]);
+            const float qc = fminf(fmaxf(__fmul_rn(x[i], rj), kLo), kHi);
+            const float r = __fsub_rn(__fadd_rn(qc, kMagic), kMagic);  // nearest-even integer of qc
+            near_tie |= !(fabsf(__fsub_rn(qc, r)) <= 0.49996948f);
+            const double d = fma(nsd, (double)r, xd[i]);
             if (i & 1) e1 = fma(d, d, e1); else e0 = fma(d, d, e0);
+        }
+        if (near_tie) {  // some quotient of this lane sits next to a rounding tie: the whole candidate again, exactly
+            e0 = 0.0; e1 = 0.0;
+#pragma unroll
+            for (int i = 0; i < KN; ++i) {
+                const float qc = fminf(fmaxf(__fdiv_rn(x[i], sj), kLo), kHi);
+                const float r = __fsub_rn(__fadd_rn(qc, kMagic), kMagic);
+                const double d = fma(nsd, (double)r, xd[i]);
+                if (i & 1) e1 = fma(d, d, e1); else e0 = fma(d, d, e0);
+            }
         }
         double e = e0 + e1;
 #pragma unroll
