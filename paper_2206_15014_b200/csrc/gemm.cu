@@ -671,6 +671,10 @@ nm_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_con
     __syncthreads();
     ptx::tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
+    // Set-up above overlaps the tail of the kernel before this one in the stream (when launched as its
+    // programmatic dependent); nothing in global memory is read or written before this point.
+    ptx::grid_dep_wait();
+    ptx::grid_dep_launch();
 
     auto raise_timeout = [&]() {
         *abort_flag = 1;
@@ -1147,10 +1151,14 @@ static int launch_gemm_pair(const LinearArgs& a) {
     cfg.blockDim = dim3(kPairThreads, 1, 1);
     cfg.dynamicSmemBytes = Cfg::SMEM;
     cfg.stream = a.stream;
-    cudaLaunchAttribute attr[1];
+    cudaLaunchAttribute attr[2];
     attr[0].id = cudaLaunchAttributeClusterDimension;
     attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
-    cfg.attrs = attr; cfg.numAttrs = 1;
+    // the kernel's set-up may start while the previous kernel of the stream drains; it waits for that kernel
+    // (griddepcontrol.wait) before its first access to global memory
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr; cfg.numAttrs = getenv("NM_NO_PDL") ? 1 : 2;
     NM_CUDA_TRY(cudaLaunchKernelEx(&cfg, fn, tw, tx, ty, p, sched));
     return NM_OK;
 }

@@ -102,6 +102,21 @@ __device__ __forceinline__ unsigned keep_mask(const float* a) {
         }
         return mask;
     }
+    if constexpr (N == 4 && M == 8) {
+        // Four of eight: the fourth largest magnitude T from a selection network (both halves sorted with five
+        // compare-exchanges each, then the four maxima of a bitonic half-cleaner hold the four largest and their
+        // minimum is T), the support as a >= T.  Equal magnitudes at the threshold make that more than four
+        // positions; only then does the rank network below decide (lower index first).
+        auto cx = [](float& hi, float& lo) { const float h = fmaxf(hi, lo), l = fminf(hi, lo); hi = h; lo = l; };
+        float x0 = a[0], x1 = a[1], x2 = a[2], x3 = a[3], y0 = a[4], y1 = a[5], y2 = a[6], y3 = a[7];
+        cx(x0, x1); cx(x2, x3); cx(x0, x2); cx(x1, x3); cx(x1, x2);   // x0 >= x1 >= x2 >= x3
+        cx(y0, y1); cx(y2, y3); cx(y0, y2); cx(y1, y3); cx(y1, y2);   // y0 >= y1 >= y2 >= y3
+        const float T = fminf(fminf(fmaxf(x0, y3), fmaxf(x1, y2)), fminf(fmaxf(x2, y1), fmaxf(x3, y0)));
+        unsigned mask = 0;
+#pragma unroll
+        for (int i = 0; i < M; ++i) mask |= (a[i] >= T ? 1u : 0u) << i;
+        if (__popc(mask) == N) return mask;
+    }
     int rank[M];
 #pragma unroll
     for (int i = 0; i < M; ++i) rank[i] = 0;
@@ -166,6 +181,8 @@ __global__ void __launch_bounds__(MAXT, MAXT == 128 ? (DENSE_OUT ? 4 : 8) : 1) p
     extern __shared__ float4 tile[];  // [warps][256] float4, then [warps] floats for the row maximum
     const int warps = blockDim.x >> 5;
     float* red = reinterpret_cast<float*>(tile + warps * 256);
+    // a kernel launched as this one's programmatic dependent may begin its set-up on SMs this grid has left
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 
     PackJobDev job;
     if (jobs) {

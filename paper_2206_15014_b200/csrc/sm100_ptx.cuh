@@ -166,6 +166,13 @@ __device__ __forceinline__ uint32_t cluster_ctarank() {
     asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
     return r;
 }
+// Programmatic dependent launch.  grid_dep_wait: returns once the grid this one was made dependent on (launch
+// attribute "programmatic stream serialization") has finished and its writes are visible; without that
+// attribute it returns at once.  grid_dep_launch: lets a dependent grid start occupying SMs that this grid's
+// CTAs have left (it still waits in grid_dep_wait for this grid to finish).
+__device__ __forceinline__ void grid_dep_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void grid_dep_launch() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
 __device__ __forceinline__ void cluster_arrive() { asm volatile("barrier.cluster.arrive.aligned;" ::: "memory"); }
 __device__ __forceinline__ void cluster_wait() { asm volatile("barrier.cluster.wait.aligned;" ::: "memory"); }
 // shared::cluster address of the same shared-memory offset in CTA `rank` of the cluster
