@@ -11,6 +11,7 @@
 #include <vector>
 #include <mutex>
 #include <algorithm>
+#include <cstdlib>
 
 namespace nm {
 
@@ -31,6 +32,13 @@ struct PackJobDev {
 struct DenseOutDev {
     float* Z;
     float* U_next;
+};
+
+// Job tables of up to kInlineJobs entries travel as a kernel parameter: no table in device memory, no
+// host-to-device copy in front of the launch.  A single matrix is a table of one.
+static constexpr int kInlineJobs = 8;
+struct PackJobInline {
+    PackJobDev j[kInlineJobs];
 };
 
 static constexpr int kPackMinWarps = 4;
@@ -167,7 +175,7 @@ __device__ __forceinline__ void store_bytes_slow(uint8_t* dst, const unsigned* w
 // tile so that the stores are as coalesced as the loads.
 template <int N, int M, int BITS, int MAXT, bool DENSE_OUT = false>
 __global__ void __launch_bounds__(MAXT, MAXT == 128 ? (DENSE_OUT ? 4 : 8) : 1) pack_kernel(const PackJobDev* __restrict__ jobs, int njobs,
-                                                    PackJobDev single, uint32_t* status, float* __restrict__ Zout,
+                                                    const __grid_constant__ PackJobInline inl, uint32_t* status, float* __restrict__ Zout,
                                                     float* __restrict__ Unext, const DenseOutDev* __restrict__ dense_jobs,
                                                     int group_mode, int group_rows) {
     constexpr bool kDense = (N == M);
@@ -194,9 +202,16 @@ __global__ void __launch_bounds__(MAXT, MAXT == 128 ? (DENSE_OUT ? 4 : 8) : 1) p
         job = jobs[lo];
         if constexpr (DENSE_OUT) { Zout = dense_jobs[lo].Z; Unext = dense_jobs[lo].U_next; }
     } else {
-        job = single;
+        // table in the kernel's parameters (a single matrix is a table of one); entries ascend in unit_begin
+        int lo = 0;
+#pragma unroll
+        for (int i = 1; i < kInlineJobs; ++i)
+            if (i < njobs && inl.j[i].unit_begin <= blockIdx.x) lo = i;
+        job = inl.j[0];
+#pragma unroll
+        for (int i = 1; i < kInlineJobs; ++i)
+            if (lo == i) job = inl.j[i];
     }
-
     const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
     const int wpr = 1 << job.wpr_log2;
     const int row_in_block = w >> job.wpr_log2, chunk = w & (wpr - 1);
@@ -670,7 +685,7 @@ __global__ void __launch_bounds__(MAXT, MAXT == 128 ? (32 / M * N > 16 ? 4 : 5) 
 // ---------------------------------------------------------------------------------------------
 // host side
 // ---------------------------------------------------------------------------------------------
-using PackFn = void (*)(const PackJobDev*, int, PackJobDev, uint32_t*, float*, float*, const DenseOutDev*, int, int);
+using PackFn = void (*)(const PackJobDev*, int, const PackJobInline, uint32_t*, float*, float*, const DenseOutDev*, int, int);
 
 template <int N, int M, bool DENSE_OUT>
 static PackFn pick_bits(int bits, int warps) {
@@ -721,16 +736,25 @@ static PackJobDev to_dev(const nm_pack_job_t& j) {
     return d;
 }
 
+// jobs_dev != nullptr: table of njobs entries in device memory; else the first njobs (>= 1) entries of `inl`.
+static int launch_table(PackFn fn, const PackJobDev* jobs_dev, int njobs, const PackJobInline& inl, unsigned blocks,
+                        int warps, uint32_t* status, cudaStream_t stream, float* Z, float* U_next,
+                        const DenseOutDev* dense_jobs, int group_mode, int group_rows) {
+    size_t smem = (size_t)warps * (256 * sizeof(float4) + sizeof(float));
+    if (smem > 48 * 1024)
+        NM_CUDA_TRY(cudaFuncSetAttribute((const void*)fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    fn<<<blocks, warps * 32, smem, stream>>>(jobs_dev, njobs, inl, status, Z, U_next, dense_jobs, group_mode, group_rows);
+    NM_CUDA_TRY(cudaGetLastError());
+    return NM_OK;
+}
+
 static int launch(PackFn fn, const PackJobDev* jobs_dev, int njobs, const PackJobDev& single,
                   unsigned blocks, int warps, uint32_t* status, cudaStream_t stream,
                   float* Z = nullptr, float* U_next = nullptr, const DenseOutDev* dense_jobs = nullptr,
                   int group_mode = kGroupNone, int group_rows = 0) {
-    size_t smem = (size_t)warps * (256 * sizeof(float4) + sizeof(float));
-    if (smem > 48 * 1024)
-        NM_CUDA_TRY(cudaFuncSetAttribute((const void*)fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    fn<<<blocks, warps * 32, smem, stream>>>(jobs_dev, njobs, single, status, Z, U_next, dense_jobs, group_mode, group_rows);
-    NM_CUDA_TRY(cudaGetLastError());
-    return NM_OK;
+    PackJobInline inl{};
+    inl.j[0] = single;
+    return launch_table(fn, jobs_dev, njobs, inl, blocks, warps, status, stream, Z, U_next, dense_jobs, group_mode, group_rows);
 }
 
 using DistFn = void (*)(const PackJobDev*, int, PackJobDev, uint32_t*, int, int32_t*);
@@ -811,6 +835,22 @@ static int launch_batched(const nm_pack_job_t* jobs, const DenseOutDev* dense, i
             if (DENSE_OUT) dense_table.push_back(dense[i]);
         }
         group_blocks[g] = blocks;
+    }
+    // Small plain batches: every group's table fits in the kernel's parameters, nothing is copied to `ws`.
+    if (!DENSE_OUT && !grouped && dist_ncand == 0) {
+        bool fits = true;
+        for (size_t g = 0; g < keys.size(); ++g) fits = fits && groups[g].size() <= (size_t)kInlineJobs;
+        if (fits) {
+            for (size_t g = 0; g < keys.size(); ++g) {
+                PackJobInline inl{};
+                for (size_t i = 0; i < groups[g].size(); ++i) inl.j[i] = table[group_first[g] + i];
+                int rc = nm::launch_table(nm::pick_kernel<DENSE_OUT>(keys[g].n, keys[g].m, keys[g].bits, keys[g].warps), nullptr,
+                                          (int)groups[g].size(), inl, group_blocks[g], keys[g].warps, status, s, nullptr,
+                                          nullptr, nullptr, kGroupNone, 0);
+                if (rc != NM_OK) return rc;
+            }
+            return NM_OK;
+        }
     }
     // Pageable-source async copies are staged before the call returns, so `table` may go away.
     NM_CUDA_TRY(cudaMemcpyAsync(ws, table.data(), table.size() * sizeof(nm::PackJobDev),
