@@ -209,6 +209,10 @@ nm_gemm_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant
     __syncthreads();
     ptx::tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
+    // Set-up above overlaps the tail of the kernel before this one in the stream (when launched as its
+    // programmatic dependent); nothing in global memory is read or written before this point.
+    ptx::grid_dep_wait();
+    ptx::grid_dep_launch();
 
     auto raise_timeout = [&]() {
         *abort_flag = 1;
@@ -1061,8 +1065,17 @@ static int launch_gemm(const LinearArgs& a) {
     auto fn = nm_gemm_kernel<SPARSE, BN, EPI, WSRC>;
     NM_CUDA_TRY(cudaFuncSetAttribute((const void*)fn, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::SMEM));
     const int grid = p.n_tiles < sm_count() ? p.n_tiles : sm_count();
-    fn<<<grid, XF ? kXformThreads : kGemmThreads, Cfg::SMEM, a.stream>>>(tw, tx, ty, p);
-    NM_CUDA_TRY(cudaGetLastError());
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(grid, 1, 1);
+    cfg.blockDim = dim3(XF ? kXformThreads : kGemmThreads, 1, 1);
+    cfg.dynamicSmemBytes = Cfg::SMEM;
+    cfg.stream = a.stream;
+    // as for the pair kernel: set-up may overlap the previous kernel's tail, global memory waits for it
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr; cfg.numAttrs = getenv("NM_NO_PDL") ? 0 : 1;
+    NM_CUDA_TRY(cudaLaunchKernelEx(&cfg, fn, tw, tx, ty, p));
     return NM_OK;
 }
 

@@ -7,6 +7,7 @@ namespace nm {
 // Non-negative floats order like their bit patterns, so an unsigned atomicMax folds the maximum.
 __global__ void __launch_bounds__(256) absmax_kernel(const float* __restrict__ Y, size_t count,
                                                      float* __restrict__ absmax) {
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");  // a dependent kernel may begin its set-up early
     const size_t n4 = count >> 2;
     const float4* Y4 = reinterpret_cast<const float4*>(Y);
     float a = 0.0f;
@@ -41,6 +42,7 @@ __global__ void __launch_bounds__(256) quantize_act_kernel(const float* __restri
                                                            const float* __restrict__ absmax,
                                                            int8_t* __restrict__ Xq,
                                                            float* __restrict__ sx_out) {
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");  // a dependent kernel may begin its set-up early
     const float a = *absmax;
     const float s = (a == 0.0f) ? 1.0f : __fdiv_rn(a, 127.0f);
     if (sx_out && blockIdx.x == 0 && threadIdx.x == 0) *sx_out = s;
