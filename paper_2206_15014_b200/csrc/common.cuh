@@ -33,31 +33,27 @@ inline size_t meta_row_words(int in, int n, int m) {
 inline bool aligned(const void* p, size_t a) { return ((uintptr_t)p % a) == 0; }
 
 #ifdef __CUDACC__
-// Signed integer code of v / s: clamp(rne(fl32(v / s))) to BITS bits, Eq. 5 with offset 0.  The scale is
-// shared by many values, so the quotient is formed from the correctly rounded reciprocal r = RN(1 / s)
-// with one FMA correction step (q = v * r; q += r * (v - s * q)), which lands within an ulp or two of the
-// IEEE quotient.  That can only change the rounded integer when the quotient sits next to a
-// half-integer: those cases (and anything non-finite, e.g. a subnormal scale whose reciprocal
-// overflows) take the true IEEE division, so the result is the same bit for bit.
-// Rounding to the nearest-even integer is done by adding 1.5 * 2^23 (the sum's own rounding does it; the
-// quotient is first clamped one code beyond the range so that it stays where that works): ordinary
-// adds instead of the quarter-rate float -> int conversions, which otherwise bound the epilogue.
+// Signed integer code of v / s: clamp(rne(fl32(v / s))) to BITS bits, Eq. 5 with offset 0, for a scale that
+// many values share: the quotient comes from the correctly rounded reciprocal r = RN(1 / s).  `fast_ok` (once
+// per scale) says that s lies in [2^-126, 2^125], where r = RN(1 / s) is a normal number: then the plain product v * r is
+// within |q| * 1.5 * 2^-23 <= 2^-15.4 of the IEEE quotient over the clamped range, so it rounds to the same
+// integer unless it sits within 2^-15 of a half-integer; those values (6 in 100000), NaNs and scales outside
+// the range take the true division.  Clamping the quotient to [lo - 0.49, hi + 0.49] before the add of
+// 1.5 * 2^23 leaves nothing to clamp afterwards (a quotient beyond the range rounds to the end code either way).
+// The add's own rounding rounds to the nearest-even integer: ordinary adds instead of quarter-rate float -> int
+// conversions.
 template <int BITS>
-__device__ __forceinline__ int quantise_rn(float v, float s, float r) {
-    constexpr int hi = (1 << (BITS - 1)) - 1, lo = -(1 << (BITS - 1));
+__device__ __forceinline__ int quantise_shared_scale(float v, float s, float r, bool fast_ok) {
+    constexpr float kLo = -(float)(1 << (BITS - 1)) - 0.49f, kHi = (float)((1 << (BITS - 1)) - 1) + 0.49f;
     constexpr float kMagic = 12582912.0f;  // 1.5 * 2^23 = 0x4B400000
-    float q = __fmul_rn(v, r);
-    q = __fmaf_rn(__fmaf_rn(-s, q, v), r, q);
-    float qc = fminf(fmaxf(q, (float)(lo - 1)), (float)(hi + 1));
+    float qc = fminf(fmaxf(__fmul_rn(v, r), kLo), kHi);
     float t = __fadd_rn(qc, kMagic);
-    const float f = __fsub_rn(qc, __fsub_rn(t, kMagic));     // clamped quotient minus its rounded value, in [-0.5, 0.5]
-    if (!(fabsf(f) <= 0.49996948f) || !(fabsf(q) <= 3.0e38f)) {  // within 2^-15 of a tie, or not finite
-        q = __fdiv_rn(v, s);
-        qc = fminf(fmaxf(q, (float)(lo - 1)), (float)(hi + 1));
+    const float f = __fsub_rn(qc, __fsub_rn(t, kMagic));
+    if (!(fabsf(f) <= 0.49996948f) || !fast_ok) {
+        qc = fminf(fmaxf(__fdiv_rn(v, s), kLo), kHi);
         t = __fadd_rn(qc, kMagic);
     }
-    const int c = __float_as_int(t) - 0x4B400000;
-    return max(lo, min(hi, c));
+    return __float_as_int(t) - 0x4B400000;
 }
 
 // The same 8-bit code for a NORMAL scale s (>= FLT_MIN, so that r = RN(1 / s) is finite and v * r cannot be

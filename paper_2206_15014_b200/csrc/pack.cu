@@ -142,12 +142,6 @@ __device__ __forceinline__ unsigned keep_mask(const float* a) {
     return mask;
 }
 
-// Integer code of v / s as an unsigned BITS-wide field (quantise_rn: common.cuh).
-template <int BITS>
-__device__ __forceinline__ unsigned quantise_code(float v, float s, float r) {
-    return (unsigned)quantise_rn<BITS>(v, s, r) & ((1u << BITS) - 1u);
-}
-
 template <int NBYTES>
 __device__ __forceinline__ void store_bytes_vec(uint8_t* dst, const unsigned* w) {
     if constexpr (NBYTES == 2) *reinterpret_cast<uint16_t*>(dst) = (uint16_t)w[0];
@@ -280,6 +274,7 @@ __global__ void __launch_bounds__(MAXT, MAXT == 128 ? (DENSE_OUT ? 4 : 8) : 1) p
                                                     : ((amax == 0.0f) ? 1.0f : __fdiv_rn(amax, qmax));
     if (row_ok && chunk == 0 && lane == 0 && (!DENSE_OUT || job.scales)) job.scales[row] = s;
     const float rs = __frcp_rn(s);  // correctly rounded reciprocal, once per row
+    const bool fast_ok = (s >= 1.17549435e-38f) && (s <= 4.25e37f);  // rs is a normal number
 
     // ---- this lane's 32 consecutive values ----------------------------------------------------
     float v[32];
@@ -310,7 +305,7 @@ __global__ void __launch_bounds__(MAXT, MAXT == 128 ? (DENSE_OUT ? 4 : 8) : 1) p
 #pragma unroll
                 for (int p = 0; p < M; ++p) {
                     const int pos = (g * M + p) * BITS;
-                    const int code = quantise_rn<BITS>(v[g * M + p], s, rs);
+                    const int code = quantise_shared_scale<BITS>(v[g * M + p], s, rs, fast_ok);
                     vw[pos >> 5] |= ((unsigned)code & ((1u << BITS) - 1u)) << (pos & 31);
                     if constexpr (DENSE_OUT) z[g * M + p] = __fmul_rn(s, (float)code);
                 }
@@ -358,7 +353,7 @@ __global__ void __launch_bounds__(MAXT, MAXT == 128 ? (DENSE_OUT ? 4 : 8) : 1) p
 #pragma unroll
                 for (int c = 0; c < N; ++c) {
                     const int vpos = (g * N + c) * BITS, mpos = (g * N + c) * F;
-                    const int code = quantise_rn<BITS>(sel[c], s, rs);
+                    const int code = quantise_shared_scale<BITS>(sel[c], s, rs, fast_ok);
                     vw[vpos >> 5] |= ((unsigned)code & ((1u << BITS) - 1u)) << (vpos & 31);
                     mw[mpos >> 5] |= selp[c] << (mpos & 31);
                     if constexpr (DENSE_OUT) {
