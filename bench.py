@@ -394,7 +394,7 @@ def run_cuda(args):
         k2 = f"nm_gemm_pair_kernel<sparse,192,{args.out},streamed>" if bits == 8 else f"nm_gemm_kernel<sparse,192,{args.out},build-per-k-block>"
         roofline = {"kernel": k1 + " on ffn1 1024->4096", "bound": "hbm",
                     "achieved": dom["gbs"], "peak": pk["hbm_gbs"], "unit": "GB/s",
-                    "frac": dom["gbs"] / pk["hbm_gbs"], "traffic": 242189824 if full_size else None,
+                    "frac": dom["gbs"] / pk["hbm_gbs"], "traffic": 241730816 if full_size else None,
                     "algorithmic_bytes": gemm_bytes(TOKENS, 1024, 4096, n, m, bits, YB), "peak_source": pk["source"]}
         f2 = per_kernel["ffn2"]
         roofline_tensor = {"kernel": k2 + " on ffn2 4096->1024", "bound": "tensor",
@@ -402,7 +402,7 @@ def run_cuda(args):
                            "frac": f2["tops"] / sparse_peak,
                            "peak_note": "4 x measured bf16 burst (nominal int8-sparse : bf16-dense ratio)",
                            "frac_of_nominal_9000": f2["tops"] / NOMINAL_SPARSE_INT8_TOPS,
-                           "traffic": 113634816 if full_size else None}
+                           "traffic": 113428480 if full_size else None}
         line = {"metric": METRIC, "value": value, "unit": "TOPS", "n_gpus": world, "steps": args.steps,
                 "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True,
                 "scaling": "weak", "vs_baseline": None, "dtype": "int8", "data": "synthetic",
@@ -417,12 +417,12 @@ def run_cuda(args):
             line["roofline_pack"] = {"kernel": "pack_kernel<2,4,8> on the 24-layer sweep", "bound": "hbm",
                                      "achieved": pack_info["gbs"], "peak": pk["hbm_gbs"], "unit": "GB/s",
                                      "frac": pack_info["gbs"] / pk["hbm_gbs"],
-                                     "frac_of_nominal_8000": pack_info["gbs"] / NOMINAL_HBM_GBS, "traffic": 2548788096,
+                                     "frac_of_nominal_8000": pack_info["gbs"] / NOMINAL_HBM_GBS, "traffic": 2549507136,
                                      "algorithmic_bytes": pack_info["bytes"]}
             adm = pack_info["admm_step_2:4/8b"]
             line["roofline_admm"] = {"kernel": "pack_kernel<2,4,8,dense outputs> (ADMM step: Z and U_next) on the 24-layer sweep",
                                      "bound": "hbm", "achieved": adm["gbs"], "peak": pk["hbm_gbs"], "unit": "GB/s",
-                                     "frac": adm["gbs"] / pk["hbm_gbs"], "traffic": 4772343552,
+                                     "frac": adm["gbs"] / pk["hbm_gbs"], "traffic": 4772082261,
                                      "algorithmic_bytes": adm["bytes"]}
         line["cpu_baseline"] = cpu_baseline() if (world == 1 and not args.skip_cpu) else None
         print(json.dumps(line))
