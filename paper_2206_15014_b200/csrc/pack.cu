@@ -180,11 +180,24 @@ __global__ void __launch_bounds__(MAXT, MAXT == 128 ? (DENSE_OUT ? 4 : 8) : 1) p
     constexpr int MBITS = kDense ? 0 : G * N * F;      // metadata bits per lane (0, 16, 32, 64)
     constexpr int MWORDS = kDense ? 1 : (MBITS + 31) / 32;
 
-    extern __shared__ float4 tile[];  // [warps][256] float4, then [warps] floats for the row maximum
+    extern __shared__ float4 tile[];  // [warps][256] float4, [warps] floats for the row maximum, 256 u16 (4:8 positions)
     const int warps = blockDim.x >> 5;
     float* red = reinterpret_cast<float*>(tile + warps * 256);
     // a kernel launched as this one's programmatic dependent may begin its set-up on SMs this grid has left
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    // four of eight: table from the 8-bit keep mask to its four positions (4-bit fields, ascending), which is
+    // also the group's metadata; the kept values are then fetched from the warp's tile by position
+    uint16_t* pos48 = reinterpret_cast<uint16_t*>(red + warps);
+    if constexpr (N == 4 && M == 8) {
+        for (unsigned mk = threadIdx.x; mk < 256; mk += blockDim.x) {
+            unsigned r = 0, c = 0;
+#pragma unroll
+            for (unsigned p8 = 0; p8 < 8; ++p8)
+                if ((mk >> p8) & 1u) { r |= p8 << (4 * (c & 3u)); ++c; }
+            pos48[mk] = (uint16_t)r;
+        }
+        __syncthreads();
+    }
 
     PackJobDev job;
     if (jobs) {
@@ -326,6 +339,15 @@ __global__ void __launch_bounds__(MAXT, MAXT == 128 ? (DENSE_OUT ? 4 : 8) : 1) p
                 }
                 // compaction: slot c receives the c-th kept position (ascending)
                 if constexpr (kPasses) {
+                } else if constexpr (N == 4 && M == 8) {
+                    const unsigned pos4 = pos48[mask];
+                    const float* tile_f = reinterpret_cast<const float*>(mytile);
+#pragma unroll
+                    for (int c = 0; c < 4; ++c) {
+                        selp[c] = (pos4 >> (4 * c)) & 7u;
+                        const unsigned e = (unsigned)(g * 8) + selp[c];  // element of this lane, in the tile's swizzle
+                        sel[c] = tile_f[(lane * 8 + ((e >> 2) ^ (lane & 7))) * 4 + (e & 3u)];
+                    }
                 } else if constexpr (N == 2 && M == 4) {
                     // two of four: the first kept position is 0, 1 or 2, the second 3, 2 or 1
                     const float* g4 = v + g * 4;
@@ -735,7 +757,7 @@ static PackJobDev to_dev(const nm_pack_job_t& j) {
 static int launch_table(PackFn fn, const PackJobDev* jobs_dev, int njobs, const PackJobInline& inl, unsigned blocks,
                         int warps, uint32_t* status, cudaStream_t stream, float* Z, float* U_next,
                         const DenseOutDev* dense_jobs, int group_mode, int group_rows) {
-    size_t smem = (size_t)warps * (256 * sizeof(float4) + sizeof(float));
+    size_t smem = (size_t)warps * (256 * sizeof(float4) + sizeof(float)) + 512;  // + the 4:8 position table
     if (smem > 48 * 1024)
         NM_CUDA_TRY(cudaFuncSetAttribute((const void*)fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     fn<<<blocks, warps * 32, smem, stream>>>(jobs_dev, njobs, inl, status, Z, U_next, dense_jobs, group_mode, group_rows);
