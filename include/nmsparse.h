@@ -189,10 +189,12 @@ int nm_admm_project_dist(const float *W, const float *U, int out, int in, int n,
                          uint32_t *status, void *stream);
 
 /*
- * The same for a list of matrices with as few launches as their (n, m, bits) allow (one when all
- * jobs share them).  `jobs` is a host array; `ws` is device scratch of at least
+ * nm_project_pack for a list of matrices with as few launches as their (n, m, bits) allow (one when
+ * all jobs share them).  `jobs` is a host array; `ws` is device scratch of at least
  * nm_pack_workspace_bytes(njobs) bytes, 16-byte aligned, which must stay untouched until the
  * enqueued work has finished.  The host array may be reused as soon as the call returns.
+ * (Batches in which no more than eight jobs share one (n, m, bits) and block size pass their job table
+ * in the kernel's parameters and leave `ws` untouched; it must be provided all the same.)
  */
 int nm_project_pack_batched(const nm_pack_job_t *jobs, int njobs, void *ws, size_t ws_bytes,
                             uint32_t *status, void *stream);
