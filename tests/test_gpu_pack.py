@@ -61,10 +61,13 @@ def test_pack_wide_rows():
         _check(W, None, 4, 8, 4)
 
 
-def test_pack_batched_matches_single():
+@pytest.mark.parametrize("repeat", [1, 3])
+def test_pack_batched_matches_single(repeat):
+    # up to eight matrices per kernel variant travel in the kernel's parameters (repeat = 1); more go through the
+    # job table in the workspace (repeat = 3: twelve matrices share the 128-thread variant)
     import paper_2206_15014_b200 as nm
     from gpu_util import DEV, to_dev
-    shapes = [(96, 1024), (40, 4096), (64, 1024), (8, 8192), (50, 768)]
+    shapes = [(96, 1024), (40, 4096), (64, 1024), (8, 8192), (50, 768)] * repeat
     for n, m, bits in [(2, 4, 8), (1, 4, 4)]:
         jobs, refs = [], []
         for i, (out, k) in enumerate(shapes):
