@@ -153,6 +153,9 @@ typedef struct nm_admm_job_t {
 size_t nm_admm_workspace_bytes(int njobs);
 int nm_admm_project_batched(const nm_admm_job_t *jobs, int njobs, void *ws, size_t ws_bytes,
                             uint32_t *status, void *stream);
+/* nm_admm_project_dist for many matrices (one ncand for all; scales required in every job). */
+int nm_admm_project_dist_batched(const nm_admm_job_t *jobs, int njobs, int ncand, void *ws,
+                                 size_t ws_bytes, uint32_t *status, void *stream);
 /* nm_admm_project_grouped for many matrices (one group_rows for all; scales required in every job). */
 int nm_admm_project_grouped_batched(const nm_admm_job_t *jobs, int njobs, int group_rows, void *ws,
                                     size_t ws_bytes, uint32_t *status, void *stream);

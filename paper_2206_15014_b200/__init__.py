@@ -29,7 +29,7 @@ EXPORTS = (
     "nm_project_pack_batched_noalloc", "nm_admm_project", "nm_admm_project_batched", "nm_admm_workspace_bytes",
     "nm_project_pack_grouped", "nm_admm_project_grouped", "nm_project_pack_grouped_batched",
     "nm_admm_project_grouped_batched",
-    "nm_dist_scales", "nm_project_pack_dist", "nm_admm_project_dist", "nm_project_pack_dist_batched",
+    "nm_dist_scales", "nm_project_pack_dist", "nm_admm_project_dist", "nm_project_pack_dist_batched", "nm_admm_project_dist_batched",
     "nm_int_linear", "nm_int_linear_dsx", "nm_int_linear_acc", "nm_int_linear_q8", "nm_int_linear_bf16",
     "nm_int_linear_workspace_bytes",
     "nm_int_linear_check", "nm_absmax", "nm_quantize_act", "nm_poll_status", "nm_strerror",
@@ -70,6 +70,7 @@ _lib.nm_dist_scales.argtypes = [_vp, _vp, _i, _i, _i, _i, _i, _i, _vp, _vp, _vp,
 _lib.nm_project_pack_dist.argtypes = [_vp, _vp, _i, _i, _i, _i, _i, _i, _vp, _vp, _vp, _vp, _vp]
 _lib.nm_admm_project_dist.argtypes = [_vp, _vp, _i, _i, _i, _i, _i, _i, _vp, _vp, _vp, _vp, _vp, _vp, _vp]
 _lib.nm_project_pack_dist_batched.argtypes = [ctypes.POINTER(nm_pack_job_t), _i, _i, _vp, _sz, _vp, _vp]
+_lib.nm_admm_project_dist_batched.argtypes = [ctypes.POINTER(nm_admm_job_t), _i, _i, _vp, _sz, _vp, _vp]
 _lib.nm_admm_project_batched.argtypes = [ctypes.POINTER(nm_admm_job_t), _i, _vp, _sz, _vp, _vp]
 _lib.nm_admm_project.argtypes = [_vp, _vp, _i, _i, _i, _i, _i, _vp, _vp, _vp, _vp, _vp, _vp, _vp]
 _lib.nm_admm_workspace_bytes.argtypes = [_i]
@@ -203,6 +204,11 @@ def nm_admm_project_dist(W, U, out, in_, n, m, bits, ncand, Z, U_next, values, m
 def nm_project_pack_dist_batched(jobs, njobs, ncand, ws, ws_bytes, status=None, stream=None):
     _chk(_lib.nm_project_pack_dist_batched(jobs, njobs, ncand, _ptr(ws), ws_bytes, _ptr(status), _stream(stream)),
          "nm_project_pack_dist_batched")
+
+
+def nm_admm_project_dist_batched(jobs, njobs, ncand, ws, ws_bytes, status=None, stream=None):
+    _chk(_lib.nm_admm_project_dist_batched(jobs, njobs, ncand, _ptr(ws), ws_bytes, _ptr(status), _stream(stream)),
+         "nm_admm_project_dist_batched")
 
 
 def nm_project_pack_grouped(W, U, out, in_, n, m, bits, group_rows, values, meta, scales, status=None, stream=None):

@@ -1109,6 +1109,27 @@ int nm_project_pack_grouped_batched(const nm_pack_job_t* jobs, int njobs, int gr
     return nm::launch_batched<false>(jobs, nullptr, njobs, ws, status, (cudaStream_t)stream, true, group_rows);
 }
 
+int nm_admm_project_dist_batched(const nm_admm_job_t* jobs, int njobs, int ncand, void* ws, size_t ws_bytes,
+                                 uint32_t* status, void* stream) {
+    if (njobs < 0) return NM_ERR_SHAPE;
+    if (ncand < 1 || ncand > NM_DIST_MAX_CANDIDATES) return NM_ERR_SHAPE;
+    if (njobs == 0) return NM_OK;
+    if (!jobs) return NM_ERR_NULL;
+    if (!ws || ws_bytes < nm_admm_workspace_bytes(njobs)) return NM_ERR_WORKSPACE;
+    if (!nm::aligned(ws, 16)) return NM_ERR_ALIGN;
+    std::vector<nm_pack_job_t> pj(njobs);
+    std::vector<nm::DenseOutDev> dj(njobs);
+    for (int i = 0; i < njobs; ++i) {
+        const nm_admm_job_t& a = jobs[i];
+        int rc = nm::validate_admm(a.W, a.U, a.out, a.in, a.n, a.m, a.bits, a.Z, a.U_next, a.values, a.meta, a.scales);
+        if (rc != NM_OK) return rc;
+        if (!a.scales) return NM_ERR_NULL;  // the search hands its result to the projection through it
+        pj[i] = nm_pack_job_t{a.W, a.U, a.out, a.in, a.n, a.m, a.bits, a.values, a.meta, a.scales};
+        dj[i] = nm::DenseOutDev{a.Z, a.U_next};
+    }
+    return nm::launch_batched<true>(pj.data(), dj.data(), njobs, ws, status, (cudaStream_t)stream, false, 0, ncand);
+}
+
 size_t nm_admm_workspace_bytes(int njobs) {
     return njobs <= 0 ? 0 : (size_t)njobs * (sizeof(nm::PackJobDev) + sizeof(nm::DenseOutDev));
 }

@@ -183,3 +183,28 @@ def test_dist_batched_matches_single_calls_and_argument_errors():
     with pytest.raises(nm.NmError):
         nm.nm_dist_scales(W, None, 8, 64, 2, 4, 8, 4, None)
     nm.nm_dist_scales(W, None, 0, 64, 2, 4, 8, 4, s)  # nothing to do
+
+
+def test_admm_dist_batched_matches_oracle():
+    import paper_2206_15014_b200 as nm
+    from gpu_util import to_dev, DEV
+    oracle.set_threads(oracle.max_threads())
+    specs = [(64, 1024, 2, 4, 4), (20, 4096, 2, 4, 4), (33, 768, 1, 4, 8), (40, 1024, 2, 4, 4)]
+    jobs, refs = [], []
+    for i, (out, k, n, m, bits) in enumerate(specs):
+        W, U = wl.pack_sweep_matrix(12, i, out, k)
+        Wd, Ud = to_dev(W), to_dev(U)
+        Z = torch.full((out, k), float("nan"), dtype=torch.float32, device=DEV)
+        sc = torch.zeros(out, dtype=torch.float32, device=DEV)
+        jobs.append((Wd, Ud, n, m, bits, Z, Ud, None, None, sc))          # the dual is updated in place
+        refs.append(oracle.admm_step_dist(W, U, n, m, bits, 32))
+    ws_bytes = nm.nm_admm_workspace_bytes(len(jobs))
+    ws = torch.empty(ws_bytes, dtype=torch.uint8, device=DEV)
+    status = torch.zeros(1, dtype=torch.int32, device=DEV)
+    nm.nm_admm_project_dist_batched(nm.make_admm_jobs(jobs), len(jobs), 32, ws, ws_bytes, status)
+    assert nm.nm_poll_status(status) == nm.NM_OK
+    for j, (Zr, Ur, sr) in zip(jobs, refs):
+        assert np.array_equal(j[9].cpu().numpy(), sr)
+        assert np.array_equal(j[5].cpu().numpy(), Zr) and np.array_equal(j[6].cpu().numpy(), Ur)
+    with pytest.raises(nm.NmError):
+        nm.nm_admm_project_dist_batched(nm.make_admm_jobs(jobs), len(jobs), 0, ws, ws_bytes, status)
