@@ -83,9 +83,25 @@ __device__ __forceinline__ void select_passes(const float* v, float* sel, unsign
     }
 }
 
+// Two of four by a tournament on the pairs (0,1) and (2,3).  With "larger magnitude first, lower index first
+// among equals" the two kept positions are 0 and 1 when the smaller of the first pair is >= the larger of the
+// second, 2 and 3 when the smaller of the second pair is > the larger of the first, and otherwise the larger of
+// each pair (the first one of a pair on equality).  Kept values and positions come out in ascending position.
+__device__ __forceinline__ void select_2_of_4(const float* v, float* sel, unsigned* selp) {
+    const float a0 = fabsf(v[0]), a1 = fabsf(v[1]), a2 = fabsf(v[2]), a3 = fabsf(v[3]);
+    const bool i01 = a1 > a0, i23 = a3 > a2;
+    const float hi01 = fmaxf(a0, a1), lo01 = fminf(a0, a1), hi23 = fmaxf(a2, a3), lo23 = fminf(a2, a3);
+    const bool both01 = lo01 >= hi23, both23 = lo23 > hi01;
+    const float w01 = i01 ? v[1] : v[0], w23 = i23 ? v[3] : v[2];
+    sel[0] = both01 ? v[0] : (both23 ? v[2] : w01);
+    sel[1] = both01 ? v[1] : (both23 ? v[3] : w23);
+    selp[0] = both01 ? 0u : (both23 ? 2u : (i01 ? 1u : 0u));
+    selp[1] = both01 ? 1u : (both23 ? 3u : (i23 ? 3u : 2u));
+}
+
 template <int N, int M>
 __device__ __forceinline__ unsigned keep_mask(const float* a) {
-    if constexpr (N == 1 || (N == 2 && M == 8)) {  // (2:4 is faster with the 6-compare rank network below)
+    if constexpr (N == 1 || (N == 2 && M == 8)) {  // (the pack kernel's 2:4 has its own tournament, select_2_of_4)
         // One or two passes of "largest magnitude, first one on equality" (a strict > keeps the lower
         // index): the same support as the rank rule, with 7 + 7 compares instead of 28 for m = 8.
         float best = a[0];
@@ -327,9 +343,11 @@ __global__ void __launch_bounds__(MAXT, MAXT == 128 ? (DENSE_OUT ? 4 : 8) : 1) p
                 unsigned selp[N];
 #pragma unroll
                 for (int c = 0; c < N; ++c) { sel[c] = 0.0f; selp[c] = 0; }
-                constexpr bool kPasses = (N == 1) || (N == 2 && M == 8);
+                constexpr bool kPasses = (N == 1) || (N == 2 && M == 8) || (N == 2 && M == 4);
                 unsigned mask = 0;
-                if constexpr (kPasses) {
+                if constexpr (N == 2 && M == 4) {
+                    select_2_of_4(v + g * M, sel, selp);
+                } else if constexpr (kPasses) {
                     select_passes<N, M>(v + g * M, sel, selp);
                 } else {
                     float a[M];
@@ -348,14 +366,6 @@ __global__ void __launch_bounds__(MAXT, MAXT == 128 ? (DENSE_OUT ? 4 : 8) : 1) p
                         const unsigned e = (unsigned)(g * 8) + selp[c];  // element of this lane, in the tile's swizzle
                         sel[c] = tile_f[(lane * 8 + ((e >> 2) ^ (lane & 7))) * 4 + (e & 3u)];
                     }
-                } else if constexpr (N == 2 && M == 4) {
-                    // two of four: the first kept position is 0, 1 or 2, the second 3, 2 or 1
-                    const float* g4 = v + g * 4;
-                    const bool b0 = mask & 1u, b1 = mask & 2u, b2 = mask & 4u, b3 = mask & 8u;
-                    sel[0] = b0 ? g4[0] : (b1 ? g4[1] : g4[2]);
-                    selp[0] = b0 ? 0u : (b1 ? 1u : 2u);
-                    sel[1] = b3 ? g4[3] : (b2 ? g4[2] : g4[1]);
-                    selp[1] = b3 ? 3u : (b2 ? 2u : 1u);
                 } else {
 #pragma unroll
                 for (int p = 0; p < M; ++p) {
