@@ -567,6 +567,72 @@ def dist_case(bits):
     return 0 if rc == 0 else 1
 
 
+def tma_probe(args):
+    """Ceiling of the memory system for the pair GEMM's tile shapes: the kernel's TMA boxes, tile walk and stage
+    ring with no arithmetic (nm_probe_tma_stream).  One JSON line per case: chip TB/s from CUDA events, bytes per
+    clock per SM from the CTAs' own clock64 counters."""
+    import torch
+    import paper_2206_15014_b200 as nm
+    dev = torch.device("cuda:0")
+    torch.cuda.set_device(dev)
+    status = torch.zeros(1, dtype=torch.int32, device=dev)
+    clocks = torch.zeros((148, 4), dtype=torch.int64, device=dev)
+
+    def case(name, out, k, tokens, a_rows, a_row_bytes, b_rows, b_slices, stages, band=0, repeat=1, delay=0, loads=3,
+             stores=1, producers=1):
+        w_row_bytes = k // 2                       # 2:4 int8 codes
+        W = torch.randint(0, 255, (out, w_row_bytes), dtype=torch.uint8, device=dev)
+        X = torch.randint(0, 255, (tokens, k), dtype=torch.uint8, device=dev)
+        Y = torch.empty((tokens, out), dtype=torch.float32, device=dev)
+        spans, cycles, ctas = [], [], 0
+        for _ in range(4):   # the first run warms up; each run is timed by the CTAs' own clocks (launched on an idle
+            ctas = nm.nm_probe_tma_stream(W, out, w_row_bytes, X, tokens, k, Y, a_rows, a_row_bytes, b_rows, b_slices,
+                                          stages, band, repeat, delay, loads, stores, producers, 0, clocks, None, status)
+            torch.cuda.synchronize()   # GPU, an event pair would also count the host's launch latency)
+            c = clocks[:ctas].cpu().numpy()
+            spans.append(float(c[:, 3].max() - c[:, 2].min()) / 1e3)
+            cycles.append(float(np.median(c[:, 1] - c[:, 0])))
+        rc = nm.nm_poll_status(status)
+        us, cyc = float(np.median(spans[1:])), float(np.median(cycles[1:]))
+        n_out_tiles, n_tok_tiles = -(-out // (2 * a_rows)), -(-tokens // (2 * b_rows))
+        tiles = n_out_tiles * n_tok_tiles * repeat
+        kblocks = w_row_bytes // a_row_bytes
+        ld = tiles * kblocks * 2 * (((loads & 1) and a_rows * a_row_bytes) + ((loads & 2) and b_rows * 128 * b_slices))
+        st = tiles * 2 * a_rows * 2 * b_rows * 4 if stores else 0
+        print(json.dumps({"case": name, "status": rc, "span_us": round(us, 2), "tile": [2 * a_rows, 2 * b_rows],
+                          "stage_bytes": a_rows * a_row_bytes + b_rows * 128 * b_slices, "stages": stages, "producers": producers,
+                          "delay": delay, "loads": loads, "stores": stores, "repeat": repeat,
+                          "load_MB": round(ld / 1e6, 1), "store_MB": round(st / 1e6, 1), "TBps": round((ld + st) / us / 1e6, 2),
+                          "B_per_clk_per_SM": round((ld + st) / ctas / cyc, 1),
+                          "clk_per_stage": round(cyc / (tiles * kblocks / (ctas / 2)), 1),
+                          "sm_ghz": round(cyc / (us * 1e3), 3)}), flush=True)
+
+    T, K, OUT = args.tokens, 4096, 1024
+    # the streamed pair kernel's tile on FFN2 (256 channels x 192 tokens, 256 reduction elements per stage, five stages)
+    for producers in (1, 2):
+        for stores in (1, 0):
+            case("ffn2 pair tile 256x192", OUT, K, T, 128, 128, 96, 2, 5, stores=stores, producers=producers)
+    case("ffn2 pair tile 256x192, stage held 384 clk", OUT, K, T, 128, 128, 96, 2, 5, delay=384, producers=2)
+    case("ffn2 pair tile 256x192, weights only", OUT, K, T, 128, 128, 96, 2, 5, loads=1, stores=0)
+    case("ffn2 pair tile 256x192, X only", OUT, K, T, 128, 128, 96, 2, 5, loads=2, stores=0)
+    for stages in (3, 4):
+        case("ffn2 pair tile 256x192", OUT, K, T, 128, 128, 96, 2, stages, producers=2)
+    # 128 reduction elements per stage: twice the stages of half the size
+    case("ffn2 pair tile 256x192, 20 KB stages", OUT, K, T, 128, 64, 96, 1, 9, producers=2)
+    # wider tiles: 512 channels per pair
+    for b_rows in (96, 112, 128):
+        for producers in (1, 2):
+            for stores in (1, 0):
+                case(f"ffn2 pair tile 512x{2 * b_rows}", OUT, K, T, 256, 64, b_rows, 1, 6 if b_rows < 128 else 5, stores=stores,
+                     producers=producers)
+    case("ffn2 pair tile 512x224, stage held 448 clk", OUT, K, T, 256, 64, 112, 1, 6, delay=448, producers=2)
+    case("ffn2 pair tile 512x224, 4 stages", OUT, K, T, 256, 64, 112, 1, 4, producers=2)
+    # everything resident in L2: a small problem walked five times
+    case("L2-resident 256x192", OUT, K, 19 * 192, 128, 128, 96, 2, 5, repeat=5, stores=0, producers=2)
+    case("L2-resident 512x224", OUT, K, 37 * 224, 256, 64, 112, 1, 6, repeat=5, stores=0, producers=2)
+    return 0
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -581,7 +647,11 @@ def main():
     ap.add_argument("--skip-sweep", action="store_true", help="leave the 24-layer pack sweep out")
     ap.add_argument("--dist-case", type=int, default=0, choices=[0, 4, 8],
                     help="run only a small ADMM-Dist case with this code width (for profiler captures) and exit")
+    ap.add_argument("--probe-tma", action="store_true",
+                    help="run only the TMA traffic probe of the pair GEMM's tile shapes (no arithmetic) and exit")
     args = ap.parse_args()
+    if args.probe_tma:
+        return tma_probe(args)
     if args.dist_case:
         return dist_case(args.dist_case)
     if args.impl == "reference":

@@ -296,6 +296,32 @@ size_t nm_int_linear_workspace_bytes(int tokens, int out, int in, int n, int m, 
 int nm_pair_tile_plan(int n_tok_tiles, int n_out_tiles, int pairs, int resident, int band_request,
                       int *start, int *tile_out, int *tile_tok);
 
+/*
+ * Measurement aid (the paper has no counterpart): the memory traffic of the CTA-pair kernel of nm_int_linear
+ * without its arithmetic.  Every CTA pair walks the tiles nm_pair_tile_plan gives it (streamed form); per
+ * pipeline stage each CTA loads a box of `a_rows` x `a_row_bytes` (64 or 128) from W, a row-major byte matrix
+ * [w_rows, w_row_bytes], and `b_rows` tokens x `b_slices` 128-byte-wide slices from X, int8 [tokens, k_bytes],
+ * into a ring of `stages` shared-memory stages; a consumer hands every stage back once it has landed and
+ * `delay_clocks` SM clocks have passed; when `stores` != 0 eight warps write the CTA's share of the output
+ * tile to Y (fp32 [tokens, w_rows], overwritten with arbitrary values) as [16 tokens][32 channels] boxes.
+ * A pair's tile is 2 * a_rows output channels x 2 * b_rows tokens; w_row_bytes / a_row_bytes must equal
+ * k_bytes / (128 * b_slices) (the stages per tile).  `loads`: bit 0 = W boxes, bit 1 = X boxes; `producers`: 1 = one thread
+ * issues both boxes of a stage, 2 = one thread per operand.  `poll`: how the store warps wait for a tile: 0 = all
+ * lanes poll the barrier, 1 = one lane polls and sleeps between polls, 2 (only with stores == 0) = they leave at
+ * once, producer and consumer run alone.  `band`: as
+ * band_request of nm_pair_tile_plan.  `repeat`: times every pair walks its range.  `clocks` (nullable): u64
+ * [CTAs][4] = clock64 at start, at end, global timer (ns) at start, at end of every CTA.  `trace`
+ * (nullable): u64 [512][8], for the first 512 stages of CTA 0 the clock64 of the producer before and after its wait for the
+ * stage, after arming the barrier, after issuing the W load, after issuing the X load, and of the consumer when the
+ * stage had landed and when it was handed back (last word unused).  W, X, Y: device,
+ * 16-byte aligned, caller-owned; w_rows % 4 == 0.  Returns the number of CTAs launched (> 0) or a negative
+ * NM_ERR_* code.  Waits are bounded: NM_STATUS_TIMEOUT in *status (nullable) when one expired.
+ */
+int nm_probe_tma_stream(const void *W, int w_rows, int w_row_bytes, const void *X, int tokens, int k_bytes,
+                        float *Y, int a_rows, int a_row_bytes, int b_rows, int b_slices, int stages, int band,
+                        int repeat, int delay_clocks, int loads, int stores, int producers, int poll, unsigned long long *clocks,
+                        unsigned long long *trace, uint32_t *status, void *stream);
+
 /* Host-only validation of a linear-layer problem: NM_OK or the error nm_int_linear would return. */
 int nm_int_linear_check(int tokens, int out, int in, int n, int m, int bits);
 

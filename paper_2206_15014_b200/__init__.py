@@ -34,6 +34,7 @@ EXPORTS = (
     "nm_int_linear_workspace_bytes",
     "nm_int_linear_check", "nm_absmax", "nm_quantize_act", "nm_poll_status", "nm_strerror",
     "nm_last_cuda_error", "nm_version", "nm_bits_per_param", "nm_encoder_cost", "nm_pair_tile_plan",
+    "nm_probe_tma_stream",
 )
 
 
@@ -85,6 +86,7 @@ _lib.nm_int_linear_bf16.argtypes = [_vp, _i, ctypes.POINTER(nm_packed_t), _f, _v
 _lib.nm_int_linear_workspace_bytes.argtypes = [_i] * 6
 _lib.nm_int_linear_workspace_bytes.restype = _sz
 _lib.nm_int_linear_check.argtypes = [_i] * 6
+_lib.nm_probe_tma_stream.argtypes = [_vp, _i, _i, _vp, _i, _i, _vp] + [_i] * 12 + [_vp, _vp, _vp, _vp]
 _lib.nm_absmax.argtypes = [_vp, _sz, _vp, _vp]
 _lib.nm_quantize_act.argtypes = [_vp, _sz, _vp, _vp, _vp, _vp]
 _lib.nm_poll_status.argtypes = [_vp, _vp]
@@ -311,6 +313,19 @@ def nm_encoder_cost(cfg, index_bits=-1):
     comp, red = ctypes.c_double(), ctypes.c_double()
     _chk(_lib.nm_encoder_cost(arr, index_bits, ctypes.byref(comp), ctypes.byref(red)), "nm_encoder_cost")
     return comp.value, red.value
+
+
+def nm_probe_tma_stream(W, w_rows, w_row_bytes, X, tokens, k_bytes, Y, a_rows, a_row_bytes, b_rows, b_slices, stages,
+                        band=0, repeat=1, delay_clocks=0, loads=3, stores=1, producers=1, poll=0, clocks=None, trace=None,
+                        status=None, stream=None):
+    """Replays the pair GEMM's tile walk with its TMA boxes and no arithmetic; returns the number of CTAs launched
+    (`clocks`, int64 [CTAs, 4], receives clock64 at start / end and the global timer at start / end of every CTA)."""
+    rc = _lib.nm_probe_tma_stream(_ptr(W), w_rows, w_row_bytes, _ptr(X), tokens, k_bytes, _ptr(Y), a_rows, a_row_bytes,
+                                  b_rows, b_slices, stages, band, repeat, delay_clocks, loads, stores, producers, poll, _ptr(clocks), _ptr(trace),
+                                  _ptr(status), _stream(stream))
+    if rc < 0:
+        raise NmError(rc, "nm_probe_tma_stream")
+    return int(rc)
 
 
 def nm_absmax(Y, count, absmax, stream=None):

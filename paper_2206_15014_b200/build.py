@@ -8,7 +8,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libnmsparse.so")
-SOURCES = ("api.cu", "pack.cu", "quant_act.cu", "gemm.cu")
+SOURCES = ("api.cu", "pack.cu", "quant_act.cu", "gemm.cu", "probe.cu")
 FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
          "-Xcompiler", "-fPIC", "--ftz=false", "--prec-div=true",
          "--prec-sqrt=true"]

@@ -24,6 +24,8 @@
 #include "common.cuh"
 #include "sm100_ptx.cuh"
 #include "xform.cuh"
+#include "tmap.cuh"
+#include "tileplan.cuh"
 #include <cuda.h>
 #include <cuda_runtime.h>
 #include <mutex>
@@ -120,20 +122,6 @@ struct GemmParams {
     float* absmax;
     uint32_t* status;
 };
-
-// Order of the tiles of the pair kernel.  Token tiles are cut into bands of `band` tiles; inside a band the
-// tiles run output-tile-major.  With band = n_tok_tiles this is the plain output-tile-major order (one
-// long run per output tile: weights and metadata change rarely).  A band of about one pair's share
-// makes neighbouring pairs work on the SAME token tiles of different output tiles at the same time, so
-// that X is fetched from DRAM once and found in L2 by the others.
-struct TileCoord { int o, t; };
-__host__ __device__ inline TileCoord tile_coord(int tile, int n_tok_tiles, int n_out_tiles, int band) {
-    const int per_band = band * n_out_tiles;
-    const int b = tile / per_band, r = tile - b * per_band;
-    const int rest = n_tok_tiles - b * band, tb = band < rest ? band : rest;  // the last band may be short
-    const int o = r / tb;
-    return TileCoord{o, b * band + (r - o * tb)};
-}
 
 template <bool SPARSE, int BN, bool RESIDENT = false>
 struct GemmCfg {
@@ -578,14 +566,6 @@ nm_gemm_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant
 constexpr int kPairThreads = 32 * (3 + kEpiWarps);
 constexpr int kPairMaxStages = 7;   // the relay cycles through 8 named barriers (ids 1-8; 9-14 serve the narrow-output epilogue)
 
-// Tile ranges of the CTA pairs, computed on the host: start[p] .. start[p + 1] is pair p's range.  A pair
-// whose range crosses into a new output tile stalls there (weights and metadata are replaced once
-// the MMAs of the old one have drained), so such a range is made shorter by that cost.
-constexpr int kMaxPairs = 128;
-struct PairSchedule {
-    int start[kMaxPairs + 1];
-};
-
 constexpr int kPairResStages = 4;   // stages of weights a CTA can keep resident (1024 reduction elements at 2:4)
 
 template <bool SPARSE, int BN, bool RES = false>
@@ -947,57 +927,6 @@ nm_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_con
 // ---------------------------------------------------------------------------------------------
 // host side
 // ---------------------------------------------------------------------------------------------
-typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
-                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*,
-                                  CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
-                                  CUtensorMapFloatOOBfill);
-
-static EncodeTiledFn encode_tiled_fn() {
-    static EncodeTiledFn fn = nullptr;
-    static std::once_flag once;
-    std::call_once(once, [] {
-        void* p = nullptr;
-        cudaDriverEntryPointQueryResult qres;
-        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres) == cudaSuccess &&
-            qres == cudaDriverEntryPointSuccess)
-            fn = (EncodeTiledFn)p;
-        (void)cudaGetLastError();
-    });
-    return fn;
-}
-
-// 2-D matrix [rows, row_elems] of `esize`-byte elements (dense pitch), box = [box_rows, box_elems].
-static int make_map(CUtensorMap* map, const void* base, uint64_t rows, uint64_t row_elems,
-                    uint32_t box_rows, uint32_t box_elems, CUtensorMapSwizzle swz,
-                    CUtensorMapDataType dtype = CU_TENSOR_MAP_DATA_TYPE_UINT8, uint32_t esize = 1) {
-    EncodeTiledFn fn = encode_tiled_fn();
-    if (!fn) return record_text_error("cuTensorMapEncodeTiled is not available from the driver");
-    cuuint64_t dims[2] = {row_elems, rows};
-    cuuint64_t strides[1] = {row_elems * esize};
-    cuuint32_t box[2] = {box_elems, box_rows};
-    cuuint32_t estr[2] = {1, 1};
-    CUresult r = fn(map, dtype, 2, const_cast<void*>(base), dims, strides, box, estr,
-                    CU_TENSOR_MAP_INTERLEAVE_NONE, swz, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-    if (r != CUDA_SUCCESS) return record_text_error("cuTensorMapEncodeTiled failed");
-    return NM_OK;
-}
-
-// X viewed as [k-slice][token][128 bytes] so that one box covers several 128-byte-wide slices of a token tile.
-static int make_map_x3(CUtensorMap* map, const void* base, uint64_t tokens, uint64_t k_bytes, uint32_t box_rows, uint32_t box_slices) {
-    EncodeTiledFn fn = encode_tiled_fn();
-    if (!fn) return record_text_error("cuTensorMapEncodeTiled is not available from the driver");
-    cuuint64_t dims[3] = {128, tokens, k_bytes / 128};
-    cuuint64_t strides[2] = {k_bytes, 128};
-    cuuint32_t box[3] = {128, box_rows, box_slices};
-    cuuint32_t estr[3] = {1, 1, 1};
-    CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 3, const_cast<void*>(base), dims, strides, box, estr,
-                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-    if (r != CUDA_SUCCESS) return record_text_error("cuTensorMapEncodeTiled failed for the 3-D view of X");
-    return NM_OK;
-}
-
 static int sm_count() {
     static int cached[64] = {0};
     int dev = 0;
@@ -1077,34 +1006,6 @@ static int launch_gemm(const LinearArgs& a) {
     cfg.attrs = attr; cfg.numAttrs = getenv("NM_NO_PDL") ? 0 : 1;
     NM_CUDA_TRY(cudaLaunchKernelEx(&cfg, fn, tw, tx, ty, p));
     return NM_OK;
-}
-
-// Tile plan of the pair kernel: the band size of the tile order (returned) and start[0..pairs], the contiguous
-// range of every pair.  Resident weights: one long run per output tile (band = all token tiles).  Streamed
-// weights: bands of about one pair's share, unless `band_request` > 0 asks for another size.  The ranges
-// have about equal cost, a tile costing 1 and an output-tile change inside a range `crossing` tiles.
-static int plan_pair_tiles(int n_tok_tiles, int n_out_tiles, int pairs, bool resident, int band_request, int* start) {
-    const int n_tiles = n_tok_tiles * n_out_tiles;
-    int band = n_tok_tiles;
-    if (!resident) {
-        const int b = band_request > 0 ? band_request : (n_tiles + pairs / 2) / pairs;
-        band = b < 1 ? 1 : (b > n_tok_tiles ? n_tok_tiles : b);
-    }
-    const double crossing = resident ? 1.0 : 0.2;
-    auto out_of = [&](int t) { return tile_coord(t, n_tok_tiles, n_out_tiles, band).o; };
-    auto cost = [&](int t) { return 1.0 + ((t > 0 && out_of(t) != out_of(t - 1)) ? crossing : 0.0); };
-    double total = 0.0;
-    for (int t = 0; t < n_tiles; ++t) total += cost(t);
-    int t = 0;
-    double before = 0.0;  // cost of the tiles before t
-    for (int q = 0; q < pairs; ++q) {
-        const double threshold = q * total / pairs;
-        while (t < n_tiles - (pairs - q) && before + 0.5 * cost(t) < threshold) before += cost(t++);
-        if (q > 0 && t <= start[q - 1]) before += cost(t++);  // every pair gets at least one tile
-        start[q] = t;
-    }
-    start[pairs] = n_tiles;
-    return band;
 }
 
 // The plan costs a pass over all tiles on the host; layers are launched again and again with the same shape, so
