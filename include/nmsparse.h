@@ -198,6 +198,11 @@ int nm_admm_project_dist(const float *W, const float *U, int out, int in, int n,
  * enqueued work has finished.  The host array may be reused as soon as the call returns.
  * (Batches in which no more than eight jobs share one (n, m, bits) and block size pass their job table
  * in the kernel's parameters and leave `ws` untouched; it must be provided all the same.)
+ * Stream capture: a call that needs the job table in `ws` (more than eight jobs per kernel variant, and every
+ * *_batched call of the dense-output, group-wise and ADMM-Dist forms) uploads it from host memory the
+ * library owns only until the call returns, so it must not be captured into a CUDA graph: on a capturing
+ * stream such a call returns NM_ERR_UNSUPPORTED and enqueues nothing.  The same holds for
+ * nm_project_pack_batched_noalloc.
  */
 int nm_project_pack_batched(const nm_pack_job_t *jobs, int njobs, void *ws, size_t ws_bytes,
                             uint32_t *status, void *stream);
@@ -240,7 +245,8 @@ int nm_project_pack_batched_noalloc(const nm_pack_job_t *jobs, int njobs, uint32
  * W is a host struct; sw = per-channel scales from nm_project_pack; sx = activation scale.
  * 2:4, 1:4, 2:8 and 1:8 weights run on the sparse tensor-core path, 4:8 and dense weights on the
  * dense path after decompression in shared memory.  Shape and alignment requirements are those
- * nm_int_linear_check() tests; X and values 16-byte aligned; Y, sw, bias 4-byte aligned.
+ * nm_int_linear_check() tests; X, values and meta 16-byte aligned (NM_ERR_ALIGN otherwise; buffers that
+ * nm_project_pack filled meet this when they start on a 16-byte boundary); Y, sw, bias 4-byte aligned.
  * `ws`/`ws_bytes`: device scratch of nm_int_linear_workspace_bytes() (may be 0 -> ws may be NULL).
  */
 int nm_int_linear(const int8_t *X, int tokens, const nm_packed_t *W, float sx, const float *sw,
@@ -322,6 +328,28 @@ int nm_probe_tma_stream(const void *W, int w_rows, int w_row_bytes, const void *
                         int repeat, int delay_clocks, int loads, int stores, int producers, int poll, unsigned long long *clocks,
                         unsigned long long *trace, uint32_t *status, void *stream);
 
+/*
+ * Measurement and test aid (the paper has no counterpart): overrides the kernel nm_int_linear and its variants
+ * pick, process-wide, for every later call (not thread-safe against calls in flight on other host threads).
+ * All options are 0 by default = the library's own choice.  Names: "no_pdl" (launch without the programmatic-
+ * dependent-launch attribute), "no_pair" (one-CTA kernels only), "no_resident" (always stream the weights),
+ * "no_wide" (never the 512-channel pair kernel), "wide_any" (the 512-channel pair kernel whenever the shape
+ * allows it, however few tiles there are), "wide_bn" (its token-tile width, 224 or 192), "band" (band size of the streamed pair kernel's tile order).
+ * Results never depend on them.  Returns NM_ERR_UNSUPPORTED for an unknown name.
+ */
+int nm_debug_set_option(const char *name /* host */, int value);
+
+/*
+ * Profiling aid (the paper has no counterpart).  Only a library built with -DNM_TRACE accepts it (build.py
+ * --variant trace -> libnmsparse_trace.so); the product library returns NM_ERR_UNSUPPORTED and its kernels carry
+ * no time stamps.  `buffer`: device, u64 [512 + 64][8], zeroed by the caller, or NULL to switch tracing off.  Every
+ * later CTA-pair GEMM launch has its CTA 0 write clock64() values: row `it` (pipeline stage `it` < 512 of that CTA):
+ * [0] producer got the free stage, [1] issued its loads, [2] gate saw the stage full, [3] MMA thread was handed
+ * the stage, [4] had issued the stage's MMAs and commits; row 512 + i (tile i < 64 of that CTA): [0] an epilogue
+ * warp saw the accumulator full, [1] had finished the tile.
+ */
+int nm_debug_set_trace(unsigned long long *buffer);
+
 /* Host-only validation of a linear-layer problem: NM_OK or the error nm_int_linear would return. */
 int nm_int_linear_check(int tokens, int out, int in, int n, int m, int bits);
 
@@ -331,7 +359,8 @@ int nm_int_linear_check(int tokens, int out, int in, int n, int m, int bits);
  *   nm_absmax:        *absmax = max(*absmax, max_i |Y[i]|)   (caller zeroes *absmax first)
  *   nm_quantize_act:  sx = *absmax / 127 (1 if *absmax == 0);  Xq[i] = clamp(rne(Y[i] / sx), -128, 127)
  *                     *sx_out (nullable) receives sx.
- * Y and Xq must be 16-byte aligned.
+ * Y and Xq must be 16-byte aligned.  sx_out must not be the same word as absmax (other blocks still read the
+ * maximum while the scale is written): NM_ERR_SHAPE.
  */
 int nm_absmax(const float *Y, size_t count, float *absmax, void *stream);
 int nm_quantize_act(const float *Y, size_t count, const float *absmax, int8_t *Xq, float *sx_out,

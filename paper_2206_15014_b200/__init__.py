@@ -11,7 +11,9 @@ import ctypes
 import os
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_HERE, "libnmsparse.so")
+# NMSPARSE_LIB selects another build of the same library (the -DNM_TRACE build with time stamps in its kernels, the
+# build with short device-side wait limits that the timeout test uses); the default is the product library.
+LIB_PATH = os.environ.get("NMSPARSE_LIB") or os.path.join(_HERE, "libnmsparse.so")
 
 if not os.path.exists(LIB_PATH):
     raise ImportError(
@@ -34,7 +36,7 @@ EXPORTS = (
     "nm_int_linear_workspace_bytes",
     "nm_int_linear_check", "nm_absmax", "nm_quantize_act", "nm_poll_status", "nm_strerror",
     "nm_last_cuda_error", "nm_version", "nm_bits_per_param", "nm_encoder_cost", "nm_pair_tile_plan",
-    "nm_probe_tma_stream",
+    "nm_probe_tma_stream", "nm_debug_set_trace", "nm_debug_set_option",
 )
 
 
@@ -87,6 +89,8 @@ _lib.nm_int_linear_workspace_bytes.argtypes = [_i] * 6
 _lib.nm_int_linear_workspace_bytes.restype = _sz
 _lib.nm_int_linear_check.argtypes = [_i] * 6
 _lib.nm_probe_tma_stream.argtypes = [_vp, _i, _i, _vp, _i, _i, _vp] + [_i] * 12 + [_vp, _vp, _vp, _vp]
+_lib.nm_debug_set_trace.argtypes = [_vp]
+_lib.nm_debug_set_option.argtypes = [ctypes.c_char_p, _i]
 _lib.nm_absmax.argtypes = [_vp, _sz, _vp, _vp]
 _lib.nm_quantize_act.argtypes = [_vp, _sz, _vp, _vp, _vp, _vp]
 _lib.nm_poll_status.argtypes = [_vp, _vp]
@@ -326,6 +330,16 @@ def nm_probe_tma_stream(W, w_rows, w_row_bytes, X, tokens, k_bytes, Y, a_rows, a
     if rc < 0:
         raise NmError(rc, "nm_probe_tma_stream")
     return int(rc)
+
+
+def nm_debug_set_option(name, value):
+    """Kernel-choice override for measurements and tests (see nmsparse.h); 0 restores the library's own choice."""
+    _chk(_lib.nm_debug_set_option(name.encode(), int(value)), "nm_debug_set_option")
+
+
+def nm_debug_set_trace(buffer):
+    """Hands a zeroed int64 [576, 8] device tensor (or None) to the GEMM launches of an NM_TRACE build."""
+    _chk(_lib.nm_debug_set_trace(_ptr(buffer)), "nm_debug_set_trace")
 
 
 def nm_absmax(Y, count, absmax, stream=None):

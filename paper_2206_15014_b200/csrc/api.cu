@@ -18,6 +18,18 @@ int record_text_error(const char* text) {
     return NM_ERR_CUDA;
 }
 
+int sm_count() {
+    static int cached[64] = {0};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return 148;
+    if (!cached[dev]) {
+        int v = 0;
+        if (cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || v <= 0) v = 148;
+        cached[dev] = v;
+    }
+    return cached[dev];
+}
+
 int check_pattern(int out, int in, int n, int m, int bits) {
     if (out < 0 || in < 0 || n < 1 || m < 1 || n > m) return NM_ERR_SHAPE;
     if (bits != 4 && bits != 8) return NM_ERR_UNSUPPORTED;

@@ -30,6 +30,9 @@ inline size_t meta_row_words(int in, int n, int m) {
     return ((size_t)(in / m) * n * meta_field_bits(m) + 31) / 32;
 }
 
+// Multiprocessors of the current device (cached per device; 148 when the query fails).
+int sm_count();
+
 inline bool aligned(const void* p, size_t a) { return ((uintptr_t)p % a) == 0; }
 
 #ifdef __CUDACC__

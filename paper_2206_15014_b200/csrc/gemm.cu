@@ -31,6 +31,7 @@
 #include <mutex>
 #include <algorithm>
 #include <cstdlib>
+#include <cstring>
 
 namespace nm {
 
@@ -46,7 +47,10 @@ constexpr int kSmemLimit = 232448;  // 227 KB of dynamic shared memory per CTA
 constexpr int kSmemTail = 2048;     // barriers, TMEM slot, abort flag, slot tables
 constexpr int kStoreStage = 8 * 4096;  // per epilogue warp two [16 tokens][32 channels] fp32 staging tiles, used alternately
 constexpr int kMaxStages = 7;       // the relay cycles through 8 named barriers
-constexpr long long kWaitLimit = 1ll << 31;  // SM clocks (about a second)
+#ifndef NM_WAIT_LIMIT
+#define NM_WAIT_LIMIT (1ll << 31)
+#endif
+constexpr long long kWaitLimit = NM_WAIT_LIMIT;  // SM clocks per device-side wait (about a second; test builds shorten it)
 
 // What the epilogue writes: y = fma(acc, sx * sw[o], b[o]) as fp32; the raw int32 accumulators; y re-quantised
 // to 8 bits with a scale fixed ahead of time (Eq. 5, b = 8); y rounded to bfloat16.
@@ -121,7 +125,20 @@ struct GemmParams {
     float sy;              // static output scale of EPI_Q8
     float* absmax;
     uint32_t* status;
+    unsigned long long* trace;  // NM_TRACE builds: time stamps of CTA 0 (see nm_debug_set_trace); NULL otherwise
 };
+
+// Time stamps for profiling, compiled in with -DNM_TRACE only (a second library, never the product's):
+// CTA 0 writes clock64() into row `it` (one row of 8 words per pipeline stage, kTraceStages rows) or, for
+// per-tile events, into row kTraceStages + tile.  The kernels' work is unchanged.
+constexpr int kTraceStages = 512, kTraceTiles = 64;
+#ifdef NM_TRACE
+#define NM_TRACE_STAGE(it, col) do { if (p.trace && blockIdx.x == 0 && (it) < (uint32_t)kTraceStages) p.trace[8 * (size_t)(it) + (col)] = clock64(); } while (0)
+#define NM_TRACE_TILE(i, col) do { if (p.trace && blockIdx.x == 0 && (i) < kTraceTiles) p.trace[8 * (size_t)(kTraceStages + (i)) + (col)] = clock64(); } while (0)
+#else
+#define NM_TRACE_STAGE(it, col) do { } while (0)
+#define NM_TRACE_TILE(i, col) do { } while (0)
+#endif
 
 template <bool SPARSE, int BN, bool RESIDENT = false>
 struct GemmCfg {
@@ -693,13 +710,21 @@ nm_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_con
                     if (!ptx::mbar_wait_bounded(empty_bar(s), ((it / S) & 1u) ^ 1u, abort_flag, kWaitLimit)) {
                         raise_timeout(); ok = false; break;
                     }
+                    NM_TRACE_STAGE(it, 0);
                     const uint32_t a_dst = ptx::smem_u32(smem + s * Cfg::STAGE);
                     const uint32_t lead_full = ptx::map_to_cta(full_bar(s), 0);
                     if (leader) ptx::mbar_expect_tx(full_bar(s), 2 * Cfg::STAGE);  // bytes of both CTAs
                     if (!RES) ptx::tma_load_2d_pair(a_dst, &tmap_w, kb * Cfg::A_ROW, n0, lead_full);
                     // X is mapped as [k-slice][token][128 bytes]: both slices of the stage in one operation
                     ptx::tma_load_3d_pair(a_dst + Cfg::B_OFF, &tmap_x, 0, t0, kb * (Cfg::KB / 128), lead_full);
+                    NM_TRACE_STAGE(it, 1);
                 }
+            }
+            if (!ok && leader) {
+                // Copies of both CTAs that are still in flight complete on this CTA's barriers: let them land
+                // before the pair goes away (the peer stays until the cluster barrier at the end).
+                for (int j = 0; j < S; ++j) ptx::mbar_wait_bounded(full_bar(j), 0, never_flag, kWaitLimit >> 6);
+                if (RES) ptx::mbar_wait_bounded(a_full_bar, 0, never_flag, kWaitLimit >> 6);
             }
         }
     } else if (warp == kGateWarp) {
@@ -724,6 +749,7 @@ nm_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_con
                 wait(acc_empty_bar(buf), ((i >> 1) & 1u) ^ 1u);
                 for (int kb = 0; kb < p.kblocks; ++kb, ++it) {
                     wait(full_bar(it % S), (it / S) & 1u);
+                    if (lane == 0) NM_TRACE_STAGE(it, 2);
                     __syncwarp();
                     ptx::named_bar_arrive(1 + (it & 7u), 64);
                 }
@@ -744,6 +770,7 @@ nm_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_con
                     ptx::named_bar_sync(1 + (it & 7u), 64);
                     if (kb == 0) ptx::tc_fence_after();  // once per tile (see the one-CTA kernel)
                     if (lane == 0) {
+                        NM_TRACE_STAGE(it, 3);
                         const uint32_t st_addr = ptx::smem_u32(smem + s * Cfg::STAGE), b_addr = st_addr + Cfg::B_OFF;
                         const uint32_t a_addr = RES ? ptx::smem_u32(a_res + kb * Cfg::A_BYTES) : st_addr;
                         if constexpr (SPARSE) {
@@ -763,6 +790,7 @@ nm_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_con
                             ptx::tc_commit_pair(acc_full_bar(buf), 3);
                             if (last_of_out_tile) ptx::tc_commit_pair(a_free_bar, 3);  // both producers may replace the weights
                         }
+                        NM_TRACE_STAGE(it, 4);
                     }
                     __syncwarp();
                 }
@@ -790,8 +818,11 @@ nm_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_con
         auto load_meta = [&](int out_tile) {
             const int n = out_tile * (2 * kBM) + (int)rank * kBM + row;
             const uint4* src = reinterpret_cast<const uint4*>(p.meta + (size_t)n * p.mrow_words);
-            for (int c = 0; c < p.mrow_words; c += 4) {
-                uint4 w = (n < p.out) ? __ldg(src + (c >> 2)) : make_uint4(0x44444444u, 0x44444444u, 0x44444444u, 0x44444444u);
+            // A stage spans KB reduction elements; when the reduction ends inside the last stage (in % KB != 0)
+            // its remaining MMAs multiply zero-filled weights, but their index fields must still be valid 2:4
+            // patterns: the columns past the row's metadata get "positions 0,1", as rows past `out` do.
+            for (int c = 0; c < p.kblocks * (Cfg::KB / 32); c += 4) {
+                uint4 w = (n < p.out && c < p.mrow_words) ? __ldg(src + (c >> 2)) : make_uint4(0x44444444u, 0x44444444u, 0x44444444u, 0x44444444u);
                 ptx::tmem_st_32x4(lane_taddr + Cfg::META_COL + c, w.x, w.y, w.z, w.w);
             }
             ptx::tmem_st_wait();
@@ -816,6 +847,7 @@ nm_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_con
             if constexpr (kNarrow<EPI>) ok = ptx::named_bar_and(kNarrowAgree + half, 128, ok);  // the group stops together
             if (!ok) break;
             ptx::tc_fence_after();
+            if (ew == 0 && lane == 0) NM_TRACE_TILE(i, 0);
             // the next tile starts a new output tile: its metadata can go in now, the MMAs of this one are done
             if (SPARSE && half == 0 && i + 1 < tile_count) {
                 const int next_out_tile = tile_coord(tile_begin + i + 1, p.n_tok_tiles, p.n_out_tiles, p.band).o;
@@ -904,6 +936,7 @@ nm_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_con
                     }
                 }
             }
+            if (ew == 0 && lane == 0) NM_TRACE_TILE(i, 1);
         }
         if (lane == 0) ptx::bulk_wait_group<0>();
         if (EPI == EPI_F32 && p.absmax) {
@@ -924,20 +957,29 @@ nm_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_con
     }
 }
 
+}  // namespace nm
+
+#include "gemm_wide.cuh"
+
+namespace nm {
+
 // ---------------------------------------------------------------------------------------------
 // host side
 // ---------------------------------------------------------------------------------------------
-static int sm_count() {
-    static int cached[64] = {0};
-    int dev = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return 148;
-    if (!cached[dev]) {
-        int v = 0;
-        if (cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || v <= 0) v = 148;
-        cached[dev] = v;
-    }
-    return cached[dev];
-}
+// Kernel-choice overrides for measurements and tests (nm_debug_set_option); all zero = the library's own choice.
+struct DebugOptions {
+    int no_pdl;       // launch without the programmatic-dependent-launch attribute
+    int no_pair;      // one-CTA kernels only
+    int no_resident;  // always stream the weights through the stage ring
+    int no_wide;      // never the 512-channel pair kernel
+    int wide_any;     // the 512-channel pair kernel whenever the shape allows it, however few tiles there are
+    int wide_bn;      // token-tile width of that kernel: 224 or 192 (0 = automatic)
+    int band;         // band size of the streamed pair kernel's tile order (0 = automatic)
+};
+static DebugOptions g_opt = {0, 0, 0, 0, 0, 0, 0};
+
+// Trace buffer of NM_TRACE builds (device, kTraceStages + kTraceTiles rows of 8 u64), handed to every GEMM launch.
+static unsigned long long* g_trace_buffer = nullptr;
 
 struct LinearArgs {
     const int8_t* X; int tokens; const nm_packed_t* W;
@@ -990,7 +1032,7 @@ static int launch_gemm(const LinearArgs& a) {
     p.mrow_bytes = (int)meta_row_words(W.in, W.n, W.m) * 4;
     p.pat = xf::pattern_of(W.n, W.m, W.bits);
     p.sw = a.sw; p.bias = a.bias; p.sx_dev = a.sx_dev; p.sx_host = a.sx;
-    p.Y = a.Y; p.ACC = a.ACC; p.NARROW = a.NARROW; p.sy = a.sy; p.absmax = a.absmax; p.status = a.status;
+    p.Y = a.Y; p.ACC = a.ACC; p.NARROW = a.NARROW; p.sy = a.sy; p.absmax = a.absmax; p.status = a.status; p.trace = g_trace_buffer;
     auto fn = nm_gemm_kernel<SPARSE, BN, EPI, WSRC>;
     NM_CUDA_TRY(cudaFuncSetAttribute((const void*)fn, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::SMEM));
     const int grid = p.n_tiles < sm_count() ? p.n_tiles : sm_count();
@@ -1003,7 +1045,7 @@ static int launch_gemm(const LinearArgs& a) {
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
-    cfg.attrs = attr; cfg.numAttrs = getenv("NM_NO_PDL") ? 0 : 1;
+    cfg.attrs = attr; cfg.numAttrs = g_opt.no_pdl ? 0 : 1;
     NM_CUDA_TRY(cudaLaunchKernelEx(&cfg, fn, tw, tx, ty, p));
     return NM_OK;
 }
@@ -1049,7 +1091,7 @@ static int launch_gemm_pair(const LinearArgs& a) {
     p.kblocks = (W.in + Cfg::KB - 1) / Cfg::KB;
     p.meta = (const uint32_t*)W.meta; p.mrow_words = W.in / 32;
     p.sw = a.sw; p.bias = a.bias; p.sx_dev = a.sx_dev; p.sx_host = a.sx;
-    p.Y = a.Y; p.ACC = a.ACC; p.NARROW = a.NARROW; p.sy = a.sy; p.absmax = a.absmax; p.status = a.status;
+    p.Y = a.Y; p.ACC = a.ACC; p.NARROW = a.NARROW; p.sy = a.sy; p.absmax = a.absmax; p.status = a.status; p.trace = g_trace_buffer;
     auto fn = nm_gemm_pair_kernel<SPARSE, BN, EPI, RES>;
     NM_CUDA_TRY(cudaFuncSetAttribute((const void*)fn, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::SMEM));
     int pairs = p.n_tiles < sm_count() / 2 ? p.n_tiles : sm_count() / 2;
@@ -1059,7 +1101,7 @@ static int launch_gemm_pair(const LinearArgs& a) {
     // Streamed weights: a change of output tile only costs the metadata, so the tiles are banded by about
     // one pair's share and neighbouring pairs share X tiles in L2.  Resident weights: long runs.
     PairSchedule sched;
-    p.band = cached_pair_plan(p.n_tok_tiles, p.n_out_tiles, pairs, RES, getenv("NM_BAND") ? atoi(getenv("NM_BAND")) : 0, sched);
+    p.band = cached_pair_plan(p.n_tok_tiles, p.n_out_tiles, pairs, RES, g_opt.band, sched);
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(2 * pairs, 1, 1);
     cfg.blockDim = dim3(kPairThreads, 1, 1);
@@ -1072,15 +1114,83 @@ static int launch_gemm_pair(const LinearArgs& a) {
     // (griddepcontrol.wait) before its first access to global memory
     attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[1].val.programmaticStreamSerializationAllowed = 1;
-    cfg.attrs = attr; cfg.numAttrs = getenv("NM_NO_PDL") ? 1 : 2;
+    cfg.attrs = attr; cfg.numAttrs = g_opt.no_pdl ? 1 : 2;
     NM_CUDA_TRY(cudaLaunchKernelEx(&cfg, fn, tw, tx, ty, p, sched));
     return NM_OK;
+}
+
+// Wide pair kernel (512 channels x BN tokens per pair): 2:4 int8 weights streamed, fp32 / int32 outputs.
+template <int BN, int EPI>
+static int launch_gemm_wide(const LinearArgs& a) {
+    using Cfg = WideCfg<BN>;
+    constexpr int SKEW = 1;
+    const nm_packed_t& W = *a.W;
+    CUtensorMap tw, tx, ty;
+    int rc = make_map(&tw, W.values, (uint64_t)W.out, (uint64_t)W.in / 2, Cfg::A_ROWS, Cfg::A_ROW, CU_TENSOR_MAP_SWIZZLE_64B);
+    if (rc != NM_OK) return rc;
+    rc = make_map(&tx, a.X, (uint64_t)a.tokens, (uint64_t)W.in, Cfg::B_ROWS, 128, CU_TENSOR_MAP_SWIZZLE_128B);
+    if (rc != NM_OK) return rc;
+    bool tma_store = false;
+    rc = make_store_map<EPI>(&ty, a, &tma_store);
+    if (rc != NM_OK) return rc;
+    GemmParams p{};
+    p.tma_store = tma_store ? 1 : 0;
+    p.tokens = a.tokens; p.out = W.out; p.in = W.in;
+    p.n_tok_tiles = (a.tokens + BN - 1) / BN;
+    p.n_out_tiles = (W.out + 2 * Cfg::A_ROWS - 1) / (2 * Cfg::A_ROWS);
+    p.n_tiles = p.n_tok_tiles * p.n_out_tiles;
+    p.kblocks = W.in / Cfg::KB;
+    p.meta = (const uint32_t*)W.meta; p.mrow_words = W.in / 32;
+    p.sw = a.sw; p.bias = a.bias; p.sx_dev = a.sx_dev; p.sx_host = a.sx;
+    p.Y = a.Y; p.ACC = a.ACC; p.NARROW = a.NARROW; p.sy = a.sy; p.absmax = a.absmax; p.status = a.status; p.trace = g_trace_buffer;
+    auto fn = nm_gemm_wide_kernel<BN, EPI, SKEW>;
+    NM_CUDA_TRY(cudaFuncSetAttribute((const void*)fn, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::SMEM));
+    int pairs = p.n_tiles < sm_count() / 2 ? p.n_tiles : sm_count() / 2;
+    if (pairs > kMaxPairs) pairs = kMaxPairs;
+    PairSchedule sched;
+    p.band = cached_pair_plan(p.n_tok_tiles, p.n_out_tiles, pairs, false, 0, sched);
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(2 * pairs, 1, 1);
+    cfg.blockDim = dim3(kWideThreads, 1, 1);
+    cfg.dynamicSmemBytes = Cfg::SMEM;
+    cfg.stream = a.stream;
+    cudaLaunchAttribute attr[2];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr; cfg.numAttrs = g_opt.no_pdl ? 1 : 2;
+    NM_CUDA_TRY(cudaLaunchKernelEx(&cfg, fn, tw, tx, ty, p, sched));
+    return NM_OK;
+}
+
+// Token-tile width of the wide kernel: the one whose slowest pair has the least to do (tiles per pair, rounded
+// up, times the tile width); 0 = the wide kernel does not apply (short reductions keep their weights resident in
+// the 256-channel kernel; a matrix of at most 256 channels would leave one of the two blocks idle; narrow outputs
+// and small problems stay on the other kernels).
+template <int EPI>
+static int wide_bn(const LinearArgs& a) {
+    if (EPI != EPI_F32 && EPI != EPI_ACC) return 0;
+    if (g_opt.no_wide || g_opt.no_pair) return 0;
+    const nm_packed_t& W = *a.W;
+    if (W.in <= kPairResStages * PairCfg<true, 192>::KB || W.out <= 2 * kBM) return 0;
+    const long long pairs = sm_count() / 2, out_tiles = (W.out + 4 * kBM - 1) / (4 * kBM);
+    int best = 0;
+    long long best_cost = 0;
+    for (int bn : {224, 192}) {
+        if (g_opt.wide_bn && bn != g_opt.wide_bn) continue;
+        const long long tiles = out_tiles * ((a.tokens + bn - 1) / bn);
+        if (tiles < pairs && !g_opt.wide_any) continue;
+        const long long cost = ((tiles + pairs - 1) / pairs) * bn;
+        if (!best || cost < best_cost) { best = bn; best_cost = cost; }
+    }
+    return best;
 }
 
 // The pair kernel pays off when there is enough work for every SM pair; small problems stay on one CTA.
 template <bool SPARSE, int EPI>
 static bool use_pair(const LinearArgs& a) {
-    if (getenv("NM_NO_PAIR")) return false;
+    if (g_opt.no_pair) return false;
     const long long tiles = (long long)((a.W->out + 2 * kBM - 1) / (2 * kBM)) * ((a.tokens + 191) / 192);
     const bool fits = !SPARSE || a.W->in / 32 <= PairCfg<SPARSE, 192>::META_COLS;
     return fits && tiles >= sm_count() / 2;
@@ -1090,7 +1200,7 @@ static bool use_pair(const LinearArgs& a) {
 template <bool SPARSE, int EPI>
 static int pick_pair(const LinearArgs& a) {
     if constexpr (SPARSE) {
-        if (a.W->in <= kPairResStages * PairCfg<true, 192>::KB && !getenv("NM_NO_RESIDENT"))
+        if (a.W->in <= kPairResStages * PairCfg<true, 192>::KB && !g_opt.no_resident)
             return launch_gemm_pair<true, 192, EPI, true>(a);
     }
     return launch_gemm_pair<SPARSE, 192, EPI, false>(a);
@@ -1107,7 +1217,7 @@ static int pick_bn(const LinearArgs& a) {
     } else {
         // Short reductions with many token tiles per output tile: build each weight tile once and keep it.
         constexpr int BNR = SPARSE ? 192 : 128;
-        if (a.W->in / kKB <= kResidentKB && (long long)out_tiles * ((a.tokens + BNR - 1) / BNR) >= sms && !getenv("NM_NO_RESIDENT"))
+        if (a.W->in / kKB <= kResidentKB && (long long)out_tiles * ((a.tokens + BNR - 1) / BNR) >= sms && !g_opt.no_resident)
             return launch_gemm<SPARSE, BNR, EPI, W_RESIDENT>(a);
         if constexpr (SPARSE) {  // wider token tiles: each built weight tile serves more columns
             if (a.W->in / 32 <= GemmCfg<SPARSE, 192>::META_COLS && (long long)out_tiles * ((a.tokens + 191) / 192) >= sms)
@@ -1130,6 +1240,13 @@ static int check_linear(int tokens, int out, int in, int n, int m, int bits) {
 template <int EPI>
 static int run_linear_epi(const LinearArgs& a, bool xform, bool sparse) {
     if (xform) return sparse ? pick_bn<true, EPI, true>(a) : pick_bn<false, EPI, true>(a);
+    if constexpr (EPI == EPI_F32 || EPI == EPI_ACC) {
+        if (sparse) {
+            const int bn = wide_bn<EPI>(a);
+            if (bn == 224) return launch_gemm_wide<224, EPI>(a);
+            if (bn == 192) return launch_gemm_wide<192, EPI>(a);
+        }
+    }
     if (sparse) return use_pair<true, EPI>(a) ? pick_pair<true, EPI>(a) : pick_bn<true, EPI, false>(a);
     return use_pair<false, EPI>(a) ? pick_pair<false, EPI>(a) : pick_bn<false, EPI, false>(a);
 }
@@ -1177,6 +1294,27 @@ int nm_pair_tile_plan(int n_tok_tiles, int n_out_tiles, int pairs, int resident,
         if (tile_tok) tile_tok[t] = c.t;
     }
     return band;
+}
+
+int nm_debug_set_option(const char* name, int value) {
+    if (!name) return NM_ERR_NULL;
+    struct { const char* name; int* slot; } table[] = {
+        {"no_pdl", &nm::g_opt.no_pdl}, {"no_pair", &nm::g_opt.no_pair}, {"no_resident", &nm::g_opt.no_resident},
+        {"no_wide", &nm::g_opt.no_wide}, {"wide_any", &nm::g_opt.wide_any}, {"wide_bn", &nm::g_opt.wide_bn},
+        {"band", &nm::g_opt.band}};
+    for (auto& e : table)
+        if (!strcmp(name, e.name)) { *e.slot = value; return NM_OK; }
+    return NM_ERR_UNSUPPORTED;
+}
+
+int nm_debug_set_trace(unsigned long long* buffer) {
+#ifdef NM_TRACE
+    nm::g_trace_buffer = buffer;
+    return NM_OK;
+#else
+    (void)buffer;
+    return NM_ERR_UNSUPPORTED;
+#endif
 }
 
 int nm_int_linear_check(int tokens, int out, int in, int n, int m, int bits) {

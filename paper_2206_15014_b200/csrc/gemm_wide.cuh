@@ -1,0 +1,399 @@
+// Wide CTA-pair kernel for 2:4 int8 weights with a long reduction (weights streamed through the stage ring).
+//
+// A pair tile is 512 output channels x BN tokens: each CTA of the pair owns 256 channels, as two blocks of
+// 128 TMEM lanes with one accumulator each (columns [0, BN) and [BN, 2 BN)), and stages half of the X tile.
+// Against the 256 x 192 tile of nm_gemm_pair_kernel every staged byte of X feeds twice as many MACs: per
+// MAC the kernel moves 0.64x the bytes through L2 and through each SM's shared memory, issues half as many
+// TMA loads and barrier operations, and one pipeline stage (128 reduction elements: 16 KB of weights + BN/2
+// x 128 B of X) carries 448 tensor-core clocks of work at BN = 224 instead of 384 for a 40 KB stage.
+//
+// What changes with two accumulators of BN columns each in the 512 TMEM columns:
+//   * The 2:4 index metadata can no longer stay resident for the whole reduction.  Four metadata warps (one
+//     per TMEM lane quarter, both CTAs) copy the 16 bytes per weight row and block that a stage needs from
+//     the canonical metadata in global memory into a ring of TMEM slots (8 columns per stage, same slot
+//     index as the shared-memory stage) with tcgen05.st; the stage's "full" barrier also counts them.
+//   * The accumulators are single-buffered.  The MMA thread runs block 1 SKEW stages behind block 0, so that
+//     block 0's accumulator is handed to its four epilogue warps SKEW stages before block 1's and the next
+//     tile's block-0 MMAs can start while block 1's accumulator is still being read.
+//   * The MMA thread's instruction stream is kept short: descriptors are advanced with one add from values
+//     formed once, ring positions are carried instead of divided out (a single thread's dependent
+//     instructions cost several clocks each; 4 MMAs + commit took ~430 clocks in the 256 x 192 kernel).
+#pragma once
+
+namespace nm {
+
+constexpr int kWideEpiWarps = 8;     // four per accumulator, one per TMEM lane quarter
+constexpr int kWideGateWarp = 2 + kWideEpiWarps;
+constexpr int kWideMetaWarp0 = kWideGateWarp + 1;
+constexpr int kWideThreads = 32 * (kWideMetaWarp0 + 4);  // producer, MMA, epilogue warps, gate, metadata warps
+constexpr uint32_t kWideRelayIds = 12;  // named barriers 1..12 carry the gate's relays in turn; the gate is never more
+                                        // than STAGES + SKEW steps ahead of the MMA thread
+
+template <int BN>
+struct WideCfg {
+    static constexpr int KB = 128;                       // reduction elements per stage
+    static constexpr int A_ROWS = 2 * kBM;               // weight rows per CTA: two blocks of 128
+    static constexpr int A_ROW = 64;                     // stored bytes per weight row and stage (2:4)
+    static constexpr int A_BLOCK = kBM * A_ROW;          // bytes of one block's weight tile
+    static constexpr int A_BYTES = A_ROWS * A_ROW;
+    static constexpr int B_ROWS = BN / 2;                // tokens staged by each CTA
+    static constexpr int B_BYTES = B_ROWS * 128;
+    static constexpr int STAGE = A_BYTES + B_BYTES;
+    static constexpr int STORE_STAGE = kWideEpiWarps * 2 * 2048;  // two [16 tokens][32 channels] fp32 tiles per epilogue warp
+    static constexpr int FIT = (kSmemLimit - kSmemTail - STORE_STAGE - 1024) / STAGE;
+    static constexpr int STAGES = FIT < 8 ? FIT : 8;
+    static constexpr int SMEM = STAGES * STAGE + STORE_STAGE + kSmemTail + 1024;
+    static constexpr int META_COL = 2 * BN;              // first TMEM column of the metadata ring
+    static constexpr int META_SLOT = 8;                  // columns per stage: two blocks x 128 index bits per row
+    static_assert(STAGES >= 4, "pipeline too shallow");
+    static_assert(META_COL + STAGES * META_SLOT <= kTmemCols, "accumulators and metadata ring exceed TMEM");
+    static_assert(B_BYTES % 1024 == 0 && A_BYTES % 1024 == 0, "operand tiles must keep the swizzle alignment");
+    static_assert(BN % 32 == 0 && BN <= 256, "token tile");
+};
+
+template <int BN, int EPI, int SKEW>
+__global__ void __launch_bounds__(kWideThreads, 1)
+nm_gemm_wide_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant__ CUtensorMap tmap_x,
+                    const __grid_constant__ CUtensorMap tmap_y, const GemmParams p,
+                    const __grid_constant__ PairSchedule sched) {
+    using Cfg = WideCfg<BN>;
+    constexpr int S = Cfg::STAGES;
+    static_assert(SKEW >= 0 && SKEW < S - 2, "the ring must hold the stages block 1 lags behind plus loads in flight");
+    static_assert(S + SKEW < (int)kWideRelayIds, "relay barriers would be reused before the MMA thread has passed them");
+    static_assert(EPI == EPI_F32 || EPI == EPI_ACC, "32-bit outputs only");
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = reinterpret_cast<uint8_t*>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+    uint8_t* store_stage = smem + S * Cfg::STAGE;
+    uint64_t* bars = reinterpret_cast<uint64_t*>(store_stage + Cfg::STORE_STAGE);
+    const uint32_t bar0 = ptx::smem_u32(bars);
+    auto full_bar = [&](int s) { return bar0 + 8u * s; };                     // leader: TMA bytes of both CTAs + 8 metadata warps
+    auto empty_bar = [&](int s) { return bar0 + 8u * (S + s); };              // both CTAs (multicast commit)
+    auto acc_full_bar = [&](int b) { return bar0 + 8u * (2 * S + b); };       // both CTAs (multicast commit)
+    auto acc_empty_bar = [&](int b) { return bar0 + 8u * (2 * S + 2 + b); };  // leader; four warps of each CTA arrive
+    const uint32_t drained_bar = bar0 + 8u * (2 * S + 4);
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * S + 5);
+    volatile uint32_t* abort_flag = tmem_slot + 1;
+    volatile uint32_t* never_flag = tmem_slot + 2;
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t rank = ptx::cluster_ctarank();
+    const bool leader = rank == 0;
+    const int pair = blockIdx.x >> 1;
+    const int tile_begin = sched.start[pair];
+    const int tile_count = sched.start[pair + 1] - tile_begin;
+    const uint32_t total = (uint32_t)tile_count * (uint32_t)p.kblocks;  // pipeline stages this pair runs
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < S; ++s) { ptx::mbar_init(full_bar(s), 1 + 8); ptx::mbar_init(empty_bar(s), 1); }
+        for (int b = 0; b < 2; ++b) { ptx::mbar_init(acc_full_bar(b), 1); ptx::mbar_init(acc_empty_bar(b), 8); }
+        ptx::mbar_init(drained_bar, 1);
+        *abort_flag = 0;
+        *never_flag = 0;
+        ptx::fence_mbar_init();
+        ptx::prefetch_tensormap(&tmap_w);
+        ptx::prefetch_tensormap(&tmap_x);
+        if (p.tma_store) ptx::prefetch_tensormap(&tmap_y);
+    }
+    __syncthreads();
+    ptx::cluster_arrive();   // both CTAs' barriers exist before anything remote touches them
+    ptx::cluster_wait();
+    if (warp == 1) {
+        ptx::tmem_alloc_pair(ptx::smem_u32(tmem_slot), kTmemCols);
+        ptx::tmem_relinquish_pair();
+    }
+    ptx::tc_fence_before();
+    __syncthreads();
+    ptx::tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+    // Set-up above may overlap the tail of the kernel before this one in the stream; global memory is first
+    // touched below.
+    ptx::grid_dep_wait();
+    ptx::grid_dep_launch();
+
+    auto raise_timeout = [&]() {
+        *abort_flag = 1;
+        if (p.status) atomicOr(p.status, NM_STATUS_TIMEOUT);
+    };
+    const uint32_t lead_full0 = ptx::map_to_cta(full_bar(0), 0);  // stage s: + 8 s (one window per CTA, linear inside)
+
+    if (warp == 0) {
+        // ------------------------------ TMA producer (both CTAs) --------------------------------
+        if (lane == 0) {
+            uint32_t it = 0, parity = 1u;  // the first pass over the ring finds every stage free
+            int s = 0;
+            bool ok = true;
+            const uint32_t smem0 = ptx::smem_u32(smem);
+            for (int i = 0; i < tile_count && ok; ++i) {
+                const TileCoord tc = tile_coord(tile_begin + i, p.n_tok_tiles, p.n_out_tiles, p.band);
+                const int n0 = tc.o * (2 * Cfg::A_ROWS) + (int)rank * Cfg::A_ROWS;
+                const int t0 = tc.t * BN + (int)rank * Cfg::B_ROWS;
+                for (int kb = 0; kb < p.kblocks; ++kb, ++it) {
+                    if (!ptx::mbar_wait_bounded(empty_bar(s), parity, abort_flag, kWaitLimit)) {
+                        raise_timeout(); ok = false; break;
+                    }
+                    NM_TRACE_STAGE(it, 0);
+                    const uint32_t dst = smem0 + (uint32_t)s * Cfg::STAGE, lead_full = lead_full0 + 8u * s;
+                    if (leader) ptx::mbar_expect_tx(full_bar(s), 2 * Cfg::STAGE);  // bytes of both CTAs
+                    ptx::tma_load_2d_pair(dst, &tmap_w, kb * Cfg::A_ROW, n0, lead_full);
+                    ptx::tma_load_2d_pair(dst + Cfg::A_BYTES, &tmap_x, kb * 128, t0, lead_full);
+                    NM_TRACE_STAGE(it, 1);
+                    if (++s == S) { s = 0; parity ^= 1u; }
+                }
+            }
+            if (!ok && leader) {
+                // copies of both CTAs still in flight complete on this CTA's barriers: let them land (the peer
+                // stays until the cluster barrier at the end); the metadata arrivals may never come, so each
+                // wait is short
+                for (int j = 0; j < S; ++j) ptx::mbar_wait_bounded(full_bar(j), 0, never_flag, kWaitLimit >> 6);
+            }
+        }
+    } else if (warp >= kWideMetaWarp0) {
+        // ------------------------------ metadata warps (both CTAs) -------------------------------
+        // Thread = TMEM lane = weight row of both blocks.  The canonical metadata of a row is 16 bytes per
+        // stage; a batch of four stages (64 bytes, two full sectors) is fetched one batch ahead.
+        const int q = warp & 3, row = q * 32 + lane;
+        const uint32_t lane_taddr = tmem_base + ((uint32_t)(q * 32) << 16) + Cfg::META_COL;
+        const uint4 kIdle = make_uint4(0x44444444u, 0x44444444u, 0x44444444u, 0x44444444u);  // valid "positions 0,1"
+        const int row_u4 = p.mrow_words >> 2;  // 16-byte units per metadata row = stages per tile
+        struct Pos { int i, kb; };
+        auto fetch = [&](Pos at, uint4 (&w)[2][4]) {  // metadata of stages at.kb .. at.kb + 3 of tile at.i
+            int n = 0;
+            bool tile_ok = at.i < tile_count;
+            if (tile_ok) {
+                const TileCoord tc = tile_coord(tile_begin + at.i, p.n_tok_tiles, p.n_out_tiles, p.band);
+                n = tc.o * (2 * Cfg::A_ROWS) + (int)rank * Cfg::A_ROWS + row;
+            }
+#pragma unroll
+            for (int b = 0; b < 2; ++b) {
+                const int nb = n + b * kBM;
+                const bool row_ok = tile_ok && nb < p.out;  // rows past the end: their products are discarded
+                const uint4* src = reinterpret_cast<const uint4*>(p.meta) + (size_t)(row_ok ? nb : 0) * row_u4;
+#pragma unroll
+                for (int j = 0; j < 4; ++j)
+                    w[b][j] = (row_ok && at.kb + j < p.kblocks) ? __ldg(src + at.kb + j) : kIdle;
+            }
+        };
+        auto next_batch = [&](Pos at) {
+            at.kb += 4;
+            if (at.kb >= p.kblocks) { at.kb = 0; ++at.i; }
+            return at;
+        };
+        Pos at{0, 0};
+        uint4 cur[2][4], nxt[2][4];
+        fetch(at, nxt);
+        uint32_t parity = 1u;
+        int s = 0;
+        bool ok = true;
+        while (at.i < tile_count && ok) {
+#pragma unroll
+            for (int b = 0; b < 2; ++b)
+#pragma unroll
+                for (int j = 0; j < 4; ++j) cur[b][j] = nxt[b][j];
+            const Pos nx = next_batch(at);
+            fetch(nx, nxt);
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                if (at.kb + j < p.kblocks && ok) {
+                    // the MMAs that read this slot's previous contents are done (same barrier as the stage)
+                    bool got = lane != 0 || ptx::mbar_wait_bounded(empty_bar(s), parity, abort_flag, kWaitLimit);
+                    ok = __all_sync(0xffffffffu, got);
+                    if (!ok) { if (lane == 0) raise_timeout(); break; }
+                    const uint32_t col = lane_taddr + (uint32_t)s * Cfg::META_SLOT;
+                    ptx::tmem_st_32x4(col, cur[0][j].x, cur[0][j].y, cur[0][j].z, cur[0][j].w);
+                    ptx::tmem_st_32x4(col + 4, cur[1][j].x, cur[1][j].y, cur[1][j].z, cur[1][j].w);
+                    ptx::tmem_st_wait();
+                    ptx::tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) ptx::mbar_arrive_cluster(lead_full0 + 8u * s);
+                    if (++s == S) { s = 0; parity ^= 1u; }
+                }
+            }
+            at = nx;
+        }
+    } else if (warp == kWideGateWarp) {
+        // ------------------------------ gate (leader): mbarrier waits relayed to the MMA warp ------
+        // One relay per step g of the MMA thread: step g issues block 0 on stage g and block 1 on stage
+        // g - SKEW.  Runs its full trip count even after a timeout (then without waiting).
+        if (leader) {
+            bool ok = true;
+            auto wait = [&](uint32_t bar, uint32_t parity) {
+                if (lane == 0 && ok && !ptx::mbar_wait_bounded(bar, parity, abort_flag, kWaitLimit)) {
+                    raise_timeout();
+                    ok = false;
+                }
+            };
+            int s = 0, kb_l = 0, kb_t = 0;
+            uint32_t parity = 0u, tile_l = 0, tile_t = 0, relay = 1;
+            for (uint32_t g = 0; g < total + SKEW; ++g) {
+                if (g < total) {
+                    if (kb_l == 0) wait(acc_empty_bar(0), (tile_l & 1u) ^ 1u);  // block 0's accumulator read out
+                    wait(full_bar(s), parity);
+                    if (lane == 0) NM_TRACE_STAGE(g, 2);
+                    if (++s == S) { s = 0; parity ^= 1u; }
+                    if (++kb_l == p.kblocks) { kb_l = 0; ++tile_l; }
+                }
+                if (g >= (uint32_t)SKEW) {
+                    if (kb_t == 0) wait(acc_empty_bar(1), (tile_t & 1u) ^ 1u);
+                    if (++kb_t == p.kblocks) { kb_t = 0; ++tile_t; }
+                }
+                __syncwarp();
+                ptx::named_bar_arrive(relay, 64);
+                relay = relay == kWideRelayIds ? 1 : relay + 1;
+            }
+        }
+    } else if (warp == 1) {
+        // ------------------------------ MMA issuer (leader) --------------------------------------
+        if (leader) {
+            constexpr uint32_t idesc = ptx::idesc_i8(2 * kBM, BN, true);
+            const uint32_t smem0 = ptx::smem_u32(smem);
+            const uint64_t a_desc0 = ptx::smem_desc_kmajor(smem0, 64, ptx::kSwizzle64);
+            const uint64_t b_desc0 = ptx::smem_desc_kmajor(smem0 + Cfg::A_BYTES, 128, ptx::kSwizzle128);
+            const uint32_t meta0 = tmem_base + Cfg::META_COL;
+            const uint32_t last_kb = (uint32_t)p.kblocks - 1;
+            // ring position of block 0 (lead) and block 1 (trail): byte offset of the stage and metadata slot
+            uint32_t off_l = 0, off_t = 0, slot_l = 0, slot_t = 0, kb_l = 0, kb_t = 0, relay = 1;
+            for (uint32_t g = 0; g < total + SKEW; ++g) {
+                ptx::named_bar_sync(relay, 64);
+                relay = relay == kWideRelayIds ? 1 : relay + 1;
+                ptx::tc_fence_after();  // orders the MMAs after the metadata stores and accumulator reads of other threads
+                if (lane == 0) {
+                    NM_TRACE_STAGE(g, 3);
+                    if (g < total) {
+                        const uint64_t a = ptx::desc_advance(a_desc0, off_l), b = ptx::desc_advance(b_desc0, off_l);
+                        const uint32_t e = meta0 + slot_l;
+                        ptx::mma_sp_i8_pair(tmem_base, a, b, e, idesc, kb_l != 0);
+                        ptx::mma_sp_i8_pair(tmem_base, ptx::desc_advance(a, 32), ptx::desc_advance(b, 64), e + 2, idesc, 1u);
+                        if (SKEW != 0 && kb_l == last_kb) ptx::tc_commit_pair(acc_full_bar(0), 3);
+                    }
+                    if (g >= (uint32_t)SKEW) {
+                        const uint64_t a = ptx::desc_advance(a_desc0, off_t + Cfg::A_BLOCK), b = ptx::desc_advance(b_desc0, off_t);
+                        const uint32_t e = meta0 + slot_t + 4;
+                        ptx::mma_sp_i8_pair(tmem_base + BN, a, b, e, idesc, kb_t != 0);
+                        ptx::mma_sp_i8_pair(tmem_base + BN, ptx::desc_advance(a, 32), ptx::desc_advance(b, 64), e + 2, idesc, 1u);
+                        ptx::tc_commit_pair(empty_bar(slot_t >> 3), 3);  // both producers and the metadata warps may refill the stage
+                        if (kb_t == last_kb) {
+                            if (SKEW == 0) ptx::tc_commit_pair(acc_full_bar(0), 3);
+                            ptx::tc_commit_pair(acc_full_bar(1), 3);
+                        }
+                    }
+                    NM_TRACE_STAGE(g, 4);
+                }
+                if (g < total) {
+                    off_l += Cfg::STAGE; slot_l += Cfg::META_SLOT;
+                    if (slot_l == S * Cfg::META_SLOT) { off_l = 0; slot_l = 0; }
+                    kb_l = kb_l == last_kb ? 0 : kb_l + 1;
+                }
+                if (g >= (uint32_t)SKEW) {
+                    off_t += Cfg::STAGE; slot_t += Cfg::META_SLOT;
+                    if (slot_t == S * Cfg::META_SLOT) { off_t = 0; slot_t = 0; }
+                    kb_t = kb_t == last_kb ? 0 : kb_t + 1;
+                }
+                __syncwarp();
+            }
+            if (lane == 0) {  // everything issued has retired before TMEM is released
+                ptx::tc_commit_pair(drained_bar, 1);
+                ptx::mbar_wait_bounded(drained_bar, 0, never_flag, kWaitLimit);
+            }
+        }
+    } else {
+        // ------------------------------ epilogue warps (both CTAs) --------------------------------
+        // Warps 2-5 read block 0's accumulator, warps 6-9 block 1's; each its TMEM lane quarter, all BN columns.
+        constexpr int CH = BN / 32;
+        const int ew = warp - 2, q = warp & 3, blk = ew >> 2;
+        const uint32_t acc_taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)blk * BN;
+        float* my_stage = reinterpret_cast<float*>(store_stage + ew * 4096);
+        const float sx = p.sx_dev ? *p.sx_dev : p.sx_host;
+        const uint32_t lead_acc_empty = ptx::map_to_cta(acc_empty_bar(blk), 0);
+        float amax = 0.0f, c_n = 0.0f, b_n = 0.0f;
+        int scaled_out_tile = -1;
+        uint32_t n_stores = 0;
+        bool ok = true;
+        auto release_acc = [&]() {  // this warp has read all it needs from the accumulator
+            ptx::tc_fence_before();
+            __syncwarp();
+            if (lane == 0) ptx::mbar_arrive_cluster(lead_acc_empty);
+        };
+        for (int i = 0; i < tile_count && ok; ++i) {
+            const TileCoord tc = tile_coord(tile_begin + i, p.n_tok_tiles, p.n_out_tiles, p.band);
+            const int nw = tc.o * (2 * Cfg::A_ROWS) + (int)rank * Cfg::A_ROWS + blk * kBM + q * 32;  // first channel of this warp
+            const int n = nw + lane, t0 = tc.t * BN;
+            bool got = ptx::mbar_wait_bounded(acc_full_bar(blk), (uint32_t)i & 1u, abort_flag, kWaitLimit);
+            ok = __all_sync(0xffffffffu, got);
+            if (!ok) { if (lane == 0) raise_timeout(); break; }
+            ptx::tc_fence_after();
+            if (ew == 0 && lane == 0) NM_TRACE_TILE(i, 0);
+            if (ew == 4 && lane == 0) NM_TRACE_TILE(i, 2);
+            const bool n_ok = n < p.out;
+            if (EPI != EPI_ACC && tc.o != scaled_out_tile) {  // channel constants: fetched once per output tile
+                scaled_out_tile = tc.o;
+                c_n = n_ok ? __fmul_rn(sx, p.sw[n]) : 0.0f;
+                b_n = n_ok && p.bias ? p.bias[n] : 0.0f;
+            }
+            const int nact = min(CH, (p.tokens - t0 + 31) >> 5);  // chunks that hold tokens (warp-uniform)
+            uint32_t r[2][32];
+            if (nact > 0) ptx::tmem_ld_32x32(acc_taddr, r[0]);
+            else release_acc();
+#pragma unroll
+            for (int c = 0; c < CH; ++c) {
+                const int tc0 = t0 + c * 32;
+                if (c < nact) {
+                    ptx::tmem_ld_wait();
+                    if (c + 1 < nact) ptx::tmem_ld_32x32(acc_taddr + (c + 1) * 32, r[(c + 1) & 1]);
+                    else release_acc();
+                    const int jmax = n_ok ? min(32, p.tokens - tc0) : 0;  // outputs of this lane that exist
+                    auto conv = [&](int j) -> uint32_t {
+                        float y_abs;
+                        const uint32_t o = epi_convert<EPI>(r[c & 1][j], c_n, b_n, p.sy, 0.0f, y_abs);
+                        if constexpr (EPI == EPI_F32) amax = fmaxf(amax, j < jmax ? y_abs : 0.0f);
+                        return o;
+                    };
+                    if (p.tma_store) {  // separate branch-free loops for the two store paths
+#pragma unroll
+                        for (int h = 0; h < 2; ++h) {  // 16 tokens per store, alternating staging tiles
+                            if (tc0 + 16 * h >= p.tokens) continue;  // warp-uniform
+                            uint32_t* sb = reinterpret_cast<uint32_t*>(my_stage + (n_stores & 1u) * 512);
+                            if (lane == 0) ptx::bulk_wait_group_read<1>();  // the store before the last has read this tile
+                            __syncwarp();
+#pragma unroll
+                            for (int j = 0; j < 16; ++j) sb[j * 32 + lane] = conv(16 * h + j);
+                            ptx::fence_proxy_async_smem();
+                            __syncwarp();
+                            if (lane == 0) {
+                                ptx::tma_store_2d(&tmap_y, nw, tc0 + 16 * h, ptx::smem_u32(sb));
+                                ptx::bulk_commit_group();
+                            }
+                            ++n_stores;
+                        }
+                    } else {
+                        uint32_t* dst = reinterpret_cast<uint32_t*>(EPI == EPI_F32 ? (void*)p.Y : (void*)p.ACC) + (size_t)tc0 * p.out + n;
+#pragma unroll
+                        for (int j = 0; j < 32; ++j) {
+                            const uint32_t o = conv(j);
+                            if (j < jmax) dst[(size_t)j * p.out] = o;
+                        }
+                    }
+                }
+            }
+            if (ew == 0 && lane == 0) NM_TRACE_TILE(i, 1);
+            if (ew == 4 && lane == 0) NM_TRACE_TILE(i, 3);
+        }
+        if (lane == 0) ptx::bulk_wait_group<0>();
+        if (EPI == EPI_F32 && p.absmax) {
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, o));
+            if (lane == 0) atomicMax(reinterpret_cast<unsigned*>(p.absmax), __float_as_uint(amax));
+        }
+    }
+
+    // Neither CTA may release TMEM or exit while the other can still reach into it.
+    ptx::tc_fence_before();
+    __syncthreads();
+    ptx::cluster_arrive();
+    ptx::cluster_wait();
+    if (warp == 1) {
+        ptx::tc_fence_after();
+        ptx::tmem_dealloc_pair(tmem_base, kTmemCols);
+    }
+}
+
+}  // namespace nm

@@ -879,7 +879,13 @@ static int launch_batched(const nm_pack_job_t* jobs, const DenseOutDev* dense, i
             return NM_OK;
         }
     }
-    // Pageable-source async copies are staged before the call returns, so `table` may go away.
+    // The job table goes to `ws` with an asynchronous copy from this function's own (pageable) vector.  Launched
+    // eagerly the source is staged before the call returns, so `table` may go away.  Under stream capture the
+    // copy node would keep the host pointer and every replay of the graph would read freed memory (and the
+    // kernels would follow whatever pointers they find there): such a call is refused before anything is enqueued.
+    cudaStreamCaptureStatus capture = cudaStreamCaptureStatusNone;
+    NM_CUDA_TRY(cudaStreamIsCapturing(s, &capture));
+    if (capture != cudaStreamCaptureStatusNone) return NM_ERR_UNSUPPORTED;
     NM_CUDA_TRY(cudaMemcpyAsync(ws, table.data(), table.size() * sizeof(nm::PackJobDev),
                                 cudaMemcpyHostToDevice, s));
     // the dense-output table follows the job table (njobs entries were reserved for each)

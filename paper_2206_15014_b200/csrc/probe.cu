@@ -236,9 +236,7 @@ extern "C" int nm_probe_tma_stream(const void* W, int w_rows, int w_row_bytes, c
     p.repeat = repeat; p.delay = delay_clocks; p.loads = loads & 3; p.stores = stores ? 1 : 0; p.producers = producers; p.poll = poll;
     p.clocks = clocks; p.trace = trace; p.status = status;
     const long long n_tiles = (long long)p.n_tok_tiles * p.n_out_tiles;
-    int dev = 0, sms = 0;
-    NM_CUDA_TRY(cudaGetDevice(&dev));
-    NM_CUDA_TRY(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+    const int sms = sm_count();
     int pairs = sms / 2 < kMaxPairs ? sms / 2 : kMaxPairs;
     if (n_tiles < pairs) pairs = (int)n_tiles;
     PairSchedule sched;

@@ -62,7 +62,7 @@ __global__ void __launch_bounds__(256) quantize_act_kernel(const float* __restri
 
 static int grid_for(size_t units) {
     size_t blocks = (units + 255) / 256;
-    size_t cap = 148 * 8;
+    size_t cap = (size_t)sm_count() * 8;
     return (int)(blocks < 1 ? 1 : (blocks > cap ? cap : blocks));
 }
 
@@ -83,6 +83,7 @@ int nm_quantize_act(const float* Y, size_t count, const float* absmax, int8_t* X
                     void* stream) {
     if (!absmax || ((!Y || !Xq) && count)) return NM_ERR_NULL;
     if (count && (!nm::aligned(Y, 16) || !nm::aligned(Xq, 16))) return NM_ERR_ALIGN;
+    if (sx_out == absmax) return NM_ERR_SHAPE;  // one thread writes the scale while the others still read the maximum
     nm::quantize_act_kernel<<<nm::grid_for(count >> 4), 256, 0, (cudaStream_t)stream>>>(Y, count, absmax, Xq, sx_out);
     NM_CUDA_TRY(cudaGetLastError());
     return NM_OK;

@@ -140,6 +140,11 @@ def test_activation_quantiser_matches_oracle():
     Z = torch.zeros(64, dtype=torch.float32, device=DEV)
     amax = torch.zeros(1, dtype=torch.float32, device=DEV)
     Xq = torch.ones(64, dtype=torch.int8, device=DEV)
+    sx = torch.zeros(1, dtype=torch.float32, device=DEV)
     nm.nm_absmax(Z, 64, amax)
-    nm.nm_quantize_act(Z, 64, amax, Xq, amax)
-    assert amax.item() == 1.0 and not Xq.cpu().numpy().any()
+    nm.nm_quantize_act(Z, 64, amax, Xq, sx)
+    assert amax.item() == 0.0 and sx.item() == 1.0 and not Xq.cpu().numpy().any()   # all-zero tensor: scale 1
+    # the scale may not be written over the maximum other blocks are still reading
+    with pytest.raises(nm.NmError) as e:
+        nm.nm_quantize_act(Z, 64, amax, Xq, amax)
+    assert e.value.code == nm.NM_ERR_SHAPE

@@ -1,0 +1,77 @@
+"""GPU parity of the 512-channel CTA-pair kernel (2:4 int8 weights, reduction longer than 1024) against the CPU oracle.
+
+The library picks that kernel only for problems with at least one tile per SM pair; the option "wide_any"
+sends every eligible shape to it, so that small and ragged cases (one tile, a ragged last token tile, an output
+that does not fill the second block of 128 channels, few and many pipeline stages per tile, a pair that walks
+several tiles and changes output tile) reach it too.  int32 accumulators bit for bit, fp32 outputs equal.
+"""
+import numpy as np
+import pytest
+
+import oracle
+import workloads as wl
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(autouse=True, params=[224, 192])
+def wide_kernel_everywhere(request):
+    """Every test runs with both token-tile widths of the kernel."""
+    import paper_2206_15014_b200 as nm
+    nm.nm_debug_set_option("wide_any", 1)
+    nm.nm_debug_set_option("wide_bn", request.param)
+    yield request.param
+    nm.nm_debug_set_option("wide_any", 0)
+    nm.nm_debug_set_option("wide_bn", 0)
+
+
+def _run(seed, T, K, out, tie=False, bias=True):
+    from gpu_util import PackedOnDevice, gpu_int_linear, assert_close
+    oracle.set_threads(oracle.max_threads())
+    rng = np.random.default_rng(seed)
+    W = wl.tie_heavy(seed, out, K) if tie else wl.normal(rng, (out, K), 0.02)
+    b = wl.normal(rng, (out,), 0.02)
+    Xq, sx = oracle.quantize_act(wl.normal(rng, (T, K)))
+    v, meta, s = oracle.project_pack(W, None, 2, 4, 8)
+    D = oracle.unpack(v, meta, out, K, 2, 4, 8)
+    acc_ref, Y_ref = oracle.int_linear(Xq, D, sx, s, b if bias else None)
+    packed = PackedOnDevice(v, meta, s, out, K, 2, 4, 8)
+    acc, Y = gpu_int_linear(Xq, packed, sx, b if bias else None)
+    assert np.array_equal(acc, acc_ref), f"{(acc != acc_ref).sum()} accumulators differ"
+    assert_close(Y, Y_ref)
+    assert np.array_equal(Y, Y_ref)
+
+
+@pytest.mark.parametrize("T,K,out", [
+    (224, 1152, 512),      # one full tile, nine stages (more than the ring holds)
+    (100, 1152, 300),      # one ragged tile: second block partly filled, 100 of 224 tokens
+    (1, 1280, 257),        # a single token; one channel in the second block
+    (225, 2048, 513),      # two token tiles x two output tiles, the second ones almost empty
+    (448, 1536, 1024),     # four tiles
+    (700, 8192, 520),      # longest supported reduction (64 stages per tile)
+])
+def test_small_and_ragged(T, K, out):
+    _run(11 + T, T, K, out)
+
+
+def test_no_bias_and_ties():
+    _run(21, 300, 1152, 640, tie=True, bias=False)
+
+
+def test_many_tiles_per_pair():
+    # 5 output tiles x 34 token tiles = 170 tiles on 74 pairs: every pair walks two or three tiles, most change
+    # output tile inside their range; the last token tile is ragged
+    _run(22, 34 * 224 - 77, 1152, 2400)
+
+
+def test_library_choice_of_tile_width():
+    # no forced width: 12288 tokens x 1536 channels gives the slowest pair less to do with 192-token tiles
+    import paper_2206_15014_b200 as nm
+    nm.nm_debug_set_option("wide_bn", 0)
+    nm.nm_debug_set_option("wide_any", 0)
+    _run(23, 12288, 1280, 1536)
+
+
+def test_output_rows_not_16_byte_aligned():
+    # out % 4 != 0: the epilogue stores directly instead of through TMA
+    _run(24, 500, 1152, 515)
