@@ -1123,7 +1123,7 @@ static int launch_gemm_pair(const LinearArgs& a) {
 template <int BN, int EPI>
 static int launch_gemm_wide(const LinearArgs& a) {
     using Cfg = WideCfg<BN>;
-    constexpr int SKEW = 1;
+    constexpr int SKEW = 0;
     const nm_packed_t& W = *a.W;
     CUtensorMap tw, tx, ty;
     int rc = make_map(&tw, W.values, (uint64_t)W.out, (uint64_t)W.in / 2, Cfg::A_ROWS, Cfg::A_ROW, CU_TENSOR_MAP_SWIZZLE_64B);
