@@ -309,7 +309,8 @@ int nm_pair_tile_plan(int n_tok_tiles, int n_out_tiles, int pairs, int resident,
  * [w_rows, w_row_bytes], and `b_rows` tokens x `b_slices` 128-byte-wide slices from X, int8 [tokens, k_bytes],
  * into a ring of `stages` shared-memory stages; a consumer hands every stage back once it has landed and
  * `delay_clocks` SM clocks have passed; when `stores` != 0 eight warps write the CTA's share of the output
- * tile to Y (fp32 [tokens, w_rows], overwritten with arbitrary values) as [16 tokens][32 channels] boxes.
+ * tile to Y (fp32 [tokens, w_rows], overwritten with arbitrary values): stores == 1 as [16 tokens][32 channels]
+ * boxes, stores == 32 / 64 / 128 as 8 KB boxes that many channels wide.
  * A pair's tile is 2 * a_rows output channels x 2 * b_rows tokens; w_row_bytes / a_row_bytes must equal
  * k_bytes / (128 * b_slices) (the stages per tile).  `loads`: bit 0 = W boxes, bit 1 = X boxes; `producers`: 1 = one thread
  * issues both boxes of a stage, 2 = one thread per operand.  `poll`: how the store warps wait for a tile: 0 = all

@@ -1180,7 +1180,7 @@ static int wide_bn(const LinearArgs& a) {
     for (int bn : {224, 192}) {
         if (g_opt.wide_bn && bn != g_opt.wide_bn) continue;
         const long long tiles = out_tiles * ((a.tokens + bn - 1) / bn);
-        if (tiles < pairs && !g_opt.wide_any) continue;
+        if (2 * tiles < pairs && !g_opt.wide_any) continue;  // measured: with half the pairs busy it still beats the 256-channel kernel
         const long long cost = ((tiles + pairs - 1) / pairs) * bn;
         if (!best || cost < best_cost) { best = bn; best_cost = cost; }
     }

@@ -19,6 +19,7 @@ namespace nm {
 struct ProbeParams {
     int a_rows, a_row_bytes, b_rows, b_slices;
     int stages, kblocks, n_tok_tiles, n_out_tiles, band, repeat, delay, loads, stores, producers, poll;
+    int store_cols, store_rows;  // shape of the store boxes (channels x tokens; `stores` carries the channel count)
     unsigned long long* trace;   // [kProbeTrace][8] of CTA 0, clock64 per stage: producer before / after its wait, after arming the
                                  // barrier, after the W load, after the X load; consumer when the stage had landed, was handed back
     unsigned long long* clocks;  // [grid][4]: clock64 at start and end, globaltimer at start and end
@@ -27,7 +28,7 @@ struct ProbeParams {
 
 constexpr int kProbeStoreWarps = 8;
 constexpr int kProbeThreads = 32 * (3 + kProbeStoreWarps);  // producer, consumer, store warps, second producer
-constexpr int kProbeStaging = kProbeStoreWarps * 2048;  // one [16 tokens][32 channels] fp32 tile per store warp, as in the streamed GEMM
+constexpr int kProbeStaging = kProbeStoreWarps * 8192;  // one store box per store warp ([16 tokens][32 channels] fp32 in the GEMMs; up to 8 KB here)
 constexpr int kProbeTail = 1024;
 constexpr int kProbeSmemLimit = 232448;
 constexpr int kProbeMaxStages = 16;
@@ -152,8 +153,9 @@ tma_probe_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_consta
     } else {
         // ------------------------------ store warps: the epilogue's TMA stores -------------------
         const int sw = warp - 2;
-        float* my_stage = reinterpret_cast<float*>(staging + sw * 2048);
-        const int boxes_c = p.a_rows / 32, boxes_t = (2 * p.b_rows) / 16, boxes = boxes_c * boxes_t;
+        float* my_stage = reinterpret_cast<float*>(staging + sw * 8192);
+        const int boxes_c = p.a_rows / p.store_cols, boxes_t = (2 * p.b_rows) / p.store_rows, boxes = boxes_c * boxes_t;
+        const int box_words = p.store_cols * p.store_rows;
         for (int i = 0; i < total; ++i) {
             const int buf = i & 1;
             if (p.poll == 2) break;  // producer and consumer alone
@@ -177,12 +179,11 @@ tma_probe_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_consta
                     if (lane == 0) ptx::bulk_wait_group_read<0>();  // the store before this one has read the tile
                     __syncwarp();
                     const float v = (float)(i + b);
-#pragma unroll
-                    for (int j = 0; j < 16; ++j) sb[j * 32 + lane] = v;
+                    for (int j = lane; j < box_words; j += 32) sb[j] = v;
                     ptx::fence_proxy_async_smem();
                     __syncwarp();
                     if (lane == 0) {
-                        ptx::tma_store_2d(&tmap_y, n0 + bc * 32, t0 + bt * 16, ptx::smem_u32(sb));
+                        ptx::tma_store_2d(&tmap_y, n0 + bc * p.store_cols, t0 + bt * p.store_rows, ptx::smem_u32(sb));
                         ptx::bulk_commit_group();
                     }
                 }
@@ -226,14 +227,19 @@ extern "C" int nm_probe_tma_stream(const void* W, int w_rows, int w_row_bytes, c
     if (rc != NM_OK) return rc;
     rc = make_map_x3(&tx, X, (uint64_t)tokens, (uint64_t)k_bytes, (uint32_t)b_rows, (uint32_t)b_slices);
     if (rc != NM_OK) return rc;
-    rc = make_map(&ty, Y, (uint64_t)tokens, (uint64_t)w_rows, 16, 32, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4);
+    // `stores`: 0 = none, 1 = the GEMMs' [16 tokens][32 channels] boxes, else the channels per box (32, 64 or 128; boxes
+    // of 8 KB: 64, 32 or 16 tokens high)
+    const int store_cols = stores <= 1 ? 32 : stores, store_rows = stores <= 1 ? 16 : 8192 / (4 * store_cols);
+    if (store_cols != 32 && store_cols != 64 && store_cols != 128) return NM_ERR_SHAPE;
+    if (a_rows % store_cols || (2 * b_rows) % store_rows) return NM_ERR_SHAPE;
+    rc = make_map(&ty, Y, (uint64_t)tokens, (uint64_t)w_rows, (uint32_t)store_rows, (uint32_t)store_cols, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4);
     if (rc != NM_OK) return rc;
     ProbeParams p{};
     p.a_rows = a_rows; p.a_row_bytes = a_row_bytes; p.b_rows = b_rows; p.b_slices = b_slices;
     p.stages = stages; p.kblocks = w_row_bytes / a_row_bytes;
     p.n_tok_tiles = (tokens + 2 * b_rows - 1) / (2 * b_rows);
     p.n_out_tiles = (w_rows + 2 * a_rows - 1) / (2 * a_rows);
-    p.repeat = repeat; p.delay = delay_clocks; p.loads = loads & 3; p.stores = stores ? 1 : 0; p.producers = producers; p.poll = poll;
+    p.repeat = repeat; p.delay = delay_clocks; p.loads = loads & 3; p.stores = stores ? 1 : 0; p.producers = producers; p.poll = poll; p.store_cols = store_cols; p.store_rows = store_rows;
     p.clocks = clocks; p.trace = trace; p.status = status;
     const long long n_tiles = (long long)p.n_tok_tiles * p.n_out_tiles;
     const int sms = sm_count();
