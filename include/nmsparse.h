@@ -336,7 +336,10 @@ int nm_probe_tma_stream(const void *W, int w_rows, int w_row_bytes, const void *
  * dependent-launch attribute), "no_pair" (one-CTA kernels only), "no_resident" (always stream the weights),
  * "no_wide" (never the 512-channel pair kernel), "wide_any" (the 512-channel pair kernel whenever the shape
  * allows it, however few tiles there are), "wide_bn" (its token-tile width, 224 or 192), "band" (band size of the streamed pair kernel's tile order).
- * Results never depend on them.  Returns NM_ERR_UNSUPPORTED for an unknown name.
+ * Results never depend on them.  Returns NM_ERR_UNSUPPORTED for an unknown name.  A library built with
+ * -DNM_TEST_HOOKS (build.py --variant shortwait: device-side waits limited to about a millisecond) also takes
+ * "skip_stage" = 1 + the pipeline stage that CTA 0's producer leaves unissued (0 = none): the bounded waits then
+ * run out, the kernel drains and returns, and nm_poll_status reports NM_ERR_TIMEOUT.
  */
 int nm_debug_set_option(const char *name /* host */, int value);
 

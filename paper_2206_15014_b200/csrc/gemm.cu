@@ -50,6 +50,7 @@ constexpr int kMaxStages = 7;       // the relay cycles through 8 named barriers
 #ifndef NM_WAIT_LIMIT
 #define NM_WAIT_LIMIT (1ll << 31)
 #endif
+constexpr long long kAbortDrain = 1ll << 17;  // SM clocks a producer of a CTA pair waits after an expired wait so that its copies in flight land
 constexpr long long kWaitLimit = NM_WAIT_LIMIT;  // SM clocks per device-side wait (about a second; test builds shorten it)
 
 // What the epilogue writes: y = fma(acc, sx * sw[o], b[o]) as fp32; the raw int32 accumulators; y re-quantised
@@ -126,12 +127,22 @@ struct GemmParams {
     float* absmax;
     uint32_t* status;
     unsigned long long* trace;  // NM_TRACE builds: time stamps of CTA 0 (see nm_debug_set_trace); NULL otherwise
+    int skip_stage;             // NM_TEST_HOOKS builds: CTA 0's producer leaves this pipeline stage unissued (-1: none)
 };
 
 // Time stamps for profiling, compiled in with -DNM_TRACE only (a second library, never the product's):
 // CTA 0 writes clock64() into row `it` (one row of 8 words per pipeline stage, kTraceStages rows) or, for
 // per-tile events, into row kTraceStages + tile.  The kernels' work is unchanged.
 constexpr int kTraceStages = 512, kTraceTiles = 64;
+// Test hook, compiled in with -DNM_TEST_HOOKS only (the library the timeout test loads, never the product's): CTA 0's
+// producer skips pipeline stage `skip_stage` -- nothing is armed, nothing is copied, no address is touched -- so that
+// the stage's "full" barrier never completes and the bounded waits downstream run out.
+#ifdef NM_TEST_HOOKS
+#define NM_SKIP_STAGE(it) (p.skip_stage >= 0 && blockIdx.x == 0 && (it) == (uint32_t)p.skip_stage)
+#else
+#define NM_SKIP_STAGE(it) false
+#endif
+
 #ifdef NM_TRACE
 #define NM_TRACE_STAGE(it, col) do { if (p.trace && blockIdx.x == 0 && (it) < (uint32_t)kTraceStages) p.trace[8 * (size_t)(it) + (col)] = clock64(); } while (0)
 #define NM_TRACE_TILE(i, col) do { if (p.trace && blockIdx.x == 0 && (i) < kTraceTiles) p.trace[8 * (size_t)(kTraceStages + (i)) + (col)] = clock64(); } while (0)
@@ -237,6 +248,7 @@ nm_gemm_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant
                     if (!ptx::mbar_wait_bounded(empty_bar(s), ((it / S) & 1u) ^ 1u, abort_flag, kWaitLimit)) {
                         raise_timeout(); ok = false; break;
                     }
+                    if (NM_SKIP_STAGE(it)) continue;
                     const uint32_t a_dst = ptx::smem_u32(smem + s * Cfg::STAGE);
                     ptx::mbar_expect_tx(full_bar(s), XF ? Cfg::B_BYTES : Cfg::STAGE);
                     if (!XF) ptx::tma_load_2d(a_dst, &tmap_w, kb * Cfg::A_ROW, n0, full_bar(s));
@@ -677,8 +689,9 @@ nm_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_con
     ptx::grid_dep_wait();
     ptx::grid_dep_launch();
 
-    auto raise_timeout = [&]() {
+    auto raise_timeout = [&]() {  // both CTAs of the pair stop: the peer's roles see the flag in their own shared memory
         *abort_flag = 1;
+        ptx::st_cluster_u32(ptx::map_to_cta(ptx::smem_u32(const_cast<uint32_t*>(abort_flag)), rank ^ 1u), 1u);
         if (p.status) atomicOr(p.status, NM_STATUS_TIMEOUT);
     };
 
@@ -711,6 +724,7 @@ nm_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_con
                         raise_timeout(); ok = false; break;
                     }
                     NM_TRACE_STAGE(it, 0);
+                    if (NM_SKIP_STAGE(it)) continue;
                     const uint32_t a_dst = ptx::smem_u32(smem + s * Cfg::STAGE);
                     const uint32_t lead_full = ptx::map_to_cta(full_bar(s), 0);
                     if (leader) ptx::mbar_expect_tx(full_bar(s), 2 * Cfg::STAGE);  // bytes of both CTAs
@@ -720,12 +734,10 @@ nm_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_con
                     NM_TRACE_STAGE(it, 1);
                 }
             }
-            if (!ok && leader) {
-                // Copies of both CTAs that are still in flight complete on this CTA's barriers: let them land
-                // before the pair goes away (the peer stays until the cluster barrier at the end).
-                for (int j = 0; j < S; ++j) ptx::mbar_wait_bounded(full_bar(j), 0, never_flag, kWaitLimit >> 6);
-                if (RES) ptx::mbar_wait_bounded(a_full_bar, 0, never_flag, kWaitLimit >> 6);
-            }
+            // After an expired wait (here or anywhere in the pair) the MMA thread runs through its remaining steps without
+            // waiting for data, so the stages' barriers no longer say whether this producer's last copies have landed:
+            // give them time before the CTA and its shared memory go away.
+            if (!ok || *abort_flag) ptx::wait_clocks(kAbortDrain);
         }
     } else if (warp == kGateWarp) {
         // ------------------------------ gate (leader): mbarrier waits relayed to the MMA warp ------
@@ -975,8 +987,9 @@ struct DebugOptions {
     int wide_any;     // the 512-channel pair kernel whenever the shape allows it, however few tiles there are
     int wide_bn;      // token-tile width of that kernel: 224 or 192 (0 = automatic)
     int band;         // band size of the streamed pair kernel's tile order (0 = automatic)
+    int skip_stage;   // NM_TEST_HOOKS builds: 1 + the pipeline stage CTA 0's producer leaves out (0 = none)
 };
-static DebugOptions g_opt = {0, 0, 0, 0, 0, 0, 0};
+static DebugOptions g_opt = {0, 0, 0, 0, 0, 0, 0, 0};
 
 // Trace buffer of NM_TRACE builds (device, kTraceStages + kTraceTiles rows of 8 u64), handed to every GEMM launch.
 static unsigned long long* g_trace_buffer = nullptr;
@@ -1032,7 +1045,7 @@ static int launch_gemm(const LinearArgs& a) {
     p.mrow_bytes = (int)meta_row_words(W.in, W.n, W.m) * 4;
     p.pat = xf::pattern_of(W.n, W.m, W.bits);
     p.sw = a.sw; p.bias = a.bias; p.sx_dev = a.sx_dev; p.sx_host = a.sx;
-    p.Y = a.Y; p.ACC = a.ACC; p.NARROW = a.NARROW; p.sy = a.sy; p.absmax = a.absmax; p.status = a.status; p.trace = g_trace_buffer;
+    p.Y = a.Y; p.ACC = a.ACC; p.NARROW = a.NARROW; p.sy = a.sy; p.absmax = a.absmax; p.status = a.status; p.trace = g_trace_buffer; p.skip_stage = g_opt.skip_stage - 1;
     auto fn = nm_gemm_kernel<SPARSE, BN, EPI, WSRC>;
     NM_CUDA_TRY(cudaFuncSetAttribute((const void*)fn, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::SMEM));
     const int grid = p.n_tiles < sm_count() ? p.n_tiles : sm_count();
@@ -1091,7 +1104,7 @@ static int launch_gemm_pair(const LinearArgs& a) {
     p.kblocks = (W.in + Cfg::KB - 1) / Cfg::KB;
     p.meta = (const uint32_t*)W.meta; p.mrow_words = W.in / 32;
     p.sw = a.sw; p.bias = a.bias; p.sx_dev = a.sx_dev; p.sx_host = a.sx;
-    p.Y = a.Y; p.ACC = a.ACC; p.NARROW = a.NARROW; p.sy = a.sy; p.absmax = a.absmax; p.status = a.status; p.trace = g_trace_buffer;
+    p.Y = a.Y; p.ACC = a.ACC; p.NARROW = a.NARROW; p.sy = a.sy; p.absmax = a.absmax; p.status = a.status; p.trace = g_trace_buffer; p.skip_stage = g_opt.skip_stage - 1;
     auto fn = nm_gemm_pair_kernel<SPARSE, BN, EPI, RES>;
     NM_CUDA_TRY(cudaFuncSetAttribute((const void*)fn, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::SMEM));
     int pairs = p.n_tiles < sm_count() / 2 ? p.n_tiles : sm_count() / 2;
@@ -1142,7 +1155,7 @@ static int launch_gemm_wide(const LinearArgs& a) {
     p.kblocks = W.in / Cfg::KB;
     p.meta = (const uint32_t*)W.meta; p.mrow_words = W.in / 32;
     p.sw = a.sw; p.bias = a.bias; p.sx_dev = a.sx_dev; p.sx_host = a.sx;
-    p.Y = a.Y; p.ACC = a.ACC; p.NARROW = a.NARROW; p.sy = a.sy; p.absmax = a.absmax; p.status = a.status; p.trace = g_trace_buffer;
+    p.Y = a.Y; p.ACC = a.ACC; p.NARROW = a.NARROW; p.sy = a.sy; p.absmax = a.absmax; p.status = a.status; p.trace = g_trace_buffer; p.skip_stage = g_opt.skip_stage - 1;
     auto fn = nm_gemm_wide_kernel<BN, EPI, SKEW>;
     NM_CUDA_TRY(cudaFuncSetAttribute((const void*)fn, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::SMEM));
     int pairs = p.n_tiles < sm_count() / 2 ? p.n_tiles : sm_count() / 2;
@@ -1304,6 +1317,9 @@ int nm_debug_set_option(const char* name, int value) {
         {"band", &nm::g_opt.band}};
     for (auto& e : table)
         if (!strcmp(name, e.name)) { *e.slot = value; return NM_OK; }
+#ifdef NM_TEST_HOOKS
+    if (!strcmp(name, "skip_stage")) { nm::g_opt.skip_stage = value; return NM_OK; }
+#endif
     return NM_ERR_UNSUPPORTED;
 }
 

@@ -110,8 +110,9 @@ nm_gemm_wide_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_con
     ptx::grid_dep_wait();
     ptx::grid_dep_launch();
 
-    auto raise_timeout = [&]() {
+    auto raise_timeout = [&]() {  // both CTAs of the pair stop: the peer's roles see the flag in their own shared memory
         *abort_flag = 1;
+        ptx::st_cluster_u32(ptx::map_to_cta(ptx::smem_u32(const_cast<uint32_t*>(abort_flag)), rank ^ 1u), 1u);
         if (p.status) atomicOr(p.status, NM_STATUS_TIMEOUT);
     };
     const uint32_t lead_full0 = ptx::map_to_cta(full_bar(0), 0);  // stage s: + 8 s (one window per CTA, linear inside)
@@ -132,6 +133,7 @@ nm_gemm_wide_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_con
                         raise_timeout(); ok = false; break;
                     }
                     NM_TRACE_STAGE(it, 0);
+                    if (NM_SKIP_STAGE(it)) { if (++s == S) { s = 0; parity ^= 1u; } continue; }
                     const uint32_t dst = smem0 + (uint32_t)s * Cfg::STAGE, lead_full = lead_full0 + 8u * s;
                     if (leader) ptx::mbar_expect_tx(full_bar(s), 2 * Cfg::STAGE);  // bytes of both CTAs
                     ptx::tma_load_2d_pair(dst, &tmap_w, kb * Cfg::A_ROW, n0, lead_full);
@@ -140,12 +142,10 @@ nm_gemm_wide_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_con
                     if (++s == S) { s = 0; parity ^= 1u; }
                 }
             }
-            if (!ok && leader) {
-                // copies of both CTAs still in flight complete on this CTA's barriers: let them land (the peer
-                // stays until the cluster barrier at the end); the metadata arrivals may never come, so each
-                // wait is short
-                for (int j = 0; j < S; ++j) ptx::mbar_wait_bounded(full_bar(j), 0, never_flag, kWaitLimit >> 6);
-            }
+            // After an expired wait (here or anywhere in the pair) the MMA thread runs through its remaining steps without
+            // waiting for data, so the stages' barriers no longer say whether this producer's last copies have landed:
+            // give them time before the CTA and its shared memory go away.
+            if (!ok || *abort_flag) ptx::wait_clocks(kAbortDrain);
         }
     } else if (warp >= kWideMetaWarp0) {
         // ------------------------------ metadata warps (both CTAs) -------------------------------

@@ -187,6 +187,17 @@ __device__ __forceinline__ uint32_t map_to_cta(uint32_t smem_addr, uint32_t rank
     asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(smem_addr), "r"(rank));
     return r;
 }
+// 32-bit store into the shared memory of a CTA of the cluster (address from map_to_cta).
+__device__ __forceinline__ void st_cluster_u32(uint32_t cluster_addr, uint32_t value) {
+    asm volatile("st.shared::cluster.u32 [%0], %1;" ::"r"(cluster_addr), "r"(value) : "memory");
+}
+// Lets bulk copies that may still be in flight land before the CTA's shared memory goes away: waits `clocks`
+// SM clocks (copies complete within a few microseconds; only used on the way out after an expired wait, when the
+// barriers that would normally tell are no longer reliable).
+__device__ __forceinline__ void wait_clocks(long long clocks) {
+    const long long t0 = clock64();
+    while (clock64() - t0 < clocks) { }
+}
 __device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
     asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
 }

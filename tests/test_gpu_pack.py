@@ -89,6 +89,80 @@ def test_pack_batched_matches_single(repeat):
             assert np.array_equal(job[7].cpu().numpy(), s_ref)
 
 
+# one encoder's six components per configuration row, as in the paper's Table 4: Q4 / Q8 dense, S4 / S8 2:4 sparse
+_TABLE4_STYLE = {"Q4": (4, 4, 4), "Q8": (4, 4, 8), "S4": (2, 4, 4), "S8": (2, 4, 8), "T8": (1, 4, 8), "E4": (4, 8, 4), "P8": (2, 8, 8)}
+
+
+@pytest.mark.parametrize("layers", [1, 4])
+def test_pack_batched_whole_model_to_a_heterogeneous_configuration(layers):
+    """The search's inner step (Sec. 4, Eq. 6): every matrix of an encoder stack projected to its component's own
+    (n, m, bits) in ONE call.  layers = 1: at most eight matrices share a kernel variant (job tables in the kernel's
+    parameters); layers = 4: 24 matrices, several variants with more than eight jobs each (job table in the
+    workspace), variants with a single job, and all of it in one launch sequence.  Bit for bit against the oracle."""
+    import paper_2206_15014_b200 as nm
+    from gpu_util import DEV, to_dev
+    oracle.set_threads(oracle.max_threads())
+    hidden = 256  # small hidden size, BERT's component shapes: Q, K, V, attention output h x h, FFN1 4h x h, FFN2 h x 4h
+    shapes = [(hidden, hidden)] * 4 + [(4 * hidden, hidden), (hidden, 4 * hidden)]
+    per_layer = [["S8", "S8", "Q8", "Q4", "S4", "S4"], ["Q8", "T8", "S8", "S8", "E4", "P8"],
+                 ["S4", "S4", "S4", "Q8", "S8", "Q4"], ["S8", "Q8", "S8", "S8", "S8", "S8"]]
+    jobs, refs = [], []
+    for layer in range(layers):
+        for comp, (out, k) in enumerate(shapes):
+            n, m, bits = _TABLE4_STYLE[per_layer[layer][comp]]
+            W, U = wl.pack_sweep_matrix(40 + layer, comp, out, k)
+            vb, mb = nm.nm_packed_sizes(out, k, n, m, bits)
+            bufs = (torch.zeros(vb, dtype=torch.uint8, device=DEV), torch.zeros(max(mb // 4, 1), dtype=torch.int32, device=DEV),
+                    torch.zeros(out, dtype=torch.float32, device=DEV))
+            jobs.append((to_dev(W), to_dev(U), n, m, bits, bufs[0], bufs[1] if mb else None, bufs[2]))
+            refs.append(oracle.project_pack(W, U, n, m, bits))
+    ws_bytes = nm.nm_pack_workspace_bytes(len(jobs))
+    ws = torch.empty(ws_bytes, dtype=torch.uint8, device=DEV)
+    status = torch.zeros(1, dtype=torch.int32, device=DEV)
+    nm.nm_project_pack_batched(nm.make_pack_jobs(jobs), len(jobs), ws, ws_bytes, status)
+    assert nm.nm_poll_status(status) == 0
+    for i, (job, (v_ref, m_ref, s_ref)) in enumerate(zip(jobs, refs)):
+        assert np.array_equal(job[5].cpu().numpy().reshape(v_ref.shape), v_ref), f"job {i}: values"
+        if job[6] is not None:
+            assert np.array_equal(job[6].cpu().numpy().view(np.uint32).reshape(m_ref.shape), m_ref), f"job {i}: metadata"
+        assert np.array_equal(job[7].cpu().numpy(), s_ref), f"job {i}: scales"
+
+
+def test_batched_call_with_uploaded_job_table_refuses_stream_capture():
+    """More than eight jobs per kernel variant need the job table copied from host memory that lives only until the
+    call returns: under stream capture the call must refuse (a replayed graph would read freed memory) and enqueue
+    nothing.  The capture is ended without ever launching the graph."""
+    import paper_2206_15014_b200 as nm
+    from gpu_util import DEV, to_dev
+    jobs = []
+    for i in range(10):
+        W, U = wl.pack_sweep_matrix(50, i, 16, 256)
+        vb, mb = nm.nm_packed_sizes(16, 256, 2, 4, 8)
+        jobs.append((to_dev(W), to_dev(U), 2, 4, 8, torch.zeros(vb, dtype=torch.uint8, device=DEV),
+                     torch.zeros(mb // 4, dtype=torch.int32, device=DEV), torch.zeros(16, dtype=torch.float32, device=DEV)))
+    arr = nm.make_pack_jobs(jobs)
+    ws_bytes = nm.nm_pack_workspace_bytes(len(jobs))
+    ws = torch.empty(ws_bytes, dtype=torch.uint8, device=DEV)
+    stream = torch.cuda.Stream()
+    graph = torch.cuda.CUDAGraph()
+    torch.cuda.synchronize()
+    with torch.cuda.stream(stream):
+        graph.capture_begin()
+        try:
+            with pytest.raises(nm.NmError) as e:
+                nm.nm_project_pack_batched(arr, len(jobs), ws, ws_bytes, None, stream=stream.cuda_stream)
+            assert e.value.code == nm.NM_ERR_UNSUPPORTED
+            # eight jobs travel in the kernel's parameters: capturing that call is fine
+            nm.nm_project_pack_batched(nm.make_pack_jobs(jobs[:8]), 8, ws, ws_bytes, None, stream=stream.cuda_stream)
+        finally:
+            graph.capture_end()
+    torch.cuda.synchronize()
+    assert not jobs[0][5].any(), "the refused call, or the capture itself, ran a kernel"
+    # outside capture the same call works
+    nm.nm_project_pack_batched(arr, len(jobs), ws, ws_bytes, None)
+    assert nm.nm_poll_status() == 0 and jobs[9][5].any()
+
+
 def test_pack_flags_nonfinite_and_rejects_bad_arguments():
     import paper_2206_15014_b200 as nm
     from gpu_util import gpu_project_pack, DEV

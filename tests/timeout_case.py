@@ -1,0 +1,70 @@
+"""Child process of test_gpu_timeout.py: runs against the library built with short device-side wait limits and the
+skipped-stage test hook (NMSPARSE_LIB points at it).  For one kernel family per invocation: a launch whose CTA 0 never
+issues one pipeline stage must come back with NM_ERR_TIMEOUT (no hang, no fault, context usable), and a normal launch
+on the same stream right afterwards must match the CPU oracle.  Prints "ok <family>" on success."""
+import os
+import sys
+
+import numpy as np
+import torch
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+sys.path.insert(0, ROOT)
+import oracle  # noqa: E402
+import workloads as wl  # noqa: E402
+import paper_2206_15014_b200 as nm  # noqa: E402
+
+# family -> (tokens, K, out, options, int8 output?)
+FAMILIES = {
+    "one_cta": (64, 512, 128, {}, False),                       # one tile, four stages, nm_gemm_kernel
+    "one_cta_narrow": (64, 512, 128, {}, True),                 # the same through the int8-output epilogue's group agreement
+    "pair": (74 * 192, 1024, 256, {}, False),                   # one tile of four stages per SM pair, resident weights: pair 0 stalls alone
+    "pair_streamed": (74 * 192, 1024, 256, {"no_resident": 1}, False),
+    "wide": (224, 1152, 512, {"wide_any": 1}, False),           # one 512 x 224 tile, nine stages
+}
+
+
+def main(family):
+    T, K, out, options, narrow = FAMILIES[family]
+    dev = torch.device("cuda:0")
+    oracle.set_threads(oracle.max_threads())
+    rng = np.random.default_rng(7)
+    W = wl.normal(rng, (out, K), 0.02)
+    b = wl.normal(rng, (out,), 0.02)
+    Xq, sx = oracle.quantize_act(wl.normal(rng, (T, K)))
+    v, meta, s = oracle.project_pack(W, None, 2, 4, 8)
+    D = oracle.unpack(v, meta, out, K, 2, 4, 8)
+    _, Y_ref = oracle.int_linear(Xq, D, sx, s, b, want_acc=False)
+    sy = np.float32(np.abs(Y_ref).max()) / np.float32(127.0)
+    td = lambda a: torch.from_numpy(np.ascontiguousarray(a)).to(dev)
+    Xd, vd, md, sd, bd = td(Xq), td(v.reshape(-1)), td(meta.reshape(-1).view(np.int32)), td(s), td(b)
+    desc = nm.make_packed(out, K, 2, 4, 8, vd, md)
+    status = torch.zeros(1, dtype=torch.int32, device=dev)
+    for k_, v_ in options.items():
+        nm.nm_debug_set_option(k_, v_)
+
+    def launch():
+        if narrow:
+            Y = torch.zeros((T, out), dtype=torch.int8, device=dev)
+            nm.nm_int_linear_q8(Xd, T, desc, float(sx), sd, bd, float(sy), Y, status=status)
+        else:
+            Y = torch.zeros((T, out), dtype=torch.float32, device=dev)
+            nm.nm_int_linear(Xd, T, desc, float(sx), sd, bd, Y, status=status)
+        return Y
+
+    nm.nm_debug_set_option("skip_stage", 2)   # CTA 0 never issues its second pipeline stage
+    launch()
+    rc = nm.nm_poll_status(status)
+    assert rc == nm.NM_ERR_TIMEOUT, f"expected a timeout, got {nm.nm_strerror(rc)}"
+    nm.nm_debug_set_option("skip_stage", 0)
+    status.zero_()
+    Y = launch()                              # same stream, same context: a normal call works and is right
+    rc = nm.nm_poll_status(status)
+    assert rc == nm.NM_OK, nm.nm_strerror(rc)
+    ref = oracle.requantize_static(Y_ref, sy) if narrow else Y_ref
+    assert np.array_equal(Y.cpu().numpy(), ref), "the call after the timeout does not match the oracle"
+    print("ok", family)
+
+
+if __name__ == "__main__":
+    main(sys.argv[1])
