@@ -123,28 +123,30 @@ class ClockSampler:
 # reference arm: the CPU oracle, as it stands, on a bounded sample of the same workload
 # ------------------------------------------------------------------------------------------------
 def oracle_step(sample_tokens, state):
-    """One bounded step of the oracle: pack the attn_out matrix (1024x1024) and run every GEMM of
-    the layer on `sample_tokens` tokens.  Returns (seconds, dense-equivalent ops)."""
+    """One step of the oracle on the benchmark's workload: projection + quantise + pack of the four weight matrices of
+    the layer (W + U), then the four GEMMs on the first `sample_tokens` tokens.  Returns (seconds, dense-equivalent ops,
+    seconds of the pack part)."""
     import oracle
     import workloads as wl
     n, m, bits = PATTERN
-    if "packed" not in state:
+    if "layer" not in state:
         oracle.set_threads(oracle.max_threads())
         rng = np.random.default_rng(2)
-        state["packed"], state["X"] = [], []
+        state["layer"] = []
         for name, k, out in wl.BERT_LARGE_GEMMS:
             W = wl.normal(rng, (out, k), wl.W_STD)
-            v, meta, s = oracle.project_pack(W, None, n, m, bits)
-            state["packed"].append((oracle.unpack(v, meta, out, k, n, m, bits), s, wl.normal(rng, (out,), wl.W_STD)))
-            state["X"].append(wl.random_int8(5, (sample_tokens, k)))
-        state["W_pack"], state["U_pack"] = wl.pack_sweep_matrix(3, 1, 1024, 1024)
+            U = wl.normal(rng, (out, k), wl.U_STD)
+            b = wl.normal(rng, (out,), wl.W_STD)
+            state["layer"].append((W, U, b, wl.random_int8([5, k, out], (TOKENS, k))))
     t0 = time.perf_counter()
-    oracle.project_pack(state["W_pack"], state["U_pack"], n, m, bits)
+    packed = [oracle.project_pack(W, U, n, m, bits) for (W, U, b, X) in state["layer"]]
+    t_pack = time.perf_counter() - t0
     ops = 0.0
-    for (D, s, b), X in zip(state["packed"], state["X"]):
-        oracle.int_linear(X, D, 0.03, s, b, want_acc=False)
-        ops += gemm_ops(X.shape[0], D.shape[1], D.shape[0])
-    return time.perf_counter() - t0, ops
+    for (v, meta, s), (W, U, b, X) in zip(packed, state["layer"]):
+        D = oracle.unpack(v, meta, W.shape[0], W.shape[1], n, m, bits)
+        oracle.int_linear(X[:sample_tokens], D, 0.03, s, b, want_acc=False)
+        ops += gemm_ops(sample_tokens, W.shape[1], W.shape[0])
+    return time.perf_counter() - t0, ops, t_pack
 
 
 def run_reference(args):
@@ -158,12 +160,12 @@ def run_reference(args):
         oracle_step(sample_tokens, state)
     secs, ops = 0.0, 0.0
     for _ in range(args.steps):
-        s, o = oracle_step(sample_tokens, state)
+        s, o, _ = oracle_step(sample_tokens, state)
         secs += s
         ops += o
     value = ops / secs / 1e12
     cores = oracle.max_threads()
-    sample = f"pack of one 1024x1024 matrix + the four BERT-large GEMMs on the first {sample_tokens} tokens per step"
+    sample = f"pack of the layer's four matrices + its four GEMMs on the first {sample_tokens} of 16384 tokens per step"
     line = {"impl": "reference", "metric": METRIC, "value": value, "unit": "TOPS", "n_gpus": args.gpus,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * secs / args.steps,
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "int8",
@@ -175,19 +177,47 @@ def run_reference(args):
     return 0
 
 
-def cpu_baseline(budget_s=15.0):
-    """The oracle timed on the host cores on a bounded sample (~budget_s of CPU work)."""
+def cpu_baseline(budget_s=25.0):
+    """The oracle, as it stands, on the host cores: the SAME step the GPU runs (four matrices packed, four GEMMs) on
+    as many of the 16384 tokens as fit the budget (all of them on the usual 16 cores), and the projection/pack of the
+    24-layer sweep (timed in full when it fits the budget, else one layer scaled by 24 and marked)."""
     import oracle
+    import workloads as wl
     state = {}
-    probe, _ = oracle_step(16, state)          # includes building the inputs' first touch
-    probe, ops = oracle_step(16, state)
-    tokens = int(max(16, min(16384, 16 * budget_s / max(probe, 1e-3))))
-    state = {}
-    oracle_step(tokens, state)
-    secs, ops = oracle_step(tokens, state)
-    return {"value": ops / secs / 1e12, "unit": "TOPS", "cores": oracle.max_threads(), "kind": "oracle",
-            "sample": f"pack of one 1024x1024 matrix + the four BERT-large GEMMs on the first {tokens} tokens "
-                      f"({secs:.1f} s)"}
+    oracle_step(16, state)                       # builds the inputs
+    probe, _, _ = oracle_step(64, state)
+    _, _, t_pack = oracle_step(16, state)
+    per_token = max(probe - t_pack, 1e-4) / 64
+    tokens = int(max(64, min(TOKENS, (budget_s - t_pack) / per_token)))
+    secs, ops, t_pack = oracle_step(tokens, state)
+    full = tokens == TOKENS
+    out = {"value": ops / secs / 1e12, "unit": "TOPS", "cores": oracle.max_threads(), "kind": "oracle",
+           "seconds": secs, "pack_seconds": t_pack,
+           "sample": (f"the whole step: pack of the layer's four matrices + its four GEMMs on all {TOKENS} tokens"
+                      if full else f"pack of the layer's four matrices + its four GEMMs on the first {tokens} of "
+                                   f"{TOKENS} tokens (GEMM time scales with the tokens: extrapolated to "
+                                   f"{t_pack + (secs - t_pack) * TOKENS / tokens:.1f} s for the whole step)") + f" ({secs:.1f} s)"}
+    # projection/pack sweep: 96 matrices, 302 M parameters, 2:4 / 8 bit
+    n, m, bits = PATTERN
+    shapes = wl.pack_sweep_shapes()
+    layer_s = t_pack
+    if layer_s * 24 <= budget_s:
+        t0 = time.perf_counter()
+        for i, (o, k) in enumerate(shapes):
+            W, U = wl.pack_sweep_matrix(3, i % 4, o, k)   # the matrices' values do not change the oracle's work
+            oracle.project_pack(W, U, n, m, bits)
+        # drawing the inputs is not the method's work: time it separately and take it off
+        t_all = time.perf_counter() - t0
+        t0 = time.perf_counter()
+        for i, (o, k) in enumerate(shapes):
+            wl.pack_sweep_matrix(3, i % 4, o, k)
+        t_draw = time.perf_counter() - t0
+        out["pack_sweep"] = {"seconds": t_all - t_draw, "gbs": sum(pack_bytes(o, k, n, m, bits) for o, k in shapes) / (t_all - t_draw) / 1e9,
+                             "extrapolated": False}
+    else:
+        out["pack_sweep"] = {"seconds": layer_s * 24, "gbs": sum(pack_bytes(o, k, n, m, bits) for o, k in shapes) / (layer_s * 24) / 1e9,
+                             "extrapolated": True, "note": "one layer (4 of 96 matrices) timed, scaled by 24"}
+    return out
 
 
 def reduce_max_ms(ms, world, device="cpu"):
@@ -209,6 +239,201 @@ def whole_job_tops(ops_per_rank_step, world, ms_per_step):
 # ------------------------------------------------------------------------------------------------
 # CUDA arm
 # ------------------------------------------------------------------------------------------------
+def source_hash():
+    """Hash of the kernel sources: ties the DRAM-traffic figures under profiles/ to the kernels they were taken from."""
+    import hashlib
+    h = hashlib.sha256()
+    csrc = os.path.join(ROOT, "paper_2206_15014_b200", "csrc")
+    for name in sorted(os.listdir(csrc)):
+        if name.endswith((".cu", ".cuh")):
+            h.update(open(os.path.join(csrc, name), "rb").read())
+    return h.hexdigest()[:16]
+
+
+def recorded_traffic():
+    """DRAM bytes per launch from the ncu capture summarised in profiles/dram_traffic.txt ("key bytes" lines under a
+    "sources <hash>" line).  Empty when the kernels have changed since the capture: the figures would be stale."""
+    path = os.path.join(ROOT, "profiles", "dram_traffic.txt")
+    out, ok = {}, False
+    if os.path.exists(path):
+        for line in open(path):
+            f = line.split()
+            if len(f) >= 2 and f[0] == "sources":
+                ok = f[1] == source_hash()
+            elif len(f) >= 2 and not line.startswith("#") and f[1].isdigit():
+                out[f[0]] = int(f[1])
+    return out if ok else {}
+
+
+def gemm_entry(us, tokens, k, out, pk, n=2, m=4, bits=8, ybytes=4):
+    """Time of one GEMM launch with its three roofline fractions: of the sparse INT8 tensor peak, of the HBM peak,
+    and of the bound that applies, min(tensor, HBM) = the longer of the two ideal times."""
+    ops, byt = gemm_ops(tokens, k, out), gemm_bytes(tokens, k, out, n, m, bits, ybytes)
+    sparse_peak = 4.0 * pk["bf16_tflops"]
+    t_tensor, t_hbm = ops / sparse_peak / 1e6, byt / pk["hbm_gbs"] / 1e3   # microseconds
+    return {"us": us, "tops": ops / us / 1e6, "gbs": byt / us / 1e3,
+            "frac_sparse_int8_peak_measured": ops / us / 1e6 / sparse_peak,
+            "frac_sparse_int8_peak_nominal": ops / us / 1e6 / NOMINAL_SPARSE_INT8_TOPS,
+            "frac_hbm_measured": byt / us / 1e3 / pk["hbm_gbs"],
+            "frac_min_bound": max(t_tensor, t_hbm) / us, "bound": "tensor" if t_tensor > t_hbm else "hbm"}
+
+
+def time_stream(torch, fn, iters, warm=20):
+    """Average microseconds of fn() launched back to back `iters` times on the current stream."""
+    for i in range(warm):
+        fn(i)
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for i in range(iters):
+        fn(i)
+    e1.record()
+    torch.cuda.synchronize()
+    return e0.elapsed_time(e1) / iters * 1e3
+
+
+def packed_layer(nm, torch, dev, gemms, tokens, n, m, bits, seed, sets=4):
+    """Device buffers of one encoder layer's GEMMs with weights projected and packed by the library: `sets` rotating
+    X / Y buffer sets per GEMM (so that back-to-back launches really write to HBM), one packed weight each."""
+    import workloads as wl
+    rng = np.random.default_rng(seed)
+    layer, status = [], torch.zeros(1, dtype=torch.int32, device=dev)
+    for name, k, out in gemms:
+        W = torch.from_numpy(wl.normal(rng, (out, k), wl.W_STD)).to(dev)
+        b = torch.from_numpy(wl.normal(rng, (out,), wl.W_STD)).to(dev)
+        vb, mb = nm.nm_packed_sizes(out, k, n, m, bits)
+        values = torch.empty(vb, dtype=torch.uint8, device=dev)
+        meta = torch.empty(max(mb // 4, 1), dtype=torch.int32, device=dev)
+        scales = torch.empty(out, dtype=torch.float32, device=dev)
+        nm.nm_project_pack(W, None, out, k, n, m, bits, values, meta if mb else None, scales, status)
+        X = [torch.from_numpy(wl.random_int8([5, k, out, i], (tokens, k))).to(dev) for i in range(sets)]
+        Y = [torch.empty((tokens, out), dtype=torch.float32, device=dev) for _ in range(sets)]
+        layer.append({"name": name, "k": k, "out": out, "b": b, "scales": scales, "X": X, "Y": Y,
+                      "keep": (values, meta), "desc": nm.make_packed(out, k, n, m, bits, values, meta if mb else None)})
+    assert nm.nm_poll_status(status) == nm.NM_OK
+    return layer
+
+
+def extra_configs(nm, torch, dev, pk, status):
+    """Timed entries for the other workload configurations (each also a parity-test case): the single 128 x 768
+    projection (a latency, in microseconds), the BERT-base layer at 4096 tokens, the BERT-large layer at 4096 tokens
+    and with packed 4-bit codes at 16384 tokens, the 48-GEMM heterogeneous chain at 6144 tokens with its re-quantise
+    steps, and the whole-model projection of the search (Sec. 4)."""
+    import workloads as wl
+    out = {}
+    sx = 0.03
+    # ---- configuration 1: one BERT-base attention output projection, 128 tokens: latency --------------------------
+    lay = packed_layer(nm, torch, dev, (("attn_out", 768, 768),), 128, 2, 4, 8, seed=0)[0]
+    call = lambda i: nm.nm_int_linear(lay["X"][i % 4], 128, lay["desc"], sx, lay["scales"], lay["b"], lay["Y"][i % 4], status=status)
+    lat = []
+    for i in range(60):
+        torch.cuda.synchronize()
+        t0 = time.perf_counter()
+        call(i)
+        torch.cuda.synchronize()
+        lat.append((time.perf_counter() - t0) * 1e6)
+    out["single_projection_128x768"] = {"latency_us_call_to_completion": float(np.median(lat[10:])),
+                                        "us_back_to_back": time_stream(torch, call, 400),
+                                        "note": "all operands resident in L2: a latency figure, no roofline"}
+    # ---- configurations 2 and 3: encoder-layer GEMMs, one launch after the other ------------------------------------
+    for key, gemms, tokens, bits in (("bert_base_4096tok_int8", wl.BERT_BASE_GEMMS, 4096, 8),
+                                     ("bert_large_4096tok_int8", wl.BERT_LARGE_GEMMS, 4096, 8),
+                                     ("bert_large_16384tok_int4", wl.BERT_LARGE_GEMMS, 16384, 4)):
+        layer = packed_layer(nm, torch, dev, gemms, tokens, 2, 4, bits, seed=1 if gemms is wl.BERT_BASE_GEMMS else 2)
+        entry, total = {}, 0.0
+        for g in layer:
+            us = time_stream(torch, lambda i, g=g: nm.nm_int_linear(g["X"][i % 4], tokens, g["desc"], sx, g["scales"], g["b"],
+                                                                     g["Y"][i % 4], status=status), 200)
+            entry[g["name"]] = gemm_entry(us, tokens, g["k"], g["out"], pk, bits=bits)
+            total += us
+        def whole(i, layer=layer):
+            for g in layer:
+                nm.nm_int_linear(g["X"][i % 4], tokens, g["desc"], sx, g["scales"], g["b"], g["Y"][i % 4], status=status)
+        entry["layer_us"] = time_stream(torch, whole, 100)
+        entry["layer_tops"] = sum(gemm_ops(tokens, g["k"], g["out"]) for g in layer) / entry["layer_us"] / 1e6
+        out[key] = entry
+        del layer
+        torch.cuda.empty_cache()
+    # ---- configuration 5: heterogeneous 12-layer chain, 6144 tokens, re-quantised between GEMMs ------------------------
+    T, hidden = 6144, 768
+    modes, h0, weights = wl.chain_case(4, layers=12, tokens=T)
+    chain = []
+    for layer_modes, wrow in zip(modes, weights):
+        for mode, (W, b) in zip(layer_modes, wrow):
+            n, m, bits = wl.CHAIN_MODES[mode]
+            o, k = W.shape
+            vb, mb = nm.nm_packed_sizes(o, k, n, m, bits)
+            values = torch.empty(vb, dtype=torch.uint8, device=dev)
+            meta = torch.empty(max(mb // 4, 1), dtype=torch.int32, device=dev)
+            scales = torch.empty(o, dtype=torch.float32, device=dev)
+            nm.nm_project_pack(torch.from_numpy(W).to(dev), None, o, k, n, m, bits, values, meta if mb else None, scales, status)
+            chain.append({"out": o, "k": k, "b": torch.from_numpy(b).to(dev), "scales": scales, "keep": (values, meta),
+                          "desc": nm.make_packed(o, k, n, m, bits, values, meta if mb else None), "mode": (n, m, bits)})
+    Ybuf = torch.empty((T, 3072), dtype=torch.float32, device=dev)      # widest output
+    Vbuf = torch.empty((T, hidden), dtype=torch.float32, device=dev)
+    Xbuf = [torch.empty((T, 3072), dtype=torch.int8, device=dev) for _ in range(2)]
+    amax = torch.zeros(2, dtype=torch.float32, device=dev)
+    sxd = torch.empty(2, dtype=torch.float32, device=dev)
+    H0 = torch.from_numpy(h0).to(dev)
+
+    def run_chain(_):
+        amax.zero_()
+        nm.nm_absmax(H0, H0.numel(), amax[0:1])
+        nm.nm_quantize_act(H0, H0.numel(), amax[0:1], Xbuf[0], sxd[0:1])
+        cur = 0
+        for i, g in enumerate(chain):
+            o, k = g["out"], g["k"]
+            Y = Ybuf.view(-1)[: T * o].view(T, o)
+            X = Xbuf[cur].view(-1)[: T * k].view(T, k)
+            nxt = cur ^ 1
+            amax[nxt:nxt + 1].zero_()
+            if i % 4 == 0:   # QKV: only the V slice feeds the next GEMM (a copy, no arithmetic), then its own maximum
+                nm.nm_int_linear_dsx(X, T, g["desc"], sxd[cur:cur + 1], g["scales"], g["b"], Y, None, status=status)
+                Vbuf.copy_(Y[:, 2 * hidden:])
+                nm.nm_absmax(Vbuf, Vbuf.numel(), amax[nxt:nxt + 1])
+                src, cnt = Vbuf, Vbuf.numel()
+            else:            # the GEMM's own running max|Y| feeds the quantiser
+                nm.nm_int_linear_dsx(X, T, g["desc"], sxd[cur:cur + 1], g["scales"], g["b"], Y, amax[nxt:nxt + 1], status=status)
+                src, cnt = Y, Y.numel()
+            nm.nm_quantize_act(src, cnt, amax[nxt:nxt + 1], Xbuf[nxt], sxd[nxt:nxt + 1])
+            cur = nxt
+
+    chain_us = time_stream(torch, run_chain, 20, warm=3)
+    chain_ops = sum(gemm_ops(T, g["k"], g["out"]) for g in chain)
+    out["hetero_chain_48gemm_6144tok"] = {
+        "us": chain_us, "tops_dense_equivalent": chain_ops / chain_us / 1e6, "gemms": len(chain),
+        "modes": {f"{n}:{m}/{b}b": int(sum(1 for g in chain if g["mode"] == (n, m, b))) for (n, m, b) in wl.CHAIN_MODES},
+        "note": "48 GEMM launches + 48 re-quantise launches (+ 12 slice copies and 13 absmax launches), device-resident scales"}
+    del chain, Ybuf, Vbuf, Xbuf
+    torch.cuda.empty_cache()
+    # ---- search support: a whole BERT-base encoder stack projected to a heterogeneous configuration in one call ---------
+    cfgs = {"Q4": (4, 4, 4), "Q8": (4, 4, 8), "S4": (2, 4, 4), "S8": (2, 4, 8)}
+    row = ["S8", "S8", "Q8", "Q4", "S4", "S4"]       # one Table-4-style row: Q, K, V, attention output, FFN1, FFN2
+    shapes6 = [(768, 768)] * 4 + [(3072, 768), (768, 3072)]
+    gen = torch.Generator(device=dev)
+    gen.manual_seed(6)
+    jobs, nbytes = [], 0.0
+    for layer in range(12):
+        for comp, (o, k) in enumerate(shapes6):
+            n, m, bits = cfgs[row[(comp + layer) % 6]]   # the components' formats rotate from layer to layer
+            W = torch.empty((o, k), dtype=torch.float32, device=dev).normal_(0.0, 0.02, generator=gen)
+            vb, mb = nm.nm_packed_sizes(o, k, n, m, bits)
+            jobs.append((W, None, n, m, bits, torch.empty(vb, dtype=torch.uint8, device=dev),
+                         torch.empty(max(mb // 4, 1), dtype=torch.int32, device=dev) if mb else None,
+                         torch.empty(o, dtype=torch.float32, device=dev)))
+            nbytes += pack_bytes(o, k, n, m, bits, with_u=False)
+    arr = nm.make_pack_jobs(jobs)
+    ws_bytes = nm.nm_pack_workspace_bytes(len(jobs))
+    ws = torch.empty(ws_bytes, dtype=torch.uint8, device=dev)
+    us = time_stream(torch, lambda i: nm.nm_project_pack_batched(arr, len(jobs), ws, ws_bytes, status), 50, warm=5)
+    out["whole_model_projection_bert_base"] = {
+        "us_per_configuration": us, "matrices": len(jobs), "gbs": nbytes / us / 1e3,
+        "frac_hbm_measured": nbytes / us / 1e3 / pk["hbm_gbs"],
+        "seconds_for_905_configurations": 905 * us / 1e6,
+        "note": "72 matrices (85 M parameters, 340 MB: larger than L2), four formats rotating over the components, one call"}
+    return out
+
+
 def run_cuda(args):
     TOKENS = args.tokens
     PATTERN = (2, 4, args.bits)
@@ -239,12 +464,10 @@ def run_cuda(args):
         Xq = wl.random_int8([5, rank, k, out], (TOKENS, k))
         layer.append((name, k, out, W, U, b, Xq))
 
-    host = []  # pinned host copies for the end-to-end leg
+    host = []  # pinned host copies for the end-to-end leg: inputs, and every result of the step
     devbuf = []
     for name, k, out, W, U, b, Xq in layer:
         hW, hU, hX = (torch.from_numpy(a).pin_memory() for a in (W, U, Xq))
-        hY = torch.empty((TOKENS, out), dtype=YDTYPE).pin_memory()
-        host.append((hW, hU, hX, hY))
         vb, mb = nm.nm_packed_sizes(out, k, n, m, bits)
         d = {"W": hW.to(dev), "U": hU.to(dev), "X": hX.to(dev), "b": torch.from_numpy(b).to(dev),
              "values": torch.empty(vb, dtype=torch.uint8, device=dev),
@@ -252,6 +475,8 @@ def run_cuda(args):
              "scales": torch.empty(out, dtype=torch.float32, device=dev),
              "Y": torch.empty((TOKENS, out), dtype=YDTYPE, device=dev), "k": k, "out": out, "name": name}
         d["desc"] = nm.make_packed(out, k, n, m, bits, d["values"], d["meta"])
+        hres = {key: torch.empty(d[key].shape, dtype=d[key].dtype).pin_memory() for key in ("Y", "values", "meta", "scales")}
+        host.append((hW, hU, hX, hres))
         devbuf.append(d)
     status = torch.zeros(1, dtype=torch.int32, device=dev)
     jobs = nm.make_pack_jobs([(d["W"], d["U"], n, m, bits, d["values"], d["meta"], d["scales"]) for d in devbuf])
@@ -265,27 +490,29 @@ def run_cuda(args):
     for d in devbuf:
         kernel_events[d["name"]] = []
 
-    def step(record=False):
-        if record:
-            e0, e1 = ev(), ev()
-            e0.record()
-        nm.nm_project_pack_batched(jobs, len(devbuf), ws, ws_bytes, status)
-        if record:
-            e1.record()
-            kernel_events["pack"].append((e0, e1))
-        for d in devbuf:
-            if record:
+    def linear(d):
+        if args.out == "f32":
+            nm.nm_int_linear(d["X"], TOKENS, d["desc"], sx, d["scales"], d["b"], d["Y"], status=status)
+        elif args.out == "int8":
+            nm.nm_int_linear_q8(d["X"], TOKENS, d["desc"], sx, d["scales"], d["b"], SY, d["Y"], status=status)
+        else:
+            nm.nm_int_linear_bf16(d["X"], TOKENS, d["desc"], sx, d["scales"], d["b"], d["Y"], status=status)
+
+    names = ["pack"] + [d["name"] for d in devbuf]
+
+    def step(record=None):
+        """One step.  record = the name of ONE launch to put an event pair around (the other four stay chained)."""
+        for name in names:
+            if name == record:
                 e0, e1 = ev(), ev()
                 e0.record()
-            if args.out == "f32":
-                nm.nm_int_linear(d["X"], TOKENS, d["desc"], sx, d["scales"], d["b"], d["Y"], status=status)
-            elif args.out == "int8":
-                nm.nm_int_linear_q8(d["X"], TOKENS, d["desc"], sx, d["scales"], d["b"], SY, d["Y"], status=status)
+            if name == "pack":
+                nm.nm_project_pack_batched(jobs, len(devbuf), ws, ws_bytes, status)
             else:
-                nm.nm_int_linear_bf16(d["X"], TOKENS, d["desc"], sx, d["scales"], d["b"], d["Y"], status=status)
-            if record:
+                linear(next(d for d in devbuf if d["name"] == name))
+            if name == record:
                 e1.record()
-                kernel_events[d["name"]].append((e0, e1))
+                kernel_events[name].append((e0, e1))
 
     def barrier():
         if world > 1:
@@ -295,7 +522,7 @@ def run_cuda(args):
     def max_over_ranks(ms):
         return reduce_max_ms(ms, world, dev)
 
-    # ---- device-resident timing -----------------------------------------------------------------
+    # ---- headline: device-resident timing, nothing but the step's five launches in the timed region ------------------
     for _ in range(max(args.warmup, 3)):
         step()
     barrier()
@@ -306,8 +533,8 @@ def run_cuda(args):
     barrier()
     t0, t1 = ev(), ev()
     t0.record()
-    for k_ in range(args.steps):
-        step(record=k_ < 200)
+    for _ in range(args.steps):
+        step()
     t1.record()
     barrier()
     ms = max_over_ranks(t0.elapsed_time(t1))
@@ -318,11 +545,22 @@ def run_cuda(args):
     ops_step = sum(gemm_ops(TOKENS, d["k"], d["out"]) for d in devbuf)
     value = whole_job_tops(ops_step, world, ms_per_step)
 
+    # ---- the same steps once more, each with an event pair around ONE of its five launches in turn: the per-kernel
+    # breakdown.  (An event between two launches keeps the second from starting its set-up during the first one's tail,
+    # so a bracketed launch reads a little longer than it takes inside the headline region.) ----
+    prof_steps = 5 * max(8, min(args.steps // 5, 40))
+    p0, p1 = ev(), ev()
+    p0.record()
+    for j in range(prof_steps):
+        step(record=names[j % 5])
+    p1.record()
+    barrier()
+    profiled_ms_per_step = p0.elapsed_time(p1) / prof_steps
     kern = {}
     for name, pairs in kernel_events.items():
         kern[name] = float(np.mean([a.elapsed_time(b) for a, b in pairs])) * 1e3  # microseconds
 
-    # ---- end to end: pinned host buffers in, Y out, every step ------------------------------------
+    # ---- end to end: pinned host buffers in, every result of the step out (Y and the packed weights), every step --------
     # Copies run on their own streams: the inputs of step i + 1 go in (after step i's kernels have read the
     # old ones) while the outputs of step i are still leaving; the kernels of step i + 1 wait for both.
     main = torch.cuda.current_stream()
@@ -332,7 +570,7 @@ def run_cuda(args):
     def e2e_step():
         s_in.wait_event(ev_comp)
         with torch.cuda.stream(s_in):
-            for (hW, hU, hX, hY), d in zip(host, devbuf):
+            for (hW, hU, hX, hres), d in zip(host, devbuf):
                 d["W"].copy_(hW, non_blocking=True)
                 d["U"].copy_(hU, non_blocking=True)
                 d["X"].copy_(hX, non_blocking=True)
@@ -343,11 +581,12 @@ def run_cuda(args):
         ev_comp.record(main)
         s_out.wait_event(ev_comp)
         with torch.cuda.stream(s_out):
-            for (hW, hU, hX, hY), d in zip(host, devbuf):
-                hY.copy_(d["Y"], non_blocking=True)
+            for (hW, hU, hX, hres), d in zip(host, devbuf):
+                for key, h in hres.items():
+                    h.copy_(d[key], non_blocking=True)
             ev_out.record(s_out)
 
-    e2e_steps = max(1, min(args.steps, 5))
+    e2e_steps = max(3, min(args.steps, 20))
     e2e_step()
     main.wait_event(ev_out)
     barrier()
@@ -358,51 +597,81 @@ def run_cuda(args):
     t1.record()
     barrier()
     e2e_ms = max_over_ranks(t0.elapsed_time(t1)) / e2e_steps
-    h2d = sum(hW.numel() * 4 + hU.numel() * 4 + hX.numel() for hW, hU, hX, hY in host)
-    d2h = sum(hY.numel() * YB for hW, hU, hX, hY in host)
+    h2d = sum(hW.numel() * 4 + hU.numel() * 4 + hX.numel() for hW, hU, hX, hres in host)
+    d2h = sum(h.numel() * h.element_size() for hW, hU, hX, hres in host for h in hres.values())
     clocks = sampler.stop() if rank == 0 else None
 
     # ---- projection/pack on the full 24-layer sweep (its own roofline), rank 0 only ---------------
     pack_info = None
     if rank == 0 and not args.skip_sweep:
         pack_info = pack_sweep(nm, torch, dev, status)
+    # ---- the dominant GEMMs launched alone, back to back over rotating buffers; write-only bandwidth of the device ------
+    alone = {}
+    write_gbs = None
+    if rank == 0:
+        for d in devbuf:
+            Ys = [d["Y"]] + [torch.empty_like(d["Y"]) for _ in range(2)]
+            def one(i, d=d, Ys=Ys):
+                saved, d["Y"] = d["Y"], Ys[i % 3]
+                linear(d)
+                d["Y"] = saved
+            alone[d["name"]] = time_stream(torch, one, 100)
+            del Ys
+        fill = torch.empty(1 << 30, dtype=torch.uint8, device=dev)
+        write_gbs = (1 << 30) / time_stream(torch, lambda i: fill.zero_(), 10, warm=2) / 1e3
+        del fill
+        torch.cuda.empty_cache()
+    extras = None
+    if rank == 0 and not args.skip_configs and TOKENS == 16384 and bits == 8 and args.out == "f32":
+        for d in devbuf:   # make room: the extra configurations bring their own buffers
+            d.pop("W"); d.pop("U")
+        torch.cuda.empty_cache()
+        extras = extra_configs(nm, torch, dev, pk, status)
+        rc = nm.nm_poll_status(status)
+        if rc != nm.NM_OK:
+            raise RuntimeError("device status in the extra configurations: " + nm.nm_strerror(rc))
 
     if rank == 0:
         sparse_peak = 4.0 * pk["bf16_tflops"]
+        traffic = recorded_traffic()
+        full_size = TOKENS == 16384 and bits == 8 and args.out == "f32"
         per_kernel = {}
         for d in devbuf:
-            us = kern[d["name"]]
-            ops, byt = gemm_ops(TOKENS, d["k"], d["out"]), gemm_bytes(TOKENS, d["k"], d["out"], n, m, bits, YB)
-            per_kernel[d["name"]] = {
-                "us": us, "tops": ops / us / 1e6, "gbs": byt / us / 1e3,
-                "frac_sparse_int8_peak_measured": ops / us / 1e6 / sparse_peak,
-                "frac_sparse_int8_peak_nominal": ops / us / 1e6 / NOMINAL_SPARSE_INT8_TOPS,
-                "frac_hbm_measured": byt / us / 1e3 / pk["hbm_gbs"]}
+            e = gemm_entry(kern[d["name"]], TOKENS, d["k"], d["out"], pk, n, m, bits, YB)
+            e["us_launched_alone"] = alone[d["name"]]
+            per_kernel[d["name"]] = e
         pbytes = sum(pack_bytes(d["out"], d["k"], n, m, bits) for d in devbuf)
         per_kernel["pack_layer"] = {"us": kern["pack"], "gbs": pbytes / kern["pack"] / 1e3,
                                     "frac_hbm_measured": pbytes / kern["pack"] / 1e3 / pk["hbm_gbs"]}
         if pack_info:
             per_kernel["pack_sweep"] = pack_info
-        # dominant kernel of the step: the FFN1 GEMM launch (longest; bound by the fp32 Y write).
-        # `traffic` = dram__bytes_read.sum + dram__bytes_write.sum of one launch at this size (ncu, see
-        # profiles/); part of Y is still in the 126 MB L2 when the kernel ends, hence below the algorithmic bytes.
-        full_size = TOKENS == 16384 and bits == 8 and args.out == "f32"
+        # dominant kernel of the step: the FFN1 GEMM launch (longest).  Its bytes are 93 % fp32 Y written; a plain fill of
+        # 1 GiB on the same device gives the write-only rate such a kernel can reach (`write_only_gbs`, below the copy
+        # figure that `peak` is).  `traffic` = dram__bytes_read.sum + dram__bytes_write.sum of one launch at this size
+        # (ncu; part of Y is still in the 126 MB L2 when the kernel ends, hence below the algorithmic bytes).
         dom = per_kernel["ffn1"]
-        # kernel variant the library picks at this size: CTA pairs with resident / streamed weights for
-        # int8 2:4; for 4-bit codes the one-CTA kernel whose builder warps widen them in shared memory
         k1 = f"nm_gemm_pair_kernel<sparse,192,{args.out},resident>" if bits == 8 else f"nm_gemm_kernel<sparse,192,{args.out},build-resident>"
-        k2 = f"nm_gemm_pair_kernel<sparse,192,{args.out},streamed>" if bits == 8 else f"nm_gemm_kernel<sparse,192,{args.out},build-per-k-block>"
+        if bits != 8:
+            k2 = f"nm_gemm_kernel<sparse,192,{args.out},build-per-k-block>"
+        elif args.out == "f32":
+            k2 = "nm_gemm_wide_kernel<224,f32>"
+        else:
+            k2 = f"nm_gemm_pair_kernel<sparse,192,{args.out},streamed>"
         roofline = {"kernel": k1 + " on ffn1 1024->4096", "bound": "hbm",
                     "achieved": dom["gbs"], "peak": pk["hbm_gbs"], "unit": "GB/s",
-                    "frac": dom["gbs"] / pk["hbm_gbs"], "traffic": 241730816 if full_size else None,
-                    "algorithmic_bytes": gemm_bytes(TOKENS, 1024, 4096, n, m, bits, YB), "peak_source": pk["source"]}
+                    "frac": dom["gbs"] / pk["hbm_gbs"], "traffic": traffic.get("ffn1") if full_size else None,
+                    "algorithmic_bytes": gemm_bytes(TOKENS, 1024, 4096, n, m, bits, YB), "peak_source": pk["source"],
+                    "write_only_gbs": write_gbs,
+                    "frac_of_write_only": dom["gbs"] / write_gbs if write_gbs else None}
         f2 = per_kernel["ffn2"]
         roofline_tensor = {"kernel": k2 + " on ffn2 4096->1024", "bound": "tensor",
                            "achieved": f2["tops"], "peak": sparse_peak, "unit": "TOP/s",
                            "frac": f2["tops"] / sparse_peak,
                            "peak_note": "4 x measured bf16 burst (nominal int8-sparse : bf16-dense ratio)",
                            "frac_of_nominal_9000": f2["tops"] / NOMINAL_SPARSE_INT8_TOPS,
-                           "traffic": 113428480 if full_size else None}
+                           "frac_launched_alone": gemm_ops(TOKENS, 4096, 1024) / alone["ffn2"] / 1e6 / sparse_peak,
+                           "frac_min_bound": f2["frac_min_bound"],
+                           "traffic": traffic.get("ffn2") if full_size else None}
         line = {"metric": METRIC, "value": value, "unit": "TOPS", "n_gpus": world, "steps": args.steps,
                 "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True,
                 "scaling": "weak", "vs_baseline": None, "dtype": "int8", "data": "synthetic",
@@ -410,19 +679,23 @@ def run_cuda(args):
                            "l2": "inputs+outputs per step (715 MB) exceed L2; no flush needed"},
                 "clocks": clocks,
                 "e2e": {"value": whole_job_tops(ops_step, world, e2e_ms), "unit": "TOPS",
-                        "ms_per_step": e2e_ms, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
+                        "ms_per_step": e2e_ms, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": e2e_steps},
                 "gpu_launches": 5 * args.steps,
+                "profiled_pass": {"steps": prof_steps, "ms_per_step": profiled_ms_per_step,
+                                  "note": "per-kernel times come from this separate pass: every step has an event pair around one of its five launches"},
                 "roofline": roofline, "roofline_tensor": roofline_tensor, "kernels": per_kernel}
+        if extras:
+            line["configs"] = extras
         if pack_info:
             line["roofline_pack"] = {"kernel": "pack_kernel<2,4,8> on the 24-layer sweep", "bound": "hbm",
                                      "achieved": pack_info["gbs"], "peak": pk["hbm_gbs"], "unit": "GB/s",
                                      "frac": pack_info["gbs"] / pk["hbm_gbs"],
-                                     "frac_of_nominal_8000": pack_info["gbs"] / NOMINAL_HBM_GBS, "traffic": 2549617536,
+                                     "frac_of_nominal_8000": pack_info["gbs"] / NOMINAL_HBM_GBS, "traffic": traffic.get("pack_sweep"),
                                      "algorithmic_bytes": pack_info["bytes"]}
             adm = pack_info["admm_step_2:4/8b"]
             line["roofline_admm"] = {"kernel": "pack_kernel<2,4,8,dense outputs> (ADMM step: Z and U_next) on the 24-layer sweep",
                                      "bound": "hbm", "achieved": adm["gbs"], "peak": pk["hbm_gbs"], "unit": "GB/s",
-                                     "frac": adm["gbs"] / pk["hbm_gbs"], "traffic": 4771902805,
+                                     "frac": adm["gbs"] / pk["hbm_gbs"], "traffic": traffic.get("admm_sweep"),
                                      "algorithmic_bytes": adm["bytes"]}
         line["cpu_baseline"] = cpu_baseline() if (world == 1 and not args.skip_cpu) else None
         print(json.dumps(line))
@@ -636,7 +909,7 @@ def tma_probe(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=2000)
+    ap.add_argument("--steps", type=int, default=1000)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
     ap.add_argument("--bits", type=int, default=8, choices=[8, 4], help="weight code width of the 2:4 weights (default 8)")
@@ -645,6 +918,7 @@ def main():
     ap.add_argument("--tokens", type=int, default=TOKENS, help="tokens per GEMM (default: the full workload)")
     ap.add_argument("--skip-cpu", action="store_true", help="leave the CPU-oracle baseline out")
     ap.add_argument("--skip-sweep", action="store_true", help="leave the 24-layer pack sweep out")
+    ap.add_argument("--skip-configs", action="store_true", help="leave the timed entries of the other workload configurations out")
     ap.add_argument("--dist-case", type=int, default=0, choices=[0, 4, 8],
                     help="run only a small ADMM-Dist case with this code width (for profiler captures) and exit")
     ap.add_argument("--probe-tma", action="store_true",

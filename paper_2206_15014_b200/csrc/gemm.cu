@@ -994,6 +994,23 @@ static DebugOptions g_opt = {0, 0, 0, 0, 0, 0, 0, 0};
 // Trace buffer of NM_TRACE builds (device, kTraceStages + kTraceTiles rows of 8 u64), handed to every GEMM launch.
 static unsigned long long* g_trace_buffer = nullptr;
 
+// cudaFuncSetAttribute(max dynamic shared memory) once per kernel and device instead of on every launch.
+static cudaError_t allow_dynamic_smem(const void* fn, int bytes) {
+    struct Done { const void* fn; int dev; };
+    static Done done[64];
+    static int n_done = 0;
+    static std::mutex mu;
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    std::lock_guard<std::mutex> lock(mu);
+    for (int i = 0; i < n_done; ++i)
+        if (done[i].fn == fn && done[i].dev == dev) return cudaSuccess;
+    e = cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+    if (e == cudaSuccess && n_done < 64) done[n_done++] = Done{fn, dev};
+    return e;
+}
+
 struct LinearArgs {
     const int8_t* X; int tokens; const nm_packed_t* W;
     float sx; const float* sx_dev; const float* sw; const float* bias;
@@ -1047,7 +1064,7 @@ static int launch_gemm(const LinearArgs& a) {
     p.sw = a.sw; p.bias = a.bias; p.sx_dev = a.sx_dev; p.sx_host = a.sx;
     p.Y = a.Y; p.ACC = a.ACC; p.NARROW = a.NARROW; p.sy = a.sy; p.absmax = a.absmax; p.status = a.status; p.trace = g_trace_buffer; p.skip_stage = g_opt.skip_stage - 1;
     auto fn = nm_gemm_kernel<SPARSE, BN, EPI, WSRC>;
-    NM_CUDA_TRY(cudaFuncSetAttribute((const void*)fn, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::SMEM));
+    NM_CUDA_TRY(allow_dynamic_smem((const void*)fn, Cfg::SMEM));
     const int grid = p.n_tiles < sm_count() ? p.n_tiles : sm_count();
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(grid, 1, 1);
@@ -1106,7 +1123,7 @@ static int launch_gemm_pair(const LinearArgs& a) {
     p.sw = a.sw; p.bias = a.bias; p.sx_dev = a.sx_dev; p.sx_host = a.sx;
     p.Y = a.Y; p.ACC = a.ACC; p.NARROW = a.NARROW; p.sy = a.sy; p.absmax = a.absmax; p.status = a.status; p.trace = g_trace_buffer; p.skip_stage = g_opt.skip_stage - 1;
     auto fn = nm_gemm_pair_kernel<SPARSE, BN, EPI, RES>;
-    NM_CUDA_TRY(cudaFuncSetAttribute((const void*)fn, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::SMEM));
+    NM_CUDA_TRY(allow_dynamic_smem((const void*)fn, Cfg::SMEM));
     int pairs = p.n_tiles < sm_count() / 2 ? p.n_tiles : sm_count() / 2;
     if (pairs > kMaxPairs) pairs = kMaxPairs;
     // Contiguous tile ranges of about equal cost: a tile costs 1, entering a new output tile inside a range
@@ -1157,7 +1174,7 @@ static int launch_gemm_wide(const LinearArgs& a) {
     p.sw = a.sw; p.bias = a.bias; p.sx_dev = a.sx_dev; p.sx_host = a.sx;
     p.Y = a.Y; p.ACC = a.ACC; p.NARROW = a.NARROW; p.sy = a.sy; p.absmax = a.absmax; p.status = a.status; p.trace = g_trace_buffer; p.skip_stage = g_opt.skip_stage - 1;
     auto fn = nm_gemm_wide_kernel<BN, EPI, SKEW>;
-    NM_CUDA_TRY(cudaFuncSetAttribute((const void*)fn, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::SMEM));
+    NM_CUDA_TRY(allow_dynamic_smem((const void*)fn, Cfg::SMEM));
     int pairs = p.n_tiles < sm_count() / 2 ? p.n_tiles : sm_count() / 2;
     if (pairs > kMaxPairs) pairs = kMaxPairs;
     PairSchedule sched;
