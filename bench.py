@@ -900,9 +900,67 @@ def tma_probe(args):
                      producers=producers)
     case("ffn2 pair tile 512x224, stage held 448 clk", OUT, K, T, 256, 64, 112, 1, 6, delay=448, producers=2)
     case("ffn2 pair tile 512x224, 4 stages", OUT, K, T, 256, 64, 112, 1, 4, producers=2)
+    # stores alone (the producer arms its stages without loading anything): [16 tokens][32 channels] boxes as in the GEMMs,
+    # then 8 KB boxes 32, 64 and 128 channels wide
+    for stores in (1, 32, 64, 128):
+        case("stores only, 512x256 tiles", OUT, K, T, 256, 64, 128, 1, 5, loads=0, stores=stores)
     # everything resident in L2: a small problem walked five times
     case("L2-resident 256x192", OUT, K, 19 * 192, 128, 128, 96, 2, 5, repeat=5, stores=0, producers=2)
     case("L2-resident 512x224", OUT, K, 37 * 224, 256, 64, 112, 1, 6, repeat=5, stores=0, producers=2)
+    return 0
+
+
+def trace_gemm(args):
+    """Role-by-role time stamps of one GEMM launch from the library built with -DNM_TRACE (build.py --variant trace;
+    run as NMSPARSE_LIB=paper_2206_15014_b200/libnmsparse_trace.so python bench.py --trace-gemm TOKENS,K,OUT).  CTA 0
+    stamps clock64() per pipeline stage (producer got the stage / issued its loads, gate saw it full, MMA thread was
+    handed it / had issued its MMAs) and per tile (accumulators full, epilogue done).  Prints one JSON line of medians
+    and the per-tile rows; the launch itself is the product's kernel with the stamps added."""
+    import torch
+    import paper_2206_15014_b200 as nm
+    dev = torch.device("cuda:0")
+    T, K, OUT = (int(x) for x in args.trace_gemm.split(","))
+    for kv in args.option:
+        k, v = kv.split("=")
+        nm.nm_debug_set_option(k, int(v))
+    X = torch.randint(-127, 127, (T, K), dtype=torch.int8, device=dev)
+    vals = torch.randint(-127, 127, (OUT, K // 2), dtype=torch.int8, device=dev)
+    meta = torch.full((OUT, K // 32), 0x4E4E4E4E, dtype=torch.int32, device=dev)   # valid 2:4 positions (2,3) and (0,1)
+    sw, b = torch.ones(OUT, device=dev), torch.zeros(OUT, device=dev)
+    Y = torch.empty((T, OUT), device=dev)
+    status = torch.zeros(1, dtype=torch.int32, device=dev)
+    desc = nm.make_packed(OUT, K, 2, 4, 8, vals, meta)
+    trace = torch.zeros((576, 8), dtype=torch.int64, device=dev)
+    for _ in range(3):
+        nm.nm_int_linear(X, T, desc, 0.01, sw, b, Y, status=status)
+    nm.nm_debug_set_trace(trace)
+    nm.nm_int_linear(X, T, desc, 0.01, sw, b, Y, status=status)
+    torch.cuda.synchronize()
+    nm.nm_debug_set_trace(None)
+    rc = nm.nm_poll_status(status)
+    tr = trace.cpu().numpy()
+    st = tr[:512]
+    n = int((st[:, 3] > 0).sum())
+    if n == 0:
+        print(json.dumps({"error": "no time stamps: this shape runs on a kernel without them (only the CTA-pair kernels have them)"}))
+        return 1
+    st = st[:n]
+    t0 = st[0, 0]
+    d = (st[:, :5] - t0).astype(np.float64)
+    ok = st[:, 0] > 0     # the last steps of the wide kernel have no load of their own
+    med = lambda x: float(np.median(x))
+    tl = tr[512:]
+    tiles = []
+    for i in range(int((tl[:, 0] > 0).sum())):
+        row = {"tile": i, "accumulator_full": int(tl[i, 0] - t0), "epilogue_done": int(tl[i, 1] - t0)}
+        if tl[i, 2] > 0:
+            row.update(second_accumulator_full=int(tl[i, 2] - t0), second_epilogue_done=int(tl[i, 3] - t0))
+        tiles.append(row)
+    print(json.dumps({"shape": [T, K, OUT], "status": rc, "stages_of_cta0": n,
+                      "producer_issue_clk": med((d[:, 1] - d[:, 0])[ok]), "load_issue_to_full_clk": med((d[:, 2] - d[:, 1])[ok]),
+                      "gate_to_mma_handoff_clk": med((d[:, 3] - d[:, 2])[ok]), "mma_issue_clk": med(d[:, 4] - d[:, 3]),
+                      "clk_per_stage_steady": med(np.diff(d[:, 3])), "first_stage_full_clk": float(d[0, 2]),
+                      "last_mma_issued_clk": float(d[-1, 4]), "tiles": tiles}))
     return 0
 
 
@@ -923,7 +981,13 @@ def main():
                     help="run only a small ADMM-Dist case with this code width (for profiler captures) and exit")
     ap.add_argument("--probe-tma", action="store_true",
                     help="run only the TMA traffic probe of the pair GEMM's tile shapes (no arithmetic) and exit")
+    ap.add_argument("--trace-gemm", default="", metavar="TOKENS,K,OUT",
+                    help="time stamps of one 2:4 int8 GEMM launch (needs the NM_TRACE build of the library, see trace_gemm)")
+    ap.add_argument("--option", action="append", default=[], metavar="NAME=VALUE",
+                    help="kernel-choice override for --trace-gemm (nm_debug_set_option), e.g. no_wide=1")
     args = ap.parse_args()
+    if args.trace_gemm:
+        return trace_gemm(args)
     if args.probe_tma:
         return tma_probe(args)
     if args.dist_case:

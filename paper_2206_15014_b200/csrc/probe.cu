@@ -28,7 +28,8 @@ struct ProbeParams {
 
 constexpr int kProbeStoreWarps = 8;
 constexpr int kProbeThreads = 32 * (3 + kProbeStoreWarps);  // producer, consumer, store warps, second producer
-constexpr int kProbeStaging = kProbeStoreWarps * 8192;  // one store box per store warp ([16 tokens][32 channels] fp32 in the GEMMs; up to 8 KB here)
+// one store box per store warp: [16 tokens][32 channels] fp32 (2 KB) as in the GEMMs, or the 8 KB boxes of the wider shapes
+__host__ __device__ inline int probe_staging(int store_cols, int store_rows) { return kProbeStoreWarps * store_cols * store_rows * 4; }
 constexpr int kProbeTail = 1024;
 constexpr int kProbeSmemLimit = 232448;
 constexpr int kProbeMaxStages = 16;
@@ -51,7 +52,7 @@ tma_probe_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_consta
     const uint32_t a_bytes = (uint32_t)p.a_rows * p.a_row_bytes, b_bytes = (uint32_t)p.b_rows * 128u * p.b_slices;
     const uint32_t stage_bytes = a_bytes + b_bytes;
     uint8_t* staging = smem + (size_t)S * stage_bytes;
-    uint64_t* bars = reinterpret_cast<uint64_t*>(staging + kProbeStaging);
+    uint64_t* bars = reinterpret_cast<uint64_t*>(staging + probe_staging(p.store_cols, p.store_rows));
     const uint32_t bar0 = ptx::smem_u32(bars);
     auto full_bar = [&](int s) { return bar0 + 8u * s; };
     auto empty_bar = [&](int s) { return bar0 + 8u * (S + s); };
@@ -153,7 +154,7 @@ tma_probe_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_consta
     } else {
         // ------------------------------ store warps: the epilogue's TMA stores -------------------
         const int sw = warp - 2;
-        float* my_stage = reinterpret_cast<float*>(staging + sw * 8192);
+        float* my_stage = reinterpret_cast<float*>(staging + sw * (p.store_cols * p.store_rows * 4));
         const int boxes_c = p.a_rows / p.store_cols, boxes_t = (2 * p.b_rows) / p.store_rows, boxes = boxes_c * boxes_t;
         const int box_words = p.store_cols * p.store_rows;
         for (int i = 0; i < total; ++i) {
@@ -219,8 +220,6 @@ extern "C" int nm_probe_tma_stream(const void* W, int w_rows, int w_row_bytes, c
     if (poll < 0 || poll > 2 || (poll == 2 && stores) || producers < 1 || producers > 2 || stages < 2 || stages > kProbeMaxStages || repeat < 1 || delay_clocks < 0 || delay_clocks > (1 << 20)) return NM_ERR_SHAPE;
     const int stage_bytes = a_rows * a_row_bytes + b_rows * 128 * b_slices;
     if (stage_bytes % 1024) return NM_ERR_SHAPE;
-    const int smem = stages * stage_bytes + kProbeStaging + kProbeTail + 1024;
-    if (smem > kProbeSmemLimit) return NM_ERR_UNSUPPORTED;
     CUtensorMap tw, tx, ty;
     int rc = make_map(&tw, W, (uint64_t)w_rows, (uint64_t)w_row_bytes, (uint32_t)a_rows, (uint32_t)a_row_bytes,
                       a_row_bytes == 128 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_64B);
@@ -232,6 +231,8 @@ extern "C" int nm_probe_tma_stream(const void* W, int w_rows, int w_row_bytes, c
     const int store_cols = stores <= 1 ? 32 : stores, store_rows = stores <= 1 ? 16 : 8192 / (4 * store_cols);
     if (store_cols != 32 && store_cols != 64 && store_cols != 128) return NM_ERR_SHAPE;
     if (a_rows % store_cols || (2 * b_rows) % store_rows) return NM_ERR_SHAPE;
+    const int smem = stages * stage_bytes + probe_staging(store_cols, store_rows) + kProbeTail + 1024;
+    if (smem > kProbeSmemLimit) return NM_ERR_UNSUPPORTED;
     rc = make_map(&ty, Y, (uint64_t)tokens, (uint64_t)w_rows, (uint32_t)store_rows, (uint32_t)store_cols, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4);
     if (rc != NM_OK) return rc;
     ProbeParams p{};
