@@ -1022,7 +1022,7 @@ struct LinearArgs {
 // through TMA when the output can be described by a tensor map (16-byte aligned base and row pitch);
 // otherwise *tma_store is cleared, the threads store directly and the map describes X as a stand-in.
 template <int EPI>
-static int make_store_map(CUtensorMap* ty, const LinearArgs& a, bool* tma_store) {
+static int make_store_map(CUtensorMap* ty, const LinearArgs& a, bool* tma_store, uint32_t box_rows = 16) {
     const nm_packed_t& W = *a.W;
     constexpr uint32_t es = (uint32_t)sizeof(typename EpiOut<EPI>::type);
     void* ybase = EPI == EPI_F32 ? (void*)a.Y : EPI == EPI_ACC ? (void*)a.ACC : a.NARROW;
@@ -1031,7 +1031,7 @@ static int make_store_map(CUtensorMap* ty, const LinearArgs& a, bool* tma_store)
                                  : EPI == EPI_Q8 ? CU_TENSOR_MAP_DATA_TYPE_UINT8 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16;
     if (!*tma_store)
         return make_map(ty, a.X, (uint64_t)a.tokens, (uint64_t)W.in / 4, 16, 32, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_DATA_TYPE_INT32, 4);
-    return make_map(ty, ybase, (uint64_t)a.tokens, (uint64_t)W.out, 16, kNarrow<EPI> ? 128 : 32, CU_TENSOR_MAP_SWIZZLE_NONE, dt, es);
+    return make_map(ty, ybase, (uint64_t)a.tokens, (uint64_t)W.out, kNarrow<EPI> ? 16 : box_rows, kNarrow<EPI> ? 128 : 32, CU_TENSOR_MAP_SWIZZLE_NONE, dt, es);
 }
 
 template <bool SPARSE, int BN, int EPI, int WSRC>
@@ -1161,7 +1161,7 @@ static int launch_gemm_wide(const LinearArgs& a) {
     rc = make_map(&tx, a.X, (uint64_t)a.tokens, (uint64_t)W.in, Cfg::B_ROWS, 128, CU_TENSOR_MAP_SWIZZLE_128B);
     if (rc != NM_OK) return rc;
     bool tma_store = false;
-    rc = make_store_map<EPI>(&ty, a, &tma_store);
+    rc = make_store_map<EPI>(&ty, a, &tma_store, 32);
     if (rc != NM_OK) return rc;
     GemmParams p{};
     p.tma_store = tma_store ? 1 : 0;

@@ -39,7 +39,11 @@ struct WideCfg {
     static constexpr int B_ROWS = BN / 2;                // tokens staged by each CTA
     static constexpr int B_BYTES = B_ROWS * 128;
     static constexpr int STAGE = A_BYTES + B_BYTES;
-    static constexpr int STORE_STAGE = kWideEpiWarps * 2 * 2048;  // two [16 tokens][32 channels] fp32 tiles per epilogue warp
+    // One [32 tokens][32 channels] 32-bit staging tile per epilogue warp: a whole accumulator chunk leaves with one TMA
+    // store.  The SM's TMA unit takes about 40 clocks per store plus 2.5 per 128-byte row (measured: 112 stores of 16
+    // rows per tile 9.3 k clocks, 56 of 32 rows 6.9 k, with 8 or 16 warps alike), and here the epilogue is exposed, so
+    // fewer, taller boxes pay; a second tile per warp would cost a ring stage, which costs more (measured).
+    static constexpr int STORE_STAGE = kWideEpiWarps * 4096;
     static constexpr int FIT = (kSmemLimit - kSmemTail - STORE_STAGE - 1024) / STAGE;
     static constexpr int STAGES = FIT < 8 ? FIT : 8;
     static constexpr int SMEM = STAGES * STAGE + STORE_STAGE + kSmemTail + 1024;
@@ -301,12 +305,11 @@ nm_gemm_wide_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_con
         constexpr int CH = BN / 32;
         const int ew = warp - 2, q = warp & 3, blk = ew >> 2;
         const uint32_t acc_taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)blk * BN;
-        float* my_stage = reinterpret_cast<float*>(store_stage + ew * 4096);
+        uint32_t* my_stage = reinterpret_cast<uint32_t*>(store_stage + ew * 4096);
         const float sx = p.sx_dev ? *p.sx_dev : p.sx_host;
         const uint32_t lead_acc_empty = ptx::map_to_cta(acc_empty_bar(blk), 0);
         float amax = 0.0f, c_n = 0.0f, b_n = 0.0f;
         int scaled_out_tile = -1;
-        uint32_t n_stores = 0;
         bool ok = true;
         auto release_acc = [&]() {  // this warp has read all it needs from the accumulator
             ptx::tc_fence_before();
@@ -348,21 +351,16 @@ nm_gemm_wide_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_con
                         return o;
                     };
                     if (p.tma_store) {  // separate branch-free loops for the two store paths
+                        // rows of the tile past the last token are clipped by the store
+                        if (lane == 0) ptx::bulk_wait_group_read<0>();  // the store before this one has read the tile
+                        __syncwarp();
 #pragma unroll
-                        for (int h = 0; h < 2; ++h) {  // 16 tokens per store, alternating staging tiles
-                            if (tc0 + 16 * h >= p.tokens) continue;  // warp-uniform
-                            uint32_t* sb = reinterpret_cast<uint32_t*>(my_stage + (n_stores & 1u) * 512);
-                            if (lane == 0) ptx::bulk_wait_group_read<1>();  // the store before the last has read this tile
-                            __syncwarp();
-#pragma unroll
-                            for (int j = 0; j < 16; ++j) sb[j * 32 + lane] = conv(16 * h + j);
-                            ptx::fence_proxy_async_smem();
-                            __syncwarp();
-                            if (lane == 0) {
-                                ptx::tma_store_2d(&tmap_y, nw, tc0 + 16 * h, ptx::smem_u32(sb));
-                                ptx::bulk_commit_group();
-                            }
-                            ++n_stores;
+                        for (int j = 0; j < 32; ++j) my_stage[j * 32 + lane] = conv(j);
+                        ptx::fence_proxy_async_smem();
+                        __syncwarp();
+                        if (lane == 0) {
+                            ptx::tma_store_2d(&tmap_y, nw, tc0, ptx::smem_u32(my_stage));
+                            ptx::bulk_commit_group();
                         }
                     } else {
                         uint32_t* dst = reinterpret_cast<uint32_t*>(EPI == EPI_F32 ? (void*)p.Y : (void*)p.ACC) + (size_t)tc0 * p.out + n;

