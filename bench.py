@@ -924,12 +924,12 @@ def trace_gemm(args):
         k, v = kv.split("=")
         nm.nm_debug_set_option(k, int(v))
     X = torch.randint(-127, 127, (T, K), dtype=torch.int8, device=dev)
-    vals = torch.randint(-127, 127, (OUT, K // 2), dtype=torch.int8, device=dev)
+    vals = torch.randint(-127, 127, (OUT, K // 2 * args.bits // 8), dtype=torch.int8, device=dev)   # 8-bit or packed 4-bit codes
     meta = torch.full((OUT, K // 32), 0x4E4E4E4E, dtype=torch.int32, device=dev)   # valid 2:4 positions (2,3) and (0,1)
     sw, b = torch.ones(OUT, device=dev), torch.zeros(OUT, device=dev)
     Y = torch.empty((T, OUT), device=dev)
     status = torch.zeros(1, dtype=torch.int32, device=dev)
-    desc = nm.make_packed(OUT, K, 2, 4, 8, vals, meta)
+    desc = nm.make_packed(OUT, K, 2, 4, args.bits, vals, meta)
     trace = torch.zeros((576, 8), dtype=torch.int64, device=dev)
     for _ in range(3):
         nm.nm_int_linear(X, T, desc, 0.01, sw, b, Y, status=status)

@@ -1150,13 +1150,15 @@ static int launch_gemm_pair(const LinearArgs& a) {
 }
 
 // Wide pair kernel (512 channels x BN tokens per pair): 2:4 int8 weights streamed, fp32 / int32 outputs.
-template <int BN, int EPI>
+template <int BN, int EPI, bool W4 = false>
 static int launch_gemm_wide(const LinearArgs& a) {
     using Cfg = WideCfg<BN>;
     constexpr int SKEW = 0;
     const nm_packed_t& W = *a.W;
     CUtensorMap tw, tx, ty;
-    int rc = make_map(&tw, W.values, (uint64_t)W.out, (uint64_t)W.in / 2, Cfg::A_ROWS, Cfg::A_ROW, CU_TENSOR_MAP_SWIZZLE_64B);
+    // packed 4-bit codes are read by the builder warps, not by TMA: the weight map then describes X as a stand-in
+    int rc = W4 ? make_map(&tw, a.X, (uint64_t)a.tokens, (uint64_t)W.in, Cfg::B_ROWS, 128, CU_TENSOR_MAP_SWIZZLE_128B)
+                : make_map(&tw, W.values, (uint64_t)W.out, (uint64_t)W.in / 2, Cfg::A_ROWS, Cfg::A_ROW, CU_TENSOR_MAP_SWIZZLE_64B);
     if (rc != NM_OK) return rc;
     rc = make_map(&tx, a.X, (uint64_t)a.tokens, (uint64_t)W.in, Cfg::B_ROWS, 128, CU_TENSOR_MAP_SWIZZLE_128B);
     if (rc != NM_OK) return rc;
@@ -1171,9 +1173,10 @@ static int launch_gemm_wide(const LinearArgs& a) {
     p.n_tiles = p.n_tok_tiles * p.n_out_tiles;
     p.kblocks = W.in / Cfg::KB;
     p.meta = (const uint32_t*)W.meta; p.mrow_words = W.in / 32;
+    p.values = (const uint8_t*)W.values; p.vrow_bytes = (int)values_row_bytes(W.in, W.n, W.m, W.bits);
     p.sw = a.sw; p.bias = a.bias; p.sx_dev = a.sx_dev; p.sx_host = a.sx;
     p.Y = a.Y; p.ACC = a.ACC; p.NARROW = a.NARROW; p.sy = a.sy; p.absmax = a.absmax; p.status = a.status; p.trace = g_trace_buffer; p.skip_stage = g_opt.skip_stage - 1;
-    auto fn = nm_gemm_wide_kernel<BN, EPI, SKEW>;
+    auto fn = nm_gemm_wide_kernel<BN, EPI, SKEW, W4>;
     NM_CUDA_TRY(allow_dynamic_smem((const void*)fn, Cfg::SMEM));
     int pairs = p.n_tiles < sm_count() / 2 ? p.n_tiles : sm_count() / 2;
     if (pairs > kMaxPairs) pairs = kMaxPairs;
@@ -1181,7 +1184,7 @@ static int launch_gemm_wide(const LinearArgs& a) {
     p.band = cached_pair_plan(p.n_tok_tiles, p.n_out_tiles, pairs, false, 0, sched);
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(2 * pairs, 1, 1);
-    cfg.blockDim = dim3(kWideThreads, 1, 1);
+    cfg.blockDim = dim3(kWideThreadsOf<W4>, 1, 1);
     cfg.dynamicSmemBytes = Cfg::SMEM;
     cfg.stream = a.stream;
     cudaLaunchAttribute attr[2];
@@ -1269,14 +1272,14 @@ static int check_linear(int tokens, int out, int in, int n, int m, int bits) {
 
 template <int EPI>
 static int run_linear_epi(const LinearArgs& a, bool xform, bool sparse) {
-    if (xform) return sparse ? pick_bn<true, EPI, true>(a) : pick_bn<false, EPI, true>(a);
     if constexpr (EPI == EPI_F32 || EPI == EPI_ACC) {
-        if (sparse) {
+        if (sparse && (!xform || xf::pattern_of(a.W->n, a.W->m, a.W->bits) == xf::P24_4)) {  // 2:4 with 8-bit or packed 4-bit codes
             const int bn = wide_bn<EPI>(a);
-            if (bn == 224) return launch_gemm_wide<224, EPI>(a);
-            if (bn == 192) return launch_gemm_wide<192, EPI>(a);
+            if (bn == 224) return xform ? launch_gemm_wide<224, EPI, true>(a) : launch_gemm_wide<224, EPI>(a);
+            if (bn == 192) return xform ? launch_gemm_wide<192, EPI, true>(a) : launch_gemm_wide<192, EPI>(a);
         }
     }
+    if (xform) return sparse ? pick_bn<true, EPI, true>(a) : pick_bn<false, EPI, true>(a);
     if (sparse) return use_pair<true, EPI>(a) ? pick_pair<true, EPI>(a) : pick_bn<true, EPI, false>(a);
     return use_pair<false, EPI>(a) ? pick_pair<false, EPI>(a) : pick_bn<false, EPI, false>(a);
 }

@@ -26,6 +26,14 @@ constexpr int kWideEpiWarps = 8;     // four per accumulator, one per TMEM lane 
 constexpr int kWideGateWarp = 2 + kWideEpiWarps;
 constexpr int kWideMetaWarp0 = kWideGateWarp + 1;
 constexpr int kWideThreads = 32 * (kWideMetaWarp0 + 4);  // producer, MMA, epilogue warps, gate, metadata warps
+// W4 (2:4 weights stored as packed 4-bit codes): the weight tile of a stage is not copied by TMA but built in shared
+// memory by eight more warps, one thread per weight row of the CTA: 32 bytes of nibbles per row and stage (fetched one
+// stage ahead) widened to the 64 int8 slot bytes and written in the tile's swizzle; the stage's "full" barrier counts
+// those warps too.  The 2:4 index metadata is the same as for 8-bit codes.  (Measured: a stage then takes ~980 clocks
+// instead of 582, with eight or with sixteen builder warps alike: the generic-proxy stores and fences compete for the
+// shared-memory bandwidth the MMAs and TMA already use up.)
+constexpr int kWideBuildWarps = 8;
+template <bool W4> constexpr int kWideThreadsOf = kWideThreads + (W4 ? 32 * kWideBuildWarps : 0);
 constexpr uint32_t kWideRelayIds = 12;  // named barriers 1..12 carry the gate's relays in turn; the gate is never more
                                         // than STAGES + SKEW steps ahead of the MMA thread
 
@@ -55,8 +63,8 @@ struct WideCfg {
     static_assert(BN % 32 == 0 && BN <= 256, "token tile");
 };
 
-template <int BN, int EPI, int SKEW>
-__global__ void __launch_bounds__(kWideThreads, 1)
+template <int BN, int EPI, int SKEW, bool W4>
+__global__ void __launch_bounds__(kWideThreadsOf<W4>, 1)
 nm_gemm_wide_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant__ CUtensorMap tmap_x,
                     const __grid_constant__ CUtensorMap tmap_y, const GemmParams p,
                     const __grid_constant__ PairSchedule sched) {
@@ -88,7 +96,7 @@ nm_gemm_wide_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_con
     const uint32_t total = (uint32_t)tile_count * (uint32_t)p.kblocks;  // pipeline stages this pair runs
 
     if (threadIdx.x == 0) {
-        for (int s = 0; s < S; ++s) { ptx::mbar_init(full_bar(s), 1 + 8); ptx::mbar_init(empty_bar(s), 1); }
+        for (int s = 0; s < S; ++s) { ptx::mbar_init(full_bar(s), 1 + 8 + (W4 ? 2 * kWideBuildWarps : 0)); ptx::mbar_init(empty_bar(s), 1); }
         for (int b = 0; b < 2; ++b) { ptx::mbar_init(acc_full_bar(b), 1); ptx::mbar_init(acc_empty_bar(b), 8); }
         ptx::mbar_init(drained_bar, 1);
         *abort_flag = 0;
@@ -139,8 +147,8 @@ nm_gemm_wide_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_con
                     NM_TRACE_STAGE(it, 0);
                     if (NM_SKIP_STAGE(it)) { if (++s == S) { s = 0; parity ^= 1u; } continue; }
                     const uint32_t dst = smem0 + (uint32_t)s * Cfg::STAGE, lead_full = lead_full0 + 8u * s;
-                    if (leader) ptx::mbar_expect_tx(full_bar(s), 2 * Cfg::STAGE);  // bytes of both CTAs
-                    ptx::tma_load_2d_pair(dst, &tmap_w, kb * Cfg::A_ROW, n0, lead_full);
+                    if (leader) ptx::mbar_expect_tx(full_bar(s), 2 * (W4 ? Cfg::B_BYTES : Cfg::STAGE));  // bytes of both CTAs
+                    if (!W4) ptx::tma_load_2d_pair(dst, &tmap_w, kb * Cfg::A_ROW, n0, lead_full);
                     ptx::tma_load_2d_pair(dst + Cfg::A_BYTES, &tmap_x, kb * 128, t0, lead_full);
                     NM_TRACE_STAGE(it, 1);
                     if (++s == S) { s = 0; parity ^= 1u; }
@@ -150,6 +158,49 @@ nm_gemm_wide_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_con
             // waiting for data, so the stages' barriers no longer say whether this producer's last copies have landed:
             // give them time before the CTA and its shared memory go away.
             if (!ok || *abort_flag) ptx::wait_clocks(kAbortDrain);
+        }
+    } else if (W4 && warp >= kWideMetaWarp0 + 4) {
+        // ------------------------------ weight-tile builders (W4, both CTAs) ---------------------
+        // Thread = one of the CTA's 256 weight rows (block = row / 128).  Per stage: the row's 32 bytes of packed
+        // nibbles (128 reduction elements at 2:4 = 64 codes), fetched one stage ahead, become the 64 slot bytes.
+        const int r256 = (warp - (kWideMetaWarp0 + 4)) * 32 + lane;
+        uint8_t* const my_rows = smem + (r256 >> 7) * Cfg::A_BLOCK;  // this thread's block within a stage
+        // the row's packed codes: pointer of the current tile, recomputed only when the tile changes (a single
+        // thread's integer divisions cost hundreds of clocks)
+        auto row_of_tile = [&](int i) -> const uint4* {
+            if (i >= tile_count) return nullptr;
+            const TileCoord tc = tile_coord(tile_begin + i, p.n_tok_tiles, p.n_out_tiles, p.band);
+            const int n = tc.o * (2 * Cfg::A_ROWS) + (int)rank * Cfg::A_ROWS + r256;
+            return n < p.out ? reinterpret_cast<const uint4*>(p.values + (size_t)n * p.vrow_bytes) : nullptr;  // rows past the end: zeros
+        };
+        auto fetch = [&](const uint4* row, int kb, uint4 (&raw)[2]) {
+            if (row) { raw[0] = __ldg(row + 2 * kb); raw[1] = __ldg(row + 2 * kb + 1); }
+            else raw[0] = raw[1] = make_uint4(0u, 0u, 0u, 0u);
+        };
+        int i = 0, kb = 0;
+        const uint4* row = row_of_tile(0);
+        uint4 cur[2], nxt[2];
+        fetch(row, 0, nxt);
+        uint32_t parity = 1u;
+        int s = 0;
+        while (i < tile_count) {
+            cur[0] = nxt[0]; cur[1] = nxt[1];
+            int ni = i, nkb = kb + 1;
+            const uint4* nrow = row;
+            if (nkb == p.kblocks) { nkb = 0; ++ni; nrow = row_of_tile(ni); }
+            fetch(nrow, nkb, nxt);  // the next stage's codes travel while this one is built
+            bool got = lane != 0 || ptx::mbar_wait_bounded(empty_bar(s), parity, abort_flag, kWaitLimit);
+            if (!__all_sync(0xffffffffu, got)) { if (lane == 0) raise_timeout(); break; }
+            uint32_t w[16];
+            const uint32_t cw[8] = {cur[0].x, cur[0].y, cur[0].z, cur[0].w, cur[1].x, cur[1].y, cur[1].z, cur[1].w};
+#pragma unroll
+            for (int j = 0; j < 8; ++j) xf::widen8(cw[j], w[2 * j], w[2 * j + 1]);
+            xf::store_row<true>(my_rows + (size_t)s * Cfg::STAGE, r256 & 127, w);
+            ptx::fence_proxy_async_smem();  // the MMA reads the tile through the async proxy
+            __syncwarp();
+            if (lane == 0) ptx::mbar_arrive_cluster(lead_full0 + 8u * s);
+            if (++s == S) { s = 0; parity ^= 1u; }
+            i = ni; kb = nkb; row = nrow;
         }
     } else if (warp >= kWideMetaWarp0) {
         // ------------------------------ metadata warps (both CTAs) -------------------------------
@@ -333,20 +384,22 @@ nm_gemm_wide_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_con
                 b_n = n_ok && p.bias ? p.bias[n] : 0.0f;
             }
             const int nact = min(CH, (p.tokens - t0 + 31) >> 5);  // chunks that hold tokens (warp-uniform)
-            uint32_t r[2][32];
-            if (nact > 0) ptx::tmem_ld_32x32(acc_taddr, r[0]);
-            else release_acc();
+            constexpr int RB = W4 ? 1 : 2;  // chunk read one ahead of its conversion, except where registers are short
+            uint32_t r[RB][32];
+            if (nact == 0) release_acc();
+            else if (RB == 2) ptx::tmem_ld_32x32(acc_taddr, r[0]);
 #pragma unroll
             for (int c = 0; c < CH; ++c) {
                 const int tc0 = t0 + c * 32;
                 if (c < nact) {
+                    if (RB == 1) ptx::tmem_ld_32x32(acc_taddr + c * 32, r[0]);
                     ptx::tmem_ld_wait();
-                    if (c + 1 < nact) ptx::tmem_ld_32x32(acc_taddr + (c + 1) * 32, r[(c + 1) & 1]);
-                    else release_acc();
+                    if (c + 1 >= nact) release_acc();
+                    else if (RB == 2) ptx::tmem_ld_32x32(acc_taddr + (c + 1) * 32, r[(c + 1) & (RB - 1)]);
                     const int jmax = n_ok ? min(32, p.tokens - tc0) : 0;  // outputs of this lane that exist
                     auto conv = [&](int j) -> uint32_t {
                         float y_abs;
-                        const uint32_t o = epi_convert<EPI>(r[c & 1][j], c_n, b_n, p.sy, 0.0f, y_abs);
+                        const uint32_t o = epi_convert<EPI>(r[c & (RB - 1)][j], c_n, b_n, p.sy, 0.0f, y_abs);
                         if constexpr (EPI == EPI_F32) amax = fmaxf(amax, j < jmax ? y_abs : 0.0f);
                         return o;
                     };

@@ -1,4 +1,5 @@
-"""GPU parity of the 512-channel CTA-pair kernel (2:4 int8 weights, reduction longer than 1024) against the CPU oracle.
+"""GPU parity of the 512-channel CTA-pair kernel (2:4 weights with 8-bit codes, or packed 4-bit codes widened in shared
+memory by its builder warps; reduction longer than 1024) against the CPU oracle.
 
 The library picks that kernel only for problems with at least one tile per SM pair; the option "wide_any"
 sends every eligible shape to it, so that small and ragged cases (one tile, a ragged last token tile, an output
@@ -25,17 +26,17 @@ def wide_kernel_everywhere(request):
     nm.nm_debug_set_option("wide_bn", 0)
 
 
-def _run(seed, T, K, out, tie=False, bias=True):
+def _run(seed, T, K, out, tie=False, bias=True, bits=8):
     from gpu_util import PackedOnDevice, gpu_int_linear, assert_close
     oracle.set_threads(oracle.max_threads())
     rng = np.random.default_rng(seed)
     W = wl.tie_heavy(seed, out, K) if tie else wl.normal(rng, (out, K), 0.02)
     b = wl.normal(rng, (out,), 0.02)
     Xq, sx = oracle.quantize_act(wl.normal(rng, (T, K)))
-    v, meta, s = oracle.project_pack(W, None, 2, 4, 8)
-    D = oracle.unpack(v, meta, out, K, 2, 4, 8)
+    v, meta, s = oracle.project_pack(W, None, 2, 4, bits)
+    D = oracle.unpack(v, meta, out, K, 2, 4, bits)
     acc_ref, Y_ref = oracle.int_linear(Xq, D, sx, s, b if bias else None)
-    packed = PackedOnDevice(v, meta, s, out, K, 2, 4, 8)
+    packed = PackedOnDevice(v, meta, s, out, K, 2, 4, bits)
     acc, Y = gpu_int_linear(Xq, packed, sx, b if bias else None)
     assert np.array_equal(acc, acc_ref), f"{(acc != acc_ref).sum()} accumulators differ"
     assert_close(Y, Y_ref)
@@ -50,18 +51,24 @@ def _run(seed, T, K, out, tie=False, bias=True):
     (448, 1536, 1024),     # four tiles
     (700, 8192, 520),      # longest supported reduction (64 stages per tile)
 ])
-def test_small_and_ragged(T, K, out):
-    _run(11 + T, T, K, out)
+@pytest.mark.parametrize("bits", [8, 4])
+def test_small_and_ragged(T, K, out, bits):
+    _run(11 + T, T, K, out, bits=bits)
 
 
-def test_no_bias_and_ties():
-    _run(21, 300, 1152, 640, tie=True, bias=False)
+@pytest.mark.parametrize("bits", [8, 4])
+def test_no_bias_and_ties(bits):
+    _run(21, 300, 1152, 640, tie=True, bias=False, bits=bits)
 
 
 def test_many_tiles_per_pair():
     # 5 output tiles x 34 token tiles = 170 tiles on 74 pairs: every pair walks two or three tiles, most change
     # output tile inside their range; the last token tile is ragged
     _run(22, 34 * 224 - 77, 1152, 2400)
+
+
+def test_many_tiles_per_pair_packed_4_bit():
+    _run(25, 34 * 224 - 77, 1152, 2400, bits=4)
 
 
 def test_library_choice_of_tile_width():
@@ -75,3 +82,4 @@ def test_library_choice_of_tile_width():
 def test_output_rows_not_16_byte_aligned():
     # out % 4 != 0: the epilogue stores directly instead of through TMA
     _run(24, 500, 1152, 515)
+    _run(26, 500, 1152, 515, bits=4)
