@@ -593,6 +593,8 @@ nm_gemm_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant
 // as a cluster before the first remote operation and before TMEM is released.
 // ---------------------------------------------------------------------------------------------
 constexpr int kPairThreads = 32 * (3 + kEpiWarps);
+constexpr int kPairBuildWarps = 8;  // two groups of four (one thread per weight row of the CTA) taking alternate 128-wide k-blocks
+template <bool BUILD> constexpr int kPairThreadsOf = kPairThreads + (BUILD ? 32 * kPairBuildWarps : 0);
 constexpr int kPairMaxStages = 7;   // the relay cycles through 8 named barriers (ids 1-8; 9-14 serve the narrow-output epilogue)
 
 constexpr int kPairResStages = 4;   // stages of weights a CTA can keep resident (1024 reduction elements at 2:4)
@@ -626,8 +628,12 @@ struct PairCfg {
     static_assert(BN % 32 == 0 && BN <= 256, "token tile");
 };
 
-template <bool SPARSE, int BN, int EPI, bool RES>
-__global__ void __launch_bounds__(kPairThreads, 1)
+// BUILD (with RES, sparse target): the weights are not stored in the tensor core's form (packed 4-bit codes, 1:4, 2:8,
+// 1:8).  Instead of a TMA copy, eight builder warps rebuild the CTA's 128 weight rows for the whole reduction in the resident
+// region once per output tile (xform.cuh: widening, placement into 2-of-4 slots), and the metadata warps derive the
+// hardware metadata from the canonical one; everything else is the resident-weight kernel.
+template <bool SPARSE, int BN, int EPI, bool RES, bool BUILD = false>
+__global__ void __launch_bounds__(kPairThreadsOf<BUILD>, 1)
 nm_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant__ CUtensorMap tmap_x,
                     const __grid_constant__ CUtensorMap tmap_y, const GemmParams p,
                     const __grid_constant__ PairSchedule sched) {
@@ -651,6 +657,8 @@ nm_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_con
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * S + 8);
     volatile uint32_t* abort_flag = tmem_slot + 1;
     volatile uint32_t* never_flag = tmem_slot + 2;
+    uint32_t* lut = reinterpret_cast<uint32_t*>(reinterpret_cast<uint8_t*>(bars) + 512);  // BUILD: slot tables (xform.cuh)
+    static_assert(!BUILD || (RES && SPARSE), "weights are rebuilt only in the resident-weight, sparse-target form");
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t rank = ptx::cluster_ctarank();
@@ -664,7 +672,7 @@ nm_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_con
         for (int b = 0; b < 2; ++b) { ptx::mbar_init(acc_full_bar(b), 1); ptx::mbar_init(acc_empty_bar(b), 2 * EW); }
         ptx::mbar_init(meta_bar, 8);
         ptx::mbar_init(drained_bar, 1);
-        ptx::mbar_init(a_full_bar, 1);
+        ptx::mbar_init(a_full_bar, BUILD ? 2 * kPairBuildWarps : 1);  // the builder warps of both CTAs, or the TMA bytes
         ptx::mbar_init(a_free_bar, 1);
         *abort_flag = 0;
         *never_flag = 0;
@@ -673,6 +681,7 @@ nm_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_con
         ptx::prefetch_tensormap(&tmap_x);
         if (p.tma_store) ptx::prefetch_tensormap(&tmap_y);
     }
+    if (BUILD) xf::build_lut(lut, threadIdx.x, blockDim.x);
     __syncthreads();
     ptx::cluster_arrive();   // both CTAs' barriers exist before anything remote touches them
     ptx::cluster_wait();
@@ -706,7 +715,7 @@ nm_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_con
                 const TileCoord tc = tile_coord(tile, p.n_tok_tiles, p.n_out_tiles, p.band);
                 const int n0 = tc.o * (2 * kBM) + (int)rank * kBM;
                 const int t0 = tc.t * BN + (int)rank * Cfg::B_ROWS;
-                if (RES && tc.o != prev_out_tile) {
+                if (RES && !BUILD && tc.o != prev_out_tile) {
                     // new output tile: once the MMAs of the previous one are done, fetch this CTA's weight rows for the whole reduction
                     prev_out_tile = tc.o;
                     if (!ptx::mbar_wait_bounded(a_free_bar, free_parity, abort_flag, kWaitLimit)) {
@@ -738,6 +747,42 @@ nm_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_con
             // waiting for data, so the stages' barriers no longer say whether this producer's last copies have landed:
             // give them time before the CTA and its shared memory go away.
             if (!ok || *abort_flag) ptx::wait_clocks(kAbortDrain);
+        }
+    } else if (BUILD && warp > kGateWarp) {
+        // ------------------------------ weight builders (both CTAs) ------------------------------
+        // One thread = one of the CTA's 128 weight rows; group g builds the 128-wide k-blocks g, g + 2, ... of the row
+        // into the resident region (two k-blocks per 128-byte row of a stage), once per output tile.
+        const int bw = warp - (kGateWarp + 1), grp = bw >> 2, tr = (bw & 3) * 32 + lane;
+        const int cb = xf::code_bytes(p.pat), mb = xf::meta_bytes(p.pat);
+        const uint8_t* meta8 = reinterpret_cast<const uint8_t*>(p.meta);
+        const int kb_real = p.in >> 7, kb_all = 2 * p.kblocks;  // k-blocks of the reduction / of the stages (a last half stage gets zeros)
+        const uint32_t lead_a_full = ptx::map_to_cta(a_full_bar, 0);
+        int prev_out_tile = -1;
+        uint32_t free_parity = 1u;  // nothing reads the region before the first build
+        for (int i = 0; i < tile_count; ++i) {
+            const int out_tile = tile_coord(tile_begin + i, p.n_tok_tiles, p.n_out_tiles, p.band).o;
+            if (out_tile == prev_out_tile) continue;
+            prev_out_tile = out_tile;
+            const int n = out_tile * (2 * kBM) + (int)rank * kBM + tr;
+            const bool row_ok = n < p.out;
+            const uint8_t* v = p.values + (size_t)(row_ok ? n : 0) * p.vrow_bytes;
+            const uint8_t* m = meta8 + (size_t)(row_ok ? n : 0) * p.mrow_bytes;
+            xf::Raw cur = xf::load_raw(p.pat, v + (size_t)grp * cb, m + (size_t)grp * mb, row_ok && grp < kb_real);
+            // the MMAs of the previous output tile have finished reading the region
+            bool got = lane != 0 || ptx::mbar_wait_bounded(a_free_bar, free_parity, abort_flag, kWaitLimit);
+            free_parity ^= 1u;
+            if (!__all_sync(0xffffffffu, got)) { if (lane == 0) raise_timeout(); break; }
+            for (int kb = grp; kb < kb_all; kb += 2) {
+                const int nkb = kb + 2;
+                xf::Raw nxt = xf::load_raw(p.pat, v + (size_t)nkb * cb, m + (size_t)nkb * mb, row_ok && nkb < kb_real);
+                uint32_t w[16];
+                xf::build_row<true>(p.pat, cur, lut, w);
+                xf::store_half_row128(a_res + (kb >> 1) * Cfg::A_BYTES, tr, kb & 1, w);
+                cur = nxt;
+            }
+            ptx::fence_proxy_async_smem();  // the MMA reads the tile through the async proxy
+            __syncwarp();
+            if (lane == 0) ptx::mbar_arrive_cluster(lead_a_full);
         }
     } else if (warp == kGateWarp) {
         // ------------------------------ gate (leader): mbarrier waits relayed to the MMA warp ------
@@ -834,7 +879,11 @@ nm_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_con
             // its remaining MMAs multiply zero-filled weights, but their index fields must still be valid 2:4
             // patterns: the columns past the row's metadata get "positions 0,1", as rows past `out` do.
             for (int c = 0; c < p.kblocks * (Cfg::KB / 32); c += 4) {
-                uint4 w = (n < p.out && c < p.mrow_words) ? __ldg(src + (c >> 2)) : make_uint4(0x44444444u, 0x44444444u, 0x44444444u, 0x44444444u);
+                uint4 w = make_uint4(0x44444444u, 0x44444444u, 0x44444444u, 0x44444444u);
+                if (n < p.out && c < p.mrow_words) {
+                    if constexpr (BUILD) w = xf::hw_meta(p.pat, reinterpret_cast<const uint8_t*>(p.meta) + (size_t)n * p.mrow_bytes + (size_t)(c >> 2) * xf::meta_bytes(p.pat), lut);
+                    else w = __ldg(src + (c >> 2));
+                }
                 ptx::tmem_st_32x4(lane_taddr + Cfg::META_COL + c, w.x, w.y, w.z, w.w);
             }
             ptx::tmem_st_wait();
@@ -872,21 +921,25 @@ nm_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_con
                 b_n = n_ok && p.bias ? p.bias[n] : 0.0f;
             }
             const int nact = min(CH, (p.tokens - t0 + 31) >> 5);
-            uint32_t r[2][32];
-            if (half < nact) ptx::tmem_ld_32x32(lane_taddr + buf * BN + half * 32, r[0]);
-            else release_acc(buf);
+            // chunks are read one ahead of their conversion; with the builder warps present registers are short and
+            // every chunk is read when it is due
+            constexpr int RB = BUILD ? 1 : 2;
+            uint32_t r[RB][32];
+            if (half >= nact) release_acc(buf);
+            else if (RB == 2) ptx::tmem_ld_32x32(lane_taddr + buf * BN + half * 32, r[0]);
 #pragma unroll
             for (int ci = 0; ci < CI; ++ci) {
                 const int c = half + ci * EWH, tc0 = t0 + c * 32;
                 if (c < nact) {
+                    if (RB == 1) ptx::tmem_ld_32x32(lane_taddr + buf * BN + c * 32, r[0]);
                     ptx::tmem_ld_wait();
-                    if (c + EWH < nact) ptx::tmem_ld_32x32(lane_taddr + buf * BN + (c + EWH) * 32, r[(ci + 1) & 1]);
-                    else release_acc(buf);
+                    if (c + EWH >= nact) release_acc(buf);
+                    else if (RB == 2) ptx::tmem_ld_32x32(lane_taddr + buf * BN + (c + EWH) * 32, r[(ci + 1) & (RB - 1)]);
                     const int jmax = n_ok ? min(32, p.tokens - tc0) : 0;  // outputs of this lane that exist
                     using OT = typename EpiOut<EPI>::type;
                     auto conv = [&](int j) -> OT {
                         float y_abs;
-                        const OT o = epi_convert<EPI>(r[ci & 1][j], c_n, b_n, p.sy, rsy, y_abs);
+                        const OT o = epi_convert<EPI>(r[ci & (RB - 1)][j], c_n, b_n, p.sy, rsy, y_abs);
                         if constexpr (EPI == EPI_F32) amax = fmaxf(amax, j < jmax ? y_abs : 0.0f);
                         return o;
                     };
@@ -903,7 +956,7 @@ nm_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_con
                                     int j_tie = 0, n_tie = 0;
 #pragma unroll
                                     for (int j = 0; j < 16; ++j)
-                                        sb[j * 128 + q * 32 + lane] = epi_convert_q8_fast(r[ci & 1][16 * h + j], c_n, b_n, rsy, j, y_tie, j_tie, n_tie);
+                                        sb[j * 128 + q * 32 + lane] = epi_convert_q8_fast(r[ci & (RB - 1)][16 * h + j], c_n, b_n, rsy, j, y_tie, j_tie, n_tie);
                                     if (__any_sync(0xffffffffu, n_tie != 0)) {  // rare (3 % of these tiles): repair with the exact division
                                         if (n_tie == 1) {
                                             sb[j_tie * 128 + q * 32 + lane] = (uint8_t)(int8_t)quantise8_exact(y_tie, p.sy);
@@ -1099,13 +1152,15 @@ static int cached_pair_plan(int n_tok_tiles, int n_out_tiles, int pairs, bool re
     return e.band;
 }
 
-template <bool SPARSE, int BN, int EPI, bool RES>
+template <bool SPARSE, int BN, int EPI, bool RES, bool BUILD = false>
 static int launch_gemm_pair(const LinearArgs& a) {
     using Cfg = PairCfg<SPARSE, BN, RES>;
     const nm_packed_t& W = *a.W;
     CUtensorMap tw, tx, ty;
-    int rc = make_map(&tw, W.values, (uint64_t)W.out, (uint64_t)(SPARSE ? W.in / 2 : W.in), kBM, Cfg::A_ROW,
-                      CU_TENSOR_MAP_SWIZZLE_128B);
+    // rebuilt weights are read by the builder warps, not by TMA: the weight map then describes X as a stand-in
+    int rc = BUILD ? make_map(&tw, a.X, (uint64_t)a.tokens, (uint64_t)W.in, kBM, 128, CU_TENSOR_MAP_SWIZZLE_128B)
+                   : make_map(&tw, W.values, (uint64_t)W.out, (uint64_t)(SPARSE ? W.in / 2 : W.in), kBM, Cfg::A_ROW,
+                              CU_TENSOR_MAP_SWIZZLE_128B);
     if (rc != NM_OK) return rc;
     rc = make_map_x3(&tx, a.X, (uint64_t)a.tokens, (uint64_t)W.in, Cfg::B_ROWS, Cfg::KB / 128);
     if (rc != NM_OK) return rc;
@@ -1120,9 +1175,13 @@ static int launch_gemm_pair(const LinearArgs& a) {
     p.n_tiles = p.n_tok_tiles * p.n_out_tiles;
     p.kblocks = (W.in + Cfg::KB - 1) / Cfg::KB;
     p.meta = (const uint32_t*)W.meta; p.mrow_words = W.in / 32;
+    p.values = (const uint8_t*)W.values;
+    p.vrow_bytes = (int)values_row_bytes(W.in, W.n, W.m, W.bits);
+    p.mrow_bytes = (int)meta_row_words(W.in, W.n, W.m) * 4;
+    p.pat = xf::pattern_of(W.n, W.m, W.bits);
     p.sw = a.sw; p.bias = a.bias; p.sx_dev = a.sx_dev; p.sx_host = a.sx;
     p.Y = a.Y; p.ACC = a.ACC; p.NARROW = a.NARROW; p.sy = a.sy; p.absmax = a.absmax; p.status = a.status; p.trace = g_trace_buffer; p.skip_stage = g_opt.skip_stage - 1;
-    auto fn = nm_gemm_pair_kernel<SPARSE, BN, EPI, RES>;
+    auto fn = nm_gemm_pair_kernel<SPARSE, BN, EPI, RES, BUILD>;
     NM_CUDA_TRY(allow_dynamic_smem((const void*)fn, Cfg::SMEM));
     int pairs = p.n_tiles < sm_count() / 2 ? p.n_tiles : sm_count() / 2;
     if (pairs > kMaxPairs) pairs = kMaxPairs;
@@ -1134,7 +1193,7 @@ static int launch_gemm_pair(const LinearArgs& a) {
     p.band = cached_pair_plan(p.n_tok_tiles, p.n_out_tiles, pairs, RES, g_opt.band, sched);
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(2 * pairs, 1, 1);
-    cfg.blockDim = dim3(kPairThreads, 1, 1);
+    cfg.blockDim = dim3(kPairThreadsOf<BUILD>, 1, 1);
     cfg.dynamicSmemBytes = Cfg::SMEM;
     cfg.stream = a.stream;
     cudaLaunchAttribute attr[2];
@@ -1248,6 +1307,13 @@ static int pick_bn(const LinearArgs& a) {
         if ((long long)out_tiles * ((a.tokens + 127) / 128) >= sms) return launch_gemm<SPARSE, 128, EPI, W_TMA>(a);
         return launch_gemm<SPARSE, 64, EPI, W_TMA>(a);
     } else {
+        // Sparse-target formats with a short reduction and work for every SM pair: the CTA-pair kernel with the weights
+        // rebuilt once per output tile into its resident region (32-bit outputs).
+        if constexpr (SPARSE && (EPI == EPI_F32 || EPI == EPI_ACC)) {
+            const long long pair_tiles = (long long)((a.W->out + 2 * kBM - 1) / (2 * kBM)) * ((a.tokens + 191) / 192);
+            if (a.W->in <= kPairResStages * PairCfg<true, 192>::KB && pair_tiles >= sms / 2 && !g_opt.no_pair && !g_opt.no_resident)
+                return launch_gemm_pair<true, 192, EPI, true, true>(a);
+        }
         // Short reductions with many token tiles per output tile: build each weight tile once and keep it.
         constexpr int BNR = SPARSE ? 192 : 128;
         if (a.W->in / kKB <= kResidentKB && (long long)out_tiles * ((a.tokens + BNR - 1) / BNR) >= sms && !g_opt.no_resident)

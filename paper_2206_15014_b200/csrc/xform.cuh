@@ -194,6 +194,16 @@ __device__ __forceinline__ void store_row(uint8_t* tile, int row, const uint32_t
         *reinterpret_cast<uint4*>(base + ((c ^ x) << 4)) = make_uint4(w[4 * c], w[4 * c + 1], w[4 * c + 2], w[4 * c + 3]);
 }
 
+// The 64 operand bytes of one row and one 128-wide k-block into a tile whose rows are 128 bytes wide (two k-blocks side by
+// side: `half` says which) with the 128-byte swizzle: 16-byte chunk c of row r lands at chunk c ^ (r & 7).
+__device__ __forceinline__ void store_half_row128(uint8_t* tile, int row, int half, const uint32_t (&w)[16]) {
+    uint8_t* base = tile + row * 128;
+    const int x = row & 7;
+#pragma unroll
+    for (int c = 0; c < 4; ++c)
+        *reinterpret_cast<uint4*>(base + (((half * 4 + c) ^ x) << 4)) = make_uint4(w[4 * c], w[4 * c + 1], w[4 * c + 2], w[4 * c + 3]);
+}
+
 // Hardware metadata words (4 per k-block) of one row from its canonical metadata.
 __device__ __forceinline__ uint4 hw_meta(int pat, const uint8_t* msrc, const uint32_t* lut) {
     if (pat == P24_4) return ldg16(msrc);
