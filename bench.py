@@ -449,6 +449,9 @@ def run_cuda(args):
     dev = torch.device("cuda", local)
     if world > 1:
         dist.init_process_group("nccl", device_id=dev)
+    for kv in args.option:   # A/B runs of a kernel choice; recorded in the line's config
+        k, v = kv.split("=")
+        nm.nm_debug_set_option(k, int(v))   # raises on an unknown name
     n, m, bits = PATTERN
     pk = peaks()
     YDTYPE = {"f32": torch.float32, "int8": torch.int8, "bf16": torch.bfloat16}[args.out]
@@ -617,6 +620,15 @@ def run_cuda(args):
                 d["Y"] = saved
             alone[d["name"]] = time_stream(torch, one, 100)
             del Ys
+        # the projection launched alone: two more copies of W and U, so that no launch finds its inputs in L2
+        sets = [jobs]
+        extra = []
+        for _ in range(2):
+            cp = [(d["W"].clone(), d["U"].clone()) for d in devbuf]
+            extra.append(cp)
+            sets.append(nm.make_pack_jobs([(W, U, n, m, bits, d["values"], d["meta"], d["scales"]) for (W, U), d in zip(cp, devbuf)]))
+        alone["pack"] = time_stream(torch, lambda i: nm.nm_project_pack_batched(sets[i % 3], len(devbuf), ws, ws_bytes, status), 100)
+        del sets, extra
         fill = torch.empty(1 << 30, dtype=torch.uint8, device=dev)
         write_gbs = (1 << 30) / time_stream(torch, lambda i: fill.zero_(), 10, warm=2) / 1e3
         del fill
@@ -641,8 +653,12 @@ def run_cuda(args):
             e["us_launched_alone"] = alone[d["name"]]
             per_kernel[d["name"]] = e
         pbytes = sum(pack_bytes(d["out"], d["k"], n, m, bits) for d in devbuf)
+        # in the step the launch follows FFN2 and FFN1, whose last outputs are still dirty in L2 and are written back
+        # while it reads; launched alone (inputs rotating, never in L2) it only moves its own bytes
         per_kernel["pack_layer"] = {"us": kern["pack"], "gbs": pbytes / kern["pack"] / 1e3,
-                                    "frac_hbm_measured": pbytes / kern["pack"] / 1e3 / pk["hbm_gbs"]}
+                                    "frac_hbm_measured": pbytes / kern["pack"] / 1e3 / pk["hbm_gbs"],
+                                    "us_launched_alone": alone["pack"],
+                                    "frac_hbm_launched_alone": pbytes / alone["pack"] / 1e3 / pk["hbm_gbs"]}
         if pack_info:
             per_kernel["pack_sweep"] = pack_info
         # dominant kernel of the step: the FFN1 GEMM launch (longest).  Its bytes are 93 % fp32 Y written; a plain fill of
@@ -676,7 +692,8 @@ def run_cuda(args):
                 "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True,
                 "scaling": "weak", "vs_baseline": None, "dtype": "int8", "data": "synthetic",
                 "config": {"workload": WORKLOAD if TOKENS == 16384 else WORKLOAD + f" (reduced to {TOKENS} tokens)", "tokens": TOKENS, "pattern": "2:4", "bits": bits, "out": args.out,
-                           "l2": "inputs+outputs per step (715 MB) exceed L2; no flush needed"},
+                           "l2": "inputs+outputs per step (715 MB) exceed L2; no flush needed",
+                           **({"options": list(args.option)} if args.option else {})},
                 "clocks": clocks,
                 "e2e": {"value": whole_job_tops(ops_step, world, e2e_ms), "unit": "TOPS",
                         "ms_per_step": e2e_ms, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": e2e_steps},
@@ -984,7 +1001,7 @@ def main():
     ap.add_argument("--trace-gemm", default="", metavar="TOKENS,K,OUT",
                     help="time stamps of one 2:4 int8 GEMM launch (needs the NM_TRACE build of the library, see trace_gemm)")
     ap.add_argument("--option", action="append", default=[], metavar="NAME=VALUE",
-                    help="kernel-choice override for --trace-gemm (nm_debug_set_option), e.g. no_wide=1")
+                    help="kernel-choice override (nm_debug_set_option) for A/B runs, e.g. no_wide=1 or pack_form=2")
     args = ap.parse_args()
     if args.trace_gemm:
         return trace_gemm(args)

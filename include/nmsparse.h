@@ -90,7 +90,10 @@ int nm_packed_sizes(int out, int in, int n, int m, int bits, size_t *values_byte
  * Accepted: (n, m) in {1:4, 2:4, 1:8, 2:8, 4:8} or n == m; bits in {4, 8}; in <= 32768.
  * W, U, values 16-byte aligned, meta and scales 4-byte aligned.
  * Sets NM_STATUS_NONFINITE in *status (nullable) when W + U holds NaN/Inf; outputs of such rows are
- * unspecified.  One pass over W and U; outputs are written once.
+ * unspecified.  One pass over W and U; outputs are written once.  Rows of at most 4096 values reach the
+ * kernel through bulk copies whose arrival a warp awaits for about a second at most: NM_STATUS_TIMEOUT in
+ * *status when such a wait expired (the outputs are then void); the same holds for every entry point below
+ * that projects.
  */
 int nm_project_pack(const float *W, const float *U, int out, int in, int n, int m, int bits,
                     void *values, void *meta, float *scales, uint32_t *status, void *stream);
@@ -331,11 +334,13 @@ int nm_probe_tma_stream(const void *W, int w_rows, int w_row_bytes, const void *
 
 /*
  * Measurement and test aid (the paper has no counterpart): overrides the kernel nm_int_linear and its variants
- * pick, process-wide, for every later call (not thread-safe against calls in flight on other host threads).
+ * (and, with "pack_form", the projection entry points) pick, process-wide, for every later call (not thread-safe against calls in flight on other host threads).
  * All options are 0 by default = the library's own choice.  Names: "no_pdl" (launch without the programmatic-
  * dependent-launch attribute), "no_pair" (one-CTA kernels only), "no_resident" (always stream the weights),
  * "no_wide" (never the 512-channel pair kernel), "wide_any" (the 512-channel pair kernel whenever the shape
- * allows it, however few tiles there are), "wide_bn" (its token-tile width, 224 or 192), "band" (band size of the streamed pair kernel's tile order).
+ * allows it, however few tiles there are), "wide_bn" (its token-tile width, 224 or 192), "band" (band size of the streamed pair kernel's tile order),
+ * "pack_form" (form of the projection kernel in blocks of four warps: 1 = one unit per block, 2 = persistent with
+ * chunks staged in shared memory by bulk copies, 3 = persistent with the next chunk asked for ahead into L2).
  * Results never depend on them.  Returns NM_ERR_UNSUPPORTED for an unknown name.  A library built with
  * -DNM_TEST_HOOKS (build.py --variant shortwait: device-side waits limited to about a millisecond) also takes
  * "skip_stage" = 1 + the pipeline stage that CTA 0's producer leaves unissued (0 = none): the bounded waits then

@@ -30,6 +30,9 @@ inline size_t meta_row_words(int in, int n, int m) {
     return ((size_t)(in / m) * n * meta_field_bits(m) + 31) / 32;
 }
 
+// Form of the projection kernel forced by nm_debug_set_option("pack_form") (0 = automatic).
+extern int g_pack_form;
+
 // Multiprocessors of the current device (cached per device; 148 when the query fails).
 int sm_count();
 

@@ -1400,7 +1400,7 @@ int nm_debug_set_option(const char* name, int value) {
     struct { const char* name; int* slot; } table[] = {
         {"no_pdl", &nm::g_opt.no_pdl}, {"no_pair", &nm::g_opt.no_pair}, {"no_resident", &nm::g_opt.no_resident},
         {"no_wide", &nm::g_opt.no_wide}, {"wide_any", &nm::g_opt.wide_any}, {"wide_bn", &nm::g_opt.wide_bn},
-        {"band", &nm::g_opt.band}};
+        {"band", &nm::g_opt.band}, {"pack_form", &nm::g_pack_form}};
     for (auto& e : table)
         if (!strcmp(name, e.name)) { *e.slot = value; return NM_OK; }
 #ifdef NM_TEST_HOOKS

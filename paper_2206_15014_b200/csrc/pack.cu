@@ -7,6 +7,7 @@
 // of 4 or 4 groups of 8).  From there everything is lane-local: the lane's share of the packed
 // values and of the metadata is a whole number of bytes, written with one vector store each.
 #include "common.cuh"
+#include "sm100_ptx.cuh"
 #include <cuda_runtime.h>
 #include <vector>
 #include <mutex>
@@ -42,6 +43,10 @@ struct PackJobInline {
 };
 
 static constexpr int kPackMinWarps = 4;
+#ifndef NM_WAIT_LIMIT
+#define NM_WAIT_LIMIT (1ll << 31)
+#endif
+static constexpr long long kPackWaitLimit = NM_WAIT_LIMIT;  // SM clocks a warp waits for its staged chunk (about a second)
 // group_mode of pack_kernel: scale per row from the row itself; only fold the row maxima per group into
 // `scales`; take the scales found in `scales`.
 enum { kGroupNone = 0, kGroupMaxPass = 1, kGroupScalesGiven = 2 };
@@ -183,11 +188,72 @@ __device__ __forceinline__ void store_bytes_slow(uint8_t* dst, const unsigned* w
 // null) the packed outputs the kernel writes Z = s * code as dense fp32, zero where pruned, and, when
 // U_next is not null, the dual update U_next = (W + U) - Z.  Both go back through the shared-memory
 // tile so that the stores are as coalesced as the loads.
-template <int N, int M, int BITS, int MAXT, bool DENSE_OUT = false>
-__global__ void __launch_bounds__(MAXT, MAXT == 128 ? (DENSE_OUT ? 4 : 8) : 1) pack_kernel(const PackJobDev* __restrict__ jobs, int njobs,
-                                                    const __grid_constant__ PackJobInline inl, uint32_t* status, float* __restrict__ Zout,
-                                                    float* __restrict__ Unext, const DenseOutDev* __restrict__ dense_jobs,
-                                                    int group_mode, int group_rows) {
+//
+// A "unit" is what one block does at a time: `warps >> wpr_log2` rows of one job, one 1024-value chunk per warp.
+// PIPE (blocks of four warps): the grid is persistent, block b takes the units b, b + gridDim.x, ...; every warp
+// fetches the chunk of its NEXT unit (W and U, 4 KB each) with two bulk copies into the other half of a
+// double buffer in shared memory while it works on the current one, so that loading and arithmetic overlap
+// inside a warp and not only between blocks that happen to be out of step.  Without PIPE one block = one unit
+// and the chunk is loaded with 16-byte global loads.
+
+// Where a warp stands inside a unit of a job.
+struct UnitPos {
+    long long row;
+    int chunk, row_in_block, elems;  // elems: values of the chunk that lie inside the row (0 when the row does not exist)
+    bool row_ok;
+};
+
+__device__ __forceinline__ UnitPos unit_pos(const PackJobDev& job, unsigned unit, int w, int warps) {
+    UnitPos u;
+    const int wpr = 1 << job.wpr_log2;
+    u.row_in_block = w >> job.wpr_log2;
+    u.chunk = w & (wpr - 1);
+    u.row = (long long)(unit - job.unit_begin) * (warps >> job.wpr_log2) + u.row_in_block;
+    u.row_ok = u.row < job.out;
+    u.elems = u.row_ok ? max(0, min(1024, job.in - u.chunk * 1024)) : 0;
+    return u;
+}
+
+// The job whose units contain `unit` (tables ascend in unit_begin) and its number in the table.
+__device__ __forceinline__ PackJobDev find_job(const PackJobDev* __restrict__ jobs, int njobs, const PackJobInline& inl,
+                                               unsigned unit, int& index) {
+    PackJobDev job;
+    if (jobs) {
+        int lo = 0, hi = njobs - 1;  // last job whose unit_begin <= unit
+        while (lo < hi) {
+            int mid = (lo + hi + 1) >> 1;
+            if (jobs[mid].unit_begin <= unit) lo = mid; else hi = mid - 1;
+        }
+        job = jobs[lo];
+        index = lo;
+    } else {
+        // table in the kernel's parameters (a single matrix is a table of one)
+        int lo = 0;
+#pragma unroll
+        for (int i = 1; i < kInlineJobs; ++i)
+            if (i < njobs && inl.j[i].unit_begin <= unit) lo = i;
+        job = inl.j[0];
+#pragma unroll
+        for (int i = 1; i < kInlineJobs; ++i)
+            if (lo == i) job = inl.j[i];
+        index = lo;
+    }
+    return job;
+}
+
+// Units of a job in a launch whose blocks have `warps` warps.
+__device__ __forceinline__ unsigned units_of(const PackJobDev& job, int warps) {
+    const int rpb = warps >> job.wpr_log2;
+    return (unsigned)((job.out + rpb - 1) / rpb);
+}
+
+// Everything after the load: `mytile` holds the warp's chunk of V = W + U in the swizzled layout, `amax` and
+// `poison` are the lane's running |max| and non-finite detector.  `red` is this unit's slot array for the row
+// maximum across the warps of a row.  Every warp of the block calls it (block-wide barrier when a row spans warps).
+template <int N, int M, int BITS, bool DENSE_OUT>
+__device__ __forceinline__ void pack_finish(const PackJobDev& job, const UnitPos& up, int lane, int w, float4* mytile,
+                                            float* red, const uint16_t* pos48, float amax, float poison, uint32_t* status,
+                                            float* __restrict__ Zout, float* __restrict__ Unext, int group_mode, int group_rows) {
     constexpr bool kDense = (N == M);
     constexpr int G = 32 / M;                          // groups per lane
     constexpr int F = (M == 4) ? 2 : 4;                // metadata field width
@@ -195,86 +261,11 @@ __global__ void __launch_bounds__(MAXT, MAXT == 128 ? (DENSE_OUT ? 4 : 8) : 1) p
     constexpr int VWORDS = (VBITS + 31) / 32;
     constexpr int MBITS = kDense ? 0 : G * N * F;      // metadata bits per lane (0, 16, 32, 64)
     constexpr int MWORDS = kDense ? 1 : (MBITS + 31) / 32;
-
-    extern __shared__ float4 tile[];  // [warps][256] float4, [warps] floats for the row maximum, 256 u16 (4:8 positions)
-    const int warps = blockDim.x >> 5;
-    float* red = reinterpret_cast<float*>(tile + warps * 256);
-    // a kernel launched as this one's programmatic dependent may begin its set-up on SMs this grid has left
-    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-    // four of eight: table from the 8-bit keep mask to its four positions (4-bit fields, ascending), which is
-    // also the group's metadata; the kept values are then fetched from the warp's tile by position
-    uint16_t* pos48 = reinterpret_cast<uint16_t*>(red + warps);
-    if constexpr (N == 4 && M == 8) {
-        for (unsigned mk = threadIdx.x; mk < 256; mk += blockDim.x) {
-            unsigned r = 0, c = 0;
-#pragma unroll
-            for (unsigned p8 = 0; p8 < 8; ++p8)
-                if ((mk >> p8) & 1u) { r |= p8 << (4 * (c & 3u)); ++c; }
-            pos48[mk] = (uint16_t)r;
-        }
-        __syncthreads();
-    }
-
-    PackJobDev job;
-    if (jobs) {
-        int lo = 0, hi = njobs - 1;  // last job whose unit_begin <= blockIdx.x
-        while (lo < hi) {
-            int mid = (lo + hi + 1) >> 1;
-            if (jobs[mid].unit_begin <= blockIdx.x) lo = mid; else hi = mid - 1;
-        }
-        job = jobs[lo];
-        if constexpr (DENSE_OUT) { Zout = dense_jobs[lo].Z; Unext = dense_jobs[lo].U_next; }
-    } else {
-        // table in the kernel's parameters (a single matrix is a table of one); entries ascend in unit_begin
-        int lo = 0;
-#pragma unroll
-        for (int i = 1; i < kInlineJobs; ++i)
-            if (i < njobs && inl.j[i].unit_begin <= blockIdx.x) lo = i;
-        job = inl.j[0];
-#pragma unroll
-        for (int i = 1; i < kInlineJobs; ++i)
-            if (lo == i) job = inl.j[i];
-    }
-    const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
     const int wpr = 1 << job.wpr_log2;
-    const int row_in_block = w >> job.wpr_log2, chunk = w & (wpr - 1);
-    const int rows_per_block = warps >> job.wpr_log2;
-    const long long row = (long long)(blockIdx.x - job.unit_begin) * rows_per_block + row_in_block;
-    const bool row_ok = row < job.out;
+    const int row_in_block = up.row_in_block, chunk = up.chunk;
+    const long long row = up.row;
+    const bool row_ok = up.row_ok;
     const int in4 = job.in >> 2;
-
-    // ---- load V = W + U (coalesced), running |max| and non-finite detector -------------------
-    float4* mytile = tile + w * 256;
-    float amax = 0.0f, poison = 0.0f;
-    {
-        const float4* W4 = reinterpret_cast<const float4*>(job.W) + (row_ok ? row * in4 : 0);
-        const float4* U4 = job.U ? reinterpret_cast<const float4*>(job.U) + (row_ok ? row * in4 : 0) : nullptr;
-        float4 v[8];
-#pragma unroll
-        for (int j = 0; j < 8; ++j) {
-            int f = chunk * 256 + j * 32 + lane;
-            v[j] = (row_ok && f < in4) ? ld_stream(W4 + f) : make_float4(0.f, 0.f, 0.f, 0.f);
-        }
-        if (U4) {
-#pragma unroll
-            for (int j = 0; j < 8; ++j) {
-                int f = chunk * 256 + j * 32 + lane;
-                if (row_ok && f < in4) {
-                    float4 u = ld_stream(U4 + f);
-                    v[j].x = __fadd_rn(v[j].x, u.x); v[j].y = __fadd_rn(v[j].y, u.y);
-                    v[j].z = __fadd_rn(v[j].z, u.z); v[j].w = __fadd_rn(v[j].w, u.w);
-                }
-            }
-        }
-#pragma unroll
-        for (int j = 0; j < 8; ++j) {
-            amax = fmaxf(amax, fmaxf(fmaxf(fabsf(v[j].x), fabsf(v[j].y)), fmaxf(fabsf(v[j].z), fabsf(v[j].w))));
-            poison = __fmaf_rn(v[j].x, 0.0f, poison); poison = __fmaf_rn(v[j].y, 0.0f, poison);
-            poison = __fmaf_rn(v[j].z, 0.0f, poison); poison = __fmaf_rn(v[j].w, 0.0f, poison);
-            int fl = j * 32 + lane, owner = fl >> 3, jj = fl & 7;
-            mytile[owner * 8 + (jj ^ (owner & 7))] = v[j];
-        }
-    }
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, o));
     const bool bad = __any_sync(0xffffffffu, poison != poison) || !(amax <= 3.402823466e+38f);
@@ -446,6 +437,216 @@ __global__ void __launch_bounds__(MAXT, MAXT == 128 ? (DENSE_OUT ? 4 : 8) : 1) p
             const unsigned wpad[3] = {mw[0], MWORDS > 1 ? mw[MWORDS - 1] : 0u, 0u};
             store_bytes_slow<MB + 4>(dst, wpad, last ? (int)min(row_bytes - lane_off, (unsigned)(MB + 4)) : MB);
         }
+    }
+}
+
+// Loads the warp's chunk with coalesced 16-byte global loads, leaves V = W + U in `mytile` (swizzled).
+__device__ __forceinline__ void load_chunk_global(const PackJobDev& job, const UnitPos& up, int lane, float4* mytile,
+                                                  float& amax, float& poison) {
+    const int in4 = job.in >> 2;
+    const float4* W4 = reinterpret_cast<const float4*>(job.W) + (up.row_ok ? up.row * in4 : 0);
+    const float4* U4 = job.U ? reinterpret_cast<const float4*>(job.U) + (up.row_ok ? up.row * in4 : 0) : nullptr;
+    float4 v[8];
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+        int f = up.chunk * 256 + j * 32 + lane;
+        v[j] = (up.row_ok && f < in4) ? ld_stream(W4 + f) : make_float4(0.f, 0.f, 0.f, 0.f);
+    }
+    if (U4) {
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            int f = up.chunk * 256 + j * 32 + lane;
+            if (up.row_ok && f < in4) {
+                float4 u = ld_stream(U4 + f);
+                v[j].x = __fadd_rn(v[j].x, u.x); v[j].y = __fadd_rn(v[j].y, u.y);
+                v[j].z = __fadd_rn(v[j].z, u.z); v[j].w = __fadd_rn(v[j].w, u.w);
+            }
+        }
+    }
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+        amax = fmaxf(amax, fmaxf(fmaxf(fabsf(v[j].x), fabsf(v[j].y)), fmaxf(fabsf(v[j].z), fabsf(v[j].w))));
+        poison = __fmaf_rn(v[j].x, 0.0f, poison); poison = __fmaf_rn(v[j].y, 0.0f, poison);
+        poison = __fmaf_rn(v[j].z, 0.0f, poison); poison = __fmaf_rn(v[j].w, 0.0f, poison);
+        int fl = j * 32 + lane, owner = fl >> 3, jj = fl & 7;
+        mytile[owner * 8 + (jj ^ (owner & 7))] = v[j];
+    }
+}
+
+// The same from the chunk that the bulk copies left in shared memory (`wbuf`, `ubuf`: 256 float4 each, in
+// memory order); V = W + U replaces W in place, swizzled inside each 128-byte row.
+__device__ __forceinline__ void load_chunk_staged(const PackJobDev& job, const UnitPos& up, int lane, float4* wbuf,
+                                                  const float4* ubuf, float& amax, float& poison) {
+    const int n4 = up.elems >> 2;  // float4 of the chunk that the copy brought
+    float4 v[8];
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+        const int fl = j * 32 + lane;
+        v[j] = fl < n4 ? wbuf[fl] : make_float4(0.f, 0.f, 0.f, 0.f);
+        if (job.U && fl < n4) {
+            const float4 u = ubuf[fl];
+            v[j].x = __fadd_rn(v[j].x, u.x); v[j].y = __fadd_rn(v[j].y, u.y);
+            v[j].z = __fadd_rn(v[j].z, u.z); v[j].w = __fadd_rn(v[j].w, u.w);
+        }
+    }
+    __syncwarp();  // every lane has read its part before the rows are rewritten in place
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+        amax = fmaxf(amax, fmaxf(fmaxf(fabsf(v[j].x), fabsf(v[j].y)), fmaxf(fabsf(v[j].z), fabsf(v[j].w))));
+        poison = __fmaf_rn(v[j].x, 0.0f, poison); poison = __fmaf_rn(v[j].y, 0.0f, poison);
+        poison = __fmaf_rn(v[j].z, 0.0f, poison); poison = __fmaf_rn(v[j].w, 0.0f, poison);
+        int fl = j * 32 + lane, owner = fl >> 3, jj = fl & 7;
+        wbuf[owner * 8 + (jj ^ (owner & 7))] = v[j];
+    }
+}
+
+// Forms of the kernel.  kDirect: one block = one unit, 16-byte global loads.  kStaged2: persistent, two chunk
+// buffers per warp (16 KB), the next unit's copies are issued before the current unit is touched; for the forms that
+// keep using the tile to the end of the unit (4:8, dense outputs).
+// kAhead: persistent, 16-byte global loads as in kDirect, but every warp first asks for its NEXT unit's chunk to be
+// brought into L2 (a bulk prefetch: no registers, no shared memory), so that DRAM streams from the first cycle on and
+// the loads of all units but the first are L2 hits.
+enum { kDirect = 0, kStaged2 = 1, kAhead = 2 };
+__host__ __device__ constexpr int pack_blocks_per_sm(int pipe) { return pipe == kStaged2 ? 3 : 8; }
+
+template <int N, int M, int BITS, int MAXT, bool DENSE_OUT = false, int PIPE = kDirect>
+__global__ void __launch_bounds__(MAXT, PIPE != kDirect ? pack_blocks_per_sm(PIPE) : (MAXT == 128 ? (DENSE_OUT ? 4 : 8) : 1))
+pack_kernel(const PackJobDev* __restrict__ jobs, int njobs, const __grid_constant__ PackJobInline inl, uint32_t* status,
+            float* __restrict__ Zout, float* __restrict__ Unext, const DenseOutDev* __restrict__ dense_jobs,
+            int group_mode, int group_rows, unsigned nunits) {
+    static_assert(PIPE == kDirect || MAXT == 128, "the staged forms are built for blocks of four warps");
+    // staged: [warps][2 buffers][W, U][256] float4; else [warps][256] float4.  Then [2][warps] floats for the row
+    // maximum, 256 u16 (4:8 positions), and for the staged forms [warps][2] mbarriers and the abort flag.
+    extern __shared__ float4 tile[];
+    const int warps = blockDim.x >> 5;
+    float* red = reinterpret_cast<float*>(tile + warps * (PIPE == kStaged2 ? 1024 : 256));
+    // a kernel launched as this one's programmatic dependent may begin its set-up on SMs this grid has left
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    // four of eight: table from the 8-bit keep mask to its four positions (4-bit fields, ascending), which is
+    // also the group's metadata; the kept values are then fetched from the warp's tile by position
+    uint16_t* pos48 = reinterpret_cast<uint16_t*>(red + 2 * warps);
+    if constexpr (N == 4 && M == 8) {
+        for (unsigned mk = threadIdx.x; mk < 256; mk += blockDim.x) {
+            unsigned r = 0, c = 0;
+#pragma unroll
+            for (unsigned p8 = 0; p8 < 8; ++p8)
+                if ((mk >> p8) & 1u) { r |= p8 << (4 * (c & 3u)); ++c; }
+            pos48[mk] = (uint16_t)r;
+        }
+        __syncthreads();
+    }
+    const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+
+    if constexpr (PIPE == kAhead) {
+        float4* mytile = tile + w * 256;
+        auto ask = [&](const PackJobDev& j, const UnitPos& up) {
+            if (up.elems == 0 || lane != 0) return;
+            const size_t first = (size_t)up.row * j.in + (size_t)up.chunk * 1024;
+            ptx::bulk_prefetch_l2(j.W + first, (uint32_t)up.elems * 4u);
+            if (j.U) ptx::bulk_prefetch_l2(j.U + first, (uint32_t)up.elems * 4u);
+        };
+        int index = 0;
+        unsigned unit = blockIdx.x;
+        PackJobDev job{};
+        if (unit < nunits) job = find_job(jobs, njobs, inl, unit, index);
+        for (int it = 0; unit < nunits; ++it, unit += gridDim.x) {
+            const UnitPos up = unit_pos(job, unit, w, warps);
+            const unsigned next = unit + gridDim.x;
+            PackJobDev njob = job;
+            int nindex = index;
+            if (next < nunits) {
+                if (next - job.unit_begin >= units_of(job, warps)) njob = find_job(jobs, njobs, inl, next, nindex);
+                ask(njob, unit_pos(njob, next, w, warps));
+            }
+            if constexpr (DENSE_OUT) {
+                if (jobs) { Zout = dense_jobs[index].Z; Unext = dense_jobs[index].U_next; }
+            }
+            float amax = 0.0f, poison = 0.0f;
+            load_chunk_global(job, up, lane, mytile, amax, poison);
+            pack_finish<N, M, BITS, DENSE_OUT>(job, up, lane, w, mytile, red + (it & 1) * warps, pos48, amax, poison,
+                                              status, Zout, Unext, group_mode, group_rows);
+            __syncwarp();  // the tile is rewritten by the next unit
+            job = njob; index = nindex;
+        }
+    } else if constexpr (PIPE == kDirect) {
+        int index = 0;
+        const PackJobDev job = find_job(jobs, njobs, inl, blockIdx.x, index);
+        if constexpr (DENSE_OUT) {
+            if (jobs) { Zout = dense_jobs[index].Z; Unext = dense_jobs[index].U_next; }
+        }
+        const UnitPos up = unit_pos(job, blockIdx.x, w, warps);
+        float4* mytile = tile + w * 256;
+        float amax = 0.0f, poison = 0.0f;
+        load_chunk_global(job, up, lane, mytile, amax, poison);
+        pack_finish<N, M, BITS, DENSE_OUT>(job, up, lane, w, mytile, red, pos48, amax, poison, status, Zout, Unext,
+                                          group_mode, group_rows);
+    } else {
+        uint64_t* bars = reinterpret_cast<uint64_t*>(pos48 + 256);       // [warps][2]
+        volatile uint32_t* abort_flag = reinterpret_cast<volatile uint32_t*>(bars + 2 * warps);
+        float4* mybuf = tile + w * 1024;                                  // [buffer][W, U][256]
+        const uint32_t bar0 = ptx::smem_u32(bars + 2 * w);
+        if (lane == 0) {
+            ptx::mbar_init(bar0, 1);
+            ptx::mbar_init(bar0 + 8, 1);
+            if (threadIdx.x == 0) *abort_flag = 0;
+            ptx::fence_mbar_init();
+        }
+        __syncthreads();
+        // every lane calls it; lane 0 issues one bulk copy per operand, completion counted in bytes on the buffer's barrier
+        auto issue = [&](const PackJobDev& j, const UnitPos& up, int buf) {
+            if (up.elems == 0) return;      // the same for the whole warp; the unit then waits for nothing
+            ptx::fence_proxy_async_smem();  // this lane's generic accesses to the buffer before the copy's writes
+            __syncwarp();                   // the buffer's last reader is done
+            if (lane == 0) {
+                const uint32_t bytes = (uint32_t)up.elems * 4u, bar = bar0 + 8u * buf;
+                const size_t first = (size_t)up.row * j.in + (size_t)up.chunk * 1024;
+                ptx::mbar_expect_tx(bar, j.U ? 2 * bytes : bytes);
+                ptx::bulk_load(ptx::smem_u32(mybuf + buf * 512), j.W + first, bytes, bar);
+                if (j.U) ptx::bulk_load(ptx::smem_u32(mybuf + buf * 512 + 256), j.U + first, bytes, bar);
+            }
+        };
+        int index = 0;
+        unsigned unit = blockIdx.x;
+        PackJobDev job{};
+        UnitPos up{};
+        if (unit < nunits) {
+            job = find_job(jobs, njobs, inl, unit, index);
+            up = unit_pos(job, unit, w, warps);
+            issue(job, up, 0);
+        }
+        uint32_t phase = 0;  // bit b: parity of buffer b's next completion
+        for (int it = 0; unit < nunits; ++it, unit += gridDim.x) {
+            const int buf = it & 1;
+            // the next unit's chunk goes into the other buffer while this one is worked on
+            const unsigned next = unit + gridDim.x;
+            PackJobDev njob = job;
+            int nindex = index;
+            UnitPos nup{};
+            if (next < nunits) {
+                if (next - job.unit_begin >= units_of(job, warps)) njob = find_job(jobs, njobs, inl, next, nindex);
+                nup = unit_pos(njob, next, w, warps);
+                issue(njob, nup, buf ^ 1);
+            }
+            if constexpr (DENSE_OUT) {
+                if (jobs) { Zout = dense_jobs[index].Z; Unext = dense_jobs[index].U_next; }
+            }
+            if (up.elems != 0) {
+                if (!ptx::mbar_wait_bounded(bar0 + 8u * buf, (phase >> buf) & 1u, abort_flag, kPackWaitLimit)) {
+                    // recorded; the unit is then worked on with whatever the buffer holds (in bounds, results void)
+                    *abort_flag = 1u;
+                    if (status) atomicOr(status, NM_STATUS_TIMEOUT);
+                }
+                phase ^= 1u << buf;
+            }
+            float4* mytile = mybuf + buf * 512;
+            float amax = 0.0f, poison = 0.0f;
+            load_chunk_staged(job, up, lane, mytile, mytile + 256, amax, poison);
+            pack_finish<N, M, BITS, DENSE_OUT>(job, up, lane, w, mytile, red + (it & 1) * warps, pos48, amax, poison,
+                                              status, Zout, Unext, group_mode, group_rows);
+            job = njob; index = nindex; up = nup;
+        }
+        // after an expired wait a copy may still be on its way into this block's shared memory
+        if (*abort_flag) ptx::wait_clocks(1 << 17);
     }
 }
 
@@ -712,26 +913,46 @@ __global__ void __launch_bounds__(MAXT, MAXT == 128 ? (32 / M * N > 16 ? 4 : 5) 
 // ---------------------------------------------------------------------------------------------
 // host side
 // ---------------------------------------------------------------------------------------------
-using PackFn = void (*)(const PackJobDev*, int, const PackJobInline, uint32_t*, float*, float*, const DenseOutDev*, int, int);
+using PackFnPtr = void (*)(const PackJobDev*, int, const PackJobInline, uint32_t*, float*, float*, const DenseOutDev*, int, int, unsigned);
+struct PackFn { PackFnPtr fn; int form; };  // kernel and its form (kDirect, kStaged2, kAhead)
+
+// nm_debug_set_option("pack_form"): 0 = automatic, 1 = kDirect, 2 = kStaged2, 3 = kAhead for blocks of four warps.
+int g_pack_form = 0;
+
+template <int N, int M, bool DENSE_OUT, int FORM>
+static PackFn pick_form(int bits) {
+    return bits == 8 ? PackFn{(PackFnPtr)pack_kernel<N, M, 8, 128, DENSE_OUT, FORM>, FORM}
+                     : PackFn{(PackFnPtr)pack_kernel<N, M, 4, 128, DENSE_OUT, FORM>, FORM};
+}
 
 template <int N, int M, bool DENSE_OUT>
-static PackFn pick_bits(int bits, int warps) {
-    if (warps <= kPackMinWarps)
-        return bits == 8 ? (PackFn)pack_kernel<N, M, 8, 128, DENSE_OUT> : (PackFn)pack_kernel<N, M, 4, 128, DENSE_OUT>;
+static PackFn pick_bits(int bits, int warps, unsigned blocks) {
+    if (warps <= kPackMinWarps) {
+        // Blocks of four warps, persistent.  Staged chunks for the dense-output form (0.83 -> 0.95 of the copy rate on the
+        // 24-layer sweep) and for launches of a few rounds per resident block, where loads and arithmetic of blocks that
+        // start together would otherwise alternate (one layer alone: 26.8 -> 24.7 us); chunks asked for ahead on long
+        // launches, where the staged form's twelve warps per SM are too few (sweep: 0.82 against 0.89).
+        const bool few_rounds = blocks <= 16u * (unsigned)(sm_count() * pack_blocks_per_sm(kStaged2));
+        const int form = g_pack_form == 1 ? kDirect : g_pack_form == 2 ? kStaged2 : g_pack_form == 3 ? kAhead
+                                          : ((DENSE_OUT || few_rounds) ? kStaged2 : kAhead);
+        if (form == kDirect) return pick_form<N, M, DENSE_OUT, kDirect>(bits);
+        if (form == kStaged2) return pick_form<N, M, DENSE_OUT, kStaged2>(bits);
+        return pick_form<N, M, DENSE_OUT, kAhead>(bits);
+    }
     if constexpr (DENSE_OUT) {  // the dense outputs need ~128 registers: blocks of at most 512 threads get them
         if (warps <= 16)
-            return bits == 8 ? (PackFn)pack_kernel<N, M, 8, 512, true> : (PackFn)pack_kernel<N, M, 4, 512, true>;
+            return bits == 8 ? PackFn{(PackFnPtr)pack_kernel<N, M, 8, 512, true>, kDirect} : PackFn{(PackFnPtr)pack_kernel<N, M, 4, 512, true>, kDirect};
     }
-    return bits == 8 ? (PackFn)pack_kernel<N, M, 8, 1024, DENSE_OUT> : (PackFn)pack_kernel<N, M, 4, 1024, DENSE_OUT>;
+    return bits == 8 ? PackFn{(PackFnPtr)pack_kernel<N, M, 8, 1024, DENSE_OUT>, kDirect} : PackFn{(PackFnPtr)pack_kernel<N, M, 4, 1024, DENSE_OUT>, kDirect};
 }
 
 template <bool DENSE_OUT = false>
-static PackFn pick_kernel(int n, int m, int bits, int warps) {
-    if (n == m) return pick_bits<4, 4, DENSE_OUT>(bits, warps);
-    if (m == 4) return n == 1 ? pick_bits<1, 4, DENSE_OUT>(bits, warps) : pick_bits<2, 4, DENSE_OUT>(bits, warps);
-    if (n == 1) return pick_bits<1, 8, DENSE_OUT>(bits, warps);
-    if (n == 2) return pick_bits<2, 8, DENSE_OUT>(bits, warps);
-    return pick_bits<4, 8, DENSE_OUT>(bits, warps);
+static PackFn pick_kernel(int n, int m, int bits, int warps, unsigned blocks) {
+    if (n == m) return pick_bits<4, 4, DENSE_OUT>(bits, warps, blocks);
+    if (m == 4) return n == 1 ? pick_bits<1, 4, DENSE_OUT>(bits, warps, blocks) : pick_bits<2, 4, DENSE_OUT>(bits, warps, blocks);
+    if (n == 1) return pick_bits<1, 8, DENSE_OUT>(bits, warps, blocks);
+    if (n == 2) return pick_bits<2, 8, DENSE_OUT>(bits, warps, blocks);
+    return pick_bits<4, 8, DENSE_OUT>(bits, warps, blocks);
 }
 
 static int validate_job(const nm_pack_job_t& j) {
@@ -764,13 +985,31 @@ static PackJobDev to_dev(const nm_pack_job_t& j) {
 }
 
 // jobs_dev != nullptr: table of njobs entries in device memory; else the first njobs (>= 1) entries of `inl`.
-static int launch_table(PackFn fn, const PackJobDev* jobs_dev, int njobs, const PackJobInline& inl, unsigned blocks,
+static int launch_table(PackFn k, const PackJobDev* jobs_dev, int njobs, const PackJobInline& inl, unsigned blocks,
                         int warps, uint32_t* status, cudaStream_t stream, float* Z, float* U_next,
                         const DenseOutDev* dense_jobs, int group_mode, int group_rows) {
-    size_t smem = (size_t)warps * (256 * sizeof(float4) + sizeof(float)) + 512;  // + the 4:8 position table
-    if (smem > 48 * 1024)
-        NM_CUDA_TRY(cudaFuncSetAttribute((const void*)fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    fn<<<blocks, warps * 32, smem, stream>>>(jobs_dev, njobs, inl, status, Z, U_next, dense_jobs, group_mode, group_rows);
+    // chunk tile(s), two sets of row-maximum slots, the 4:8 position table; staged form: also two barriers per warp
+    // and the abort flag, and a grid that stays resident
+    const bool staged = k.form == kStaged2, persistent = k.form != kDirect;
+    size_t smem = (size_t)warps * ((staged ? 1024 : 256) * sizeof(float4) + 2 * sizeof(float)) + 512 +
+                  (staged ? (size_t)warps * 16 + 16 : 0);
+    const PackFnPtr fn = k.fn;
+    if (smem > 48 * 1024) {  // the attribute is set once per kernel and device
+        struct Done { const void* fn; int dev; };
+        static std::mutex mu;
+        static std::vector<Done> done;
+        int dev = 0;
+        NM_CUDA_TRY(cudaGetDevice(&dev));
+        std::lock_guard<std::mutex> lock(mu);
+        bool found = false;
+        for (const Done& d : done) found = found || (d.fn == (const void*)fn && d.dev == dev);
+        if (!found) {
+            NM_CUDA_TRY(cudaFuncSetAttribute((const void*)fn, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
+            done.push_back(Done{(const void*)fn, dev});
+        }
+    }
+    const unsigned grid = persistent ? std::min(blocks, (unsigned)(sm_count() * pack_blocks_per_sm(k.form))) : blocks;
+    fn<<<grid, warps * 32, smem, stream>>>(jobs_dev, njobs, inl, status, Z, U_next, dense_jobs, group_mode, group_rows, blocks);
     NM_CUDA_TRY(cudaGetLastError());
     return NM_OK;
 }
@@ -871,7 +1110,7 @@ static int launch_batched(const nm_pack_job_t* jobs, const DenseOutDev* dense, i
             for (size_t g = 0; g < keys.size(); ++g) {
                 PackJobInline inl{};
                 for (size_t i = 0; i < groups[g].size(); ++i) inl.j[i] = table[group_first[g] + i];
-                int rc = nm::launch_table(nm::pick_kernel<DENSE_OUT>(keys[g].n, keys[g].m, keys[g].bits, keys[g].warps), nullptr,
+                int rc = nm::launch_table(nm::pick_kernel<DENSE_OUT>(keys[g].n, keys[g].m, keys[g].bits, keys[g].warps, group_blocks[g]), nullptr,
                                           (int)groups[g].size(), inl, group_blocks[g], keys[g].warps, status, s, nullptr,
                                           nullptr, nullptr, kGroupNone, 0);
                 if (rc != NM_OK) return rc;
@@ -899,7 +1138,7 @@ static int launch_batched(const nm_pack_job_t* jobs, const DenseOutDev* dense, i
             const nm::PackJobDev* dev = reinterpret_cast<const nm::PackJobDev*>(ws) + group_first[g];
             group_prepare_kernel<<<(unsigned)groups[g].size(), 256, 0, s>>>(dev, group_rows, keys[g].bits, 0);
             NM_CUDA_TRY(cudaGetLastError());
-            int rc = nm::launch(nm::pick_kernel<DENSE_OUT>(keys[g].n, keys[g].m, keys[g].bits, keys[g].warps), dev,
+            int rc = nm::launch(nm::pick_kernel<DENSE_OUT>(keys[g].n, keys[g].m, keys[g].bits, keys[g].warps, group_blocks[g]), dev,
                                 (int)groups[g].size(), nm::PackJobDev{}, group_blocks[g], keys[g].warps, status, s,
                                 nullptr, nullptr, DENSE_OUT ? dense_dev + group_first[g] : nullptr, kGroupMaxPass, group_rows);
             if (rc != NM_OK) return rc;
@@ -919,7 +1158,7 @@ static int launch_batched(const nm_pack_job_t* jobs, const DenseOutDev* dense, i
     }
     for (size_t g = 0; g < keys.size(); ++g) {
         const nm::PackJobDev* dev = reinterpret_cast<const nm::PackJobDev*>(ws) + group_first[g];
-        int rc = nm::launch(nm::pick_kernel<DENSE_OUT>(keys[g].n, keys[g].m, keys[g].bits, keys[g].warps), dev,
+        int rc = nm::launch(nm::pick_kernel<DENSE_OUT>(keys[g].n, keys[g].m, keys[g].bits, keys[g].warps, group_blocks[g]), dev,
                             (int)groups[g].size(), nm::PackJobDev{}, group_blocks[g], keys[g].warps,
                             status, s, nullptr, nullptr, DENSE_OUT ? dense_dev + group_first[g] : nullptr,
                             (grouped || dist_ncand > 0) ? kGroupScalesGiven : kGroupNone, group_rows);
@@ -955,7 +1194,7 @@ int nm_project_pack(const float* W, const float* U, int out, int in, int n, int 
     int warps = std::max(nm::kPackMinWarps, 1 << d.wpr_log2);
     int rows_per_block = warps >> d.wpr_log2;
     unsigned blocks = (unsigned)((out + rows_per_block - 1) / rows_per_block);
-    return nm::launch(nm::pick_kernel(n, m, bits, warps), nullptr, 0, d, blocks, warps, status, (cudaStream_t)stream);
+    return nm::launch(nm::pick_kernel(n, m, bits, warps, blocks), nullptr, 0, d, blocks, warps, status, (cudaStream_t)stream);
 }
 
 int nm_admm_project(const float* W, const float* U, int out, int in, int n, int m, int bits, float* Z,
@@ -968,7 +1207,7 @@ int nm_admm_project(const float* W, const float* U, int out, int in, int n, int 
     int warps = std::max(nm::kPackMinWarps, 1 << d.wpr_log2);
     int rows_per_block = warps >> d.wpr_log2;
     unsigned blocks = (unsigned)((out + rows_per_block - 1) / rows_per_block);
-    return nm::launch(nm::pick_kernel<true>(n, m, bits, warps), nullptr, 0, d, blocks, warps, status,
+    return nm::launch(nm::pick_kernel<true>(n, m, bits, warps, blocks), nullptr, 0, d, blocks, warps, status,
                       (cudaStream_t)stream, Z, U_next);
 }
 
@@ -985,7 +1224,7 @@ int nm_project_pack_grouped(const float* W, const float* U, int out, int in, int
     int warps = std::max(nm::kPackMinWarps, 1 << d.wpr_log2);
     int rows_per_block = warps >> d.wpr_log2;
     unsigned blocks = (unsigned)((out + rows_per_block - 1) / rows_per_block);
-    return nm::launch(nm::pick_kernel(n, m, bits, warps), nullptr, 0, d, blocks, warps, status, (cudaStream_t)stream,
+    return nm::launch(nm::pick_kernel(n, m, bits, warps, blocks), nullptr, 0, d, blocks, warps, status, (cudaStream_t)stream,
                       nullptr, nullptr, nullptr, nm::kGroupScalesGiven, group_rows);
 }
 
@@ -1003,7 +1242,7 @@ int nm_admm_project_grouped(const float* W, const float* U, int out, int in, int
     int warps = std::max(nm::kPackMinWarps, 1 << d.wpr_log2);
     int rows_per_block = warps >> d.wpr_log2;
     unsigned blocks = (unsigned)((out + rows_per_block - 1) / rows_per_block);
-    return nm::launch(nm::pick_kernel<true>(n, m, bits, warps), nullptr, 0, d, blocks, warps, status,
+    return nm::launch(nm::pick_kernel<true>(n, m, bits, warps, blocks), nullptr, 0, d, blocks, warps, status,
                       (cudaStream_t)stream, Z, U_next, nullptr, nm::kGroupScalesGiven, group_rows);
 }
 
@@ -1035,7 +1274,7 @@ int nm_project_pack_dist(const float* W, const float* U, int out, int in, int n,
     int warps = std::max(nm::kPackMinWarps, 1 << d.wpr_log2);
     int rows_per_block = warps >> d.wpr_log2;
     unsigned blocks = (unsigned)((out + rows_per_block - 1) / rows_per_block);
-    return nm::launch(nm::pick_kernel(n, m, bits, warps), nullptr, 0, d, blocks, warps, status, (cudaStream_t)stream,
+    return nm::launch(nm::pick_kernel(n, m, bits, warps, blocks), nullptr, 0, d, blocks, warps, status, (cudaStream_t)stream,
                       nullptr, nullptr, nullptr, nm::kGroupScalesGiven, 0);
 }
 
@@ -1054,7 +1293,7 @@ int nm_admm_project_dist(const float* W, const float* U, int out, int in, int n,
     int warps = std::max(nm::kPackMinWarps, 1 << d.wpr_log2);
     int rows_per_block = warps >> d.wpr_log2;
     unsigned blocks = (unsigned)((out + rows_per_block - 1) / rows_per_block);
-    return nm::launch(nm::pick_kernel<true>(n, m, bits, warps), nullptr, 0, d, blocks, warps, status,
+    return nm::launch(nm::pick_kernel<true>(n, m, bits, warps, blocks), nullptr, 0, d, blocks, warps, status,
                       (cudaStream_t)stream, Z, U_next, nullptr, nm::kGroupScalesGiven, 0);
 }
 

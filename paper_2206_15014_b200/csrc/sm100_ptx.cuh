@@ -67,6 +67,16 @@ __device__ __forceinline__ void tma_load_3d(uint32_t dst, const void* tmap, int 
         "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
         ::"r"(dst), "l"((uint64_t)tmap), "r"(c0), "r"(c1), "r"(c2), "r"(bar) : "memory");
 }
+// Untiled bulk copy global -> shared (both addresses 16-byte aligned, `bytes` a multiple of 16), completion
+// counted in bytes on `bar`.
+__device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(dst), "l"((uint64_t)src), "r"(bytes), "r"(bar) : "memory");
+}
+// Asks for `bytes` (a multiple of 16) from a 16-byte aligned global address to be brought into L2.
+__device__ __forceinline__ void bulk_prefetch_l2(const void* src, uint32_t bytes) {
+    asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"((uint64_t)src), "r"(bytes) : "memory");
+}
 // 2-D tiled store shared -> global (bulk async group of the issuing thread).  Rows/columns of the
 // box that fall outside the tensor are clipped by the hardware.
 __device__ __forceinline__ void tma_store_2d(const void* tmap, int c0, int c1, uint32_t src) {
