@@ -434,6 +434,27 @@ def extra_configs(nm, torch, dev, pk, status):
     return out
 
 
+def ffn1_stream_probe(nm, torch, dev, d, tokens, status):
+    """The resident-weight pair kernel's traffic on one GEMM without its arithmetic (nm_probe_tma_stream): X loads
+    through the ring + Y stores, and Y stores alone.  Times from the CTAs' own globaltimer stamps, median of three."""
+    import numpy as np
+    clocks = torch.zeros((148, 4), dtype=torch.int64, device=dev)
+    out, k = d["out"], d["k"]
+    res = {}
+    for name, loads, stores in (("loads_and_stores_us", 2, 1), ("stores_only_us", 0, 1)):
+        spans = []
+        for _ in range(4):
+            ctas = nm.nm_probe_tma_stream(d["values"], out, k // 2, d["X"], tokens, k, d["Y"], 128, 128, 96, 2, 5, 0, 1, 0,
+                                          loads, stores, 1, 0, clocks, None, status)
+            torch.cuda.synchronize()
+            c = clocks[:ctas].cpu().numpy()
+            spans.append(float(c[:, 3].max() - c[:, 2].min()) / 1e3)
+        res[name] = float(np.median(spans[1:]))
+    ybytes = tokens * out * 4
+    res["stores_only_gbs"] = ybytes / res["stores_only_us"] / 1e3
+    return res
+
+
 def run_cuda(args):
     TOKENS = args.tokens
     PATTERN = (2, 4, args.bits)
@@ -610,7 +631,7 @@ def run_cuda(args):
         pack_info = pack_sweep(nm, torch, dev, status)
     # ---- the dominant GEMMs launched alone, back to back over rotating buffers; write-only bandwidth of the device ------
     alone = {}
-    write_gbs = None
+    stream_probe = None
     if rank == 0:
         for d in devbuf:
             Ys = [d["Y"]] + [torch.empty_like(d["Y"]) for _ in range(2)]
@@ -629,9 +650,11 @@ def run_cuda(args):
             sets.append(nm.make_pack_jobs([(W, U, n, m, bits, d["values"], d["meta"], d["scales"]) for (W, U), d in zip(cp, devbuf)]))
         alone["pack"] = time_stream(torch, lambda i: nm.nm_project_pack_batched(sets[i % 3], len(devbuf), ws, ws_bytes, status), 100)
         del sets, extra
-        fill = torch.empty(1 << 30, dtype=torch.uint8, device=dev)
-        write_gbs = (1 << 30) / time_stream(torch, lambda i: fill.zero_(), 10, warm=2) / 1e3
-        del fill
+        # what FFN1's byte stream costs with no arithmetic: the library's traffic probe walks the same tiles in the same
+        # order with the same TMA operations (X through a five-stage ring, Y in [16 tokens][32 channels] boxes) --
+        # stores alone, and loads + stores.  fp32 outputs and 8-bit weights only (the probe's tile is that kernel's).
+        if args.out == "f32" and bits == 8:
+            stream_probe = ffn1_stream_probe(nm, torch, dev, next(d for d in devbuf if d["name"] == "ffn1"), TOKENS, status)
         torch.cuda.empty_cache()
     extras = None
     if rank == 0 and not args.skip_configs and TOKENS == 16384 and bits == 8 and args.out == "f32":
@@ -661,24 +684,24 @@ def run_cuda(args):
                                     "frac_hbm_launched_alone": pbytes / alone["pack"] / 1e3 / pk["hbm_gbs"]}
         if pack_info:
             per_kernel["pack_sweep"] = pack_info
-        # dominant kernel of the step: the FFN1 GEMM launch (longest).  Its bytes are 93 % fp32 Y written; a plain fill of
-        # 1 GiB on the same device gives the write-only rate such a kernel can reach (`write_only_gbs`, below the copy
-        # figure that `peak` is).  `traffic` = dram__bytes_read.sum + dram__bytes_write.sum of one launch at this size
+        # dominant kernel of the step: the FFN1 GEMM launch (longest).  Its bytes are 93 % fp32 Y written in tiles of
+        # 128 channels x 192 tokens; `stream_probe` says what that byte stream costs on this device with no arithmetic
+        # (`frac_of_stream_probe` = probe time / kernel time launched alone).  `traffic` = dram__bytes_read.sum + dram__bytes_write.sum of one launch at this size
         # (ncu; part of Y is still in the 126 MB L2 when the kernel ends, hence below the algorithmic bytes).
         dom = per_kernel["ffn1"]
-        k1 = f"nm_gemm_pair_kernel<sparse,192,{args.out},resident>" if bits == 8 else f"nm_gemm_kernel<sparse,192,{args.out},build-resident>"
-        if bits != 8:
-            k2 = f"nm_gemm_kernel<sparse,192,{args.out},build-per-k-block>"
-        elif args.out == "f32":
-            k2 = "nm_gemm_wide_kernel<224,f32>"
-        else:
+        k1 = f"nm_gemm_pair_kernel<sparse,192,{args.out},resident" + (">" if bits == 8 else ",builder warps>")
+        if args.out == "f32":
+            k2 = "nm_gemm_wide_kernel<224,f32" + (">" if bits == 8 else ",packed 4-bit codes>")
+        elif bits == 8:
             k2 = f"nm_gemm_pair_kernel<sparse,192,{args.out},streamed>"
+        else:
+            k2 = f"nm_gemm_kernel<sparse,192,{args.out},build-per-k-block>"
         roofline = {"kernel": k1 + " on ffn1 1024->4096", "bound": "hbm",
                     "achieved": dom["gbs"], "peak": pk["hbm_gbs"], "unit": "GB/s",
                     "frac": dom["gbs"] / pk["hbm_gbs"], "traffic": traffic.get("ffn1") if full_size else None,
                     "algorithmic_bytes": gemm_bytes(TOKENS, 1024, 4096, n, m, bits, YB), "peak_source": pk["source"],
-                    "write_only_gbs": write_gbs,
-                    "frac_of_write_only": dom["gbs"] / write_gbs if write_gbs else None}
+                    "stream_probe": stream_probe,
+                    "frac_of_stream_probe": (stream_probe["loads_and_stores_us"] / alone["ffn1"]) if stream_probe else None}
         f2 = per_kernel["ffn2"]
         roofline_tensor = {"kernel": k2 + " on ffn2 4096->1024", "bound": "tensor",
                            "achieved": f2["tops"], "peak": sparse_peak, "unit": "TOP/s",
@@ -921,6 +944,10 @@ def tma_probe(args):
     # then 8 KB boxes 32, 64 and 128 channels wide
     for stores in (1, 32, 64, 128):
         case("stores only, 512x256 tiles", OUT, K, T, 256, 64, 128, 1, 5, loads=0, stores=stores)
+    # FFN1 (1024 -> 4096), where the weights stay in shared memory: the ring carries X only and Y is four times as large
+    for loads, stores in ((2, 1), (2, 0), (0, 1)):
+        case("ffn1 resident-weight tile 256x192 (X loads only)", 4096, 1024, T, 128, 128, 96, 2, 5, loads=loads, stores=stores)
+    case("ffn1 resident-weight tile 256x192, stage held 640 clk", 4096, 1024, T, 128, 128, 96, 2, 5, loads=2, delay=640)
     # everything resident in L2: a small problem walked five times
     case("L2-resident 256x192", OUT, K, 19 * 192, 128, 128, 96, 2, 5, repeat=5, stores=0, producers=2)
     case("L2-resident 512x224", OUT, K, 37 * 224, 256, 64, 112, 1, 6, repeat=5, stores=0, producers=2)
@@ -972,6 +999,9 @@ def trace_gemm(args):
         row = {"tile": i, "accumulator_full": int(tl[i, 0] - t0), "epilogue_done": int(tl[i, 1] - t0)}
         if tl[i, 2] > 0:
             row.update(second_accumulator_full=int(tl[i, 2] - t0), second_epilogue_done=int(tl[i, 3] - t0))
+        elif tl[i, 3:8].sum() > 0:   # the 256-channel pair kernel: the first epilogue warp's phases, summed over the tile
+            row["epilogue_warp0_clk"] = dict(zip(["accumulator_chunk_wait", "staging_free_wait", "convert_and_fill", "proxy_fence", "store_issue"],
+                                                 (int(x) for x in tl[i, 3:8])))
         tiles.append(row)
     print(json.dumps({"shape": [T, K, OUT], "status": rc, "stages_of_cta0": n,
                       "producer_issue_clk": med((d[:, 1] - d[:, 0])[ok]), "load_issue_to_full_clk": med((d[:, 2] - d[:, 1])[ok]),

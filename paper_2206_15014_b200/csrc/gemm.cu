@@ -146,9 +146,19 @@ constexpr int kTraceStages = 512, kTraceTiles = 64;
 #ifdef NM_TRACE
 #define NM_TRACE_STAGE(it, col) do { if (p.trace && blockIdx.x == 0 && (it) < (uint32_t)kTraceStages) p.trace[8 * (size_t)(it) + (col)] = clock64(); } while (0)
 #define NM_TRACE_TILE(i, col) do { if (p.trace && blockIdx.x == 0 && (i) < kTraceTiles) p.trace[8 * (size_t)(kTraceStages + (i)) + (col)] = clock64(); } while (0)
+// Phases of the first epilogue warp's work on a tile, summed per tile into columns 3..7 of the tile's row: waiting for the
+// accumulator chunk, waiting for the staging tile to be free, converting and filling it, the proxy fence, issuing the store.
+#define NM_TRACE_EPI_DECL long long tr_t = clock64(), tr_acc[5] = {0, 0, 0, 0, 0}
+#define NM_TRACE_EPI_MARK() do { tr_t = clock64(); } while (0)
+#define NM_TRACE_EPI_ADD(k) do { const long long tr_now = clock64(); tr_acc[k] += tr_now - tr_t; tr_t = tr_now; } while (0)
+#define NM_TRACE_EPI_FLUSH(i) do { if (p.trace && blockIdx.x == 0 && (i) < kTraceTiles) { for (int k = 0; k < 5; ++k) { p.trace[8 * (size_t)(kTraceStages + (i)) + 3 + k] = tr_acc[k]; tr_acc[k] = 0; } } } while (0)
 #else
 #define NM_TRACE_STAGE(it, col) do { } while (0)
 #define NM_TRACE_TILE(i, col) do { } while (0)
+#define NM_TRACE_EPI_DECL do { } while (0)
+#define NM_TRACE_EPI_MARK() do { } while (0)
+#define NM_TRACE_EPI_ADD(k) do { } while (0)
+#define NM_TRACE_EPI_FLUSH(i) do { } while (0)
 #endif
 
 template <bool SPARSE, int BN, bool RESIDENT = false>
@@ -897,6 +907,7 @@ nm_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_con
             if (lane == 0) ptx::mbar_arrive_cluster(ptx::map_to_cta(acc_empty_bar(buf), 0));
         };
 
+        NM_TRACE_EPI_DECL;
         for (int i = 0; i < tile_count && ok; ++i) {
             const TileCoord tc = tile_coord(tile_begin + i, p.n_tok_tiles, p.n_out_tiles, p.band);
             const int out_tile = tc.o, tok_tile = tc.t, buf = i & 1;
@@ -909,6 +920,7 @@ nm_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_con
             if (!ok) break;
             ptx::tc_fence_after();
             if (ew == 0 && lane == 0) NM_TRACE_TILE(i, 0);
+            NM_TRACE_EPI_MARK();
             // the next tile starts a new output tile: its metadata can go in now, the MMAs of this one are done
             if (SPARSE && half == 0 && i + 1 < tile_count) {
                 const int next_out_tile = tile_coord(tile_begin + i + 1, p.n_tok_tiles, p.n_out_tiles, p.band).o;
@@ -933,6 +945,7 @@ nm_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_con
                 if (c < nact) {
                     if (RB == 1) ptx::tmem_ld_32x32(lane_taddr + buf * BN + c * 32, r[0]);
                     ptx::tmem_ld_wait();
+                    NM_TRACE_EPI_ADD(0);
                     if (c + EWH >= nact) release_acc(buf);
                     else if (RB == 2) ptx::tmem_ld_32x32(lane_taddr + buf * BN + (c + EWH) * 32, r[(ci + 1) & (RB - 1)]);
                     const int jmax = n_ok ? min(32, p.tokens - tc0) : 0;  // outputs of this lane that exist
@@ -980,14 +993,18 @@ nm_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_con
                                 OT* sb = reinterpret_cast<OT*>(my_stage + (NB == 2 ? (n_stores & 1u) * 512 : 0));
                                 if (lane == 0) ptx::bulk_wait_group_read<NB - 1>();  // the store that last used this tile has read it
                                 __syncwarp();
+                                NM_TRACE_EPI_ADD(1);
 #pragma unroll
                                 for (int j = 0; j < 16; ++j) sb[j * 32 + lane] = conv(16 * h + j);
+                                NM_TRACE_EPI_ADD(2);
                                 ptx::fence_proxy_async_smem();
                                 __syncwarp();
+                                NM_TRACE_EPI_ADD(3);
                                 if (lane == 0) {
                                     ptx::tma_store_2d(&tmap_y, n0 + q * 32, tc0 + 16 * h, ptx::smem_u32(sb));
                                     ptx::bulk_commit_group();
                                 }
+                                NM_TRACE_EPI_ADD(4);
                                 ++n_stores;
                             }
                         }
@@ -1001,7 +1018,7 @@ nm_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_con
                     }
                 }
             }
-            if (ew == 0 && lane == 0) NM_TRACE_TILE(i, 1);
+            if (ew == 0 && lane == 0) { NM_TRACE_TILE(i, 1); NM_TRACE_EPI_FLUSH(i); }
         }
         if (lane == 0) ptx::bulk_wait_group<0>();
         if (EPI == EPI_F32 && p.absmax) {
