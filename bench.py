@@ -975,10 +975,18 @@ def trace_gemm(args):
     status = torch.zeros(1, dtype=torch.int32, device=dev)
     desc = nm.make_packed(OUT, K, 2, 4, args.bits, vals, meta)
     trace = torch.zeros((576, 8), dtype=torch.int64, device=dev)
+    if args.out == "int8":
+        Y = torch.empty((T, OUT), dtype=torch.int8, device=dev)
+        run = lambda: nm.nm_int_linear_q8(X, T, desc, 0.01, sw, b, 0.05, Y, status=status)
+    elif args.out == "bf16":
+        Y = torch.empty((T, OUT), dtype=torch.bfloat16, device=dev)
+        run = lambda: nm.nm_int_linear_bf16(X, T, desc, 0.01, sw, b, Y, status=status)
+    else:
+        run = lambda: nm.nm_int_linear(X, T, desc, 0.01, sw, b, Y, status=status)
     for _ in range(3):
-        nm.nm_int_linear(X, T, desc, 0.01, sw, b, Y, status=status)
+        run()
     nm.nm_debug_set_trace(trace)
-    nm.nm_int_linear(X, T, desc, 0.01, sw, b, Y, status=status)
+    run()
     torch.cuda.synchronize()
     nm.nm_debug_set_trace(None)
     rc = nm.nm_poll_status(status)

@@ -77,6 +77,9 @@ __device__ __forceinline__ uint8_t epi_convert_q8_fast(uint32_t acc, float c_n, 
     return (uint8_t)(int8_t)code;
 }
 
+// The exact quantiser as a call: the repair of near-ties runs for a few values in 10^5, its code stays out of the loops.
+__device__ __noinline__ int quantise8_exact_call(float y, float sy) { return quantise8_exact(y, sy); }
+
 template <int EPI> constexpr bool kNarrow = EPI == EPI_Q8 || EPI == EPI_BF16;
 constexpr uint32_t kNarrowFree = 9, kNarrowFull = 11, kNarrowAgree = 13;
 
@@ -490,11 +493,13 @@ nm_gemm_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant
             const int nact = min(CH, (p.tokens - t0 + 31) >> 5);  // chunks that hold tokens (warp-uniform)
             // Accumulator chunks are read one ahead of their conversion (two register buffers); the
             // transform kernels, short of registers with their extra warps, read each chunk when it is due.
-            constexpr int RB = XF ? 1 : 2;
+            // narrow outputs: the conversion code of one chunk is long; the chunk loop stays a loop (one copy of that code
+            // instead of CI, which no longer fit the instruction cache) and every chunk is read when it is due
+            constexpr int RB = (XF || kNarrow<EPI>) ? 1 : 2;
             uint32_t r[RB][32];
             if (half >= nact) release_acc(buf);
             else if (RB == 2) ptx::tmem_ld_32x32(lane_taddr + buf * BN + half * 32, r[0]);
-#pragma unroll
+#pragma unroll (kNarrow<EPI> ? 1 : CI)
             for (int ci = 0; ci < CI; ++ci) {
                 const int c = half + ci * EWH, tc0 = t0 + c * 32;
                 if (c < nact) {
@@ -531,10 +536,12 @@ nm_gemm_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant
                                         sb[j * 128 + q * 32 + lane] = epi_convert_q8_fast(r[ci & (RB - 1)][16 * h + j], c_n, b_n, rsy, j, y_tie, j_tie, n_tie);
                                     if (__any_sync(0xffffffffu, n_tie != 0)) {  // rare (3 % of these tiles): repair with the exact division
                                         if (n_tie == 1) {
-                                            sb[j_tie * 128 + q * 32 + lane] = (uint8_t)(int8_t)quantise8_exact(y_tie, p.sy);
+                                            sb[j_tie * 128 + q * 32 + lane] = (uint8_t)(int8_t)quantise8_exact_call(y_tie, p.sy);
                                         } else if (n_tie > 1) {
 #pragma unroll
-                                            for (int j = 0; j < 16; ++j) sb[j * 128 + q * 32 + lane] = conv(16 * h + j);
+                                            for (int j = 0; j < 16; ++j)
+                                                sb[j * 128 + q * 32 + lane] = (uint8_t)(int8_t)quantise8_exact_call(
+                                                    __fmaf_rn((float)(int)r[ci & (RB - 1)][16 * h + j], c_n, b_n), p.sy);
                                         }
                                     }
                                 } else {
@@ -935,11 +942,11 @@ nm_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_con
             const int nact = min(CH, (p.tokens - t0 + 31) >> 5);
             // chunks are read one ahead of their conversion; with the builder warps present registers are short and
             // every chunk is read when it is due
-            constexpr int RB = BUILD ? 1 : 2;
+            constexpr int RB = (BUILD || kNarrow<EPI>) ? 1 : 2;  // narrow outputs: see the one-CTA kernel
             uint32_t r[RB][32];
             if (half >= nact) release_acc(buf);
             else if (RB == 2) ptx::tmem_ld_32x32(lane_taddr + buf * BN + half * 32, r[0]);
-#pragma unroll
+#pragma unroll (kNarrow<EPI> ? 1 : CI)
             for (int ci = 0; ci < CI; ++ci) {
                 const int c = half + ci * EWH, tc0 = t0 + c * 32;
                 if (c < nact) {
@@ -964,6 +971,7 @@ nm_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_con
                                 OT* sb = reinterpret_cast<OT*>(store_stage) + (half * 2 + (n_stores & 1u)) * (16 * 128);
                                 if (q == 0 && lane == 0) ptx::bulk_wait_group_read<1>();  // the store before the last has read this tile
                                 ptx::named_bar_sync(kNarrowFree + half, 128);
+                                NM_TRACE_EPI_ADD(1);
                                 if constexpr (EPI == EPI_Q8) {
                                     float y_tie = 0.0f;
                                     int j_tie = 0, n_tie = 0;
@@ -972,22 +980,27 @@ nm_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_con
                                         sb[j * 128 + q * 32 + lane] = epi_convert_q8_fast(r[ci & (RB - 1)][16 * h + j], c_n, b_n, rsy, j, y_tie, j_tie, n_tie);
                                     if (__any_sync(0xffffffffu, n_tie != 0)) {  // rare (3 % of these tiles): repair with the exact division
                                         if (n_tie == 1) {
-                                            sb[j_tie * 128 + q * 32 + lane] = (uint8_t)(int8_t)quantise8_exact(y_tie, p.sy);
+                                            sb[j_tie * 128 + q * 32 + lane] = (uint8_t)(int8_t)quantise8_exact_call(y_tie, p.sy);
                                         } else if (n_tie > 1) {
 #pragma unroll
-                                            for (int j = 0; j < 16; ++j) sb[j * 128 + q * 32 + lane] = conv(16 * h + j);
+                                            for (int j = 0; j < 16; ++j)
+                                                sb[j * 128 + q * 32 + lane] = (uint8_t)(int8_t)quantise8_exact_call(
+                                                    __fmaf_rn((float)(int)r[ci & (RB - 1)][16 * h + j], c_n, b_n), p.sy);
                                         }
                                     }
                                 } else {
 #pragma unroll
                                     for (int j = 0; j < 16; ++j) sb[j * 128 + q * 32 + lane] = conv(16 * h + j);
                                 }
+                                NM_TRACE_EPI_ADD(2);
                                 ptx::fence_proxy_async_smem();
                                 ptx::named_bar_sync(kNarrowFull + half, 128);
+                                NM_TRACE_EPI_ADD(3);
                                 if (q == 0 && lane == 0) {
                                     ptx::tma_store_2d(&tmap_y, n0, tc0 + 16 * h, ptx::smem_u32(sb));
                                     ptx::bulk_commit_group();
                                 }
+                                NM_TRACE_EPI_ADD(4);
                                 ++n_stores;
                             } else {
                                 OT* sb = reinterpret_cast<OT*>(my_stage + (NB == 2 ? (n_stores & 1u) * 512 : 0));

@@ -76,6 +76,32 @@ def test_int8_chain_of_two_layers():
     assert np.array_equal(gacc2, acc2) and np.array_equal(gY2, Y2)
 
 
+@pytest.mark.parametrize("T,K,out", [(300, 4096, 128), (8960, 1024, 512), (8960, 4096, 512)])
+@pytest.mark.parametrize("n,m,bits", [(2, 4, 8), (4, 4, 8), (2, 4, 4)])
+def test_accumulators_from_zero_to_the_largest(n, m, bits, T, K, out):
+    """Constant rows of X against all-ones weights give every token its own accumulator value, from 0 up to the
+    largest the operands allow (beyond 2^22 and 2^24 in magnitude for 8-bit codes, where int -> float rounds): fp32,
+    int8 and bfloat16 outputs bit for bit on the one-CTA, resident-weight pair and 512-channel pair kernels."""
+    from gpu_util import PackedOnDevice, gpu_int_linear, gpu_int_linear_q8, gpu_int_linear_bf16
+    oracle.set_threads(oracle.max_threads())
+    W = np.ones((out, K), np.float32)
+    b = wl.normal(np.random.default_rng(31), (out,), 0.5)
+    v, meta, s = oracle.project_pack(W, None, n, m, bits)
+    D = oracle.unpack(v, meta, out, K, n, m, bits)
+    c = ((np.arange(T) * 37) % 256 - 128).astype(np.int8)
+    Xq = np.repeat(c[:, None], K, axis=1)
+    sx = np.float32(2e-4)
+    acc_ref, Y = oracle.int_linear(Xq, D, sx, s, b)
+    if bits == 8:
+        assert np.abs(acc_ref).max() > (1 << 22)
+    packed = PackedOnDevice(v, meta, s, out, K, n, m, bits)
+    acc, Yg = gpu_int_linear(Xq, packed, sx, b)
+    assert np.array_equal(acc, acc_ref) and np.array_equal(Yg, Y)
+    sy = np.float32(np.abs(Y).max()) / np.float32(127.0)
+    assert np.array_equal(gpu_int_linear_q8(Xq, packed, sx, b, sy), oracle.requantize_static(Y, sy))
+    assert np.array_equal(gpu_int_linear_bf16(Xq, packed, sx, b), oracle.to_bf16(Y))
+
+
 def test_narrow_outputs_reject_bad_arguments():
     import torch
     import paper_2206_15014_b200 as nm
