@@ -727,6 +727,7 @@ nm_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_con
             uint32_t it = 0, free_parity = 1u;  // nothing reads the resident region before the first load
             int prev_out_tile = -1;
             bool ok = true;
+            const uint64_t keep = ptx::policy_evict_last();  // X is read again for every output tile
             for (int i = 0; i < tile_count && ok; ++i) {
                 const int tile = tile_begin + i;
                 const TileCoord tc = tile_coord(tile, p.n_tok_tiles, p.n_out_tiles, p.band);
@@ -756,7 +757,7 @@ nm_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_con
                     if (leader) ptx::mbar_expect_tx(full_bar(s), 2 * Cfg::STAGE);  // bytes of both CTAs
                     if (!RES) ptx::tma_load_2d_pair(a_dst, &tmap_w, kb * Cfg::A_ROW, n0, lead_full);
                     // X is mapped as [k-slice][token][128 bytes]: both slices of the stage in one operation
-                    ptx::tma_load_3d_pair(a_dst + Cfg::B_OFF, &tmap_x, 0, t0, kb * (Cfg::KB / 128), lead_full);
+                    ptx::tma_load_3d_pair_hint(a_dst + Cfg::B_OFF, &tmap_x, 0, t0, kb * (Cfg::KB / 128), lead_full, keep);
                     NM_TRACE_STAGE(it, 1);
                 }
             }
@@ -913,6 +914,7 @@ nm_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_con
             __syncwarp();
             if (lane == 0) ptx::mbar_arrive_cluster(ptx::map_to_cta(acc_empty_bar(buf), 0));
         };
+        const uint64_t stream_out = ptx::policy_evict_first();  // Y is written once and not read here
 
         NM_TRACE_EPI_DECL;
         for (int i = 0; i < tile_count && ok; ++i) {
@@ -1014,7 +1016,7 @@ nm_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_con
                                 __syncwarp();
                                 NM_TRACE_EPI_ADD(3);
                                 if (lane == 0) {
-                                    ptx::tma_store_2d(&tmap_y, n0 + q * 32, tc0 + 16 * h, ptx::smem_u32(sb));
+                                    ptx::tma_store_2d_hint(&tmap_y, n0 + q * 32, tc0 + 16 * h, ptx::smem_u32(sb), stream_out);
                                     ptx::bulk_commit_group();
                                 }
                                 NM_TRACE_EPI_ADD(4);

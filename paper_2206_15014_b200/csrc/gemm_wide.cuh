@@ -133,6 +133,7 @@ nm_gemm_wide_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_con
         // ------------------------------ TMA producer (both CTAs) --------------------------------
         if (lane == 0) {
             uint32_t it = 0, parity = 1u;  // the first pass over the ring finds every stage free
+            const uint64_t keep = ptx::policy_evict_last();  // weights and X are read again by other pairs
             int s = 0;
             bool ok = true;
             const uint32_t smem0 = ptx::smem_u32(smem);
@@ -148,8 +149,8 @@ nm_gemm_wide_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_con
                     if (NM_SKIP_STAGE(it)) { if (++s == S) { s = 0; parity ^= 1u; } continue; }
                     const uint32_t dst = smem0 + (uint32_t)s * Cfg::STAGE, lead_full = lead_full0 + 8u * s;
                     if (leader) ptx::mbar_expect_tx(full_bar(s), 2 * (W4 ? Cfg::B_BYTES : Cfg::STAGE));  // bytes of both CTAs
-                    if (!W4) ptx::tma_load_2d_pair(dst, &tmap_w, kb * Cfg::A_ROW, n0, lead_full);
-                    ptx::tma_load_2d_pair(dst + Cfg::A_BYTES, &tmap_x, kb * 128, t0, lead_full);
+                    if (!W4) ptx::tma_load_2d_pair_hint(dst, &tmap_w, kb * Cfg::A_ROW, n0, lead_full, keep);
+                    ptx::tma_load_2d_pair_hint(dst + Cfg::A_BYTES, &tmap_x, kb * 128, t0, lead_full, keep);
                     NM_TRACE_STAGE(it, 1);
                     if (++s == S) { s = 0; parity ^= 1u; }
                 }
@@ -357,6 +358,7 @@ nm_gemm_wide_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_con
         const int ew = warp - 2, q = warp & 3, blk = ew >> 2;
         const uint32_t acc_taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)blk * BN;
         uint32_t* my_stage = reinterpret_cast<uint32_t*>(store_stage + ew * 4096);
+        const uint64_t stream_out = ptx::policy_evict_first();  // Y is written once and not read here
         const float sx = p.sx_dev ? *p.sx_dev : p.sx_host;
         const uint32_t lead_acc_empty = ptx::map_to_cta(acc_empty_bar(blk), 0);
         float amax = 0.0f, c_n = 0.0f, b_n = 0.0f;
@@ -412,7 +414,7 @@ nm_gemm_wide_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_con
                         ptx::fence_proxy_async_smem();
                         __syncwarp();
                         if (lane == 0) {
-                            ptx::tma_store_2d(&tmap_y, nw, tc0, ptx::smem_u32(my_stage));
+                            ptx::tma_store_2d_hint(&tmap_y, nw, tc0, ptx::smem_u32(my_stage), stream_out);
                             ptx::bulk_commit_group();
                         }
                     } else {
