@@ -63,18 +63,19 @@ template <> struct EpiOut<EPI_BF16> { using type = uint16_t; };
 // group fill together (rows of 128 / 256 bytes instead of 32 / 64): named barriers kNarrowFree + half and
 // kNarrowFull + half order the fills against the one warp that issues the TMA store, kNarrowAgree + half
 // makes the group take a timed-out wait together so that nobody is left alone on a barrier.
-// EPI_Q8 without a branch per value: code from the reciprocal rsy = RN(1 / sy).  A value for which only the
-// exact division decides (within 2^-15 of a rounding tie: 6 in 100000) is remembered in (y_tie, j_tie) and
-// counted; the caller repairs it afterwards with one exact division.
-__device__ __forceinline__ uint8_t epi_convert_q8_fast(uint32_t acc, float c_n, float b_n, float rsy, int j,
-                                                       float& y_tie, int& j_tie, int& n_tie) {
+// EPI_Q8 without a branch per value: the code from the reciprocal rsy = RN(1 / sy), exact unless the product sits
+// within 2^-15 of a rounding tie (6 values in 100000), where only the IEEE division decides.  `worst` keeps the largest
+// distance of a product from its rounded integer over a run of values; beyond 0.49996948 the caller fills the run again
+// with the exact quantiser.  The clamp to [-128.49, 127.49] before the add of 1.5 * 2^23 (whose own rounding rounds to
+// the nearest-even integer) leaves nothing to clamp afterwards, and the low byte of the sum's bit pattern
+// 0x4B400000 + code is the code.
+__device__ __forceinline__ uint8_t epi_convert_q8_fast(uint32_t acc, float c_n, float b_n, float rsy, float& worst) {
+    constexpr float kMagic = 12582912.0f;
     const float y = __fmaf_rn((float)(int)acc, c_n, b_n);
-    bool near_tie = false;
-    const int code = quantise8_fast(y, rsy, near_tie);
-    y_tie = near_tie ? y : y_tie;
-    j_tie = near_tie ? j : j_tie;
-    n_tie += near_tie ? 1 : 0;
-    return (uint8_t)(int8_t)code;
+    const float qc = fminf(fmaxf(__fmul_rn(y, rsy), -128.49f), 127.49f);
+    const float t = __fadd_rn(qc, kMagic);
+    worst = fmaxf(worst, fabsf(__fsub_rn(qc, __fsub_rn(t, kMagic))));
+    return (uint8_t)__float_as_uint(t);
 }
 
 // The exact quantiser as a call: the repair of near-ties runs for a few values in 10^5, its code stays out of the loops.
@@ -529,17 +530,17 @@ nm_gemm_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant
                                 if (q == 0 && lane == 0) ptx::bulk_wait_group_read<1>();  // the store before the last has read this tile
                                 ptx::named_bar_sync(kNarrowFree + half, 128);
                                 if constexpr (EPI == EPI_Q8) {
-                                    float y_tie = 0.0f;
-                                    int j_tie = 0, n_tie = 0;
+                                    float worst = 0.0f;
 #pragma unroll
                                     for (int j = 0; j < 16; ++j)
-                                        sb[j * 128 + q * 32 + lane] = epi_convert_q8_fast(r[ci & (RB - 1)][16 * h + j], c_n, b_n, rsy, j, y_tie, j_tie, n_tie);
-                                    if (__any_sync(0xffffffffu, n_tie != 0)) {  // rare (3 % of these tiles): repair with the exact division
-                                        if (n_tie == 1) {
-                                            sb[j_tie * 128 + q * 32 + lane] = (uint8_t)(int8_t)quantise8_exact_call(y_tie, p.sy);
-                                        } else if (n_tie > 1) {
+                                        sb[j * 128 + q * 32 + lane] = epi_convert_q8_fast(r[ci & (RB - 1)][16 * h + j], c_n, b_n, rsy, worst);
+                                    if (__any_sync(0xffffffffu, !(worst <= 0.49996948f))) {  // rare (3 % of the runs)
+                                        // find the values in question again; the exact division decides those
 #pragma unroll
-                                            for (int j = 0; j < 16; ++j)
+                                        for (int j = 0; j < 16; ++j) {
+                                            float w1 = 0.0f;
+                                            (void)epi_convert_q8_fast(r[ci & (RB - 1)][16 * h + j], c_n, b_n, rsy, w1);
+                                            if (!(w1 <= 0.49996948f))
                                                 sb[j * 128 + q * 32 + lane] = (uint8_t)(int8_t)quantise8_exact_call(
                                                     __fmaf_rn((float)(int)r[ci & (RB - 1)][16 * h + j], c_n, b_n), p.sy);
                                         }
@@ -612,6 +613,12 @@ nm_gemm_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant
 constexpr int kPairThreads = 32 * (3 + kEpiWarps);
 constexpr int kPairBuildWarps = 8;  // two groups of four (one thread per weight row of the CTA) taking alternate 128-wide k-blocks
 template <bool BUILD> constexpr int kPairThreadsOf = kPairThreads + (BUILD ? 32 * kPairBuildWarps : 0);
+// Narrow outputs from resident weights: the epilogue sets the pace there and is a chain of waits (accumulator read, staging
+// tile, fence, store issue) that eight warps do not overlap; sixteen epilogue warps in four groups take 16-token units.
+// The second eight sit behind the gate warp, where the builder warps of the BUILD form are.
+template <int EPI, bool RES, bool BUILD> constexpr int kPairEpiWarps = (kNarrow<EPI> && RES && !BUILD) ? 16 : kEpiWarps;
+template <int EPI, bool RES, bool BUILD> constexpr int kPairThreadsFor = kPairThreadsOf<BUILD> + 32 * (kPairEpiWarps<EPI, RES, BUILD> - kEpiWarps);
+constexpr uint32_t kNarrowGroup = 9;  // named barriers 9-12: one per group of four epilogue warps in that form
 constexpr int kPairMaxStages = 7;   // the relay cycles through 8 named barriers (ids 1-8; 9-14 serve the narrow-output epilogue)
 
 constexpr int kPairResStages = 4;   // stages of weights a CTA can keep resident (1024 reduction elements at 2:4)
@@ -650,13 +657,13 @@ struct PairCfg {
 // region once per output tile (xform.cuh: widening, placement into 2-of-4 slots), and the metadata warps derive the
 // hardware metadata from the canonical one; everything else is the resident-weight kernel.
 template <bool SPARSE, int BN, int EPI, bool RES, bool BUILD = false>
-__global__ void __launch_bounds__(kPairThreadsOf<BUILD>, 1)
+__global__ void __launch_bounds__(kPairThreadsFor<EPI, RES, BUILD>, 1)
 nm_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant__ CUtensorMap tmap_x,
                     const __grid_constant__ CUtensorMap tmap_y, const GemmParams p,
                     const __grid_constant__ PairSchedule sched) {
     using Cfg = PairCfg<SPARSE, BN, RES>;
     constexpr int S = Cfg::STAGES;
-    constexpr int EW = kEpiWarps, kGateWarp = 2 + EW;
+    constexpr int EW = kPairEpiWarps<EPI, RES, BUILD>, kGateWarp = 2 + kEpiWarps;
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
     uint8_t* a_res = smem + S * Cfg::STAGE;  // resident weight rows: kPairResStages stages of A_BYTES
@@ -878,7 +885,7 @@ nm_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_con
     } else {
         // ------------------------------ metadata + epilogue warps (both CTAs) ----------------------
         constexpr int EWH = EW / 4, CH = BN / 32, CI = (CH + EWH - 1) / EWH;
-        const int ew = warp - 2, q = warp & 3, half = ew >> 2, row = q * 32 + lane;
+        const int ew = warp - 2 - (warp > kGateWarp ? 1 : 0), q = warp & 3, half = ew >> 2, row = q * 32 + lane;
         const uint32_t lane_taddr = tmem_base + ((uint32_t)(q * 32) << 16);
         constexpr int NB = Cfg::STORE_BUFS;
         float* my_stage = reinterpret_cast<float*>(store_stage + ew * (NB * 2048));
@@ -925,7 +932,7 @@ nm_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_con
             bool got = ptx::mbar_wait_bounded(acc_full_bar(buf), (i >> 1) & 1u, abort_flag, kWaitLimit);
             ok = __all_sync(0xffffffffu, got);
             if (!ok && lane == 0) raise_timeout();
-            if constexpr (kNarrow<EPI>) ok = ptx::named_bar_and(kNarrowAgree + half, 128, ok);  // the group stops together
+            if constexpr (kNarrow<EPI>) ok = ptx::named_bar_and(EW == 16 ? kNarrowGroup + half : kNarrowAgree + half, 128, ok);  // the group stops together
             if (!ok) break;
             ptx::tc_fence_after();
             if (ew == 0 && lane == 0) NM_TRACE_TILE(i, 0);
@@ -940,6 +947,75 @@ nm_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_con
                 scaled_out_tile = out_tile;
                 c_n = n_ok ? __fmul_rn(sx, p.sw[n]) : 0.0f;
                 b_n = n_ok && p.bias ? p.bias[n] : 0.0f;
+            }
+            if constexpr (EW == 16) {
+                // Four groups of four warps (one per TMEM lane quarter); group g takes the 16-token units g, g + 4, ... of the
+                // tile: reads 16 accumulator columns, fills its quarter of the group's [16 tokens][128 channels] staging tile
+                // (two per group, used alternately), and the group's warp of lane quarter 0 issues the store.
+                using OT = typename EpiOut<EPI>::type;
+                constexpr int UNITS = BN / 16;
+                const int nunits = min(UNITS, (p.tokens - t0 + 15) >> 4);  // units that hold tokens (the same for the whole group)
+                const uint32_t gbar = kNarrowGroup + half;
+                bool released = false;
+#pragma unroll 1
+                for (int u = half; u < nunits; u += 4) {
+                    const int tc0 = t0 + 16 * u;
+                    uint32_t r[16];
+                    ptx::tmem_ld_32x16(lane_taddr + buf * BN + 16 * u, r);
+                    ptx::tmem_ld_wait();
+                    NM_TRACE_EPI_ADD(0);
+                    if (u + 4 >= nunits) { release_acc(buf); released = true; }
+                    if (p.tma_store) {
+                        OT* sb = reinterpret_cast<OT*>(store_stage) + (half * 2 + (n_stores & 1u)) * (16 * 128);
+                        if (q == 0 && lane == 0) ptx::bulk_wait_group_read<1>();  // the store before the last has read this tile
+                        ptx::named_bar_sync(gbar, 128);
+                        NM_TRACE_EPI_ADD(1);
+                        if constexpr (EPI == EPI_Q8) {
+                            float worst = 0.0f;
+#pragma unroll
+                            for (int j = 0; j < 16; ++j) sb[j * 128 + q * 32 + lane] = epi_convert_q8_fast(r[j], c_n, b_n, rsy, worst);
+                            if (__any_sync(0xffffffffu, !(worst <= 0.49996948f))) {  // rare (3 % of the runs)
+                                // find the values in question again; the exact division decides those
+#pragma unroll
+                                for (int j = 0; j < 16; ++j) {
+                                    float w1 = 0.0f;
+                                    (void)epi_convert_q8_fast(r[j], c_n, b_n, rsy, w1);
+                                    if (!(w1 <= 0.49996948f))
+                                        sb[j * 128 + q * 32 + lane] =
+                                            (uint8_t)(int8_t)quantise8_exact_call(__fmaf_rn((float)(int)r[j], c_n, b_n), p.sy);
+                                }
+                            }
+                        } else {
+#pragma unroll
+                            for (int j = 0; j < 16; ++j) {
+                                float y_abs;
+                                sb[j * 128 + q * 32 + lane] = epi_convert<EPI>(r[j], c_n, b_n, p.sy, rsy, y_abs);
+                            }
+                        }
+                        NM_TRACE_EPI_ADD(2);
+                        ptx::fence_proxy_async_smem();
+                        ptx::named_bar_sync(gbar, 128);
+                        NM_TRACE_EPI_ADD(3);
+                        if (q == 0 && lane == 0) {
+                            ptx::tma_store_2d_hint(&tmap_y, n0, tc0, ptx::smem_u32(sb), stream_out);
+                            ptx::bulk_commit_group();
+                        }
+                        NM_TRACE_EPI_ADD(4);
+                        ++n_stores;
+                    } else {
+                        const int jmax = n_ok ? min(16, p.tokens - tc0) : 0;  // outputs of this lane that exist
+                        OT* dst = reinterpret_cast<OT*>(p.NARROW) + (size_t)tc0 * p.out + n;
+#pragma unroll
+                        for (int j = 0; j < 16; ++j) {
+                            float y_abs;
+                            const OT o = epi_convert<EPI>(r[j], c_n, b_n, p.sy, rsy, y_abs);
+                            if (j < jmax) dst[(size_t)j * p.out] = o;
+                        }
+                    }
+                }
+                if (!released) release_acc(buf);
+                if (ew == 0 && lane == 0) { NM_TRACE_TILE(i, 1); NM_TRACE_EPI_FLUSH(i); }
+                continue;
             }
             const int nact = min(CH, (p.tokens - t0 + 31) >> 5);
             // chunks are read one ahead of their conversion; with the builder warps present registers are short and
@@ -975,17 +1051,17 @@ nm_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_con
                                 ptx::named_bar_sync(kNarrowFree + half, 128);
                                 NM_TRACE_EPI_ADD(1);
                                 if constexpr (EPI == EPI_Q8) {
-                                    float y_tie = 0.0f;
-                                    int j_tie = 0, n_tie = 0;
+                                    float worst = 0.0f;
 #pragma unroll
                                     for (int j = 0; j < 16; ++j)
-                                        sb[j * 128 + q * 32 + lane] = epi_convert_q8_fast(r[ci & (RB - 1)][16 * h + j], c_n, b_n, rsy, j, y_tie, j_tie, n_tie);
-                                    if (__any_sync(0xffffffffu, n_tie != 0)) {  // rare (3 % of these tiles): repair with the exact division
-                                        if (n_tie == 1) {
-                                            sb[j_tie * 128 + q * 32 + lane] = (uint8_t)(int8_t)quantise8_exact_call(y_tie, p.sy);
-                                        } else if (n_tie > 1) {
+                                        sb[j * 128 + q * 32 + lane] = epi_convert_q8_fast(r[ci & (RB - 1)][16 * h + j], c_n, b_n, rsy, worst);
+                                    if (__any_sync(0xffffffffu, !(worst <= 0.49996948f))) {  // rare (3 % of the runs)
+                                        // find the values in question again; the exact division decides those
 #pragma unroll
-                                            for (int j = 0; j < 16; ++j)
+                                        for (int j = 0; j < 16; ++j) {
+                                            float w1 = 0.0f;
+                                            (void)epi_convert_q8_fast(r[ci & (RB - 1)][16 * h + j], c_n, b_n, rsy, w1);
+                                            if (!(w1 <= 0.49996948f))
                                                 sb[j * 128 + q * 32 + lane] = (uint8_t)(int8_t)quantise8_exact_call(
                                                     __fmaf_rn((float)(int)r[ci & (RB - 1)][16 * h + j], c_n, b_n), p.sy);
                                         }
@@ -1225,7 +1301,7 @@ static int launch_gemm_pair(const LinearArgs& a) {
     p.band = cached_pair_plan(p.n_tok_tiles, p.n_out_tiles, pairs, RES, g_opt.band, sched);
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(2 * pairs, 1, 1);
-    cfg.blockDim = dim3(kPairThreadsOf<BUILD>, 1, 1);
+    cfg.blockDim = dim3(kPairThreadsFor<EPI, RES, BUILD>, 1, 1);
     cfg.dynamicSmemBytes = Cfg::SMEM;
     cfg.stream = a.stream;
     cudaLaunchAttribute attr[2];
