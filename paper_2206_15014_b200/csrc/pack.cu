@@ -928,13 +928,20 @@ static PackFn pick_form(int bits) {
 template <int N, int M, bool DENSE_OUT>
 static PackFn pick_bits(int bits, int warps, unsigned blocks) {
     if (warps <= kPackMinWarps) {
-        // Blocks of four warps, persistent.  Staged chunks for the dense-output form (0.83 -> 0.95 of the copy rate on the
-        // 24-layer sweep) and for launches of a few rounds per resident block, where loads and arithmetic of blocks that
-        // start together would otherwise alternate (one layer alone: 26.8 -> 24.7 us); chunks asked for ahead on long
-        // launches, where the staged form's twelve warps per SM are too few (sweep: 0.82 against 0.89).
-        const bool few_rounds = blocks <= 16u * (unsigned)(sm_count() * pack_blocks_per_sm(kStaged2));
-        const int form = g_pack_form == 1 ? kDirect : g_pack_form == 2 ? kStaged2 : g_pack_form == 3 ? kAhead
-                                          : ((DENSE_OUT || few_rounds) ? kStaged2 : kAhead);
+        // Blocks of four warps.  Measured choices (GB/s on the 24-layer sweep, one unit per block / staged / ahead:
+        // 1:4 6231 / 5916 / 6011, 2:4 5520 / 5276 / 5746, 2:8 5643 / 5175 / 5282, 4:8 5090 / 4435 / 5046; one 2:4 layer
+        // alone 26.8 / 24.7 / 25.1 us; 72 matrices in four formats, four launches: 130 / 197 / 156 us; dense outputs on
+        // the sweep 0.83 / 0.95 / 0.60 of the copy rate):
+        //  - dense outputs: staged;
+        //  - 2:4: staged for launches of a few rounds per resident block (blocks that start together otherwise alternate
+        //    between loading and arithmetic), ahead for very long ones, one unit per block between;
+        //  - every other pattern: one unit per block.
+        const unsigned staged_blocks = (unsigned)(sm_count() * pack_blocks_per_sm(kStaged2));
+        const unsigned ahead_blocks = (unsigned)(sm_count() * pack_blocks_per_sm(kAhead));
+        int form = kDirect;
+        if (DENSE_OUT) form = kStaged2;
+        else if (N == 2 && M == 4) form = blocks <= 8u * staged_blocks ? kStaged2 : (blocks >= 32u * ahead_blocks ? kAhead : kDirect);
+        if (g_pack_form >= 1 && g_pack_form <= 3) form = g_pack_form == 1 ? kDirect : g_pack_form == 2 ? kStaged2 : kAhead;
         if (form == kDirect) return pick_form<N, M, DENSE_OUT, kDirect>(bits);
         if (form == kStaged2) return pick_form<N, M, DENSE_OUT, kStaged2>(bits);
         return pick_form<N, M, DENSE_OUT, kAhead>(bits);
