@@ -344,7 +344,9 @@ int nm_probe_tma_stream(const void *W, int w_rows, int w_row_bytes, const void *
  * Results never depend on them.  Returns NM_ERR_UNSUPPORTED for an unknown name.  A library built with
  * -DNM_TEST_HOOKS (build.py --variant shortwait: device-side waits limited to about a millisecond) also takes
  * "skip_stage" = 1 + the pipeline stage that CTA 0's producer leaves unissued (0 = none): the bounded waits then
- * run out, the kernel drains and returns, and nm_poll_status reports NM_ERR_TIMEOUT.
+ * run out, the kernel drains and returns, and nm_poll_status reports NM_ERR_TIMEOUT.  The same build takes
+ * "skip_pack_copy" = 1 + the unit (counted per block) whose bulk copies warp 0 of block 0 of the staged projection
+ * kernel leaves unissued, with the same outcome for the projection entry points.
  */
 int nm_debug_set_option(const char *name /* host */, int value);
 

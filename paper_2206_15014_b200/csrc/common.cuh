@@ -33,6 +33,11 @@ inline size_t meta_row_words(int in, int n, int m) {
 // Form of the projection kernel forced by nm_debug_set_option("pack_form") (0 = automatic).
 extern int g_pack_form;
 
+#ifdef NM_TEST_HOOKS
+// Timeout test only: the unit (per block) whose copies warp 0 of block 0 of the staged projection kernel leaves unissued.
+int pack_set_skip_unit(int unit);
+#endif
+
 // Multiprocessors of the current device (cached per device; 148 when the query fails).
 int sm_count();
 

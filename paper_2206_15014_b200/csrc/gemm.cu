@@ -1513,6 +1513,7 @@ int nm_debug_set_option(const char* name, int value) {
         if (!strcmp(name, e.name)) { *e.slot = value; return NM_OK; }
 #ifdef NM_TEST_HOOKS
     if (!strcmp(name, "skip_stage")) { nm::g_opt.skip_stage = value; return NM_OK; }
+    if (!strcmp(name, "skip_pack_copy")) return nm::pack_set_skip_unit(value - 1);
 #endif
     return NM_ERR_UNSUPPORTED;
 }

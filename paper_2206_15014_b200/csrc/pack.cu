@@ -47,6 +47,20 @@ static constexpr int kPackMinWarps = 4;
 #define NM_WAIT_LIMIT (1ll << 31)
 #endif
 static constexpr long long kPackWaitLimit = NM_WAIT_LIMIT;  // SM clocks a warp waits for its staged chunk (about a second)
+
+// Test hook, compiled in with -DNM_TEST_HOOKS only (the library the timeout test loads, never the product's): in the
+// staged form, warp 0 of block 0 leaves the copies of its unit number `d_pack_skip_unit` (counted per block) unissued --
+// nothing is armed, nothing is copied, no address is touched -- so that the wait for that chunk runs out.
+#ifdef NM_TEST_HOOKS
+__device__ int d_pack_skip_unit = -1;
+int pack_set_skip_unit(int unit) {
+    NM_CUDA_TRY(cudaMemcpyToSymbol(d_pack_skip_unit, &unit, sizeof(unit)));
+    return NM_OK;
+}
+#define NM_PACK_SKIP(iter) (blockIdx.x == 0 && w == 0 && (iter) == d_pack_skip_unit)
+#else
+#define NM_PACK_SKIP(iter) false
+#endif
 // group_mode of pack_kernel: scale per row from the row itself; only fold the row maxima per group into
 // `scales`; take the scales found in `scales`.
 enum { kGroupNone = 0, kGroupMaxPass = 1, kGroupScalesGiven = 2 };
@@ -593,8 +607,9 @@ pack_kernel(const PackJobDev* __restrict__ jobs, int njobs, const __grid_constan
         }
         __syncthreads();
         // every lane calls it; lane 0 issues one bulk copy per operand, completion counted in bytes on the buffer's barrier
-        auto issue = [&](const PackJobDev& j, const UnitPos& up, int buf) {
+        auto issue = [&](const PackJobDev& j, const UnitPos& up, int buf, int iter) {
             if (up.elems == 0) return;      // the same for the whole warp; the unit then waits for nothing
+            if (NM_PACK_SKIP(iter)) return;
             ptx::fence_proxy_async_smem();  // this lane's generic accesses to the buffer before the copy's writes
             __syncwarp();                   // the buffer's last reader is done
             if (lane == 0) {
@@ -612,7 +627,7 @@ pack_kernel(const PackJobDev* __restrict__ jobs, int njobs, const __grid_constan
         if (unit < nunits) {
             job = find_job(jobs, njobs, inl, unit, index);
             up = unit_pos(job, unit, w, warps);
-            issue(job, up, 0);
+            issue(job, up, 0, 0);
         }
         uint32_t phase = 0;  // bit b: parity of buffer b's next completion
         for (int it = 0; unit < nunits; ++it, unit += gridDim.x) {
@@ -625,7 +640,7 @@ pack_kernel(const PackJobDev* __restrict__ jobs, int njobs, const __grid_constan
             if (next < nunits) {
                 if (next - job.unit_begin >= units_of(job, warps)) njob = find_job(jobs, njobs, inl, next, nindex);
                 nup = unit_pos(njob, next, w, warps);
-                issue(njob, nup, buf ^ 1);
+                issue(njob, nup, buf ^ 1, it + 1);
             }
             if constexpr (DENSE_OUT) {
                 if (jobs) { Zout = dense_jobs[index].Z; Unext = dense_jobs[index].U_next; }
@@ -918,6 +933,7 @@ struct PackFn { PackFnPtr fn; int form; };  // kernel and its form (kDirect, kSt
 
 // nm_debug_set_option("pack_form"): 0 = automatic, 1 = kDirect, 2 = kStaged2, 3 = kAhead for blocks of four warps.
 int g_pack_form = 0;
+
 
 template <int N, int M, bool DENSE_OUT, int FORM>
 static PackFn pick_form(int bits) {

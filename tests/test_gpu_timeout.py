@@ -4,7 +4,8 @@ A second build of the library (short wait limits, plus a test hook that makes CT
 stage unissued: nothing armed, nothing in flight, no address touched) runs in a child process; the stage's barrier
 never completes, the gate's wait expires after about a millisecond, the kernel raises NM_STATUS_TIMEOUT, drains and
 returns, and the next call on the same stream matches the oracle.  One case per kernel family that this form has been
-shown to be safe for (the 512-channel pair kernel's case is not run: see timeout_case.py)."""
+shown to be safe for (the 512-channel pair kernel's case is not run: see timeout_case.py), and one for the staged projection
+kernel, where a warp leaves the bulk copies of one chunk unissued and its wait for the chunk expires."""
 import os
 import subprocess
 import sys
@@ -23,7 +24,7 @@ def _shortwait_lib():
     return mod.build(variant="shortwait")
 
 
-@pytest.mark.parametrize("family", ["one_cta", "one_cta_narrow", "pair", "pair_streamed"])
+@pytest.mark.parametrize("family", ["one_cta", "one_cta_narrow", "pair", "pair_streamed", "pack_staged"])
 def test_expired_wait_reports_timeout_and_leaves_the_context_usable(family):
     env = dict(os.environ, NMSPARSE_LIB=_shortwait_lib())
     r = subprocess.run([sys.executable, os.path.join(ROOT, "tests", "timeout_case.py"), family], env=env,

@@ -27,7 +27,45 @@ FAMILIES = {
 }
 
 
+def pack_staged():
+    """The staged projection kernel: warp 0 of block 0 never issues the copies of its second unit; its wait for that
+    chunk expires, the launch reports the time-out, the next call is right."""
+    dev = torch.device("cuda:0")
+    oracle.set_threads(oracle.max_threads())
+    out, k = 2048, 1024                       # 512 units: block 0 of the 444 resident blocks takes units 0 and 444
+    W, U = wl.pack_sweep_matrix(5, 0, out, k)
+    v_ref, meta_ref, s_ref = oracle.project_pack(W, U, 2, 4, 8)
+    td = lambda a: torch.from_numpy(np.ascontiguousarray(a)).to(dev)
+    Wd, Ud = td(W), td(U)
+    vb, mb = nm.nm_packed_sizes(out, k, 2, 4, 8)
+    status = torch.zeros(1, dtype=torch.int32, device=dev)
+
+    def launch():
+        values = torch.zeros(vb, dtype=torch.uint8, device=dev)
+        meta = torch.zeros(mb // 4, dtype=torch.int32, device=dev)
+        scales = torch.zeros(out, dtype=torch.float32, device=dev)
+        nm.nm_project_pack(Wd, Ud, out, k, 2, 4, 8, values, meta, scales, status)
+        return values, meta, scales
+
+    nm.nm_debug_set_option("pack_form", 2)
+    nm.nm_debug_set_option("skip_pack_copy", 2)
+    launch()
+    rc = nm.nm_poll_status(status)
+    assert rc == nm.NM_ERR_TIMEOUT, f"expected a timeout, got {nm.nm_strerror(rc)} {nm.nm_last_cuda_error()}"
+    nm.nm_debug_set_option("skip_pack_copy", 0)
+    status.zero_()
+    values, meta, scales = launch()
+    rc = nm.nm_poll_status(status)
+    assert rc == nm.NM_OK, nm.nm_strerror(rc)
+    assert np.array_equal(values.cpu().numpy().reshape(v_ref.shape), v_ref)
+    assert np.array_equal(meta.cpu().numpy().view(np.uint32).reshape(meta_ref.shape), meta_ref)
+    assert np.array_equal(scales.cpu().numpy(), s_ref), "the call after the timeout does not match the oracle"
+    print("ok pack_staged")
+
+
 def main(family):
+    if family == "pack_staged":
+        return pack_staged()
     T, K, out, options, narrow = FAMILIES[family]
     dev = torch.device("cuda:0")
     oracle.set_threads(oracle.max_threads())
