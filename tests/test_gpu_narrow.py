@@ -16,7 +16,8 @@ pytestmark = pytest.mark.gpu
 MODES = [(2, 4, 8), (4, 4, 8), (2, 4, 4), (1, 4, 8), (2, 8, 8), (4, 8, 8)]
 # (tokens, K, out): one tile; ragged, out % 16 != 0 (plain stores) ; out % 16 == 0 but ragged tokens;
 # many tiles with resident weights and output-tile changes; long reduction with streamed weights
-SHAPES = [(64, 128, 128), (100, 384, 200), (77, 256, 208), (4096 + 37, 512, 1280), (6000 + 3, 2048, 640)]
+# the last one: resident weights on CTA pairs with rows that no TMA store can address (plain stores from sixteen warps)
+SHAPES = [(64, 128, 128), (100, 384, 200), (77, 256, 208), (4096 + 37, 512, 1280), (6000 + 3, 2048, 640), (7680 + 5, 512, 516)]
 
 
 def _setup(seed, T, K, out, n, m, bits):
