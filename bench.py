@@ -696,12 +696,7 @@ def run_cuda(args):
         # (ncu; part of Y is still in the 126 MB L2 when the kernel ends, hence below the algorithmic bytes).
         dom = per_kernel["ffn1"]
         k1 = f"nm_gemm_pair_kernel<sparse,192,{args.out},resident" + (">" if bits == 8 else ",builder warps>")
-        if args.out == "f32":
-            k2 = "nm_gemm_wide_kernel<224,f32" + (">" if bits == 8 else ",packed 4-bit codes>")
-        elif bits == 8:
-            k2 = f"nm_gemm_pair_kernel<sparse,192,{args.out},streamed>"
-        else:
-            k2 = f"nm_gemm_kernel<sparse,192,{args.out},build-per-k-block>"
+        k2 = f"nm_gemm_wide_kernel<224,{args.out}" + (">" if bits == 8 else ",packed 4-bit codes>")
         roofline = {"kernel": k1 + " on ffn1 1024->4096", "bound": "hbm",
                     "achieved": dom["gbs"], "peak": pk["hbm_gbs"], "unit": "GB/s",
                     "frac": dom["gbs"] / pk["hbm_gbs"], "traffic": traffic.get("ffn1") if full_size else None,

@@ -1192,7 +1192,7 @@ static int make_store_map(CUtensorMap* ty, const LinearArgs& a, bool* tma_store,
                                  : EPI == EPI_Q8 ? CU_TENSOR_MAP_DATA_TYPE_UINT8 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16;
     if (!*tma_store)
         return make_map(ty, a.X, (uint64_t)a.tokens, (uint64_t)W.in / 4, 16, 32, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_DATA_TYPE_INT32, 4);
-    return make_map(ty, ybase, (uint64_t)a.tokens, (uint64_t)W.out, kNarrow<EPI> ? 16 : box_rows, kNarrow<EPI> ? 128 : 32, CU_TENSOR_MAP_SWIZZLE_NONE, dt, es);
+    return make_map(ty, ybase, (uint64_t)a.tokens, (uint64_t)W.out, box_rows, kNarrow<EPI> ? 128 : 32, CU_TENSOR_MAP_SWIZZLE_NONE, dt, es);
 }
 
 template <bool SPARSE, int BN, int EPI, int WSRC>
@@ -1370,7 +1370,6 @@ static int launch_gemm_wide(const LinearArgs& a) {
 // and small problems stay on the other kernels).
 template <int EPI>
 static int wide_bn(const LinearArgs& a) {
-    if (EPI != EPI_F32 && EPI != EPI_ACC) return 0;
     if (g_opt.no_wide || g_opt.no_pair) return 0;
     const nm_packed_t& W = *a.W;
     if (W.in <= kPairResStages * PairCfg<true, 192>::KB || W.out <= 2 * kBM) return 0;
@@ -1446,12 +1445,10 @@ static int check_linear(int tokens, int out, int in, int n, int m, int bits) {
 
 template <int EPI>
 static int run_linear_epi(const LinearArgs& a, bool xform, bool sparse) {
-    if constexpr (EPI == EPI_F32 || EPI == EPI_ACC) {
-        if (sparse && (!xform || xf::pattern_of(a.W->n, a.W->m, a.W->bits) == xf::P24_4)) {  // 2:4 with 8-bit or packed 4-bit codes
-            const int bn = wide_bn<EPI>(a);
-            if (bn == 224) return xform ? launch_gemm_wide<224, EPI, true>(a) : launch_gemm_wide<224, EPI>(a);
-            if (bn == 192) return xform ? launch_gemm_wide<192, EPI, true>(a) : launch_gemm_wide<192, EPI>(a);
-        }
+    if (sparse && (!xform || xf::pattern_of(a.W->n, a.W->m, a.W->bits) == xf::P24_4)) {  // 2:4 with 8-bit or packed 4-bit codes
+        const int bn = wide_bn<EPI>(a);
+        if (bn == 224) return xform ? launch_gemm_wide<224, EPI, true>(a) : launch_gemm_wide<224, EPI>(a);
+        if (bn == 192) return xform ? launch_gemm_wide<192, EPI, true>(a) : launch_gemm_wide<192, EPI>(a);
     }
     if (xform) return sparse ? pick_bn<true, EPI, true>(a) : pick_bn<false, EPI, true>(a);
     if (sparse) return use_pair<true, EPI>(a) ? pick_pair<true, EPI>(a) : pick_bn<true, EPI, false>(a);

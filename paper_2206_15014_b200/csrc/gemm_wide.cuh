@@ -34,6 +34,7 @@ constexpr int kWideThreads = 32 * (kWideMetaWarp0 + 4);  // producer, MMA, epilo
 // shared-memory bandwidth the MMAs and TMA already use up.)
 constexpr int kWideBuildWarps = 8;
 template <bool W4> constexpr int kWideThreadsOf = kWideThreads + (W4 ? 32 * kWideBuildWarps : 0);
+constexpr uint32_t kWideNarrowBar = 13;  // named barriers 13 and 14: the four epilogue warps of block 0 / block 1 (narrow outputs)
 constexpr uint32_t kWideRelayIds = 12;  // named barriers 1..12 carry the gate's relays in turn; the gate is never more
                                         // than STAGES + SKEW steps ahead of the MMA thread
 
@@ -72,7 +73,6 @@ nm_gemm_wide_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_con
     constexpr int S = Cfg::STAGES;
     static_assert(SKEW >= 0 && SKEW < S - 2, "the ring must hold the stages block 1 lags behind plus loads in flight");
     static_assert(S + SKEW < (int)kWideRelayIds, "relay barriers would be reused before the MMA thread has passed them");
-    static_assert(EPI == EPI_F32 || EPI == EPI_ACC, "32-bit outputs only");
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
     uint8_t* store_stage = smem + S * Cfg::STAGE;
@@ -362,6 +362,8 @@ nm_gemm_wide_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_con
         const float sx = p.sx_dev ? *p.sx_dev : p.sx_host;
         const uint32_t lead_acc_empty = ptx::map_to_cta(acc_empty_bar(blk), 0);
         float amax = 0.0f, c_n = 0.0f, b_n = 0.0f;
+        const float rsy = EPI == EPI_Q8 ? __frcp_rn(p.sy) : 0.0f;
+        uint32_t n_stores = 0;
         int scaled_out_tile = -1;
         bool ok = true;
         auto release_acc = [&]() {  // this warp has read all it needs from the accumulator
@@ -375,7 +377,9 @@ nm_gemm_wide_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_con
             const int n = nw + lane, t0 = tc.t * BN;
             bool got = ptx::mbar_wait_bounded(acc_full_bar(blk), (uint32_t)i & 1u, abort_flag, kWaitLimit);
             ok = __all_sync(0xffffffffu, got);
-            if (!ok) { if (lane == 0) raise_timeout(); break; }
+            if (!ok && lane == 0) raise_timeout();
+            if constexpr (kNarrow<EPI>) ok = ptx::named_bar_and(kWideNarrowBar + blk, 128, ok);  // the block's four warps stop together
+            if (!ok) break;
             ptx::tc_fence_after();
             if (ew == 0 && lane == 0) NM_TRACE_TILE(i, 0);
             if (ew == 4 && lane == 0) NM_TRACE_TILE(i, 2);
@@ -386,6 +390,73 @@ nm_gemm_wide_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_con
                 b_n = n_ok && p.bias ? p.bias[n] : 0.0f;
             }
             const int nact = min(CH, (p.tokens - t0 + 31) >> 5);  // chunks that hold tokens (warp-uniform)
+            if constexpr (kNarrow<EPI>) {
+                // int8 / bfloat16 outputs: the four warps of a block fill one [32 tokens][128 channels] staging tile per chunk
+                // together (two tiles per block, used alternately: rows of 128 / 256 bytes for the store), the warp of lane
+                // quarter 0 issues the store.  One named barrier per block orders the fills against the store.
+                using OT = typename EpiOut<EPI>::type;
+                const uint32_t gbar = kWideNarrowBar + blk;
+                const int n0b = nw - q * 32;  // first channel of the block
+                if (nact == 0) release_acc();
+#pragma unroll 1
+                for (int c = 0; c < nact; ++c) {
+                    const int tc0 = t0 + c * 32;
+                    uint32_t r[32];
+                    ptx::tmem_ld_32x32(acc_taddr + c * 32, r);
+                    ptx::tmem_ld_wait();
+                    if (c + 1 >= nact) release_acc();
+                    if (p.tma_store) {
+                        OT* sb = reinterpret_cast<OT*>(store_stage) + (blk * 2 + (n_stores & 1u)) * (32 * 128);
+                        if (q == 0 && lane == 0) ptx::bulk_wait_group_read<1>();  // the store before the last has read this tile
+                        ptx::named_bar_sync(gbar, 128);
+                        OT* mine = sb + q * 32 + lane;
+#pragma unroll
+                        for (int h = 0; h < 2; ++h) {
+                            if constexpr (EPI == EPI_Q8) {
+                                float worst = 0.0f;
+#pragma unroll
+                                for (int j = 0; j < 16; ++j) mine[(16 * h + j) * 128] = epi_convert_q8_fast(r[16 * h + j], c_n, b_n, rsy, worst);
+                                if (__any_sync(0xffffffffu, !(worst <= 0.49996948f))) {  // rare (3 % of the runs)
+                                    // find the values in question again; the exact division decides those
+#pragma unroll
+                                    for (int j = 0; j < 16; ++j) {
+                                        float w1 = 0.0f;
+                                        (void)epi_convert_q8_fast(r[16 * h + j], c_n, b_n, rsy, w1);
+                                        if (!(w1 <= 0.49996948f))
+                                            mine[(16 * h + j) * 128] =
+                                                (uint8_t)(int8_t)quantise8_exact_call(__fmaf_rn((float)(int)r[16 * h + j], c_n, b_n), p.sy);
+                                    }
+                                }
+                            } else {
+#pragma unroll
+                                for (int j = 0; j < 16; ++j) {
+                                    float y_abs;
+                                    mine[(16 * h + j) * 128] = epi_convert<EPI>(r[16 * h + j], c_n, b_n, p.sy, rsy, y_abs);
+                                }
+                            }
+                        }
+                        ptx::fence_proxy_async_smem();
+                        ptx::named_bar_sync(gbar, 128);
+                        if (q == 0 && lane == 0) {
+                            ptx::tma_store_2d_hint(&tmap_y, n0b, tc0, ptx::smem_u32(sb), stream_out);
+                            ptx::bulk_commit_group();
+                        }
+                        ++n_stores;
+                    } else {
+                        const int jmax = n_ok ? min(32, p.tokens - tc0) : 0;  // outputs of this lane that exist
+                        OT* dst = reinterpret_cast<OT*>(p.NARROW) + (size_t)tc0 * p.out + n;
+#pragma unroll
+                        for (int j = 0; j < 32; ++j) {
+                            float y_abs;
+                            const OT o = epi_convert<EPI>(r[j], c_n, b_n, p.sy, rsy, y_abs);
+                            if (j < jmax) dst[(size_t)j * p.out] = o;
+                        }
+                    }
+                }
+                if (ew == 0 && lane == 0) NM_TRACE_TILE(i, 1);
+                if (ew == 4 && lane == 0) NM_TRACE_TILE(i, 3);
+                continue;
+            }
             constexpr int RB = W4 ? 1 : 2;  // chunk read one ahead of its conversion, except where registers are short
             uint32_t r[RB][32];
             if (nact == 0) release_acc();

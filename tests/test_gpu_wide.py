@@ -4,7 +4,8 @@ memory by its builder warps; reduction longer than 1024) against the CPU oracle.
 The library picks that kernel only for problems with at least one tile per SM pair; the option "wide_any"
 sends every eligible shape to it, so that small and ragged cases (one tile, a ragged last token tile, an output
 that does not fill the second block of 128 channels, few and many pipeline stages per tile, a pair that walks
-several tiles and changes output tile) reach it too.  int32 accumulators bit for bit, fp32 outputs equal.
+several tiles and changes output tile) reach it too.  int32 accumulators bit for bit, fp32 outputs equal, and the
+kernel's int8 and bfloat16 outputs bit for bit.
 """
 import numpy as np
 import pytest
@@ -26,7 +27,7 @@ def wide_kernel_everywhere(request):
     nm.nm_debug_set_option("wide_bn", 0)
 
 
-def _run(seed, T, K, out, tie=False, bias=True, bits=8):
+def _run(seed, T, K, out, tie=False, bias=True, bits=8, narrow=True):
     from gpu_util import PackedOnDevice, gpu_int_linear, assert_close
     oracle.set_threads(oracle.max_threads())
     rng = np.random.default_rng(seed)
@@ -41,6 +42,15 @@ def _run(seed, T, K, out, tie=False, bias=True, bits=8):
     assert np.array_equal(acc, acc_ref), f"{(acc != acc_ref).sum()} accumulators differ"
     assert_close(Y, Y_ref)
     assert np.array_equal(Y, Y_ref)
+    if narrow:   # the same kernel's int8 (two scales: full range; two thirds of the outputs clamp) and bfloat16 outputs
+        from gpu_util import gpu_int_linear_q8, gpu_int_linear_bf16
+        amax = np.float32(np.abs(Y_ref).max())
+        for sy in (amax / np.float32(127.0), amax / np.float32(40.0)):
+            ref = oracle.requantize_static(Y_ref, sy)
+            got = gpu_int_linear_q8(Xq, packed, sx, b if bias else None, sy)
+            assert np.array_equal(got, ref), f"{(got != ref).sum()} of {ref.size} codes differ at sy={sy}"
+        got = gpu_int_linear_bf16(Xq, packed, sx, b if bias else None)
+        assert np.array_equal(got, oracle.to_bf16(Y_ref)), "bfloat16 patterns differ"
 
 
 @pytest.mark.parametrize("T,K,out", [
