@@ -1183,7 +1183,7 @@ struct LinearArgs {
 // through TMA when the output can be described by a tensor map (16-byte aligned base and row pitch);
 // otherwise *tma_store is cleared, the threads store directly and the map describes X as a stand-in.
 template <int EPI>
-static int make_store_map(CUtensorMap* ty, const LinearArgs& a, bool* tma_store, uint32_t box_rows = 16) {
+static int make_store_map(CUtensorMap* ty, const LinearArgs& a, bool* tma_store, uint32_t box_rows = 16, uint32_t box_cols = 0) {
     const nm_packed_t& W = *a.W;
     constexpr uint32_t es = (uint32_t)sizeof(typename EpiOut<EPI>::type);
     void* ybase = EPI == EPI_F32 ? (void*)a.Y : EPI == EPI_ACC ? (void*)a.ACC : a.NARROW;
@@ -1192,7 +1192,7 @@ static int make_store_map(CUtensorMap* ty, const LinearArgs& a, bool* tma_store,
                                  : EPI == EPI_Q8 ? CU_TENSOR_MAP_DATA_TYPE_UINT8 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16;
     if (!*tma_store)
         return make_map(ty, a.X, (uint64_t)a.tokens, (uint64_t)W.in / 4, 16, 32, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_DATA_TYPE_INT32, 4);
-    return make_map(ty, ybase, (uint64_t)a.tokens, (uint64_t)W.out, box_rows, kNarrow<EPI> ? 128 : 32, CU_TENSOR_MAP_SWIZZLE_NONE, dt, es);
+    return make_map(ty, ybase, (uint64_t)a.tokens, (uint64_t)W.out, box_rows, box_cols ? box_cols : (kNarrow<EPI> ? 128 : 32), CU_TENSOR_MAP_SWIZZLE_NONE, dt, es);
 }
 
 template <bool SPARSE, int BN, int EPI, int WSRC>

@@ -355,6 +355,9 @@ nm_gemm_wide_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_con
         // ------------------------------ epilogue warps (both CTAs) --------------------------------
         // Warps 2-5 read block 0's accumulator, warps 6-9 block 1's; each its TMEM lane quarter, all BN columns.
         constexpr int CH = BN / 32;
+        // narrow outputs leave through staging tiles that a block's four warps share; for 32-bit outputs that form (one
+        // 16 KB tile per block) was measured slower than a tile per warp (FFN2 alone 44.6 against 42.5 us)
+        constexpr bool kGroupEpi = kNarrow<EPI>;
         const int ew = warp - 2, q = warp & 3, blk = ew >> 2;
         const uint32_t acc_taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)blk * BN;
         uint32_t* my_stage = reinterpret_cast<uint32_t*>(store_stage + ew * 4096);
@@ -378,7 +381,7 @@ nm_gemm_wide_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_con
             bool got = ptx::mbar_wait_bounded(acc_full_bar(blk), (uint32_t)i & 1u, abort_flag, kWaitLimit);
             ok = __all_sync(0xffffffffu, got);
             if (!ok && lane == 0) raise_timeout();
-            if constexpr (kNarrow<EPI>) ok = ptx::named_bar_and(kWideNarrowBar + blk, 128, ok);  // the block's four warps stop together
+            if constexpr (kGroupEpi) ok = ptx::named_bar_and(kWideNarrowBar + blk, 128, ok);  // the block's four warps stop together
             if (!ok) break;
             ptx::tc_fence_after();
             if (ew == 0 && lane == 0) NM_TRACE_TILE(i, 0);
@@ -390,7 +393,7 @@ nm_gemm_wide_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_con
                 b_n = n_ok && p.bias ? p.bias[n] : 0.0f;
             }
             const int nact = min(CH, (p.tokens - t0 + 31) >> 5);  // chunks that hold tokens (warp-uniform)
-            if constexpr (kNarrow<EPI>) {
+            if constexpr (kGroupEpi) {
                 // int8 / bfloat16 outputs: the four warps of a block fill one [32 tokens][128 channels] staging tile per chunk
                 // together (two tiles per block, used alternately: rows of 128 / 256 bytes for the store), the warp of lane
                 // quarter 0 issues the store.  One named barrier per block orders the fills against the store.
@@ -406,8 +409,10 @@ nm_gemm_wide_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_con
                     ptx::tmem_ld_wait();
                     if (c + 1 >= nact) release_acc();
                     if (p.tma_store) {
-                        OT* sb = reinterpret_cast<OT*>(store_stage) + (blk * 2 + (n_stores & 1u)) * (32 * 128);
-                        if (q == 0 && lane == 0) ptx::bulk_wait_group_read<1>();  // the store before the last has read this tile
+                        constexpr int NBUF = sizeof(OT) == 4 ? 1 : 2;  // 32 KB of staging: one 16 KB tile per block, or two smaller ones
+                        OT* sb = reinterpret_cast<OT*>(store_stage) + (blk * NBUF + (NBUF == 2 ? (n_stores & 1u) : 0u)) * (32 * 128);
+                        const int jmax = n_ok ? min(32, p.tokens - tc0) : 0;  // outputs of this lane that exist
+                        if (q == 0 && lane == 0) ptx::bulk_wait_group_read<NBUF - 1>();  // the store that last used this tile has read it
                         ptx::named_bar_sync(gbar, 128);
                         OT* mine = sb + q * 32 + lane;
 #pragma unroll
@@ -432,6 +437,7 @@ nm_gemm_wide_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_con
                                 for (int j = 0; j < 16; ++j) {
                                     float y_abs;
                                     mine[(16 * h + j) * 128] = epi_convert<EPI>(r[16 * h + j], c_n, b_n, p.sy, rsy, y_abs);
+                                    if constexpr (EPI == EPI_F32) amax = fmaxf(amax, 16 * h + j < jmax ? y_abs : 0.0f);
                                 }
                             }
                         }
@@ -444,11 +450,12 @@ nm_gemm_wide_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_con
                         ++n_stores;
                     } else {
                         const int jmax = n_ok ? min(32, p.tokens - tc0) : 0;  // outputs of this lane that exist
-                        OT* dst = reinterpret_cast<OT*>(p.NARROW) + (size_t)tc0 * p.out + n;
+                        OT* dst = reinterpret_cast<OT*>(EPI == EPI_F32 ? (void*)p.Y : EPI == EPI_ACC ? (void*)p.ACC : p.NARROW) + (size_t)tc0 * p.out + n;
 #pragma unroll
                         for (int j = 0; j < 32; ++j) {
                             float y_abs;
                             const OT o = epi_convert<EPI>(r[j], c_n, b_n, p.sy, rsy, y_abs);
+                            if constexpr (EPI == EPI_F32) amax = fmaxf(amax, j < jmax ? y_abs : 0.0f);
                             if (j < jmax) dst[(size_t)j * p.out] = o;
                         }
                     }
