@@ -2,7 +2,7 @@
 that every kernel variant (CTA pairs with resident or streamed weights, one-CTA kernels with 192 / 128 / 64
 token tiles, weight tiles built in shared memory per k-block or once per output tile) meets ragged token
 and channel tails, single tiles and ranges that cross output tiles.  Accumulators bit for bit, fp32
-outputs equal, int8 outputs bit for bit."""
+outputs equal, int8 and bfloat16 outputs bit for bit (every third seed each)."""
 import numpy as np
 import pytest
 
@@ -56,6 +56,9 @@ def test_random_shape(seed):
     if seed % 3 == 0:
         sy = np.float32(max(np.abs(Y_ref).max(), 1e-3)) / np.float32(100.0)
         assert np.array_equal(gpu_int_linear_q8(Xq, packed, sx, b, sy), oracle.requantize_static(Y_ref, sy)), tag
+    if seed % 3 == 1:
+        from gpu_util import gpu_int_linear_bf16
+        assert np.array_equal(gpu_int_linear_bf16(Xq, packed, sx, b), oracle.to_bf16(Y_ref)), tag
 
 
 PACK_PATTERNS = [(1, 4), (2, 4), (1, 8), (2, 8), (4, 8), (4, 4)]
