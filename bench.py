@@ -1017,7 +1017,10 @@ def trace_gemm(args):
                       "producer_issue_clk": med((d[:, 1] - d[:, 0])[ok]), "load_issue_to_full_clk": med((d[:, 2] - d[:, 1])[ok]),
                       "gate_to_mma_handoff_clk": med((d[:, 3] - d[:, 2])[ok]), "mma_issue_clk": med(d[:, 4] - d[:, 3]),
                       "clk_per_stage_steady": med(np.diff(d[:, 3])), "first_stage_full_clk": float(d[0, 2]),
-                      "last_mma_issued_clk": float(d[-1, 4]), "tiles": tiles}))
+                      "last_mma_issued_clk": float(d[-1, 4]), "tiles": tiles,
+                      # per stage: when the MMA thread was handed it, and how long its loads took from issue to arrival
+                      "stage_handed_to_mma_clk": [int(x) for x in d[:, 3]],
+                      "stage_load_clk": [int(x) if k else -1 for x, k in zip(d[:, 2] - d[:, 1], ok)]}))
     return 0
 
 
