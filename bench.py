@@ -332,8 +332,29 @@ def extra_configs(nm, torch, dev, pk, status):
         call(i)
         torch.cuda.synchronize()
         lat.append((time.perf_counter() - t0) * 1e6)
+    # the same launches replayed from a CUDA graph: what the device needs per launch without the host's share
+    # (Python, ctypes and the launch call cost more than this kernel runs)
+    graph_us = None
+    try:
+        side = torch.cuda.Stream()
+        side.wait_stream(torch.cuda.current_stream())
+        with torch.cuda.stream(side):
+            for i in range(8):
+                call(i)
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g, stream=side):
+                for i in range(64):
+                    call(i)
+            torch.cuda.synchronize()
+            graph_us = time_stream(torch, lambda i: g.replay(), 20, warm=3) / 64
+        torch.cuda.current_stream().wait_stream(side)
+        torch.cuda.synchronize()
+    except Exception as e:   # a capture failure must not cost the benchmark line
+        graph_us = None
+        print("graph replay of the single projection failed: " + repr(e), file=sys.stderr)
     out["single_projection_128x768"] = {"latency_us_call_to_completion": float(np.median(lat[10:])),
                                         "us_back_to_back": time_stream(torch, call, 400),
+                                        "us_back_to_back_from_a_graph": graph_us,
                                         "note": "all operands resident in L2: a latency figure, no roofline"}
     # ---- configurations 2 and 3: encoder-layer GEMMs, one launch after the other ------------------------------------
     for key, gemms, tokens, bits in (("bert_base_4096tok_int8", wl.BERT_BASE_GEMMS, 4096, 8),
