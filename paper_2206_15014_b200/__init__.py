@@ -114,14 +114,15 @@ def _chk(code, where):
 
 
 def _ptr(t):
-    return None if t is None else ctypes.c_void_p(t.data_ptr())
+    # a plain int converts to void* through the declared argtypes; no ctypes object per argument
+    return None if t is None else t.data_ptr()
 
 
 def _stream(stream=None):
     if stream is None:
         import torch
-        return ctypes.c_void_p(torch.cuda.current_stream().cuda_stream)
-    return ctypes.c_void_p(int(stream))
+        return torch.cuda.current_stream().cuda_stream
+    return int(stream)
 
 
 def nm_strerror(code):
