@@ -138,6 +138,31 @@ def test_bert_large_full_size(name, k, out, bits):
     assert np.array_equal(Yh[:T], Yr), f"{(Yh[:T] != Yr).sum()} of {Yr.size} outputs differ"
 
 
+@pytest.mark.parametrize("name,k,out", wl.BERT_LARGE_GEMMS)
+def test_bert_large_full_size_narrow_outputs(name, k, out):
+    """16384 tokens, 2:4 int8 weights, the launch configurations `bench.py --out int8 | bf16` times (sixteen epilogue warps
+    on the resident-weight kernel, shared staging tiles on the 512-channel kernel): every int8 code and every bfloat16
+    pattern of the launch against the oracle."""
+    from gpu_util import PackedOnDevice, gpu_int_linear_q8, gpu_int_linear_bf16
+    oracle.set_threads(oracle.max_threads())
+    T = 16384
+    rng = np.random.default_rng([6, k, out])
+    W = wl.normal(rng, (out, k), wl.W_STD)
+    b = wl.normal(rng, (out,), wl.W_STD)
+    Xq = wl.random_int8([7, k, out], (T, k))
+    v, meta, s = oracle.project_pack(W, None, 2, 4, 8)
+    D = oracle.unpack(v, meta, out, k, 2, 4, 8)
+    _, Yr = oracle.int_linear(Xq, D, 0.03, s, b, want_acc=False)
+    packed = PackedOnDevice(v, meta, s, out, k, 2, 4, 8)
+    sy = np.float32(np.abs(Yr).max()) / np.float32(100.0)       # a few outputs clamp
+    got = gpu_int_linear_q8(Xq, packed, 0.03, b, sy)
+    ref = oracle.requantize_static(Yr, sy)
+    assert np.array_equal(got, ref), f"{(got != ref).sum()} of {ref.size} int8 codes differ"
+    got = gpu_int_linear_bf16(Xq, packed, 0.03, b)
+    ref = oracle.to_bf16(Yr)
+    assert np.array_equal(got, ref), f"{(got != ref).sum()} of {ref.size} bfloat16 patterns differ"
+
+
 def test_pack_sweep_full_size_batched():
     """One batched launch over a full BERT-large layer (2:4, 8 bit) against the oracle, bit for bit."""
     import paper_2206_15014_b200 as nm
