@@ -384,7 +384,7 @@ nm_gemm_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant
             for (int kb = 0; kb < p.kblocks; ++kb, ++it) {
                 wait(full_bar(it % S), (it / S) & 1u);
                 __syncwarp();
-                ptx::named_bar_arrive(1 + (it & 7u), 64);
+                ptx::relay_step(1 + (it & 7u), abort_flag);
             }
         }
     } else if (warp == 1) {
@@ -833,7 +833,7 @@ nm_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_con
                     wait(full_bar(it % S), (it / S) & 1u);
                     if (lane == 0) NM_TRACE_STAGE(it, 2);
                     __syncwarp();
-                    ptx::named_bar_arrive(1 + (it & 7u), 64);
+                    ptx::relay_step(1 + (it & 7u), abort_flag);
                 }
             }
         }

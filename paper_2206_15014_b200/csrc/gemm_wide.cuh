@@ -296,7 +296,7 @@ nm_gemm_wide_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_con
                     if (++kb_t == p.kblocks) { kb_t = 0; ++tile_t; }
                 }
                 __syncwarp();
-                ptx::named_bar_arrive(relay, 64);
+                ptx::relay_step(relay, abort_flag);
                 relay = relay == kWideRelayIds ? 1 : relay + 1;
             }
         }

@@ -99,6 +99,15 @@ __device__ __forceinline__ void named_bar_arrive(uint32_t id, uint32_t threads) 
     asm volatile("bar.arrive %0, %1;" ::"r"(id), "r"(threads) : "memory");
 }
 
+// The gate warp's hand-off of one pipeline step to the MMA warp (two warps, 64 threads).  Normally an arrive: the gate runs
+// ahead of the MMA warp by as many steps as it has found ready.  Once a bounded wait has expired anywhere in the CTA the gate
+// no longer waits for data; it would then lap the MMA warp on the ring of named barriers (arriving twice on an id the
+// MMA warp has not reached), so from then on it meets the MMA warp at every step.
+__device__ __forceinline__ void relay_step(uint32_t id, volatile uint32_t* abort_flag) {
+    if (__any_sync(0xffffffffu, *abort_flag != 0u)) named_bar_sync(id, 64);
+    else named_bar_arrive(id, 64);
+}
+
 // Named barrier that also ANDs a predicate over its `threads` participants: everyone gets the same answer.
 __device__ __forceinline__ bool named_bar_and(uint32_t id, uint32_t threads, bool pred) {
     uint32_t out;
