@@ -36,8 +36,7 @@ constexpr int kWideThreads = 32 * (kWideMetaWarp0 + 4);  // producer, MMA, epilo
 // One builder warp per ring slot, building the slot's whole tile with a single proxy fence, 66.4 us: a lone warp needs
 // about 2.5 k clk per tile, nearly the ring's whole lead.  Two groups of four warps on alternate stages, two rows per
 // thread: 61.0 us.  Fetch distances of two and three stages: 58.6 and 59.5 us.  Six builder warps, none of them on the
-// MMA warp's scheduler: 69.5 us.  The figures fit a builder warp that needs about 300 clk per row it builds plus about 600 clk
-// per stage for the proxy fence and the arrival, i.e. 900 clk per stage as it stands.)
+// MMA warp's scheduler: 69.5 us.  Sixteen builder warps in two groups on alternate stages (64 registers per thread): 87.8 us.)
 constexpr int kWideBuildWarps = 8;
 template <bool W4> constexpr int kWideThreadsOf = kWideThreads + (W4 ? 32 * kWideBuildWarps : 0);
 constexpr uint32_t kWideNarrowBar = 13;  // named barriers 13 and 14: the four epilogue warps of block 0 / block 1 (narrow outputs)
