@@ -459,7 +459,7 @@ def ffn1_stream_probe(nm, torch, dev, d, tokens, status):
     """The resident-weight pair kernel's traffic on one GEMM without its arithmetic (nm_probe_tma_stream): X loads
     through the ring + Y stores, and Y stores alone.  Times from the CTAs' own globaltimer stamps, median of three."""
     import numpy as np
-    clocks = torch.zeros((148, 4), dtype=torch.int64, device=dev)
+    clocks = torch.zeros((torch.cuda.get_device_properties(dev).multi_processor_count, 4), dtype=torch.int64, device=dev)
     out, k = d["out"], d["k"]
     res = {}
     for name, loads, stores in (("loads_and_stores_us", 2, 1), ("stores_only_us", 0, 1)):
@@ -912,7 +912,7 @@ def tma_probe(args):
     dev = torch.device("cuda:0")
     torch.cuda.set_device(dev)
     status = torch.zeros(1, dtype=torch.int32, device=dev)
-    clocks = torch.zeros((148, 4), dtype=torch.int64, device=dev)
+    clocks = torch.zeros((torch.cuda.get_device_properties(dev).multi_processor_count, 4), dtype=torch.int64, device=dev)
 
     def case(name, out, k, tokens, a_rows, a_row_bytes, b_rows, b_slices, stages, band=0, repeat=1, delay=0, loads=3,
              stores=1, producers=1):
